@@ -1,0 +1,152 @@
+/*
+ * libmst: the unstructured-sparse fully-connected layer of Mixed Sparsity Training
+ * (arXiv 2408.11746) for NVIDIA B200 (sm_100a).
+ *
+ * One handle = one layer theta_l [O x I] (out_features x in_features, row-major, PyTorch layout)
+ * under a binary mask M (Sec. 3.2).  The layer is stored as canonical CSR (columns ascending in
+ * each row) plus a CSC view; the flat index of entry (o, i) is o*I + i.
+ *
+ * Conventions for every call
+ *   - returns mst_status_t; nothing throws, aborts, traps or spins without bound.
+ *   - every pointer named "device" is a CUDA device pointer owned by the caller; the handle owns
+ *     its sparse arrays and its scratch, sized once for nnz_capacity (never reallocated).
+ *   - leading dimensions (ld*) are in elements; activations are row-major [tokens x features].
+ *   - element type of X, Y, dY, dX, W and the stored values is the layer's dtype
+ *     (MST_F32: float; MST_BF16: 16-bit bfloat16 patterns); accumulation is always fp32.
+ *   - work is enqueued on the caller's stream and is stream-ordered; calls that return data to
+ *     host memory (stats, nnz) synchronise that stream.
+ *   - argument, shape, dtype, capacity and count errors are detected on the host before any
+ *     launch.  Problems only the device can see (a non-finite selection key, a corrupt structure)
+ *     set a sticky flag in handle-owned memory that mst_validate and mst_topology_update(stats)
+ *     report.
+ */
+#ifndef MST_H_
+#define MST_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mst_layer mst_layer_t;
+typedef void* mst_stream_t; /* a cudaStream_t; NULL = the default stream */
+
+typedef enum { MST_F32 = 0, MST_BF16 = 1 } mst_dtype_t;
+
+typedef enum {
+  MST_OK = 0,
+  MST_ERR_INVALID_ARG = 1, /* NULL pointer, negative size, value outside its range          */
+  MST_ERR_SHAPE = 2,       /* leading dimension smaller than the row, feature count > 65535   */
+  MST_ERR_DTYPE = 3,       /* unknown dtype                                                   */
+  MST_ERR_CAPACITY = 4,    /* nnz (or target nnz) exceeds the capacity given at creation      */
+  MST_ERR_INFEASIBLE = 5,  /* no prune/grow counts satisfy the request                        */
+  MST_ERR_NONFINITE = 6,   /* Inf/NaN met in |w| or |g| while selecting                       */
+  MST_ERR_CORRUPT = 7,     /* sparse structure fails validation                               */
+  MST_ERR_CUDA = 8,        /* a CUDA runtime call failed                                      */
+  MST_ERR_NOT_PACKED = 9   /* the layer has no structure yet (call mst_pack first)            */
+} mst_status_t;
+
+/* Growth rule of one topology update (Algorithm 1; Table "Comparison of different topology evolution schemes").
+ *   target_nnz          active entries after the update, (1 - s_l') N_l; < 0 keeps the current count
+ *   random_ratio        R in [0,1], share of grown links drawn at random (0 = RigL rule, 1 = SET rule)
+ *   seed, step          the random-growth ranking is a pure function of (seed, step, layer_id, flat index):
+ *                       candidates are ranked by SplitMix64 outputs (smaller first, ties by flat index)
+ *   allow_regrow_pruned 0: links pruned in this update are not candidates for growth (default reading);
+ *                       1: gradient growth may also pick just-pruned links (such a link keeps its value) */
+typedef struct {
+  int64_t target_nnz;
+  double random_ratio;
+  uint64_t seed;
+  uint64_t step;
+  int32_t allow_regrow_pruned;
+} mst_regrow_rule_t;
+
+typedef struct {
+  int64_t nnz_before, nnz_after, n_prune, n_grad, n_rand, max_row_nnz;
+} mst_update_stats_t;
+
+/* Create an empty layer.  out_features, in_features in [1, 65535]; nnz_capacity in [1, O*I].
+ * Allocates all device memory the layer will ever use on the current device. */
+mst_status_t mst_layer_create(mst_layer_t** layer, int32_t layer_id, int32_t out_features, int32_t in_features,
+                              mst_dtype_t dtype, int64_t nnz_capacity);
+mst_status_t mst_layer_destroy(mst_layer_t* layer);
+
+/* Number of active entries (host value; known after mst_pack / mst_topology_update without a sync). */
+mst_status_t mst_layer_nnz(const mst_layer_t* layer, int64_t* nnz);
+
+/* Dense mask -> sparse structure (Sec. 3.2: the binary mask M_theta; Algorithm 1: theta <- theta . M).
+ *   W_dense  device, [O x ldw] in the layer's dtype; only entries under the mask are read
+ *   mask     device, uint8 [O x I] contiguous, non-zero = active
+ * Builds CSR, the CSC view and the bit mask.  Synchronises the stream (returns nnz to the host);
+ * MST_ERR_CAPACITY if the mask holds more than nnz_capacity entries (layer left unpacked). */
+mst_status_t mst_pack(mst_layer_t* layer, const void* W_dense, int64_t ldw, const uint8_t* mask, mst_stream_t stream);
+
+/* Canonical CSR out: row_ptr int32 [O+1], col_idx int32 [nnz], vals [nnz] in the layer's dtype; all device,
+ * any of the three may be NULL to skip it. */
+mst_status_t mst_export_csr(const mst_layer_t* layer, int32_t* row_ptr, int32_t* col_idx, void* vals,
+                            mst_stream_t stream);
+/* CSC view out: col_ptr int32 [I+1], row_idx int32 [nnz] (rows ascending in each column),
+ * perm int32 [nnz] = CSR position of each CSC entry; device; any may be NULL. */
+mst_status_t mst_export_csc(const mst_layer_t* layer, int32_t* col_ptr, int32_t* row_idx, int32_t* perm,
+                            mst_stream_t stream);
+
+/* Device pointer to the stored values (CSR order, layer dtype) so an optimizer can update them in place.
+ * The pointer changes at every mst_pack / mst_topology_update. */
+mst_status_t mst_values(mst_layer_t* layer, void** vals, int64_t* nnz);
+
+/* Structure check on the device: row pointers monotone and ending at nnz, columns in range and strictly
+ * ascending, CSC consistent with CSR, bit mask consistent.  Synchronises.  MST_ERR_CORRUPT / MST_ERR_NONFINITE
+ * (sticky flag from an earlier update) or MST_OK. */
+mst_status_t mst_validate(const mst_layer_t* layer, mst_stream_t stream);
+
+/* Forward, Y[t,o] = sum_{i:(o,i) in M} W[o,i] X[t,i]   (Algorithm 1: the layer computes with theta . M; no bias;
+ * cost (1-S)(2I-1)O per token, Eq. (3)).  X device [T x ldx], Y device [T x ldy]. */
+mst_status_t mst_spmm_fwd(const mst_layer_t* layer, const void* X, int64_t ldx, int64_t T, void* Y, int64_t ldy,
+                          mst_stream_t stream);
+
+/* Input gradient, dX[t,i] = sum_{o:(o,i) in M} dY[t,o] W[o,i]   (App. "FLOP Calculation": backward = 2 x forward).
+ * dY device [T x lddy], dX device [T x lddx].  Uses the CSC view: a gather, no floating-point atomics. */
+mst_status_t mst_spmm_bwd_x(const mst_layer_t* layer, const void* dY, int64_t lddy, int64_t T, void* dX, int64_t lddx,
+                            mst_stream_t stream);
+
+/* Weight gradient on the mask only, dW[k] = sum_t dY[t,o_k] X[t,i_k] for the k-th active entry in CSR order
+ * (same passage).  dW_vals device float [nnz]. */
+mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,
+                          float* dW_vals, mst_stream_t stream);
+
+/* Dense gradient for growth, G = dY^T X, float [O x I] contiguous (Algorithm 1, gradient-growth line: |grad L| on
+ * empty slots; Sec. 2.1 "infrequent full gradient calculation").  No layer handle: a plain contraction. */
+mst_status_t mst_dense_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int32_t out_features,
+                            int32_t in_features, mst_dtype_t dtype, float* G, mst_stream_t stream);
+
+/* Counts of one update (Algorithm 1, count lines), as the library computes them on the host:
+ *   n_prune = clamp(floor(prune_frac * nnz), max(0, nnz - target), min(nnz, N - target)),
+ *   n_grow = n_prune + target - nnz, n_rand = floor(n_grow * R), n_grad = n_grow - n_rand.
+ * counts = {n_prune, n_grow, n_rand, n_grad}. */
+mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_t target_nnz, int64_t numel, double random_ratio,
+                               int64_t counts[4]);
+
+/* One Mixed-Growing topology update (Algorithm 1): prune the n_prune active entries of smallest |w|, grow the n_grad
+ * empty slots of largest |g| and n_rand more at random, rewrite the mask, drop pruned values, start grown values at
+ * +0.0, rebuild CSR/CSC in place.  Ties are broken by the smaller flat index.  Selection is bit-exact and
+ * deterministic.
+ *   prune_frac  zeta in [0,1]
+ *   G_dense     device float [O x I] contiguous; may be NULL iff n_grad == 0
+ *   stats       host, may be NULL; when given the call synchronises and reports device-side errors */
+mst_status_t mst_topology_update(mst_layer_t* layer, double prune_frac, const mst_regrow_rule_t* regrow_rule,
+                                 const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream);
+
+/* One training step of the layer from HOST buffers (pinned memory recommended): copies X [T x I] and dY [T x O]
+ * (contiguous, layer dtype) to the device, runs forward, input gradient and weight gradient, and copies
+ * Y [T x O], dX [T x I] (layer dtype) and dW_vals float [nnz] back.  Any output may be NULL to skip its copy.
+ * Staging buffers live in the handle and grow on demand.  Synchronises the stream. */
+mst_status_t mst_layer_step_host(mst_layer_t* layer, const void* X_host, const void* dY_host, int64_t T, void* Y_host,
+                                 void* dX_host, float* dW_vals_host, mst_stream_t stream);
+
+const char* mst_status_string(mst_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MST_H_ */

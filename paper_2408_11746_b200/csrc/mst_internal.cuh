@@ -1,0 +1,87 @@
+// Internal declarations shared by the translation units of libmst (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mst.h"
+
+#define MST_CUDA_TRY(expr)                       \
+  do {                                           \
+    cudaError_t e__ = (expr);                    \
+    if (e__ != cudaSuccess) return MST_ERR_CUDA; \
+  } while (0)
+
+#define MST_TRY(expr)                   \
+  do {                                  \
+    mst_status_t s__ = (expr);          \
+    if (s__ != MST_OK) return s__;      \
+  } while (0)
+
+// Device-side error flag bits (sticky, in handle-owned memory).
+enum { MST_FLAG_NONFINITE = 1, MST_FLAG_CORRUPT = 2 };
+
+// Scratch of one radix-select run (device resident; nothing comes back to the host).
+struct mst_select_state {
+  unsigned long long prefix;  // digits fixed so far (left-aligned into the low bits as they are found)
+  long long k;                // how many more entries to take among those matching the prefix
+  unsigned long long tau;     // final threshold key
+  long long rem;              // entries equal to tau to take, in index order
+};
+
+struct mst_layer {
+  int32_t layer_id, O, I;
+  mst_dtype_t dtype;
+  int64_t cap, N;
+  int32_t wpr;        // 32-bit mask words per row      = ceil(I/32)
+  int32_t wpc;        // mask words per transposed row  = ceil(O/32)
+  int64_t nwords;     // O * wpr
+  int64_t nwordsT;    // I * wpc
+  int64_t nnz;        // host copy, -1 = not packed
+  int cur;            // which of the two buffer sets is live
+
+  // live structure is set [cur]; a topology update builds set [cur^1] and flips
+  uint32_t* bits[2];     // [nwords]    bit (o, i) at word o*wpr + i/32, bit i%32
+  int32_t* wscan[2];     // [nwords+1]  exclusive scan of popc(bits): CSR position of a word's first entry
+  int32_t* row_ptr[2];   // [O+1]
+  uint16_t* col_idx[2];  // [cap]
+  void* vals[2];         // [cap] layer dtype
+
+  // CSC view of the live structure
+  uint32_t* bitsT;       // [nwordsT]
+  int32_t* wscanT;       // [nwordsT+1]
+  int32_t* col_ptr;      // [I+1]
+  uint16_t* row_idx;     // [cap]
+  int32_t* perm;         // [cap]  CSR position of each CSC entry
+
+  // scratch for selection and rebuild
+  uint32_t* pruned_bits;  // [nwords]
+  uint32_t* grad_bits;    // [nwords]
+  uint32_t* rand_bits;    // [nwords]
+  int32_t* word_cnt;      // [max(nwords, nwordsT)+1]
+  int32_t* word_scan;     // [max(nwords, nwordsT)+1]
+  int32_t* block_sums;    // scan partials
+  unsigned int* hist;     // [256]
+  mst_select_state* sel;  // [1]
+  int32_t* flags;         // [4]: error bits, max row nnz, spare
+  unsigned int* counter;  // [1] block-completion counter
+
+  // host staging for mst_layer_step_host
+  void *stg_x, *stg_dy, *stg_y, *stg_dx;
+  float* stg_dw;
+  int64_t stg_tokens;
+};
+
+static inline size_t mst_elem_size(mst_dtype_t d) { return d == MST_F32 ? 4 : 2; }
+
+// structure (mst_structure.cu)
+mst_status_t mst_scan_i32(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t s);
+int64_t mst_scan_block_sums_len(int64_t n);
+mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set, cudaStream_t s);
+mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s);
+mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
+
+// kernels' launchers
+mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in, int64_t ldin, int64_t T, void* out,
+                             int64_t ldout, cudaStream_t s);
+mst_status_t mst_launch_sddmm(const mst_layer* L, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,
+                              float* dW, cudaStream_t s);

@@ -1,0 +1,411 @@
+// Sparse structure of a layer: bit mask -> CSR (+ CSC view) by popcount, exclusive prefix scan and fill.
+//
+// The mask is kept as 32-bit words, wpr words per row.  Because canonical CSR order (rows ascending,
+// columns ascending) is the order of the flat index o*I+i, the CSR position of an entry is the number of
+// set bits before it: an exclusive scan of the per-word popcounts plus a popcount inside the word.
+// The same holds for the CSC view on the transposed bit mask.  Everything below is integer work,
+// stream-ordered, with no inter-block waiting (the scan is three plain kernels).
+#include "mst_internal.cuh"
+
+#include <cuda_bf16.h>
+
+namespace {
+
+constexpr int SCAN_THREADS = 256;
+constexpr int SCAN_ITEMS = 8;
+constexpr int SCAN_TILE = SCAN_THREADS * SCAN_ITEMS;
+
+__device__ __forceinline__ unsigned lanemask_lt() {
+  unsigned m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// ---- exclusive scan of int32, n up to 2^31: out[0..n], out[n] = total -------------------------
+__device__ int block_reduce_sum(int v, int* sh) {
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = 0;
+  if (threadIdx.x < 32) {
+    r = threadIdx.x < (blockDim.x >> 5) ? sh[threadIdx.x] : 0;
+    for (int o = 16; o; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+  }
+  __syncthreads();
+  return r;  // valid in warp 0
+}
+
+__global__ void scan_tile_sums(const int32_t* __restrict__ in, int64_t n, int32_t* __restrict__ sums) {
+  __shared__ int sh[32];
+  const int64_t base = (int64_t)blockIdx.x * SCAN_TILE;
+  int v = 0;
+  for (int j = 0; j < SCAN_ITEMS; ++j) {
+    const int64_t i = base + (int64_t)j * SCAN_THREADS + threadIdx.x;
+    if (i < n) v += in[i];
+  }
+  const int r = block_reduce_sum(v, sh);
+  if (threadIdx.x == 0) sums[blockIdx.x] = r;
+}
+
+// one block: in-place exclusive scan of the tile sums (m values)
+__global__ void scan_sums_inplace(int32_t* sums, int64_t m) {
+  __shared__ int sh[32];
+  __shared__ int carry;
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int64_t base = 0; base < m; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    const int v = i < m ? sums[i] : 0;
+    int x = v;  // inclusive scan inside the warp
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, x, o);
+      if ((threadIdx.x & 31) >= o) x += y;
+    }
+    if ((threadIdx.x & 31) == 31) sh[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      int w = threadIdx.x < (blockDim.x >> 5) ? sh[threadIdx.x] : 0;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, w, o);
+        if (threadIdx.x >= o) w += y;
+      }
+      sh[threadIdx.x] = w;  // inclusive over warps
+    }
+    __syncthreads();
+    const int warp_off = (threadIdx.x >> 5) ? sh[(threadIdx.x >> 5) - 1] : 0;
+    const int c = carry;
+    if (i < m) sums[i] = c + warp_off + x - v;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry = c + warp_off + x;
+    __syncthreads();
+  }
+}
+
+__global__ void scan_tiles(const int32_t* __restrict__ in, int64_t n, const int32_t* __restrict__ sums,
+                           int32_t* __restrict__ out) {
+  // thread owns SCAN_ITEMS consecutive elements
+  __shared__ int sh[32];
+  const int64_t base = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
+  int v[SCAN_ITEMS];
+  int t = 0;
+  for (int j = 0; j < SCAN_ITEMS; ++j) {
+    v[j] = (base + j < n) ? in[base + j] : 0;
+    t += v[j];
+  }
+  int x = t;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if ((threadIdx.x & 31) >= o) x += y;
+  }
+  if ((threadIdx.x & 31) == 31) sh[threadIdx.x >> 5] = x;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    int w = threadIdx.x < (SCAN_THREADS >> 5) ? sh[threadIdx.x] : 0;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, w, o);
+      if (threadIdx.x >= o) w += y;
+    }
+    sh[threadIdx.x] = w;
+  }
+  __syncthreads();
+  int run = sums[blockIdx.x] + ((threadIdx.x >> 5) ? sh[(threadIdx.x >> 5) - 1] : 0) + x - t;
+  for (int j = 0; j < SCAN_ITEMS; ++j) {
+    if (base + j < n) out[base + j] = run;
+    run += v[j];
+    if (base + j == n - 1) out[n] = run;
+  }
+}
+
+__global__ void scan_empty(int32_t* out) { out[0] = 0; }
+
+// ---- bit mask construction ---------------------------------------------------------------------
+// one warp per mask word: lane = column inside the word
+__global__ void mask_bytes_to_bits(const uint8_t* __restrict__ mask, int O, int I, int wpr, uint32_t* __restrict__ bits) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= (int64_t)O * wpr) return;
+  const int o = (int)(w / wpr), c = (int)(w % wpr) * 32 + lane;
+  const bool on = c < I && mask[(int64_t)o * I + c] != 0;
+  const unsigned b = __ballot_sync(0xffffffffu, on);
+  if (lane == 0) bits[w] = b;
+}
+
+__global__ void popc_words(const uint32_t* __restrict__ bits, int64_t n, int32_t* __restrict__ cnt) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) cnt[i] = __popc(bits[i]);
+}
+
+// new = (old & ~pruned) | grad | rand
+__global__ void combine_bits(const uint32_t* __restrict__ oldb, const uint32_t* __restrict__ pruned,
+                             const uint32_t* __restrict__ grad, const uint32_t* __restrict__ rnd, int64_t n,
+                             uint32_t* __restrict__ out, int32_t* __restrict__ cnt) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    const uint32_t b = (oldb[i] & ~pruned[i]) | grad[i] | rnd[i];
+    out[i] = b;
+    cnt[i] = __popc(b);
+  }
+}
+
+// ---- CSR fill: one warp per word, lane = bit ---------------------------------------------------
+// Source of a value: dense W (pack) or the previous structure (update: survivors keep their value, others +0).
+template <typename V>
+__global__ void fill_csr(const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan, int O, int I, int wpr,
+                         uint16_t* __restrict__ col_idx, V* __restrict__ vals, int32_t* __restrict__ row_ptr,
+                         const V* __restrict__ dense_W, int64_t ldw, const uint32_t* __restrict__ old_bits,
+                         const int32_t* __restrict__ old_wscan, const V* __restrict__ old_vals) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int64_t nwords = (int64_t)O * wpr;
+  if (w >= nwords) return;
+  const int o = (int)(w / wpr), wc = (int)(w % wpr);
+  const uint32_t b = bits[w];
+  const int32_t base = wscan[w];
+  if (wc == 0 && lane == 0) {
+    row_ptr[o] = base;
+    if (o == O - 1) row_ptr[O] = wscan[nwords];
+  }
+  if ((b >> lane) & 1u) {
+    const int32_t pos = base + __popc(b & lanemask_lt());
+    const int c = wc * 32 + lane;
+    col_idx[pos] = (uint16_t)c;
+    V v;
+    if (dense_W) {
+      v = dense_W[(int64_t)o * ldw + c];
+    } else {
+      const uint32_t ob = old_bits[w];
+      if ((ob >> lane) & 1u) {
+        v = old_vals[old_wscan[w] + __popc(ob & lanemask_lt())];
+      } else {
+        v = V(0);
+      }
+    }
+    vals[pos] = v;
+  }
+}
+
+// ---- bit transpose: one warp per 32x32 bit tile -------------------------------------------------
+__global__ void transpose_bits(const uint32_t* __restrict__ bits, int O, int I, int wpr, int wpc,
+                               uint32_t* __restrict__ bitsT) {
+  const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (tile >= (int64_t)wpc * wpr) return;
+  const int wr = (int)(tile / wpr), wc = (int)(tile % wpr);
+  const int o = wr * 32 + lane;
+  const uint32_t word = o < O ? bits[(int64_t)o * wpr + wc] : 0u;
+  uint32_t mine = 0;
+  for (int c = 0; c < 32; ++c) {
+    const uint32_t t = __ballot_sync(0xffffffffu, (word >> c) & 1u);
+    if (c == lane) mine = t;
+  }
+  const int i = wc * 32 + lane;
+  if (i < I) bitsT[(int64_t)i * wpc + wr] = mine;
+}
+
+__global__ void fill_csc(const uint32_t* __restrict__ bitsT, const int32_t* __restrict__ wscanT, int O, int I, int wpr,
+                         int wpc, const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan,
+                         uint16_t* __restrict__ row_idx, int32_t* __restrict__ perm, int32_t* __restrict__ col_ptr) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int64_t nwordsT = (int64_t)I * wpc;
+  if (w >= nwordsT) return;
+  const int i = (int)(w / wpc), wr = (int)(w % wpc);
+  const uint32_t b = bitsT[w];
+  const int32_t base = wscanT[w];
+  if (wr == 0 && lane == 0) {
+    col_ptr[i] = base;
+    if (i == I - 1) col_ptr[I] = wscanT[nwordsT];
+  }
+  if ((b >> lane) & 1u) {
+    const int o = wr * 32 + lane;
+    const int32_t posT = base + __popc(b & lanemask_lt());
+    const int64_t wf = (int64_t)o * wpr + (i >> 5);
+    const uint32_t fb = bits[wf];
+    row_idx[posT] = (uint16_t)o;
+    perm[posT] = wscan[wf] + __popc(fb & ((1u << (i & 31)) - 1u));
+  }
+}
+
+// ---- export / validate ---------------------------------------------------------------------------
+__global__ void widen_u16(const uint16_t* __restrict__ in, int64_t n, int32_t* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = in[i];
+}
+
+__global__ void validate_rows(const int32_t* __restrict__ row_ptr, const uint16_t* __restrict__ col_idx,
+                              const uint32_t* __restrict__ bits, int O, int I, int wpr, int64_t nnz,
+                              int32_t* __restrict__ flags) {
+  const int o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= O) return;
+  bool bad = false;
+  const int32_t a = row_ptr[o], b = row_ptr[o + 1];
+  if (o == 0 && a != 0) bad = true;
+  if (o == O - 1 && b != nnz) bad = true;
+  if (a > b || a < 0 || b > nnz) {
+    bad = true;
+  } else {
+    int prev = -1, pc = 0;
+    for (int32_t k = a; k < b; ++k) {
+      const int c = col_idx[k];
+      if (c <= prev || c >= I) { bad = true; break; }
+      if (!((bits[(int64_t)o * wpr + (c >> 5)] >> (c & 31)) & 1u)) { bad = true; break; }
+      prev = c;
+    }
+    for (int w = 0; w < wpr; ++w) pc += __popc(bits[(int64_t)o * wpr + w]);
+    if (pc != b - a) bad = true;
+  }
+  if (bad) atomicOr(&flags[0], MST_FLAG_CORRUPT);
+}
+
+__global__ void validate_cols(const int32_t* __restrict__ col_ptr, const uint16_t* __restrict__ row_idx,
+                              const int32_t* __restrict__ perm, const int32_t* __restrict__ row_ptr,
+                              const uint16_t* __restrict__ col_idx, int O, int I, int64_t nnz,
+                              int32_t* __restrict__ flags) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= I) return;
+  bool bad = false;
+  const int32_t a = col_ptr[i], b = col_ptr[i + 1];
+  if (i == 0 && a != 0) bad = true;
+  if (i == I - 1 && b != nnz) bad = true;
+  if (a > b || a < 0 || b > nnz) {
+    bad = true;
+  } else {
+    int prev = -1;
+    for (int32_t k = a; k < b; ++k) {
+      const int o = row_idx[k];
+      const int32_t p = perm[k];
+      if (o <= prev || o >= O || p < 0 || p >= nnz) { bad = true; break; }
+      if (p < row_ptr[o] || p >= row_ptr[o + 1] || col_idx[p] != i) { bad = true; break; }
+      prev = o;
+    }
+  }
+  if (bad) atomicOr(&flags[0], MST_FLAG_CORRUPT);
+}
+
+inline unsigned blocks_for(int64_t n, int per_block) { return (unsigned)((n + per_block - 1) / per_block); }
+
+}  // namespace
+
+int64_t mst_scan_block_sums_len(int64_t n) { return (n + SCAN_TILE - 1) / SCAN_TILE + 1; }
+
+mst_status_t mst_scan_i32(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t s) {
+  if (n <= 0) {
+    scan_empty<<<1, 1, 0, s>>>(out);
+    MST_CUDA_TRY(cudaGetLastError());
+    return MST_OK;
+  }
+  const int64_t tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
+  scan_tile_sums<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums);
+  scan_sums_inplace<<<1, 1024, 0, s>>>(block_sums, tiles);
+  scan_tiles<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, out);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+// bits[set] must be final.  Computes wscan[set], row_ptr[set], col_idx[set], vals[set].
+mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set,
+                                   cudaStream_t s) {
+  popc_words<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[set], L->nwords, L->word_cnt);
+  MST_TRY(mst_scan_i32(L->word_cnt, L->wscan[set], L->nwords, L->block_sums, s));
+  const unsigned grid = blocks_for(L->nwords * 32, 256);
+  if (L->dtype == MST_F32) {
+    fill_csr<float><<<grid, 256, 0, s>>>(L->bits[set], L->wscan[set], L->O, L->I, L->wpr, L->col_idx[set],
+                                         (float*)L->vals[set], L->row_ptr[set], (const float*)dense_W, ldw,
+                                         L->bits[old_set], L->wscan[old_set], (const float*)L->vals[old_set]);
+  } else {
+    fill_csr<uint16_t><<<grid, 256, 0, s>>>(L->bits[set], L->wscan[set], L->O, L->I, L->wpr, L->col_idx[set],
+                                            (uint16_t*)L->vals[set], L->row_ptr[set], (const uint16_t*)dense_W, ldw,
+                                            L->bits[old_set], L->wscan[old_set], (const uint16_t*)L->vals[old_set]);
+  }
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+// CSC view of the live set.
+mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s) {
+  const int c = L->cur;
+  transpose_bits<<<blocks_for((int64_t)L->wpc * L->wpr * 32, 256), 256, 0, s>>>(L->bits[c], L->O, L->I, L->wpr, L->wpc,
+                                                                                L->bitsT);
+  popc_words<<<blocks_for(L->nwordsT, 256), 256, 0, s>>>(L->bitsT, L->nwordsT, L->word_cnt);
+  MST_TRY(mst_scan_i32(L->word_cnt, L->wscanT, L->nwordsT, L->block_sums, s));
+  fill_csc<<<blocks_for(L->nwordsT * 32, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->O, L->I, L->wpr, L->wpc, L->bits[c],
+                                                            L->wscan[c], L->row_idx, L->perm, L->col_ptr);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+// new mask of an update from the three selection results; leaves popcounts in word_cnt
+mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s) {
+  combine_bits<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[L->cur], L->pruned_bits, L->grad_bits, L->rand_bits,
+                                                          L->nwords, L->bits[new_set], L->word_cnt);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_pack(mst_layer_t* L, const void* W_dense, int64_t ldw, const uint8_t* mask,
+                                 mst_stream_t stream) {
+  if (!L || !W_dense || !mask) return MST_ERR_INVALID_ARG;
+  if (ldw < L->I) return MST_ERR_SHAPE;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int set = L->cur;
+  L->nnz = -1;
+  mask_bytes_to_bits<<<blocks_for(L->nwords * 32, 256), 256, 0, s>>>(mask, L->O, L->I, L->wpr, L->bits[set]);
+  popc_words<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[set], L->nwords, L->word_cnt);
+  MST_TRY(mst_scan_i32(L->word_cnt, L->wscan[set], L->nwords, L->block_sums, s));
+  int32_t total = 0;
+  MST_CUDA_TRY(cudaMemcpyAsync(&total, L->wscan[set] + L->nwords, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  MST_CUDA_TRY(cudaStreamSynchronize(s));
+  if (total > L->cap) return MST_ERR_CAPACITY;
+  MST_TRY(mst_rebuild_from_bits(L, set, W_dense, ldw, set, s));
+  L->nnz = total;
+  MST_TRY(mst_build_csc(L, s));
+  MST_CUDA_TRY(cudaStreamSynchronize(s));
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_export_csr(const mst_layer_t* L, int32_t* row_ptr, int32_t* col_idx, void* vals,
+                                       mst_stream_t stream) {
+  if (!L) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int c = L->cur;
+  if (row_ptr)
+    MST_CUDA_TRY(cudaMemcpyAsync(row_ptr, L->row_ptr[c], sizeof(int32_t) * (L->O + 1), cudaMemcpyDeviceToDevice, s));
+  if (col_idx && L->nnz > 0) widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->col_idx[c], L->nnz, col_idx);
+  if (vals && L->nnz > 0)
+    MST_CUDA_TRY(cudaMemcpyAsync(vals, L->vals[c], mst_elem_size(L->dtype) * L->nnz, cudaMemcpyDeviceToDevice, s));
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_export_csc(const mst_layer_t* L, int32_t* col_ptr, int32_t* row_idx, int32_t* perm,
+                                       mst_stream_t stream) {
+  if (!L) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (col_ptr)
+    MST_CUDA_TRY(cudaMemcpyAsync(col_ptr, L->col_ptr, sizeof(int32_t) * (L->I + 1), cudaMemcpyDeviceToDevice, s));
+  if (row_idx && L->nnz > 0) widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->row_idx, L->nnz, row_idx);
+  if (perm && L->nnz > 0)
+    MST_CUDA_TRY(cudaMemcpyAsync(perm, L->perm, sizeof(int32_t) * L->nnz, cudaMemcpyDeviceToDevice, s));
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_validate(const mst_layer_t* L, mst_stream_t stream) {
+  if (!L) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int c = L->cur;
+  validate_rows<<<blocks_for(L->O, 128), 128, 0, s>>>(L->row_ptr[c], L->col_idx[c], L->bits[c], L->O, L->I, L->wpr,
+                                                     L->nnz, L->flags);
+  validate_cols<<<blocks_for(L->I, 128), 128, 0, s>>>(L->col_ptr, L->row_idx, L->perm, L->row_ptr[c], L->col_idx[c],
+                                                     L->O, L->I, L->nnz, L->flags);
+  MST_CUDA_TRY(cudaGetLastError());
+  int32_t f = 0;
+  MST_CUDA_TRY(cudaMemcpyAsync(&f, L->flags, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  MST_CUDA_TRY(cudaStreamSynchronize(s));
+  if (f & MST_FLAG_CORRUPT) return MST_ERR_CORRUPT;
+  if (f & MST_FLAG_NONFINITE) return MST_ERR_NONFINITE;
+  return MST_OK;
+}
