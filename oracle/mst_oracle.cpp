@@ -182,7 +182,7 @@ int mst_oracle_mg_update(int64_t O, int64_t I, float* W, uint8_t* M, const float
   for (int64_t f = 0; f < N; ++f)
     if (old_mask[f]) {
       const uint32_t k = abs_bits(W[f]);
-      if (k >= 0x7F800000u) return 1;
+      if (n_prune > 0 && k >= 0x7F800000u) return 1;   // keys are only examined when something is selected
       act.push_back(KI(k, f));
     }
   if (n_prune < 0 || n_prune > (int64_t)act.size() || n_grad < 0 || n_rand < 0) return 2;

@@ -1,0 +1,232 @@
+"""Python binding of libmst (argument marshalling only; every step runs in the CUDA library).
+
+The functions carry the names of the C entry points declared in ``include/mst.h``
+and take device pointers as ``torch.Tensor`` (``data_ptr()`` is used) or plain
+integers.  PyTorch appears only as the owner of device buffers and streams.
+
+Importing the package needs ``libmst.so`` (built in-tree by
+``python paper_2408_11746_b200/csrc/build.py``); there is no fallback path:
+a missing library is an ImportError.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmst.so")
+
+MST_F32, MST_BF16 = 0, 1
+MST_OK = 0
+STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "MST_ERR_DTYPE", 4: "MST_ERR_CAPACITY",
+                5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
+                9: "MST_ERR_NOT_PACKED"}
+EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
+           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad",
+           "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_status_string"]
+
+
+class MstError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (%s)" % (where, STATUS_NAMES.get(status, status), status_string(status)))
+
+
+class RegrowRule(ctypes.Structure):
+    _fields_ = [("target_nnz", ctypes.c_int64), ("random_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
+                ("step", ctypes.c_uint64), ("allow_regrow_pruned", ctypes.c_int32)]
+
+
+class UpdateStats(ctypes.Structure):
+    _fields_ = [("nnz_before", ctypes.c_int64), ("nnz_after", ctypes.c_int64), ("n_prune", ctypes.c_int64),
+                ("n_grad", ctypes.c_int64), ("n_rand", ctypes.c_int64), ("max_row_nnz", ctypes.c_int64)]
+
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError("libmst.so is not built: run `python paper_2408_11746_b200/csrc/build.py` (needs nvcc); "
+                      "there is no CPU fallback")
+_lib = ctypes.CDLL(LIB_PATH)
+
+_vp, _i32, _i64, _f64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_double
+_sig = {
+    "mst_layer_create": [ctypes.POINTER(_vp), _i32, _i32, _i32, ctypes.c_int, _i64],
+    "mst_layer_destroy": [_vp],
+    "mst_layer_nnz": [_vp, ctypes.POINTER(_i64)],
+    "mst_pack": [_vp, _vp, _i64, _vp, _vp],
+    "mst_export_csr": [_vp, _vp, _vp, _vp, _vp],
+    "mst_export_csc": [_vp, _vp, _vp, _vp, _vp],
+    "mst_values": [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_i64)],
+    "mst_validate": [_vp, _vp],
+    "mst_spmm_fwd": [_vp, _vp, _i64, _i64, _vp, _i64, _vp],
+    "mst_spmm_bwd_x": [_vp, _vp, _i64, _i64, _vp, _i64, _vp],
+    "mst_sddmm_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp],
+    "mst_dense_grad": [_vp, _i64, _vp, _i64, _i64, _i32, _i32, ctypes.c_int, _vp, _vp],
+    "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
+    "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
+    "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
+}
+for _n, _a in _sig.items():
+    getattr(_lib, _n).argtypes = _a
+    getattr(_lib, _n).restype = ctypes.c_int
+_lib.mst_status_string.argtypes = [ctypes.c_int]
+_lib.mst_status_string.restype = ctypes.c_char_p
+
+
+def status_string(status: int) -> str:
+    return _lib.mst_status_string(int(status)).decode()
+
+
+def _ptr(x) -> Optional[int]:
+    """Device (or host) address of a tensor / ndarray / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError("expected a tensor, an ndarray, an int address or None")
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _check(status: int, where: str) -> None:
+    if status != MST_OK:
+        raise MstError(status, where)
+
+
+# ---------------------------------------------------------------- C entry points, same names
+def mst_layer_create(layer_id: int, out_features: int, in_features: int, dtype: int, nnz_capacity: int) -> int:
+    h = _vp()
+    _check(_lib.mst_layer_create(ctypes.byref(h), layer_id, out_features, in_features, dtype, nnz_capacity),
+           "mst_layer_create")
+    return h.value
+
+
+def mst_layer_destroy(layer: int) -> None:
+    _check(_lib.mst_layer_destroy(layer), "mst_layer_destroy")
+
+
+def mst_layer_nnz(layer: int) -> int:
+    n = _i64()
+    _check(_lib.mst_layer_nnz(layer, ctypes.byref(n)), "mst_layer_nnz")
+    return n.value
+
+
+def mst_pack(layer: int, W_dense, ldw: int, mask, stream=None) -> None:
+    _check(_lib.mst_pack(layer, _ptr(W_dense), ldw, _ptr(mask), _stream(stream)), "mst_pack")
+
+
+def mst_export_csr(layer: int, row_ptr, col_idx, vals, stream=None) -> None:
+    _check(_lib.mst_export_csr(layer, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _stream(stream)), "mst_export_csr")
+
+
+def mst_export_csc(layer: int, col_ptr, row_idx, perm, stream=None) -> None:
+    _check(_lib.mst_export_csc(layer, _ptr(col_ptr), _ptr(row_idx), _ptr(perm), _stream(stream)), "mst_export_csc")
+
+
+def mst_values(layer: int) -> Tuple[int, int]:
+    p, n = _vp(), _i64()
+    _check(_lib.mst_values(layer, ctypes.byref(p), ctypes.byref(n)), "mst_values")
+    return p.value, n.value
+
+
+def mst_validate(layer: int, stream=None) -> None:
+    _check(_lib.mst_validate(layer, _stream(stream)), "mst_validate")
+
+
+def mst_spmm_fwd(layer: int, X, ldx: int, T: int, Y, ldy: int, stream=None) -> None:
+    _check(_lib.mst_spmm_fwd(layer, _ptr(X), ldx, T, _ptr(Y), ldy, _stream(stream)), "mst_spmm_fwd")
+
+
+def mst_spmm_bwd_x(layer: int, dY, lddy: int, T: int, dX, lddx: int, stream=None) -> None:
+    _check(_lib.mst_spmm_bwd_x(layer, _ptr(dY), lddy, T, _ptr(dX), lddx, _stream(stream)), "mst_spmm_bwd_x")
+
+
+def mst_sddmm_dw(layer: int, dY, lddy: int, X, ldx: int, T: int, dW_vals, stream=None) -> None:
+    _check(_lib.mst_sddmm_dw(layer, _ptr(dY), lddy, _ptr(X), ldx, T, _ptr(dW_vals), _stream(stream)), "mst_sddmm_dw")
+
+
+def mst_dense_grad(dY, lddy: int, X, ldx: int, T: int, out_features: int, in_features: int, dtype: int, G,
+                   stream=None) -> None:
+    _check(_lib.mst_dense_grad(_ptr(dY), lddy, _ptr(X), ldx, T, out_features, in_features, dtype, _ptr(G),
+                               _stream(stream)), "mst_dense_grad")
+
+
+def mst_update_counts(prune_frac: float, nnz: int, target_nnz: int, numel: int, random_ratio: float):
+    """(n_prune, n_grow, n_rand, n_grad)."""
+    out = (_i64 * 4)()
+    _check(_lib.mst_update_counts(prune_frac, nnz, target_nnz, numel, random_ratio, out), "mst_update_counts")
+    return tuple(int(v) for v in out)
+
+
+def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, random_ratio: float = 0.25,
+                        seed: int = 0, step: int = 0, allow_regrow_pruned: bool = False, G_dense=None,
+                        want_stats: bool = True, stream=None) -> Optional[UpdateStats]:
+    rule = RegrowRule(int(target_nnz), float(random_ratio), int(seed), int(step), int(bool(allow_regrow_pruned)))
+    stats = UpdateStats() if want_stats else None
+    _check(_lib.mst_topology_update(layer, float(prune_frac), ctypes.byref(rule), _ptr(G_dense),
+                                    ctypes.byref(stats) if want_stats else None, _stream(stream)),
+           "mst_topology_update")
+    return stats
+
+
+def mst_layer_step_host(layer: int, X_host, dY_host, T: int, Y_host, dX_host, dW_vals_host, stream=None) -> None:
+    _check(_lib.mst_layer_step_host(layer, _ptr(X_host), _ptr(dY_host), T, _ptr(Y_host), _ptr(dX_host),
+                                    _ptr(dW_vals_host), _stream(stream)), "mst_layer_step_host")
+
+
+# ---------------------------------------------------------------- small RAII convenience
+class Layer:
+    """Owns one ``mst_layer_t`` handle; methods forward to the entry points above."""
+
+    def __init__(self, layer_id: int, out_features: int, in_features: int, dtype: int, nnz_capacity: Optional[int] = None):
+        self.out_features, self.in_features, self.dtype = out_features, in_features, dtype
+        cap = out_features * in_features if nnz_capacity is None else nnz_capacity
+        self.handle = mst_layer_create(layer_id, out_features, in_features, dtype, cap)
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            mst_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def nnz(self) -> int:
+        return mst_layer_nnz(self.handle)
+
+    def pack(self, W_dense, mask, ldw: Optional[int] = None, stream=None) -> None:
+        mst_pack(self.handle, W_dense, self.in_features if ldw is None else ldw, mask, stream)
+
+    def fwd(self, X, Y, T: int, stream=None) -> None:
+        mst_spmm_fwd(self.handle, X, self.in_features, T, Y, self.out_features, stream)
+
+    def bwd_x(self, dY, dX, T: int, stream=None) -> None:
+        mst_spmm_bwd_x(self.handle, dY, self.out_features, T, dX, self.in_features, stream)
+
+    def sddmm(self, dY, X, T: int, dW_vals, stream=None) -> None:
+        mst_sddmm_dw(self.handle, dY, self.out_features, X, self.in_features, T, dW_vals, stream)
+
+    def dense_grad(self, dY, X, T: int, G, stream=None) -> None:
+        mst_dense_grad(dY, self.out_features, X, self.in_features, T, self.out_features, self.in_features, self.dtype,
+                       G, stream)
+
+    def update(self, prune_frac: float, **kw):
+        return mst_topology_update(self.handle, prune_frac, **kw)
+
+    def validate(self, stream=None) -> None:
+        mst_validate(self.handle, stream)

@@ -1,0 +1,188 @@
+// Handle management and the host-buffer convenience entry point of libmst.
+#include "mst_internal.cuh"
+
+#include <new>
+
+namespace {
+
+struct Carver {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    const size_t at = off;
+    off += (bytes + 255) & ~(size_t)255;
+    return at;
+  }
+};
+
+void free_staging(mst_layer* L) {
+  cudaFree(L->stg_x);
+  cudaFree(L->stg_dy);
+  cudaFree(L->stg_y);
+  cudaFree(L->stg_dx);
+  cudaFree(L->stg_dw);
+  L->stg_x = L->stg_dy = L->stg_y = L->stg_dx = nullptr;
+  L->stg_dw = nullptr;
+  L->stg_tokens = 0;
+}
+
+}  // namespace
+
+extern "C" const char* mst_status_string(mst_status_t st) {
+  switch (st) {
+    case MST_OK: return "ok";
+    case MST_ERR_INVALID_ARG: return "invalid argument";
+    case MST_ERR_SHAPE: return "shape or leading dimension out of range";
+    case MST_ERR_DTYPE: return "unsupported dtype";
+    case MST_ERR_CAPACITY: return "nnz exceeds the layer's capacity";
+    case MST_ERR_INFEASIBLE: return "no feasible prune/grow counts";
+    case MST_ERR_NONFINITE: return "non-finite selection key";
+    case MST_ERR_CORRUPT: return "sparse structure is corrupt";
+    case MST_ERR_CUDA: return "CUDA runtime error";
+    case MST_ERR_NOT_PACKED: return "layer has no structure yet";
+  }
+  return "unknown status";
+}
+
+extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, int32_t O, int32_t I, mst_dtype_t dtype,
+                                         int64_t cap) {
+  if (!out) return MST_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (dtype != MST_F32 && dtype != MST_BF16) return MST_ERR_DTYPE;
+  if (O < 1 || I < 1 || O > 65535 || I > 65535) return MST_ERR_SHAPE;
+  const int64_t N = (int64_t)O * I;
+  if (cap < 1 || cap > N) return MST_ERR_CAPACITY;
+  mst_layer* L = new (std::nothrow) mst_layer();
+  if (!L) return MST_ERR_INVALID_ARG;
+  L->layer_id = layer_id;
+  L->O = O;
+  L->I = I;
+  L->dtype = dtype;
+  L->cap = cap;
+  L->N = N;
+  L->wpr = (I + 31) / 32;
+  L->wpc = (O + 31) / 32;
+  L->nwords = (int64_t)O * L->wpr;
+  L->nwordsT = (int64_t)I * L->wpc;
+  L->nnz = -1;
+  L->cur = 0;
+  const int64_t wmax = L->nwords > L->nwordsT ? L->nwords : L->nwordsT;
+  const size_t es = mst_elem_size(dtype);
+
+  Carver cv;
+  size_t o_bits[2], o_wscan[2], o_rowptr[2], o_col[2], o_vals[2];
+  for (int s = 0; s < 2; ++s) {
+    o_bits[s] = cv.take(4 * (size_t)L->nwords);
+    o_wscan[s] = cv.take(4 * (size_t)(L->nwords + 1));
+    o_rowptr[s] = cv.take(4 * (size_t)(O + 1));
+    o_col[s] = cv.take(2 * (size_t)cap);
+    o_vals[s] = cv.take(es * (size_t)cap);
+  }
+  const size_t o_bitsT = cv.take(4 * (size_t)L->nwordsT);
+  const size_t o_wscanT = cv.take(4 * (size_t)(L->nwordsT + 1));
+  const size_t o_colptr = cv.take(4 * (size_t)(I + 1));
+  const size_t o_rowidx = cv.take(2 * (size_t)cap);
+  const size_t o_perm = cv.take(4 * (size_t)cap);
+  const size_t o_pruned = cv.take(4 * (size_t)L->nwords);
+  const size_t o_grad = cv.take(4 * (size_t)L->nwords);
+  const size_t o_rand = cv.take(4 * (size_t)L->nwords);
+  const size_t o_cnt = cv.take(4 * (size_t)(wmax + 1));
+  const size_t o_scan = cv.take(4 * (size_t)(wmax + 1));
+  const size_t o_bsum = cv.take(4 * (size_t)mst_scan_block_sums_len(wmax));
+  const size_t o_hist = cv.take(4 * 256);
+  const size_t o_sel = cv.take(sizeof(mst_select_state));
+  const size_t o_flags = cv.take(4 * 4);
+  const size_t o_counter = cv.take(4);
+
+  unsigned char* base = nullptr;
+  if (cudaMalloc((void**)&base, cv.off) != cudaSuccess) {
+    delete L;
+    return MST_ERR_CUDA;
+  }
+  if (cudaMemset(base, 0, cv.off) != cudaSuccess) {
+    cudaFree(base);
+    delete L;
+    return MST_ERR_CUDA;
+  }
+  for (int s = 0; s < 2; ++s) {
+    L->bits[s] = (uint32_t*)(base + o_bits[s]);
+    L->wscan[s] = (int32_t*)(base + o_wscan[s]);
+    L->row_ptr[s] = (int32_t*)(base + o_rowptr[s]);
+    L->col_idx[s] = (uint16_t*)(base + o_col[s]);
+    L->vals[s] = (void*)(base + o_vals[s]);
+  }
+  L->bitsT = (uint32_t*)(base + o_bitsT);
+  L->wscanT = (int32_t*)(base + o_wscanT);
+  L->col_ptr = (int32_t*)(base + o_colptr);
+  L->row_idx = (uint16_t*)(base + o_rowidx);
+  L->perm = (int32_t*)(base + o_perm);
+  L->pruned_bits = (uint32_t*)(base + o_pruned);
+  L->grad_bits = (uint32_t*)(base + o_grad);
+  L->rand_bits = (uint32_t*)(base + o_rand);
+  L->word_cnt = (int32_t*)(base + o_cnt);
+  L->word_scan = (int32_t*)(base + o_scan);
+  L->block_sums = (int32_t*)(base + o_bsum);
+  L->hist = (unsigned int*)(base + o_hist);
+  L->sel = (mst_select_state*)(base + o_sel);
+  L->flags = (int32_t*)(base + o_flags);
+  L->counter = (unsigned int*)(base + o_counter);
+  L->stg_x = L->stg_dy = L->stg_y = L->stg_dx = nullptr;
+  L->stg_dw = nullptr;
+  L->stg_tokens = 0;
+  *out = L;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_layer_destroy(mst_layer_t* L) {
+  if (!L) return MST_OK;
+  free_staging(L);
+  cudaFree(L->bits[0]);  // base of the single allocation
+  delete L;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_layer_nnz(const mst_layer_t* L, int64_t* nnz) {
+  if (!L || !nnz) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  *nnz = L->nnz;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_values(mst_layer_t* L, void** vals, int64_t* nnz) {
+  if (!L || !vals) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  *vals = L->vals[L->cur];
+  if (nnz) *nnz = L->nnz;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_layer_step_host(mst_layer_t* L, const void* X_host, const void* dY_host, int64_t T,
+                                            void* Y_host, void* dX_host, float* dW_host, mst_stream_t stream) {
+  if (!L || T < 0 || (T > 0 && (!X_host || !dY_host))) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t es = mst_elem_size(L->dtype);
+  if (T > L->stg_tokens || !L->stg_dw) {
+    MST_CUDA_TRY(cudaStreamSynchronize(s));
+    free_staging(L);
+    const int64_t Ta = T > 0 ? T : 1;
+    MST_CUDA_TRY(cudaMalloc(&L->stg_x, es * Ta * L->I));
+    MST_CUDA_TRY(cudaMalloc(&L->stg_dy, es * Ta * L->O));
+    MST_CUDA_TRY(cudaMalloc(&L->stg_y, es * Ta * L->O));
+    MST_CUDA_TRY(cudaMalloc(&L->stg_dx, es * Ta * L->I));
+    MST_CUDA_TRY(cudaMalloc((void**)&L->stg_dw, sizeof(float) * L->cap));
+    L->stg_tokens = Ta;
+  }
+  if (T > 0) {
+    MST_CUDA_TRY(cudaMemcpyAsync(L->stg_x, X_host, es * T * L->I, cudaMemcpyHostToDevice, s));
+    MST_CUDA_TRY(cudaMemcpyAsync(L->stg_dy, dY_host, es * T * L->O, cudaMemcpyHostToDevice, s));
+  }
+  MST_TRY(mst_launch_spmm(L, false, L->stg_x, L->I, T, L->stg_y, L->O, s));
+  MST_TRY(mst_launch_spmm(L, true, L->stg_dy, L->O, T, L->stg_dx, L->I, s));
+  MST_TRY(mst_launch_sddmm(L, L->stg_dy, L->O, L->stg_x, L->I, T, L->stg_dw, s));
+  if (T > 0 && Y_host) MST_CUDA_TRY(cudaMemcpyAsync(Y_host, L->stg_y, es * T * L->O, cudaMemcpyDeviceToHost, s));
+  if (T > 0 && dX_host) MST_CUDA_TRY(cudaMemcpyAsync(dX_host, L->stg_dx, es * T * L->I, cudaMemcpyDeviceToHost, s));
+  if (dW_host && L->nnz > 0)
+    MST_CUDA_TRY(cudaMemcpyAsync(dW_host, L->stg_dw, sizeof(float) * L->nnz, cudaMemcpyDeviceToHost, s));
+  MST_CUDA_TRY(cudaStreamSynchronize(s));
+  return MST_OK;
+}

@@ -1,0 +1,312 @@
+// Mixed-Growing topology update (Algorithm 1) on the device.
+//
+// The three selections of the algorithm (prune by smallest |w|, grow by largest |g|, grow at random) are the same
+// primitive: take the k smallest keys of a candidate set, ties broken by the smaller flat index.  Each is done by a
+// most-significant-digit radix select (8 bits per pass) that leaves a threshold key tau and the number `rem` of
+// entries equal to tau still to take; a popcount + exclusive scan over the mask words then ranks the entries equal to
+// tau in flat-index order and the first `rem` of them are taken.  Results are bit masks over the flat index space, so
+// the mask rewrite is three bitwise operations per word and the CSR rebuild is the popcount/scan/fill of
+// mst_structure.cu.  Integer keys, integer atomics only: the outcome is deterministic and bit-exact.
+//
+// Work layout: one warp per 32-bit mask word, lane = column inside the word, so reads of G and of the value array are
+// coalesced.  The last block to finish a histogram pass picks the digit (completion counter, no waiting).
+#include "mst_internal.cuh"
+
+namespace {
+
+enum { MODE_PRUNE = 0, MODE_GRAD = 1, MODE_RAND = 2 };
+
+struct SelParams {
+  const uint32_t* old_bits;
+  const int32_t* old_wscan;
+  const void* vals;
+  int bf16;
+  const float* G;
+  const uint32_t* pruned_bits;
+  const uint32_t* grad_bits;
+  int O, I, wpr, allow;
+  int64_t nwords;
+  unsigned long long stream;
+};
+
+__device__ __forceinline__ unsigned lanemask_lt() {
+  unsigned m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// SplitMix64 output function (Steele, Lea, Flood 2014)
+__device__ __forceinline__ unsigned long long sm64_mix(unsigned long long z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+constexpr unsigned long long SM64_GAMMA = 0x9E3779B97F4A7C15ULL;
+
+template <int MODE>
+struct KeyBits {
+  static constexpr int value = MODE == MODE_RAND ? 64 : 32;
+};
+
+// candidate test and key of bit `lane` of word w.  nonfinite is set when a magnitude key is Inf/NaN.
+template <int MODE>
+__device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane, unsigned long long& key,
+                                         bool& nonfinite) {
+  const int o = (int)(w / P.wpr), c = (int)(w % P.wpr) * 32 + lane;
+  nonfinite = false;
+  key = 0;
+  if (MODE == MODE_PRUNE) {
+    const uint32_t word = P.old_bits[w];
+    if (!((word >> lane) & 1u)) return false;
+    const int32_t pos = P.old_wscan[w] + __popc(word & lanemask_lt());
+    uint32_t k;
+    if (P.bf16)
+      k = ((uint32_t)(((const uint16_t*)P.vals)[pos] & 0x7FFFu)) << 16;
+    else
+      k = ((const uint32_t*)P.vals)[pos] & 0x7FFFFFFFu;
+    nonfinite = k >= 0x7F800000u;
+    key = k;
+    return true;
+  } else if (MODE == MODE_GRAD) {
+    uint32_t word = ~P.old_bits[w];
+    if (P.allow) word |= P.pruned_bits[w];
+    if (c >= P.I || !((word >> lane) & 1u)) return false;
+    const uint32_t k = __float_as_uint(P.G[(int64_t)o * P.I + c]) & 0x7FFFFFFFu;
+    nonfinite = k >= 0x7F800000u;
+    key = 0xFFFFFFFFu - k;  // largest magnitude first
+    return true;
+  } else {
+    const uint32_t word = ~P.old_bits[w] & ~P.grad_bits[w];
+    if (c >= P.I || !((word >> lane) & 1u)) return false;
+    const unsigned long long f = (unsigned long long)o * (unsigned long long)P.I + (unsigned long long)c;
+    key = sm64_mix(P.stream + SM64_GAMMA * (f + 1ULL));
+    return true;
+  }
+}
+
+__global__ void select_init(mst_select_state* st, long long k, unsigned int* hist, unsigned int* counter) {
+  if (threadIdx.x == 0) {
+    st->prefix = 0;
+    st->k = k;
+    st->tau = 0;
+    st->rem = 0;
+    *counter = 0;
+  }
+  if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(256) select_hist(SelParams P, int pass, mst_select_state* st, unsigned int* hist,
+                                                   unsigned int* counter, int32_t* flags) {
+  constexpr int KB = KeyBits<MODE>::value;
+  __shared__ unsigned int sh[256];
+  __shared__ bool is_last;
+  sh[threadIdx.x] = 0;
+  __syncthreads();
+  const unsigned long long prefix = st->prefix;
+  const int shift = KB - 8 * (pass + 1);
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  bool saw_nonfinite = false;
+  for (int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < P.nwords; w += warps) {
+    unsigned long long key;
+    bool nf;
+    const bool c = cand_key<MODE>(P, w, lane, key, nf);
+    saw_nonfinite |= (c && nf);
+    // entries whose higher digits differ from the prefix are out of the race
+    const bool live = c && (pass == 0 || (key >> (shift + 8)) == prefix);
+    const unsigned digit = live ? (unsigned)((key >> shift) & 0xFFu) : 256u;
+    const unsigned peers = __match_any_sync(0xffffffffu, digit);
+    if (live && lane == (__ffs(peers) - 1)) atomicAdd(&sh[digit], (unsigned)__popc(peers));
+  }
+  if (pass == 0 && saw_nonfinite) atomicOr(&flags[0], MST_FLAG_NONFINITE);
+  __syncthreads();
+  if (sh[threadIdx.x]) atomicAdd(&hist[threadIdx.x], sh[threadIdx.x]);
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!is_last) return;
+  // last block: every other block's histogram contribution is visible
+  __threadfence();
+  sh[threadIdx.x] = atomicAdd(&hist[threadIdx.x], 0u);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    long long k = st->k, cum = 0;
+    int bin = -1;
+    for (int b = 0; b < 256; ++b) {
+      if (cum + (long long)sh[b] >= k) { bin = b; break; }
+      cum += sh[b];
+    }
+    if (bin < 0) {  // fewer candidates than requested: the host-side counts rule this out
+      atomicOr(&flags[0], MST_FLAG_CORRUPT);
+      bin = 255;
+      cum = 0;
+      k = 0;
+    }
+    const unsigned long long np = (prefix << 8) | (unsigned long long)bin;
+    st->prefix = np;
+    st->k = k - cum;
+    if (shift == 0) {
+      st->tau = np;
+      st->rem = k - cum;
+    }
+    *counter = 0;
+  }
+  hist[threadIdx.x] = 0;
+}
+
+// cnt[w] = number of candidates in word w whose key equals tau
+template <int MODE>
+__global__ void __launch_bounds__(256) select_count_equal(SelParams P, const mst_select_state* st,
+                                                          int32_t* __restrict__ cnt) {
+  const unsigned long long tau = st->tau;
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= P.nwords) return;
+  unsigned long long key;
+  bool nf;
+  const bool c = cand_key<MODE>(P, w, lane, key, nf);
+  const unsigned eq = __ballot_sync(0xffffffffu, c && key == tau);
+  if (lane == 0) cnt[w] = __popc(eq);
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(256) select_mark(SelParams P, const mst_select_state* st,
+                                                   const int32_t* __restrict__ eq_scan, uint32_t* __restrict__ out) {
+  const unsigned long long tau = st->tau;
+  const long long rem = st->rem;
+  const int lane = threadIdx.x & 31;
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (w >= P.nwords) return;
+  unsigned long long key;
+  bool nf;
+  const bool c = cand_key<MODE>(P, w, lane, key, nf);
+  const bool iseq = c && key == tau;
+  const unsigned eq = __ballot_sync(0xffffffffu, iseq);
+  const long long rank = (long long)eq_scan[w] + __popc(eq & lanemask_lt());
+  const bool take = c && (key < tau || (iseq && rank < rem));
+  const unsigned bits = __ballot_sync(0xffffffffu, take);
+  if (lane == 0) out[w] = bits;
+}
+
+__global__ void max_row_nnz(const int32_t* __restrict__ row_ptr, int O, int32_t* flags) {
+  const int o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o < O) atomicMax(&flags[1], row_ptr[o + 1] - row_ptr[o]);
+}
+
+template <int MODE>
+mst_status_t run_select(mst_layer* L, const SelParams& P, int64_t k, uint32_t* out_bits, cudaStream_t s) {
+  if (k <= 0) {
+    MST_CUDA_TRY(cudaMemsetAsync(out_bits, 0, sizeof(uint32_t) * L->nwords, s));
+    return MST_OK;
+  }
+  constexpr int passes = KeyBits<MODE>::value / 8;
+  select_init<<<1, 256, 0, s>>>(L->sel, (long long)k, L->hist, L->counter);
+  const int64_t warps_needed = L->nwords;
+  int64_t blocks = (warps_needed * 32 + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  for (int p = 0; p < passes; ++p)
+    select_hist<MODE><<<(unsigned)blocks, 256, 0, s>>>(P, p, L->sel, L->hist, L->counter, L->flags);
+  const unsigned wgrid = (unsigned)((L->nwords * 32 + 255) / 256);
+  select_count_equal<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_cnt);
+  MST_TRY(mst_scan_i32(L->word_cnt, L->word_scan, L->nwords, L->block_sums, s));
+  select_mark<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_scan, out_bits);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+inline unsigned long long host_mix(unsigned long long z) {
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+  return z ^ (z >> 31);
+}
+
+}  // namespace
+
+extern "C" mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_t target_nnz, int64_t numel,
+                                          double random_ratio, int64_t counts[4]) {
+  if (!counts) return MST_ERR_INVALID_ARG;
+  if (!(prune_frac >= 0.0 && prune_frac <= 1.0) || !(random_ratio >= 0.0 && random_ratio <= 1.0))
+    return MST_ERR_INVALID_ARG;
+  if (nnz < 0 || nnz > numel) return MST_ERR_INVALID_ARG;
+  if (target_nnz < 0) target_nnz = nnz;
+  if (target_nnz > numel) return MST_ERR_INFEASIBLE;
+  // floor(zeta * nnz) in double; then the smallest adjustment that lets the layer reach its target count
+  int64_t n_prune = (int64_t)(prune_frac * (double)nnz);
+  const int64_t lo = nnz - target_nnz > 0 ? nnz - target_nnz : 0;
+  const int64_t hi = nnz < numel - target_nnz ? nnz : numel - target_nnz;
+  if (n_prune < lo) n_prune = lo;
+  if (n_prune > hi) n_prune = hi;
+  const int64_t n_grow = n_prune + target_nnz - nnz;
+  const int64_t n_rand = (int64_t)((double)n_grow * random_ratio);
+  counts[0] = n_prune;
+  counts[1] = n_grow;
+  counts[2] = n_rand;
+  counts[3] = n_grow - n_rand;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, const mst_regrow_rule_t* rule,
+                                            const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream) {
+  if (!L || !rule) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  cudaStream_t s = (cudaStream_t)stream;
+  int64_t cnt[4];
+  MST_TRY(mst_update_counts(prune_frac, L->nnz, rule->target_nnz, L->N, rule->random_ratio, cnt));
+  const int64_t n_prune = cnt[0], n_rand = cnt[2], n_grad = cnt[3];
+  const int64_t target = rule->target_nnz < 0 ? L->nnz : rule->target_nnz;
+  if (target > L->cap) return MST_ERR_CAPACITY;
+  if (n_grad > 0 && !G_dense) return MST_ERR_INVALID_ARG;
+
+  const int c = L->cur, n = c ^ 1;
+  MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t) * 4, s));
+
+  SelParams P;
+  P.old_bits = L->bits[c];
+  P.old_wscan = L->wscan[c];
+  P.vals = L->vals[c];
+  P.bf16 = L->dtype == MST_BF16;
+  P.G = G_dense;
+  P.pruned_bits = L->pruned_bits;
+  P.grad_bits = L->grad_bits;
+  P.O = L->O;
+  P.I = L->I;
+  P.wpr = L->wpr;
+  P.allow = rule->allow_regrow_pruned ? 1 : 0;
+  P.nwords = L->nwords;
+  {  // state of the random-growth generator for (seed, step, layer): three chained SplitMix64 first outputs
+    const unsigned long long a = host_mix(rule->seed + SM64_GAMMA);
+    const unsigned long long b = host_mix((a ^ rule->step) + SM64_GAMMA);
+    P.stream = host_mix((b ^ (unsigned long long)(int64_t)L->layer_id) + SM64_GAMMA);
+  }
+
+  MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
+  MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
+  MST_TRY(run_select<MODE_RAND>(L, P, n_rand, L->rand_bits, s));
+
+  MST_TRY(mst_combine_update_bits(L, n, s));
+  MST_TRY(mst_rebuild_from_bits(L, n, nullptr, 0, c, s));
+  L->cur = n;
+  const int64_t nnz_before = L->nnz;
+  L->nnz = target;
+  MST_TRY(mst_build_csc(L, s));
+
+  if (stats) {
+    max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
+    int32_t f[4] = {0, 0, 0, 0};
+    int32_t total = 0;
+    MST_CUDA_TRY(cudaMemcpyAsync(f, L->flags, sizeof(f), cudaMemcpyDeviceToHost, s));
+    MST_CUDA_TRY(cudaMemcpyAsync(&total, L->wscan[n] + L->nwords, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    MST_CUDA_TRY(cudaStreamSynchronize(s));
+    stats->nnz_before = nnz_before;
+    stats->nnz_after = total;
+    stats->n_prune = n_prune;
+    stats->n_grad = n_grad;
+    stats->n_rand = n_rand;
+    stats->max_row_nnz = f[1];
+    if (f[0] & MST_FLAG_NONFINITE) return MST_ERR_NONFINITE;
+    if ((f[0] & MST_FLAG_CORRUPT) || total != target) return MST_ERR_CORRUPT;
+  }
+  return MST_OK;
+}
