@@ -1,0 +1,241 @@
+"""CUDA library vs the CPU checker, element by element, on seeded inputs (needs a GPU)."""
+import numpy as np
+import pytest
+
+import mst_inputs
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if torch.cuda.is_available():
+    import paper_2408_11746_b200 as mst
+    from gpu_util import (TOL, dev, export_csc, export_csr, host, make_layer, mdtype, rel_err, tdtype, to_dev,
+                          value_bits)
+
+
+def _problem(O, I, T, dtype, density, seed, kind="uniform"):
+    f = mst_inputs.uniform_layer if kind == "uniform" else mst_inputs.zipf_layer
+    return f("t", seed % 7, O, I, T, dtype, density, seed)
+
+
+# ----------------------------------------------------------------- structure
+@pytest.mark.parametrize("O,I,dtype,density,kind", [
+    (64, 64, "f32", 0.25, "uniform"), (130, 257, "bf16", 0.1, "uniform"), (33, 31, "f32", 0.5, "uniform"),
+    (1, 1, "bf16", 1.0, "uniform"), (300, 200, "bf16", 0.0, "uniform"), (97, 160, "f32", 1.0, "uniform"),
+    (768, 768, "bf16", 0.05, "zipf"), (5, 1000, "bf16", 0.3, "uniform"), (1000, 5, "f32", 0.3, "uniform")])
+def test_pack_export_roundtrip(O, I, dtype, density, kind):
+    p = _problem(O, I, 4, dtype, density, 100 + O + I, kind)
+    L = make_layer(p)
+    assert L.nnz == p.nnz
+    L.validate()
+    rp, ci, vb = export_csr(L, dtype)
+    rp_r, ci_r, v_r = oracle.to_csr(p.W, p.mask)
+    np.testing.assert_array_equal(rp, rp_r)
+    np.testing.assert_array_equal(ci, ci_r)
+    np.testing.assert_array_equal(vb, value_bits(v_r, dtype))
+    # CSC view = CSR of the transpose; perm points back into CSR order
+    cp, ri, pm = export_csc(L)
+    cp_r, ri_r, _ = oracle.to_csr(p.W.T, p.mask.T)
+    np.testing.assert_array_equal(cp, cp_r)
+    np.testing.assert_array_equal(ri, ri_r)
+    cols_of_csc = np.repeat(np.arange(I), np.diff(cp_r))
+    np.testing.assert_array_equal(ci_r[pm], cols_of_csc)
+    rows_of_csr = np.repeat(np.arange(O), np.diff(rp_r))
+    np.testing.assert_array_equal(rows_of_csr[pm], ri_r)
+    L.close()
+
+
+def test_pack_capacity_and_padded_weights():
+    p = _problem(40, 70, 4, "f32", 0.5, 9)
+    L = mst.Layer(0, 40, 70, mst.MST_F32, p.nnz - 1)
+    with pytest.raises(mst.MstError) as e:
+        L.pack(to_dev(p, "W"), torch.from_numpy(p.mask).to(dev()))
+    assert e.value.status == 4
+    L.close()
+    L = mst.Layer(0, 40, 70, mst.MST_F32, p.nnz)
+    Wp = to_dev(p, "W", ld=96)
+    L.pack(Wp, torch.from_numpy(p.mask).to(dev()), ldw=96)
+    _, _, vb = export_csr(L, "f32")
+    np.testing.assert_array_equal(vb, value_bits(oracle.to_csr(p.W, p.mask)[2], "f32"))
+    L.close()
+
+
+# ------------------------------------------------------------------ products
+def _run_products(p, L, ldx=None, ldy=None):
+    T, O, I = p.tokens, p.out_features, p.in_features
+    X, dY = to_dev(p, "X", ldx), to_dev(p, "dY", ldy)
+    ldx, ldy = ldx or I, ldy or O
+    Y = torch.full((T, ldy), float("nan"), dtype=tdtype(p), device=dev())
+    dX = torch.full((T, ldx), float("nan"), dtype=tdtype(p), device=dev())
+    dW = torch.full((max(p.nnz, 1),), float("nan"), dtype=torch.float32, device=dev())
+    G = torch.full((O, I), float("nan"), dtype=torch.float32, device=dev())
+    mst.mst_spmm_fwd(L.handle, X, ldx, T, Y, ldy)
+    mst.mst_spmm_bwd_x(L.handle, dY, ldy, T, dX, ldx)
+    mst.mst_sddmm_dw(L.handle, dY, ldy, X, ldx, T, dW)
+    mst.mst_dense_grad(dY, ldy, X, ldx, T, O, I, mdtype(p), G)
+    torch.cuda.synchronize()
+    return host(Y)[:, :O], host(dX)[:, :I], host(dW)[: p.nnz], host(G)
+
+
+@pytest.mark.parametrize("O,I,T,dtype,density,kind,pad", [
+    (160, 200, 300, "bf16", 0.2, "uniform", 0),      # several panels/chunks, ragged tails everywhere
+    (160, 200, 300, "f32", 0.2, "uniform", 0),
+    (130, 257, 513, "bf16", 0.1, "uniform", 0),      # odd sizes: scalar staging path
+    (130, 257, 513, "f32", 0.1, "uniform", 0),
+    (128, 256, 256, "bf16", 0.25, "uniform", 8),     # padded leading dimensions
+    (64, 128, 1, "f32", 0.5, "uniform", 0),          # single token
+    (200, 96, 700, "bf16", 1.0, "uniform", 0),       # all-ones mask
+    (200, 96, 64, "bf16", 0.0, "uniform", 0),        # empty mask
+    (768, 768, 512, "bf16", 0.06, "zipf", 0),        # skewed rows: some full, many empty
+    (3, 5, 7, "f32", 0.6, "uniform", 0),
+    (70, 1100, 260, "bf16", 0.15, "uniform", 0)])
+def test_products_match_oracle(O, I, T, dtype, density, kind, pad):
+    p = _problem(O, I, T, dtype, density, 1000 + O + I + T, kind)
+    L = make_layer(p)
+    Y, dX, dW, G = _run_products(p, L, I + pad if pad else None, O + pad if pad else None)
+    tol = TOL[dtype]
+    Wm = np.where(p.mask == 1, p.W, np.float32(0))
+    assert rel_err(Y, oracle.fwd(p.X, Wm, p.mask)) <= tol
+    assert rel_err(dX, oracle.bwd_x(p.dY, Wm, p.mask)) <= tol
+    Gr = oracle.dense_grad(p.dY, p.X)
+    rows, cols = np.nonzero(p.mask)
+    assert rel_err(dW, Gr[rows, cols]) <= tol
+    assert rel_err(G, Gr) <= tol
+    L.close()
+
+
+def test_results_are_run_to_run_identical():
+    p = _problem(192, 320, 600, "bf16", 0.15, 77)
+    L = make_layer(p)
+    a = _run_products(p, L)
+    b = _run_products(p, L)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x.view(np.uint32), y.view(np.uint32))
+    L.close()
+
+
+def test_step_host_matches_device_entry_points():
+    p = _problem(160, 200, 300, "bf16", 0.2, 5)
+    L = make_layer(p)
+    Y, dX, dW, _ = _run_products(p, L)
+    Xh = torch.from_numpy(p.X_bits.view(np.int16)).pin_memory()
+    dYh = torch.from_numpy(p.dY_bits.view(np.int16)).pin_memory()
+    Yh = torch.empty((300, 160), dtype=torch.int16).pin_memory()
+    dXh = torch.empty((300, 200), dtype=torch.int16).pin_memory()
+    dWh = torch.empty((p.nnz,), dtype=torch.float32).pin_memory()
+    mst.mst_layer_step_host(L.handle, Xh, dYh, 300, Yh, dXh, dWh)
+    np.testing.assert_array_equal(mst_inputs.bf16_bits_to_f32(Yh.numpy().view(np.uint16)), Y)
+    np.testing.assert_array_equal(mst_inputs.bf16_bits_to_f32(dXh.numpy().view(np.uint16)), dX)
+    np.testing.assert_array_equal(dWh.numpy(), dW)
+    L.close()
+
+
+# ------------------------------------------------------------ topology update
+def _update_both(L, p, W, M, G, zeta, target, R, seed, step, allow=False):
+    """Run one update on the GPU and in the oracle from the same state; compare bit-exactly."""
+    O, I = M.shape
+    Gd = None if G is None else torch.from_numpy(G).to(dev())
+    st = mst.mst_topology_update(L.handle, zeta, target, R, seed, step, allow, Gd)
+    n_prune, n_grow, n_rand, n_grad = oracle.mg_counts(zeta, int(M.sum()), target, O * I, R)
+    assert (st.n_prune, st.n_rand, st.n_grad) == (n_prune, n_rand, n_grad)
+    Wn, Mn, *_ = oracle.mg_update(W, M, G, n_prune, n_grad, n_rand, seed, step, p.layer_id, allow)
+    assert st.nnz_after == int(Mn.sum()) == L.nnz
+    assert st.max_row_nnz == int(Mn.sum(1).max())
+    rp, ci, vb = export_csr(L, p.dtype)
+    rp_r, ci_r, v_r = oracle.to_csr(Wn, Mn)
+    np.testing.assert_array_equal(rp, rp_r)
+    np.testing.assert_array_equal(ci, ci_r)
+    np.testing.assert_array_equal(vb, value_bits(v_r, p.dtype))
+    L.validate()
+    return Wn, Mn
+
+
+@pytest.mark.parametrize("O,I,dtype,density,kind,zeta,R,allow", [
+    (96, 160, "f32", 0.25, "uniform", 0.3, 0.25, False), (130, 257, "bf16", 0.1, "uniform", 0.3, 0.25, False),
+    (256, 512, "bf16", 0.05, "zipf", 0.1, 0.25, False), (64, 96, "f32", 0.3, "uniform", 0.3, 0.0, False),
+    (64, 96, "bf16", 0.3, "uniform", 0.3, 1.0, False), (96, 160, "bf16", 0.25, "uniform", 0.5, 0.25, True),
+    (33, 31, "f32", 0.5, "uniform", 1.0, 0.5, False)])
+def test_update_is_bit_exact_over_consecutive_steps(O, I, dtype, density, kind, zeta, R, allow):
+    p = _problem(O, I, 4, dtype, density, 300 + O + I, kind)
+    L = make_layer(p)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    M = p.mask.copy()
+    rng = np.random.default_rng(O * I)
+    for step in range(4):     # grown weights are +0: from the second step on, ties at |w| = 0 decide the pruning
+        G = rng.standard_normal((O, I)).astype(np.float32)
+        G.reshape(-1)[::3] = np.float32(0.25)        # ties among gradient magnitudes
+        G.reshape(-1)[1::5] = np.float32(-0.25)
+        W, M = _update_both(L, p, W, M, G, zeta, -1, R, 42, step, allow)
+    L.close()
+
+
+def test_update_changes_density_both_ways_and_reaches_dense_and_empty():
+    O, I = 80, 96
+    p = _problem(O, I, 4, "bf16", 0.3, 55)
+    L = make_layer(p)        # capacity = O*I
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    M = p.mask.copy()
+    rng = np.random.default_rng(1)
+    for step, frac in enumerate([0.1, 0.04, 0.5, 1.0, 0.2, 0.0, 0.3]):
+        G = rng.standard_normal((O, I)).astype(np.float32)
+        W, M = _update_both(L, p, W, M, G, 0.3, int(round(frac * O * I)), 0.25, 7, step)
+    L.close()
+
+
+def test_update_without_gradient_and_identity():
+    p = _problem(64, 64, 4, "f32", 0.25, 66)
+    L = make_layer(p)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    M = p.mask.copy()
+    W, M = _update_both(L, p, W, M, None, 0.3, -1, 1.0, 3, 0)          # SET rule needs no gradient
+    W2, M2 = _update_both(L, p, W, M, None, 0.0, -1, 0.25, 3, 1)       # zeta = 0: nothing changes
+    np.testing.assert_array_equal(M2, M)
+    L.close()
+
+
+def test_error_statuses():
+    p = _problem(32, 32, 4, "f32", 0.25, 8)
+    # unpacked layer
+    L = mst.Layer(0, 32, 32, mst.MST_F32)
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_layer_nnz(L.handle)
+    assert e.value.status == 9
+    L.close()
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_layer_create(0, 0, 32, mst.MST_F32, 10)
+    assert e.value.status == 2
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_layer_create(0, 32, 32, 5, 10)
+    assert e.value.status == 3
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_layer_create(0, 32, 32, mst.MST_F32, 32 * 32 + 1)
+    assert e.value.status == 4
+    L = make_layer(p, capacity=p.nnz + 10)
+    X = to_dev(p, "X")
+    Y = torch.empty(4, 32, device=dev())
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_spmm_fwd(L.handle, X, 16, 4, Y, 32)          # leading dimension too small
+    assert e.value.status == 2
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_spmm_fwd(L.handle, None, 32, 4, Y, 32)
+    assert e.value.status == 1
+    G = torch.zeros(32, 32, device=dev())
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_topology_update(L.handle, 0.3, p.nnz + 11, 0.25, 0, 0, False, G)     # beyond capacity
+    assert e.value.status == 4
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_topology_update(L.handle, 0.3, 32 * 32 + 1, 0.25, 0, 0, False, G)    # beyond the layer
+    assert e.value.status == 5
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_topology_update(L.handle, 1.5, -1, 0.25, 0, 0, False, G)
+    assert e.value.status == 1
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_topology_update(L.handle, 0.3, -1, 0.25, 0, 0, False, None)          # gradient growth without G
+    assert e.value.status == 1
+    G[3, 4] = float("nan")
+    if p.mask[3, 4] == 0:
+        with pytest.raises(mst.MstError) as e:
+            mst.mst_topology_update(L.handle, 0.3, -1, 0.25, 0, 0, False, G)
+        assert e.value.status == 6
+    L.close()
