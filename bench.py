@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse fully-connected training path (one JSON line on stdout).
+
+A step = one pass of the whole path over the four FC weights of one GPT-2-small block (bf16, 8192 tokens,
+uniform masks at density 0.25): forward SpMM, input-gradient SpMM, weight-gradient SDDMM, dense gradient,
+and one Mixed-Growing topology update (counts, prune/grow selection, mask rewrite, CSR/CSC rebuild) per layer.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+value  = useful (nnz-only) FLOPs of forward + backward, 6*T*nnz per layer, divided by the time of the whole step.
+With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no exchange step).
+--impl reference times the CPU checker (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import mst_inputs  # noqa: E402
+
+METRIC = "sparse_fc_fwd_bwd_useful_tflops"
+UNIT = "TFLOP/s"
+WORKLOAD = "gpt2-small block (qkv, attn_proj, fc1, fc2), T=8192, bf16, uniform masks d=0.25"
+FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # SMs x fp32 lanes x 2 flop x max SM clock
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for ts, r in self.rows if t0 - 0.05 <= ts <= t1 + 0.15 and len(r) >= 7] or \
+               [r for _, r in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(r[0]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for j, n in enumerate(names) if any(r[3 + j].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][1]), "reasons": reasons, "samples": len(rows),
+                "power_w_max": max(float(r[2]) for r in rows)}
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def run_reference(args) -> None:
+    """Time the CPU checker, as it stands, on a bounded sample of the workload (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    oracle.build()
+    Ts = args.ref_tokens
+    layers = mst_inputs.config2(tokens=Ts)
+    cores = oracle.threads()
+
+    def step(k):
+        for p in layers:
+            Wm = np.where(p.mask == 1, p.W, np.float32(0))
+            oracle.fwd(p.X, Wm, p.mask)
+            oracle.bwd_x(p.dY, Wm, p.mask)
+            oracle.dw(p.dY, p.X, p.mask)
+            G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
+            c = oracle.mg_counts(0.3, p.nnz, -1, p.mask.size, 0.25)
+            oracle.mg_update(Wm, p.mask, G, c[0], c[3], c[2], 1, k, p.layer_id)
+
+    for k in range(args.warmup):
+        step(k)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        step(k)
+    dt = time.perf_counter() - t0
+    flops = 6.0 * Ts * sum(p.nnz for p in layers) * args.steps
+    val = flops / dt / 1e12
+    sample = "first %d of 8192 tokens of every layer, whole path per step" % Ts
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def cpu_baseline(tokens: int):
+    import oracle
+    oracle.build()
+    layers = mst_inputs.config2(tokens=tokens)
+    t0 = time.perf_counter()
+    for p in layers:
+        Wm = np.where(p.mask == 1, p.W, np.float32(0))
+        oracle.fwd(p.X, Wm, p.mask)
+        oracle.bwd_x(p.dY, Wm, p.mask)
+        oracle.dw(p.dY, p.X, p.mask)
+        G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
+        c = oracle.mg_counts(0.3, p.nnz, -1, p.mask.size, 0.25)
+        oracle.mg_update(Wm, p.mask, G, c[0], c[3], c[2], 1, 0, p.layer_id)
+    dt = time.perf_counter() - t0
+    flops = 6.0 * tokens * sum(p.nnz for p in layers)
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": "first %d of 8192 tokens of every layer, whole path once (%.1f s)" % (tokens, dt)}
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-tokens", type=int, default=48, help="tokens per layer in one reference-arm step")
+    ap.add_argument("--cpu-tokens", type=int, default=3072, help="tokens per layer in the cpu_baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2408_11746_b200 as mst
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    peaks = measured_peaks()
+    probs = mst_inputs.config2()
+    T = probs[0].tokens
+
+    def up_bits(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    class Slot:
+        pass
+
+    slots = []
+    for p in probs:
+        s = Slot()
+        s.p, s.O, s.I, s.nnz = p, p.out_features, p.in_features, p.nnz
+        s.L = mst.Layer(p.layer_id, s.O, s.I, mst.MST_BF16)
+        s.L.pack(up_bits(p.W_bits), torch.from_numpy(p.mask).to(dev))
+        s.X, s.dY = up_bits(p.X_bits), up_bits(p.dY_bits)
+        s.Y = torch.empty(T, s.O, dtype=torch.bfloat16, device=dev)
+        s.dX = torch.empty(T, s.I, dtype=torch.bfloat16, device=dev)
+        s.dW = torch.empty(s.nnz, dtype=torch.float32, device=dev)
+        s.G = torch.empty(s.O, s.I, dtype=torch.float32, device=dev)
+        # pinned host copies for the end-to-end leg
+        s.Xh = torch.from_numpy(p.X_bits.view(np.int16)).pin_memory()
+        s.dYh = torch.from_numpy(p.dY_bits.view(np.int16)).pin_memory()
+        s.Yh = torch.empty((T, s.O), dtype=torch.int16).pin_memory()
+        s.dXh = torch.empty((T, s.I), dtype=torch.int16).pin_memory()
+        s.dWh = torch.empty((s.nnz,), dtype=torch.float32).pin_memory()
+        slots.append(s)
+    stream = torch.cuda.current_stream()
+    KERNELS = ["spmm_fwd", "spmm_bwd_x", "sddmm_dw", "dense_grad", "topology_update"]
+    timers = {k: [] for k in KERNELS}
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    def step(k: int, timed: bool):
+        for s in slots:
+            marks = [ev()] if timed else None
+            s.L.fwd(s.X, s.Y, T)
+            if timed: marks.append(ev())
+            s.L.bwd_x(s.dY, s.dX, T)
+            if timed: marks.append(ev())
+            s.L.sddmm(s.dY, s.X, T, s.dW)
+            if timed: marks.append(ev())
+            s.L.dense_grad(s.dY, s.X, T, s.G)
+            if timed: marks.append(ev())
+            s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=1, step=k, G_dense=s.G, want_stats=False)
+            if timed:
+                marks.append(ev())
+                for j, name in enumerate(KERNELS):
+                    timers[name].append((s, marks[j], marks[j + 1]))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for k in range(args.warmup):
+        step(k, False)
+    barrier()
+    sampler = ClockSampler(local)
+    time.sleep(0.25)
+    w0 = time.time()
+    e0 = ev()
+    for k in range(args.steps):
+        step(args.warmup + k, True)
+    e1 = ev()
+    barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1)
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    useful = 6.0 * T * sum(s.nnz for s in slots)          # per step, per replica
+    value = useful * args.steps * world / (ms * 1e-3) / 1e12
+
+    # ---- per-kernel summary and the roofline of the dominant kernel
+    per = {}
+    for name in KERNELS:
+        tot = sum(a.elapsed_time(b) for _, a, b in timers[name])
+        per[name] = {"ms_per_step": tot / args.steps, "launches": len(timers[name])}
+    dom = max(per, key=lambda n: per[n]["ms_per_step"])
+    es = 2
+
+    def algorithmic(name, s):
+        """(flops, bytes) of one call on layer slot s."""
+        x, y, idx = T * s.I * es, T * s.O * es, s.nnz * (es + 2) + 4 * (s.O + 1)
+        if name == "spmm_fwd": return 2.0 * T * s.nnz, x + y + idx
+        if name == "spmm_bwd_x": return 2.0 * T * s.nnz, x + y + idx + 4 * s.nnz
+        if name == "sddmm_dw": return 2.0 * T * s.nnz, x + y + s.nnz * 2 + 4 * (s.O + 1) + 4 * s.nnz
+        if name == "dense_grad": return 2.0 * T * s.O * s.I, x + y + 4 * s.O * s.I
+        return 0.0, 4.0 * s.O * s.I + 2 * s.nnz * (es + 2 + 6)
+    dom_ms = sum(a.elapsed_time(b) for _, a, b in timers[dom])
+    flops = sum(algorithmic(dom, s)[0] for s, _, _ in timers[dom])
+    byts = sum(algorithmic(dom, s)[1] for s, _, _ in timers[dom])
+    t_alu = flops / (FMA_PEAK_TFLOPS * 1e12)
+    t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+    if dom == "topology_update" or t_hbm >= t_alu:
+        roof = {"bound": "hbm", "achieved": byts / (dom_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    else:
+        roof = {"bound": "alu", "achieved": flops / (dom_ms * 1e-3) / 1e12, "peak": FMA_PEAK_TFLOPS, "unit": "TFLOP/s"}
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": dom,
+                 "peak_source": peaks["source"] if roof["bound"] == "hbm" else
+                 "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"})
+    for name in KERNELS:
+        f = sum(algorithmic(name, s)[0] for s, _, _ in timers[name])
+        per[name]["useful_tflops"] = f / (per[name]["ms_per_step"] * args.steps * 1e-3) / 1e12 if f else None
+
+    # ---- end to end: host buffers in, host results out, through the C ABI
+    def e2e_step(k):
+        for s in slots:
+            mst.mst_layer_step_host(s.L.handle, s.Xh, s.dYh, T, s.Yh, s.dXh, s.dWh)
+            s.L.dense_grad(s.dY, s.X, T, s.G)
+            s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=2, step=k, G_dense=s.G, want_stats=False)
+    e2e_step(0)
+    barrier()
+    e2e_steps = max(2, min(args.steps, 5))
+    a = ev()
+    for k in range(e2e_steps):
+        e2e_step(1 + k)
+    b = ev()
+    barrier()
+    e2e_ms = a.elapsed_time(b)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = sum(T * (s.I + s.O) * es for s in slots)
+    d2h = sum(T * (s.I + s.O) * es + 4 * s.nnz for s in slots)
+    e2e = {"value": useful * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    launches_per_layer = 4 + 46       # 4 product kernels + update (3 radix selects, mask rewrite, CSR and CSC rebuild)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: four layers' distinct buffers, %.0f MB touched "
+                   "per step" % (sum(2 * T * (s.I + s.O) * es for s in slots) / 1e6),
+                   "update": "every step, zeta=0.3, R=0.25, target = current nnz", "replicas": world},
+        "clocks": clocks, "roofline": roof, "kernels": per,
+        "fwd_bwd_only_tflops": useful / ((per["spmm_fwd"]["ms_per_step"] + per["spmm_bwd_x"]["ms_per_step"] +
+                                          per["sddmm_dw"]["ms_per_step"]) * 1e-3) / 1e12,
+        "e2e": e2e, "gpu_launches": launches_per_layer * len(slots) * args.steps,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(args.cpu_tokens)
+    if rank == 0:
+        print(json.dumps(out))
+    for s in slots:
+        s.L.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
