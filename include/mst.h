@@ -144,6 +144,31 @@ mst_status_t mst_topology_update(mst_layer_t* layer, double prune_frac, const ms
 mst_status_t mst_layer_step_host(mst_layer_t* layer, const void* X_host, const void* dY_host, int64_t T, void* Y_host,
                                  void* dX_host, float* dW_vals_host, mst_stream_t stream);
 
+/* Dense mask -> canonical CSR with no handle and NO allocation (the paper has no counterpart: this entry point
+ * exists for callers that must not allocate device memory).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a host framework that has handed the whole GPU to its
+ * own memory pool and forbids plugins to allocate, a real-time or serving loop that must not take the allocator's
+ * implicit device synchronisation, or a thread working while another thread of the process is capturing a stream
+ * (allocation calls are illegal during a global-mode capture).  Those callers cannot create an mst_layer_t (creation
+ * allocates), yet still want the compressed structure of a mask.
+ *
+ * Same result as mst_pack followed by mst_export_csr, written into the caller's buffers:
+ *   W_dense  device, [O x ldw] layer dtype;  mask device uint8 [O x I]
+ *   row_ptr  device int32 [O+1]; row_ptr[O] receives the true number of active entries
+ *   col_idx  device int32 [nnz_capacity];  vals device [nnz_capacity] in `dtype`
+ * Entries at CSR positions >= nnz_capacity are not written (compare row_ptr[O] with the capacity afterwards).
+ * Work space is a fixed array inside the library (about 3 MB of device memory on every GPU that loads the library,
+ * held until the process ends), which limits the layer to O*I <= 4 194 304 entries and O*ceil(I/32) <= 262 144 mask
+ * words; larger layers return MST_ERR_CAPACITY.  The call itself allocates nothing and frees nothing.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress); make that first call
+ * outside any stream capture.  All calls share the one array: calls whose GPU work may overlap (different streams,
+ * different threads) race on it - keep them on one stream or order them with events.  Nothing in the array has to
+ * be cleared between calls; every call overwrites the part it reads.  Asynchronous on `stream`. */
+mst_status_t mst_mask_to_csr_noalloc(int32_t out_features, int32_t in_features, mst_dtype_t dtype, const void* W_dense,
+                                     int64_t ldw, const uint8_t* mask, int64_t nnz_capacity, int32_t* row_ptr,
+                                     int32_t* col_idx, void* vals, mst_stream_t stream);
+
 const char* mst_status_string(mst_status_t status);
 
 #ifdef __cplusplus

@@ -24,7 +24,8 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad",
-           "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_status_string"]
+           "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_mask_to_csr_noalloc",
+           "mst_status_string"]
 
 
 class MstError(RuntimeError):
@@ -65,6 +66,7 @@ _sig = {
     "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
     "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
+    "mst_mask_to_csr_noalloc": [_i32, _i32, ctypes.c_int, _vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp],
 }
 for _n, _a in _sig.items():
     getattr(_lib, _n).argtypes = _a
@@ -183,6 +185,19 @@ def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, ran
 def mst_layer_step_host(layer: int, X_host, dY_host, T: int, Y_host, dX_host, dW_vals_host, stream=None) -> None:
     _check(_lib.mst_layer_step_host(layer, _ptr(X_host), _ptr(dY_host), T, _ptr(Y_host), _ptr(dX_host),
                                     _ptr(dW_vals_host), _stream(stream)), "mst_layer_step_host")
+
+
+def mst_mask_to_csr_noalloc(out_features: int, in_features: int, dtype: int, W_dense, ldw: int, mask,
+                            nnz_capacity: int, row_ptr, col_idx, vals, stream=None) -> None:
+    """Dense mask -> CSR into caller-owned buffers, for callers that may not allocate device memory.
+
+    The library works in a fixed internal array instead of allocating, so the layer is limited to
+    4 194 304 entries, overlapping calls race, and the first call per device should happen outside
+    stream capture.  See ``include/mst.h``.
+    """
+    _check(_lib.mst_mask_to_csr_noalloc(out_features, in_features, dtype, _ptr(W_dense), ldw, _ptr(mask),
+                                        nnz_capacity, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _stream(stream)),
+           "mst_mask_to_csr_noalloc")
 
 
 # ---------------------------------------------------------------- small RAII convenience

@@ -409,3 +409,98 @@ extern "C" mst_status_t mst_validate(const mst_layer_t* L, mst_stream_t stream) 
   if (f & MST_FLAG_NONFINITE) return MST_ERR_NONFINITE;
   return MST_OK;
 }
+
+// ---- allocation-free mask -> CSR ------------------------------------------------------------------------------------
+// Same popcount / scan / fill pipeline as mst_pack, but with no handle and no allocation: the mask words, their
+// popcounts, the scan and the scan partials live in one file-scope device array that every GPU loading this library
+// holds until the process exits.
+namespace {
+
+constexpr int64_t NOALLOC_MAX_NUMEL = (int64_t)1 << 22;  // 4 194 304 entries, e.g. a 4096 x 1024 layer
+constexpr int64_t NOALLOC_MAX_WORDS = (int64_t)1 << 18;  // >= numel/32 + rows for every shape accepted below
+constexpr int64_t NOALLOC_SUMS = NOALLOC_MAX_WORDS / SCAN_TILE + 2;
+constexpr size_t NOALLOC_OFF_BITS = 0;
+constexpr size_t NOALLOC_OFF_CNT = NOALLOC_OFF_BITS + 4 * (size_t)NOALLOC_MAX_WORDS;
+constexpr size_t NOALLOC_OFF_SCAN = NOALLOC_OFF_CNT + 4 * (size_t)(NOALLOC_MAX_WORDS + 64);
+constexpr size_t NOALLOC_OFF_SUMS = NOALLOC_OFF_SCAN + 4 * (size_t)(NOALLOC_MAX_WORDS + 64);
+constexpr size_t NOALLOC_BYTES = NOALLOC_OFF_SUMS + 4 * (size_t)(NOALLOC_SUMS + 62);
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};
+
+// Device address of the scratch array on the current device.  g_noalloc_scratch itself is only a host-side handle
+// for the symbol: the address a kernel can use has to be asked for, once per device, with that device current.
+mst_status_t noalloc_scratch(unsigned char** out) {
+  int devi = -1;
+  MST_CUDA_TRY(cudaGetDevice(&devi));
+  if (devi < 0 || devi >= NOALLOC_MAX_DEVICES) return MST_ERR_INVALID_ARG;
+  if (!g_noalloc_ptr[devi]) {
+    void* p = nullptr;
+    MST_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+    if (!p) return MST_ERR_CUDA;
+    g_noalloc_ptr[devi] = (unsigned char*)p;
+  }
+  *out = g_noalloc_ptr[devi];
+  return MST_OK;
+}
+
+// one warp per mask word, lane = bit; entries at positions >= cap are counted but not written
+template <typename V>
+__global__ void fill_csr_external(const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan, int O, int I,
+                                  int wpr, const V* __restrict__ dense_W, int64_t ldw, int64_t cap,
+                                  int32_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx, V* __restrict__ vals) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  const int64_t nwords = (int64_t)O * wpr;
+  if (w >= nwords) return;
+  const int o = (int)(w / wpr), wc = (int)(w % wpr);
+  const uint32_t b = bits[w];
+  const int32_t base = wscan[w];
+  if (wc == 0 && lane == 0) {
+    row_ptr[o] = base;
+    if (o == O - 1) row_ptr[O] = wscan[nwords];
+  }
+  if ((b >> lane) & 1u) {
+    const int64_t pos = (int64_t)base + __popc(b & lanemask_lt());
+    if (pos < cap) {
+      const int c = wc * 32 + lane;
+      col_idx[pos] = c;
+      vals[pos] = dense_W[(int64_t)o * ldw + c];
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" mst_status_t mst_mask_to_csr_noalloc(int32_t O, int32_t I, mst_dtype_t dtype, const void* W_dense,
+                                                int64_t ldw, const uint8_t* mask, int64_t nnz_capacity,
+                                                int32_t* row_ptr, int32_t* col_idx, void* vals, mst_stream_t stream) {
+  if (!W_dense || !mask || !row_ptr || !col_idx || !vals || nnz_capacity < 0) return MST_ERR_INVALID_ARG;
+  if (dtype != MST_F32 && dtype != MST_BF16) return MST_ERR_DTYPE;
+  if (O < 1 || I < 1 || O > 65535 || I > 65535 || ldw < I) return MST_ERR_SHAPE;
+  const int wpr = (I + 31) / 32;
+  const int64_t nwords = (int64_t)O * wpr;
+  if ((int64_t)O * I > NOALLOC_MAX_NUMEL || nwords > NOALLOC_MAX_WORDS) return MST_ERR_CAPACITY;
+  unsigned char* base = nullptr;
+  MST_TRY(noalloc_scratch(&base));
+  uint32_t* bits = (uint32_t*)(base + NOALLOC_OFF_BITS);
+  int32_t* cnt = (int32_t*)(base + NOALLOC_OFF_CNT);
+  int32_t* scan = (int32_t*)(base + NOALLOC_OFF_SCAN);
+  int32_t* sums = (int32_t*)(base + NOALLOC_OFF_SUMS);
+  cudaStream_t s = (cudaStream_t)stream;
+  // every word of the scratch that the later kernels read is written first by this call: nothing needs clearing
+  mask_bytes_to_bits<<<blocks_for(nwords * 32, 256), 256, 0, s>>>(mask, O, I, wpr, bits);
+  popc_words<<<blocks_for(nwords, 256), 256, 0, s>>>(bits, nwords, cnt);
+  MST_TRY(mst_scan_i32(cnt, scan, nwords, sums, s));
+  const unsigned grid = blocks_for(nwords * 32, 256);
+  if (dtype == MST_F32)
+    fill_csr_external<float><<<grid, 256, 0, s>>>(bits, scan, O, I, wpr, (const float*)W_dense, ldw, nnz_capacity,
+                                                  row_ptr, col_idx, (float*)vals);
+  else
+    fill_csr_external<uint16_t><<<grid, 256, 0, s>>>(bits, scan, O, I, wpr, (const uint16_t*)W_dense, ldw, nnz_capacity,
+                                                     row_ptr, col_idx, (uint16_t*)vals);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
