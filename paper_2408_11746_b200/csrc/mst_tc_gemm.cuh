@@ -1,0 +1,43 @@
+// Interface of the tcgen05 (5th-generation tensor core) bf16 contraction used for the dense gradient,
+// the dense-tile SpMM path and the sampled weight gradient.  Internal to libmst.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mst.h"
+
+// C[M x N] = A * B^T-like contraction over K with fp32 accumulation in tensor memory.
+//   A operand: K-major   -> A is stored [M x K] row-major (lda elements between rows), or
+//              MN-major  -> A is stored [K x M] row-major (lda elements between K rows)
+//   B operand: K-major   -> B is stored [N x K] row-major, or MN-major -> [K x N] row-major
+// Epilogues:
+//   MST_TC_OUT_BF16     C bf16 row-major [M x ldc]
+//   MST_TC_OUT_F32      C fp32 row-major [M x ldc]; with splits > 1 writes partial sums to
+//                       partial[split][M x N] (contiguous) which mst_tc_reduce then sums in a fixed order
+//   MST_TC_OUT_SAMPLED  only entries under a bit mask are written, to their CSR position:
+//                       out[wscan[w] + rank] for mask word w = m*wpr + n/32 (needs N-tile offsets multiple of 32)
+enum { MST_TC_OUT_BF16 = 0, MST_TC_OUT_F32 = 1, MST_TC_OUT_SAMPLED = 2 };
+
+struct mst_tc_gemm_args {
+  const void* A;
+  int64_t lda;
+  int a_mn_major;
+  const void* B;
+  int64_t ldb;
+  int b_mn_major;
+  int64_t M, N, K;
+  int epilogue;
+  void* out;
+  int64_t ldc;
+  int splits;            // K is cut into `splits` contiguous ranges (F32 / SAMPLED epilogues only)
+  float* partial;        // [splits][M*N] (F32) or [splits][nnz] (SAMPLED) when splits > 1
+  const uint32_t* bits;  // SAMPLED: mask words, wpr per row
+  const int32_t* wscan;  // SAMPLED: exclusive popcount scan of the words
+  int wpr;
+  int64_t nnz;           // SAMPLED: number of stored entries (partial stride)
+};
+
+// Returns MST_ERR_SHAPE when the operands cannot be described to the TMA unit (leading dimension or base address
+// not 16-byte aligned); the caller then falls back to the CUDA-core kernel.
+mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s);
+bool mst_tc_gemm_usable(const void* A, int64_t lda, const void* B, int64_t ldb);
