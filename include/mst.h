@@ -116,7 +116,9 @@ mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy
                           float* dW_vals, mst_stream_t stream);
 
 /* Dense gradient for growth, G = dY^T X, float [O x I] contiguous (Algorithm 1, gradient-growth line: |grad L| on
- * empty slots; Sec. 2.1 "infrequent full gradient calculation").  No layer handle: a plain contraction. */
+ * empty slots; Sec. 2.1 "infrequent full gradient calculation").  No layer handle: a plain contraction.
+ * bf16 inputs with 16-byte-aligned rows run on the tensor cores and may use a process-wide scratch buffer for
+ * split partial sums (allocated on first use, grown on demand): such calls must not overlap on the GPU. */
 mst_status_t mst_dense_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int32_t out_features,
                             int32_t in_features, mst_dtype_t dtype, float* G, mst_stream_t stream);
 
@@ -168,6 +170,10 @@ mst_status_t mst_layer_step_host(mst_layer_t* layer, const void* X_host, const v
 mst_status_t mst_mask_to_csr_noalloc(int32_t out_features, int32_t in_features, mst_dtype_t dtype, const void* W_dense,
                                      int64_t ldw, const uint8_t* mask, int64_t nnz_capacity, int32_t* row_ptr,
                                      int32_t* col_idx, void* vals, mst_stream_t stream);
+
+/* Sticky error bits of kernels that run without a layer handle (bit 0: a bounded wait inside the tensor-core
+ * contraction expired and the block gave up; its output is then undefined).  Synchronises the device. */
+mst_status_t mst_device_error_flags(int32_t* flags);
 
 const char* mst_status_string(mst_status_t status);
 

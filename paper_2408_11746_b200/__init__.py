@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_mask_to_csr_noalloc",
-           "mst_status_string"]
+           "mst_device_error_flags", "mst_status_string"]
 
 
 class MstError(RuntimeError):
@@ -66,6 +66,7 @@ _sig = {
     "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
     "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
+    "mst_device_error_flags": [ctypes.POINTER(_i32)],
     "mst_mask_to_csr_noalloc": [_i32, _i32, ctypes.c_int, _vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp],
 }
 for _n, _a in _sig.items():
@@ -185,6 +186,12 @@ def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, ran
 def mst_layer_step_host(layer: int, X_host, dY_host, T: int, Y_host, dX_host, dW_vals_host, stream=None) -> None:
     _check(_lib.mst_layer_step_host(layer, _ptr(X_host), _ptr(dY_host), T, _ptr(Y_host), _ptr(dX_host),
                                     _ptr(dW_vals_host), _stream(stream)), "mst_layer_step_host")
+
+
+def mst_device_error_flags() -> int:
+    f = _i32()
+    _check(_lib.mst_device_error_flags(ctypes.byref(f)), "mst_device_error_flags")
+    return f.value
 
 
 def mst_mask_to_csr_noalloc(out_features: int, in_features: int, dtype: int, W_dense, ldw: int, mask,

@@ -1,8 +1,12 @@
 // Dense gradient for gradient-based growth:  G[o, i] = sum_t dY[t, o] * X[t, i]   (fp32 out).
 //
-// CUDA-core tiled contraction (fp32 accumulate): 64 x 64 output tile per block, 16-token slices staged in shared
-// memory in their natural layout (both operands are contiguous along the output dimensions), 4 x 4 outputs per thread.
+// bf16 operands with 16-byte-aligned rows go to the tensor cores (mst_tc_gemm.cu): both operands are MN-major there
+// (dY is [T x O], X is [T x I], the contraction runs over T), the token range is split across blocks when the output
+// has too few tiles to fill the GPU, and the partial sums are added in a fixed order.
+// Everything else (fp32, odd leading dimensions) uses the CUDA-core tiled contraction below (fp32 accumulate): 64 x 64
+// output tile per block, 16-token slices staged in shared memory in their natural layout, 4 x 4 outputs per thread.
 #include "mst_internal.cuh"
+#include "mst_tc_gemm.cuh"
 
 namespace {
 
@@ -68,6 +72,26 @@ extern "C" mst_status_t mst_dense_grad(const void* dY, int64_t lddy, const void*
   if (dtype != MST_F32 && dtype != MST_BF16) return MST_ERR_DTYPE;
   if (lddy < out_features || ldx < in_features) return MST_ERR_SHAPE;
   cudaStream_t s = (cudaStream_t)stream;
+  if (T == 0) {
+    MST_CUDA_TRY(cudaMemsetAsync(G, 0, sizeof(float) * (size_t)out_features * in_features, s));
+    return MST_OK;
+  }
+  if (dtype == MST_BF16 && mst_tc_gemm_usable(dY, lddy, X, ldx) && ((reinterpret_cast<uintptr_t>(G) & 15u) == 0)) {
+    mst_tc_gemm_args a = {};
+    a.A = dY; a.lda = lddy; a.a_mn_major = 1;
+    a.B = X; a.ldb = ldx; a.b_mn_major = 1;
+    a.M = out_features; a.N = in_features; a.K = T;
+    a.epilogue = MST_TC_OUT_F32;
+    a.out = G; a.ldc = in_features;
+    const int64_t tiles = ((int64_t)(out_features + 127) / 128) * ((in_features + 255) / 256);
+    a.splits = mst_tc_pick_splits(tiles, (T + 63) / 64);
+    if (a.splits > 1) {
+      void* ws = nullptr;
+      MST_TRY(mst_workspace(sizeof(float) * (size_t)a.splits * out_features * in_features, &ws));
+      a.partial = (float*)ws;
+    }
+    return mst_tc_gemm(a, s);
+  }
   dim3 grid((unsigned)((in_features + TN - 1) / TN), (unsigned)((out_features + TM - 1) / TM));
   if (dtype == MST_F32)
     dense_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dY, lddy, (const float*)X, ldx, T, out_features,

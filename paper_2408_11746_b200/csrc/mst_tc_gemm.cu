@@ -1,0 +1,461 @@
+// bf16 contraction on the 5th-generation tensor cores (tcgen05) with fp32 accumulators in tensor memory.
+//
+// One persistent block per SM, 192 threads in three roles:
+//   warp 0     producer: one lane issues TMA tile loads (cp.async.bulk.tensor, 128-byte swizzle) into a 4-stage
+//              shared-memory ring, signalling "full" mbarriers by transaction bytes;
+//   warp 1     one lane issues tcgen05.mma (M=128, N=256, K=16 per instruction) from shared-memory descriptors
+//              into one of two 128x256 fp32 accumulators in tensor memory, tcgen05.commit releases the smem stage
+//              ("empty") and, after the last K block, hands the accumulator to the epilogue ("tmem_full");
+//   warps 2-5  epilogue: tcgen05.ld 32 columns at a time (one row per thread), convert / sample / store, then
+//              release the accumulator ("tmem_empty") so the next tile's MMAs overlap this tile's stores.
+// Operands may be K-major ([rows x K] row-major) or MN-major ([K x rows] row-major, as dY and X are for
+// G = dY^T X): the tile is fetched with 64-element-wide boxes either way and described to the tensor core with the
+// matching canonical layout (K-major: 8-row groups 1024 B apart; MN-major: 64-wide blocks one box apart).
+// Every mbarrier wait is bounded: on expiry the block raises an abort flag, records an error bit, skips the rest
+// of its work, frees its tensor memory and returns.
+#include "mst_tc_gemm.cuh"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "mst_internal.cuh"
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2;  // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;  // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BOX_BYTES = 64 * BK * 2;  // one 64-wide MN-major box: 8 KiB
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+
+__device__ int g_tc_error = 0;  // sticky: 1 = a bounded wait expired
+
+struct Params {
+  int64_t M, N;
+  int kblocks;        // ceil(K / BK)
+  int splits;
+  int m_tiles, n_tiles;
+  int a_mn, b_mn;
+  int epilogue;
+  void* out;
+  int64_t ldc;
+  float* partial;
+  const uint32_t* bits;
+  const int32_t* wscan;
+  int wpr;
+  int64_t nnz;
+};
+
+// ------------------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the block is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (it > SPIN_LIMIT) {
+      *abort_flag = 1;
+      atomicOr(&g_tc_error, 1);
+      return false;
+    }
+    if (it > 128) __nanosleep(40);
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(tm), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptors, 128-byte swizzle, version 1 (Blackwell).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version
+  d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params P) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
+  const uint32_t bar_base = tiles_base + STAGES * STAGE_BYTES;
+  // barrier slots (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+  const uint32_t full0 = bar_base, empty0 = bar_base + 8 * STAGES, tfull0 = bar_base + 16 * STAGES,
+                 tempty0 = tfull0 + 16;
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_sh;
+  volatile int* abort_flag = &abort_sh;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    abort_sh = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull0 + 8 * a, 1);
+      mbar_init(tempty0 + 8 * a, 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+
+  const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
+  const int tiles = P.m_tiles * P.n_tiles;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      for (int64_t w = blockIdx.x; w < works && !*abort_flag; w += gridDim.x) {
+        const int split = (int)(w / tiles), t = (int)(w % tiles);
+        const int m0 = (t / P.n_tiles) * BM, n0 = (t % P.n_tiles) * BN;
+        const int kb0 = (int)((int64_t)split * P.kblocks / P.splits), kb1 = (int)((int64_t)(split + 1) * P.kblocks / P.splits);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
+          const uint32_t fb = full0 + 8 * s;
+          const uint32_t sa = tiles_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          if (P.a_mn) {
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d(sa + j * BOX_BYTES, &tmA, m0 + j * 64, kb * BK, fb);
+          } else {
+            tma_load_2d(sa, &tmA, kb * BK, m0, fb);
+          }
+          if (P.b_mn) {
+            for (int j = 0; j < BN / 64; ++j) tma_load_2d(sb + j * BOX_BYTES, &tmB, n0 + j * 64, kb * BK, fb);
+          } else {
+            tma_load_2d(sb, &tmB, kb * BK, n0, fb);
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 256, operand majors
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.a_mn ? 1 : 0) << 15) |
+                             ((uint32_t)(P.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      int s = 0, acc = 0;
+      uint32_t ph = 0, acc_ph = 0;
+      for (int64_t w = blockIdx.x; w < works && !*abort_flag; w += gridDim.x) {
+        const int split = (int)(w / tiles);
+        const int kb0 = (int)((int64_t)split * P.kblocks / P.splits), kb1 = (int)((int64_t)(split + 1) * P.kblocks / P.splits);
+        if (!mbar_wait(tempty0 + 8 * acc, acc_ph ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        bool ok = true;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = P.a_mn ? smem_desc(sa + k * (UMMA_K * 128), BOX_BYTES, 1024)
+                                       : smem_desc(sa + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = P.b_mn ? smem_desc(sb + k * (UMMA_K * 128), BOX_BYTES, 1024)
+                                       : smem_desc(sb + k * (UMMA_K * 2), 16, 1024);
+            tc_mma(d_tmem, ad, bd, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(empty0 + 8 * s);  // the smem stage is free once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull0 + 8 * acc);  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_ph = 0;
+    for (int64_t w = blockIdx.x; w < works; w += gridDim.x) {
+      const int split = (int)(w / tiles), t = (int)(w % tiles);
+      const int m0 = (t / P.n_tiles) * BM, n0 = (t % P.n_tiles) * BN;
+      if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
+      tc_fence_after();
+      const int64_t m = (int64_t)m0 + q * 32 + lane;
+      const bool row_ok = m < P.M;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int n = n0 + c * 32;
+        if (n >= P.N) break;  // uniform
+        uint32_t r[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+        if (!row_ok) continue;
+        if (P.epilogue == MST_TC_OUT_BF16) {
+          uint16_t* dst = reinterpret_cast<uint16_t*>(P.out) + m * P.ldc + n;
+          if (n + 32 <= P.N && ((P.ldc & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.out) & 15u) == 0)) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint4 o;
+              o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+              o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+              o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+              o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+              reinterpret_cast<uint4*>(dst)[v] = o;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n + j < P.N) dst[j] = (uint16_t)(pack_bf16(__uint_as_float(r[j]), 0.f) & 0xFFFFu);
+          }
+        } else if (P.epilogue == MST_TC_OUT_F32) {
+          float* base = P.splits > 1 ? P.partial + (int64_t)split * P.M * P.N + m * P.N : reinterpret_cast<float*>(P.out) + m * P.ldc;
+          float* dst = base + n;
+          const int64_t ld = P.splits > 1 ? P.N : P.ldc;
+          if (n + 32 <= P.N && ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(base) & 15u) == 0)) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+              reinterpret_cast<uint4*>(dst)[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n + j < P.N) dst[j] = __uint_as_float(r[j]);
+          }
+        } else {
+          // sampled: the 32 columns of this chunk are one mask word of row m
+          const int64_t wi = m * P.wpr + (n >> 5);
+          const uint32_t word = P.bits[wi];
+          float* dst = (P.splits > 1 ? P.partial + (int64_t)split * P.nnz : reinterpret_cast<float*>(P.out)) + P.wscan[wi];
+          int rank = 0;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if ((word >> j) & 1u) {
+              dst[rank] = __uint_as_float(r[j]);
+              ++rank;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+      if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (*abort_flag) {
+    // give copies and MMAs already in flight time to land before shared and tensor memory are released
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// out[i] = sum over splits of partial[s][i], fixed order
+__global__ void tc_reduce_kernel(const float* __restrict__ partial, int splits, int64_t n, float* __restrict__ out) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float s = partial[i];
+  for (int k = 1; k < splits; ++k) s += partial[(int64_t)k * n + i];
+  out[i] = s;
+}
+
+// ------------------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+// rows x cols (cols contiguous, ld elements between rows) bf16 matrix; box = box_rows x 64 columns
+bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1u, 1u};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+}  // namespace
+
+int mst_tc_pick_splits(int64_t tiles, int64_t kblocks) {
+  const int sms = sm_count();
+  if (tiles * 4 >= sms * 3) return 1;  // one wave is already at least three quarters full
+  int64_t sp = sms / tiles;
+  if (sp > kblocks) sp = kblocks;
+  if (sp > 16) sp = 16;
+  return sp < 1 ? 1 : (int)sp;
+}
+
+mst_status_t mst_workspace(size_t bytes, void** ptr) {
+  static void* buf = nullptr;
+  static size_t cap = 0;
+  if (bytes > cap) {
+    if (buf) {
+      MST_CUDA_TRY(cudaDeviceSynchronize());
+      MST_CUDA_TRY(cudaFree(buf));
+      buf = nullptr;
+      cap = 0;
+    }
+    const size_t want = (bytes + ((size_t)1 << 20)) & ~(((size_t)1 << 20) - 1);
+    MST_CUDA_TRY(cudaMalloc(&buf, want));
+    cap = want;
+  }
+  *ptr = buf;
+  return MST_OK;
+}
+
+bool mst_tc_gemm_usable(const void* A, int64_t lda, const void* B, int64_t ldb) {
+  return (lda % 8 == 0) && (ldb % 8 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15u) == 0) &&
+         ((reinterpret_cast<uintptr_t>(B) & 15u) == 0) && encode_fn() != nullptr;
+}
+
+mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
+  if (a.M <= 0 || a.N <= 0 || a.K <= 0) return MST_ERR_INVALID_ARG;
+  if (!mst_tc_gemm_usable(a.A, a.lda, a.B, a.ldb)) return MST_ERR_SHAPE;
+  CUtensorMap tmA, tmB;
+  // K-major: [rows x K], box 64 (K) x tile rows.  MN-major: [K x rows], box 64 (rows) x BK.
+  const bool okA = a.a_mn_major ? make_map(&tmA, a.A, a.K, a.M, a.lda, BK) : make_map(&tmA, a.A, a.M, a.K, a.lda, BM);
+  const bool okB = a.b_mn_major ? make_map(&tmB, a.B, a.K, a.N, a.ldb, BK) : make_map(&tmB, a.B, a.N, a.K, a.ldb, BN);
+  if (!okA || !okB) return MST_ERR_SHAPE;
+  Params P;
+  P.M = a.M;
+  P.N = a.N;
+  P.kblocks = (int)((a.K + BK - 1) / BK);
+  P.splits = a.splits < 1 ? 1 : a.splits;
+  if (P.splits > P.kblocks) P.splits = P.kblocks;
+  if (a.epilogue == MST_TC_OUT_BF16) P.splits = 1;
+  P.m_tiles = (int)((a.M + BM - 1) / BM);
+  P.n_tiles = (int)((a.N + BN - 1) / BN);
+  P.a_mn = a.a_mn_major;
+  P.b_mn = a.b_mn_major;
+  P.epilogue = a.epilogue;
+  P.out = a.out;
+  P.ldc = a.ldc;
+  P.partial = a.partial;
+  P.bits = a.bits;
+  P.wscan = a.wscan;
+  P.wpr = a.wpr;
+  P.nnz = a.nnz;
+  if (P.splits > 1 && !a.partial) return MST_ERR_INVALID_ARG;
+  MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+  const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
+  const int grid = (int)(works < sm_count() ? works : sm_count());
+  tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, P);
+  MST_CUDA_TRY(cudaGetLastError());
+  if (P.splits > 1) {
+    const int64_t n = a.epilogue == MST_TC_OUT_F32 ? a.M * a.N : a.nnz;
+    if (n > 0) tc_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(a.partial, P.splits, n, (float*)a.out);
+    MST_CUDA_TRY(cudaGetLastError());
+  }
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_device_error_flags(int32_t* flags) {
+  if (!flags) return MST_ERR_INVALID_ARG;
+  int v = 0;
+  MST_CUDA_TRY(cudaDeviceSynchronize());
+  MST_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)));
+  *flags = v;
+  return MST_OK;
+}

@@ -41,3 +41,10 @@ struct mst_tc_gemm_args {
 // not 16-byte aligned); the caller then falls back to the CUDA-core kernel.
 mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s);
 bool mst_tc_gemm_usable(const void* A, int64_t lda, const void* B, int64_t ldb);
+
+// How many K ranges to cut a contraction into so that `tiles` output tiles fill the GPU in one wave.
+int mst_tc_pick_splits(int64_t tiles, int64_t kblocks);
+
+// Process-wide scratch buffer for handle-less entry points (grows on demand; growing synchronises the device).
+// Calls that use it must not overlap on the GPU.
+mst_status_t mst_workspace(size_t bytes, void** ptr);

@@ -239,3 +239,20 @@ def test_error_statuses():
             mst.mst_topology_update(L.handle, 0.3, -1, 0.25, 0, 0, False, G)
         assert e.value.status == 6
     L.close()
+
+
+# ------------------------------------------------------- tensor-core dense gradient
+@pytest.mark.parametrize("O,I,T", [(300, 520, 1000), (512, 512, 4096), (128, 256, 64), (136, 264, 72), (1024, 768, 2048)])
+def test_dense_grad_tensor_core_path(O, I, T):
+    # bf16 with 16-byte-aligned rows takes the tcgen05 contraction: several tiles, ragged tails in M, N and K,
+    # token-range splitting with the fixed-order reduction
+    p = _problem(O, I, T, "bf16", 0.1, 4000 + O + I + T)
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    G = torch.full((O, I), float("nan"), dtype=torch.float32, device=dev())
+    mst.mst_dense_grad(dY, O, X, I, T, O, I, mst.MST_BF16, G)
+    G2 = torch.full((O, I), float("nan"), dtype=torch.float32, device=dev())
+    mst.mst_dense_grad(dY, O, X, I, T, O, I, mst.MST_BF16, G2)
+    assert mst.mst_device_error_flags() == 0
+    Gr = oracle.dense_grad(p.dY, p.X)
+    assert rel_err(host(G), Gr) <= 1e-5          # exact bf16 products, fp32 accumulation
+    np.testing.assert_array_equal(host(G).view(np.uint32), host(G2).view(np.uint32))     # deterministic
