@@ -72,6 +72,18 @@ mst_status_t mst_layer_create(mst_layer_t** layer, int32_t layer_id, int32_t out
                               mst_dtype_t dtype, int64_t nnz_capacity);
 mst_status_t mst_layer_destroy(mst_layer_t* layer);
 
+/* Which kernels serve forward, input gradient and weight gradient of a bf16 layer:
+ *   MST_PATH_CUDA_CORE    the sparse kernels (work proportional to nnz, fp32 FMA pipe)
+ *   MST_PATH_TENSOR_CORE  dense-tile kernels: W.M is expanded on the fly to a dense bf16 image and contracted on the
+ *                         tensor cores (work proportional to O*I, about 18x the FMA pipe's rate); the weight gradient
+ *                         is the dense contraction sampled on the mask in its epilogue.  Needs 16-byte-aligned rows
+ *                         (leading dimensions multiple of 8), otherwise the CUDA-core kernels are used.
+ *   MST_PATH_AUTO         (default) tensor cores at density >= 0.04, CUDA cores below.
+ * fp32 layers always use the CUDA-core kernels.  Results of the two paths agree within the stated tolerance, not
+ * bit for bit (different summation order). */
+typedef enum { MST_PATH_AUTO = 0, MST_PATH_CUDA_CORE = 1, MST_PATH_TENSOR_CORE = 2 } mst_compute_path_t;
+mst_status_t mst_set_compute_path(mst_layer_t* layer, mst_compute_path_t path);
+
 /* Number of active entries (host value; known after mst_pack / mst_topology_update without a sync). */
 mst_status_t mst_layer_nnz(const mst_layer_t* layer, int64_t* nnz);
 

@@ -18,11 +18,12 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmst.so")
 
 MST_F32, MST_BF16 = 0, 1
+MST_PATH_AUTO, MST_PATH_CUDA_CORE, MST_PATH_TENSOR_CORE = 0, 1, 2
 MST_OK = 0
 STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "MST_ERR_DTYPE", 4: "MST_ERR_CAPACITY",
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
                 9: "MST_ERR_NOT_PACKED"}
-EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
+EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_status_string"]
@@ -54,6 +55,7 @@ _sig = {
     "mst_layer_create": [ctypes.POINTER(_vp), _i32, _i32, _i32, ctypes.c_int, _i64],
     "mst_layer_destroy": [_vp],
     "mst_layer_nnz": [_vp, ctypes.POINTER(_i64)],
+    "mst_set_compute_path": [_vp, ctypes.c_int],
     "mst_pack": [_vp, _vp, _i64, _vp, _vp],
     "mst_export_csr": [_vp, _vp, _vp, _vp, _vp],
     "mst_export_csc": [_vp, _vp, _vp, _vp, _vp],
@@ -117,6 +119,10 @@ def mst_layer_create(layer_id: int, out_features: int, in_features: int, dtype: 
 
 def mst_layer_destroy(layer: int) -> None:
     _check(_lib.mst_layer_destroy(layer), "mst_layer_destroy")
+
+
+def mst_set_compute_path(layer: int, path: int) -> None:
+    _check(_lib.mst_set_compute_path(layer, path), "mst_set_compute_path")
 
 
 def mst_layer_nnz(layer: int) -> int:
@@ -226,6 +232,9 @@ class Layer:
             self.close()
         except Exception:
             pass
+
+    def set_path(self, path: int) -> None:
+        mst_set_compute_path(self.handle, path)
 
     @property
     def nnz(self) -> int:

@@ -92,6 +92,8 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   const size_t o_sel = cv.take(sizeof(mst_select_state));
   const size_t o_flags = cv.take(4 * 4);
   const size_t o_counter = cv.take(4);
+  const size_t o_dense = dtype == MST_BF16 ? cv.take(2 * (size_t)N) : 0;
+  const size_t o_denseT = dtype == MST_BF16 ? cv.take(2 * (size_t)N) : 0;
 
   unsigned char* base = nullptr;
   if (cudaMalloc((void**)&base, cv.off) != cudaSuccess) {
@@ -125,6 +127,9 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->sel = (mst_select_state*)(base + o_sel);
   L->flags = (int32_t*)(base + o_flags);
   L->counter = (unsigned int*)(base + o_counter);
+  L->dense_w = dtype == MST_BF16 ? (uint16_t*)(base + o_dense) : nullptr;
+  L->dense_wt = dtype == MST_BF16 ? (uint16_t*)(base + o_denseT) : nullptr;
+  L->path = MST_PATH_AUTO;
   L->stg_x = L->stg_dy = L->stg_y = L->stg_dx = nullptr;
   L->stg_dw = nullptr;
   L->stg_tokens = 0;
@@ -138,6 +143,21 @@ extern "C" mst_status_t mst_layer_destroy(mst_layer_t* L) {
   cudaFree(L->bits[0]);  // base of the single allocation
   delete L;
   return MST_OK;
+}
+
+extern "C" mst_status_t mst_set_compute_path(mst_layer_t* L, mst_compute_path_t path) {
+  if (!L || path < MST_PATH_AUTO || path > MST_PATH_TENSOR_CORE) return MST_ERR_INVALID_ARG;
+  L->path = path;
+  return MST_OK;
+}
+
+// Density above which the dense-tile tensor-core kernels beat the CUDA-core sparse kernels on B200 (measured).
+static const double kTensorPathMinDensity = 0.04;
+
+bool mst_use_tensor_path(const mst_layer* L) {
+  if (L->dtype != MST_BF16 || L->path == MST_PATH_CUDA_CORE) return false;
+  if (L->path == MST_PATH_TENSOR_CORE) return true;
+  return (double)L->nnz >= kTensorPathMinDensity * (double)L->N;
 }
 
 extern "C" mst_status_t mst_layer_nnz(const mst_layer_t* L, int64_t* nnz) {

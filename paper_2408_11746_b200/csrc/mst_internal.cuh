@@ -65,6 +65,11 @@ struct mst_layer {
   int32_t* flags;         // [4]: error bits, max row nnz, spare
   unsigned int* counter;  // [1] block-completion counter
 
+  // dense bf16 images of W.M for the tensor-core path (bf16 layers only): [O x I] and its transpose [I x O]
+  uint16_t* dense_w;
+  uint16_t* dense_wt;
+  int path;  // mst_compute_path_t
+
   // host staging for mst_layer_step_host
   void *stg_x, *stg_dy, *stg_y, *stg_dx;
   float* stg_dw;
@@ -79,6 +84,8 @@ int64_t mst_scan_block_sums_len(int64_t n);
 mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set, cudaStream_t s);
 mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s);
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
+mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s);
+bool mst_use_tensor_path(const mst_layer* L);
 
 // kernels' launchers
 mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in, int64_t ldin, int64_t T, void* out,

@@ -9,6 +9,7 @@
 // operands of a row stay in registers while consecutive entries share the row.  Every entry is owned by exactly one
 // warp and one lane, the token order is fixed: no atomics, deterministic.
 #include "mst_internal.cuh"
+#include "mst_tc_gemm.cuh"
 
 namespace {
 
@@ -190,6 +191,26 @@ mst_status_t mst_launch_sddmm(const mst_layer* L, const void* dY, int64_t lddy, 
   if (T == 0) {
     MST_CUDA_TRY(cudaMemsetAsync(dW, 0, sizeof(float) * L->nnz, s));
     return MST_OK;
+  }
+  // Tensor-core path: the dense contraction dY^T X with an epilogue that keeps only the entries under the mask and
+  // writes them to their CSR positions; the token range is split when the output has few tiles.
+  if (mst_use_tensor_path(L) && mst_tc_gemm_usable(dY, lddy, X, ldx)) {
+    const int c = L->cur;
+    mst_tc_gemm_args a = {};
+    a.A = dY; a.lda = lddy; a.a_mn_major = 1;
+    a.B = X; a.ldb = ldx; a.b_mn_major = 1;
+    a.M = L->O; a.N = L->I; a.K = T;
+    a.epilogue = MST_TC_OUT_SAMPLED;
+    a.out = dW;
+    a.bits = L->bits[c]; a.wscan = L->wscan[c]; a.wpr = L->wpr; a.nnz = L->nnz;
+    const int64_t tiles = ((int64_t)(L->O + 127) / 128) * ((L->I + 255) / 256);
+    a.splits = mst_tc_pick_splits(tiles, (T + 63) / 64);
+    if (a.splits > 1) {
+      void* ws = nullptr;
+      MST_TRY(mst_workspace(sizeof(float) * (size_t)a.splits * L->nnz, &ws));
+      a.partial = (float*)ws;
+    }
+    return mst_tc_gemm(a, s);
   }
   if (L->dtype == MST_F32) return launch<float>(L, dY, lddy, X, ldx, T, dW, s);
   return launch<uint16_t>(L, dY, lddy, X, ldx, T, dW, s);

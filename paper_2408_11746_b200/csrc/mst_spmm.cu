@@ -11,6 +11,7 @@
 // loaded 32 at a time, coalesced, and broadcast with shuffles.  Accumulation is fp32 in registers; the output tile
 // goes through shared memory so that global stores are contiguous along the feature dimension.
 #include "mst_internal.cuh"
+#include "mst_tc_gemm.cuh"
 
 namespace {
 
@@ -196,6 +197,21 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
                              int64_t ldout, cudaStream_t s) {
   if (T == 0) return MST_OK;
   const int c = L->cur;
+  // Dense-tile tensor-core path: expand W.M (or its transpose) to a dense bf16 image, then out = in * image^T.
+  if (mst_use_tensor_path(L) && (ldout % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0)) {
+    const uint16_t* image = transpose ? L->dense_wt : L->dense_w;
+    const int rows = transpose ? L->I : L->O, cols = transpose ? L->O : L->I;
+    if (mst_tc_gemm_usable(in, ldin, image, cols)) {
+      MST_TRY(mst_densify(L, transpose, s));
+      mst_tc_gemm_args a = {};
+      a.A = in; a.lda = ldin; a.a_mn_major = 0;
+      a.B = image; a.ldb = cols; a.b_mn_major = 0;
+      a.M = T; a.N = rows; a.K = cols;
+      a.epilogue = MST_TC_OUT_BF16;
+      a.out = out; a.ldc = ldout; a.splits = 1;
+      return mst_tc_gemm(a, s);
+    }
+  }
   if (!transpose) {
     if (L->dtype == MST_F32)
       return launch<float, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, out, ldout, T, L->O, L->I, s);

@@ -226,6 +226,25 @@ __global__ void fill_csc(const uint32_t* __restrict__ bitsT, const int32_t* __re
   }
 }
 
+// ---- dense bf16 image of W.M (or its transpose) for the tensor-core path: one warp per mask word ------------------
+// Writes every element (value or +0), so no separate clear is needed; stores are contiguous along the row.
+__global__ void densify_from_bits(const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan, int R, int C,
+                                  int wpr, const uint16_t* __restrict__ vals, const int32_t* __restrict__ perm,
+                                  uint16_t* __restrict__ dense) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= (int64_t)R * wpr) return;
+  const int r = (int)(w / wpr), c = (int)(w % wpr) * 32 + lane;
+  if (c >= C) return;
+  const uint32_t b = bits[w];
+  uint16_t v = 0;
+  if ((b >> lane) & 1u) {
+    const int32_t pos = wscan[w] + __popc(b & lanemask_lt());
+    v = vals[perm ? perm[pos] : pos];
+  }
+  dense[(int64_t)r * C + c] = v;
+}
+
 // ---- export / validate ---------------------------------------------------------------------------
 __global__ void widen_u16(const uint16_t* __restrict__ in, int64_t n, int32_t* __restrict__ out) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -330,6 +349,18 @@ mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s) {
   MST_TRY(mst_scan_i32(L->word_cnt, L->wscanT, L->nwordsT, L->block_sums, s));
   fill_csc<<<blocks_for(L->nwordsT * 32, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->O, L->I, L->wpr, L->wpc, L->bits[c],
                                                             L->wscan[c], L->row_idx, L->perm, L->col_ptr);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s) {
+  const int c = L->cur;
+  if (!transpose)
+    densify_from_bits<<<blocks_for(L->nwords * 32, 256), 256, 0, s>>>(L->bits[c], L->wscan[c], L->O, L->I, L->wpr,
+                                                                      (const uint16_t*)L->vals[c], nullptr, L->dense_w);
+  else
+    densify_from_bits<<<blocks_for(L->nwordsT * 32, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->I, L->O, L->wpc,
+                                                                       (const uint16_t*)L->vals[c], L->perm, L->dense_wt);
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

@@ -89,19 +89,25 @@ def _run_products(p, L, ldx=None, ldy=None):
     (200, 96, 64, "bf16", 0.0, "uniform", 0),        # empty mask
     (768, 768, 512, "bf16", 0.06, "zipf", 0),        # skewed rows: some full, many empty
     (3, 5, 7, "f32", 0.6, "uniform", 0),
-    (70, 1100, 260, "bf16", 0.15, "uniform", 0)])
+    (70, 1100, 260, "bf16", 0.15, "uniform", 0),
+    (520, 328, 900, "bf16", 0.1, "uniform", 0),      # three N tiles / two K-tail blocks on the tensor-core path
+    (1024, 768, 1024, "bf16", 0.05, "zipf", 0)])
 def test_products_match_oracle(O, I, T, dtype, density, kind, pad):
     p = _problem(O, I, T, dtype, density, 1000 + O + I + T, kind)
     L = make_layer(p)
-    Y, dX, dW, G = _run_products(p, L, I + pad if pad else None, O + pad if pad else None)
     tol = TOL[dtype]
     Wm = np.where(p.mask == 1, p.W, np.float32(0))
-    assert rel_err(Y, oracle.fwd(p.X, Wm, p.mask)) <= tol
-    assert rel_err(dX, oracle.bwd_x(p.dY, Wm, p.mask)) <= tol
-    Gr = oracle.dense_grad(p.dY, p.X)
+    Yr, dXr, Gr = oracle.fwd(p.X, Wm, p.mask), oracle.bwd_x(p.dY, Wm, p.mask), oracle.dense_grad(p.dY, p.X)
     rows, cols = np.nonzero(p.mask)
-    assert rel_err(dW, Gr[rows, cols]) <= tol
-    assert rel_err(G, Gr) <= tol
+    # both kernel families: the sparse CUDA-core kernels and the dense-tile tensor-core kernels
+    for path in (mst.MST_PATH_CUDA_CORE, mst.MST_PATH_TENSOR_CORE):
+        L.set_path(path)
+        Y, dX, dW, G = _run_products(p, L, I + pad if pad else None, O + pad if pad else None)
+        assert rel_err(Y, Yr) <= tol, path
+        assert rel_err(dX, dXr) <= tol, path
+        assert rel_err(dW, Gr[rows, cols]) <= tol, path
+        assert rel_err(G, Gr) <= tol, path
+    assert mst.mst_device_error_flags() == 0
     L.close()
 
 
