@@ -26,6 +26,8 @@ struct mst_select_state {
   long long k;                // how many more entries to take among those matching the prefix
   unsigned long long tau;     // final threshold key
   long long rem;              // entries equal to tau to take, in index order
+  int need_rank;              // 1 when more entries equal tau than are taken (their index order then decides)
+  int pad;
 };
 
 struct mst_layer {
@@ -60,7 +62,7 @@ struct mst_layer {
   int32_t* word_cnt;      // [max(nwords, nwordsT)+1]
   int32_t* word_scan;     // [max(nwords, nwordsT)+1]
   int32_t* block_sums;    // scan partials
-  unsigned int* hist;     // [256]
+  unsigned int* hist;     // [2048]
   mst_select_state* sel;  // [1]
   int32_t* flags;         // [4]: error bits, max row nnz, spare
   unsigned int* counter;  // [1] block-completion counter
@@ -81,6 +83,9 @@ static inline size_t mst_elem_size(mst_dtype_t d) { return d == MST_F32 ? 4 : 2;
 // structure (mst_structure.cu)
 mst_status_t mst_scan_i32(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t s);
 int64_t mst_scan_block_sums_len(int64_t n);
+// same scan, but every block returns at once when *enabled (device memory) is 0
+mst_status_t mst_scan_i32_if(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, const int* enabled,
+                             cudaStream_t s);
 mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set, cudaStream_t s);
 mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s);
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);

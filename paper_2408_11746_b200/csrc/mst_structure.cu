@@ -35,8 +35,10 @@ __device__ int block_reduce_sum(int v, int* sh) {
   return r;  // valid in warp 0
 }
 
-__global__ void scan_tile_sums(const int32_t* __restrict__ in, int64_t n, int32_t* __restrict__ sums) {
+__global__ void scan_tile_sums(const int32_t* __restrict__ in, int64_t n, int32_t* __restrict__ sums,
+                               const int* __restrict__ enabled) {
   __shared__ int sh[32];
+  if (enabled && !*enabled) return;
   const int64_t base = (int64_t)blockIdx.x * SCAN_TILE;
   int v = 0;
   for (int j = 0; j < SCAN_ITEMS; ++j) {
@@ -48,9 +50,10 @@ __global__ void scan_tile_sums(const int32_t* __restrict__ in, int64_t n, int32_
 }
 
 // one block: in-place exclusive scan of the tile sums (m values)
-__global__ void scan_sums_inplace(int32_t* sums, int64_t m) {
+__global__ void scan_sums_inplace(int32_t* sums, int64_t m, const int* __restrict__ enabled) {
   __shared__ int sh[32];
   __shared__ int carry;
+  if (enabled && !*enabled) return;
   if (threadIdx.x == 0) carry = 0;
   __syncthreads();
   for (int64_t base = 0; base < m; base += blockDim.x) {
@@ -82,9 +85,10 @@ __global__ void scan_sums_inplace(int32_t* sums, int64_t m) {
 }
 
 __global__ void scan_tiles(const int32_t* __restrict__ in, int64_t n, const int32_t* __restrict__ sums,
-                           int32_t* __restrict__ out) {
+                           int32_t* __restrict__ out, const int* __restrict__ enabled) {
   // thread owns SCAN_ITEMS consecutive elements
   __shared__ int sh[32];
+  if (enabled && !*enabled) return;
   const int64_t base = (int64_t)blockIdx.x * SCAN_TILE + (int64_t)threadIdx.x * SCAN_ITEMS;
   int v[SCAN_ITEMS];
   int t = 0;
@@ -307,18 +311,23 @@ inline unsigned blocks_for(int64_t n, int per_block) { return (unsigned)((n + pe
 
 int64_t mst_scan_block_sums_len(int64_t n) { return (n + SCAN_TILE - 1) / SCAN_TILE + 1; }
 
-mst_status_t mst_scan_i32(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t s) {
+mst_status_t mst_scan_i32_if(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, const int* enabled,
+                             cudaStream_t s) {
   if (n <= 0) {
     scan_empty<<<1, 1, 0, s>>>(out);
     MST_CUDA_TRY(cudaGetLastError());
     return MST_OK;
   }
   const int64_t tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
-  scan_tile_sums<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums);
-  scan_sums_inplace<<<1, 1024, 0, s>>>(block_sums, tiles);
-  scan_tiles<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, out);
+  scan_tile_sums<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, enabled);
+  scan_sums_inplace<<<1, 1024, 0, s>>>(block_sums, tiles, enabled);
+  scan_tiles<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, out, enabled);
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
+}
+
+mst_status_t mst_scan_i32(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, cudaStream_t s) {
+  return mst_scan_i32_if(in, out, n, block_sums, nullptr, s);
 }
 
 // bits[set] must be final.  Computes wscan[set], row_ptr[set], col_idx[set], vals[set].

@@ -2,14 +2,15 @@
 //
 // The three selections of the algorithm (prune by smallest |w|, grow by largest |g|, grow at random) are the same
 // primitive: take the k smallest keys of a candidate set, ties broken by the smaller flat index.  Each is done by a
-// most-significant-digit radix select (8 bits per pass) that leaves a threshold key tau and the number `rem` of
+// most-significant-digit radix select (11 bits per pass) that leaves a threshold key tau and the number `rem` of
 // entries equal to tau still to take; a popcount + exclusive scan over the mask words then ranks the entries equal to
 // tau in flat-index order and the first `rem` of them are taken.  Results are bit masks over the flat index space, so
 // the mask rewrite is three bitwise operations per word and the CSR rebuild is the popcount/scan/fill of
 // mst_structure.cu.  Integer keys, integer atomics only: the outcome is deterministic and bit-exact.
 //
 // Work layout: one warp per 32-bit mask word, lane = column inside the word, so reads of G and of the value array are
-// coalesced.  The last block to finish a histogram pass picks the digit (completion counter, no waiting).
+// coalesced.  The last block to finish a histogram pass picks the digit (completion counter, no waiting).  The tie
+// ranking (count, scan) is skipped on the device when the threshold key has no surplus ties.
 #include "mst_internal.cuh"
 
 namespace {
@@ -84,27 +85,45 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
   }
 }
 
+constexpr int RADIX_BITS = 11;
+constexpr int BINS = 1 << RADIX_BITS;  // 2048
+constexpr int HIST_THREADS = 1024;
+constexpr int BINS_PER_THREAD = BINS / HIST_THREADS;
+
+__host__ __device__ constexpr int num_passes(int key_bits) { return (key_bits + RADIX_BITS - 1) / RADIX_BITS; }
+// digit `pass` (most significant first) covers key bits [pass_shift, pass_shift + pass_width)
+__host__ __device__ constexpr int pass_shift(int key_bits, int pass) {
+  return key_bits - RADIX_BITS * (pass + 1) > 0 ? key_bits - RADIX_BITS * (pass + 1) : 0;
+}
+__host__ __device__ constexpr int pass_width(int key_bits, int pass) {
+  return key_bits - RADIX_BITS * pass < RADIX_BITS ? key_bits - RADIX_BITS * pass : RADIX_BITS;
+}
+
 __global__ void select_init(mst_select_state* st, long long k, unsigned int* hist, unsigned int* counter) {
   if (threadIdx.x == 0) {
     st->prefix = 0;
     st->k = k;
     st->tau = 0;
     st->rem = 0;
+    st->need_rank = 0;
     *counter = 0;
   }
-  if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+  for (int b = threadIdx.x; b < BINS; b += blockDim.x) hist[b] = 0;
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(256) select_hist(SelParams P, int pass, mst_select_state* st, unsigned int* hist,
+__global__ void __launch_bounds__(HIST_THREADS) select_hist(SelParams P, int pass, mst_select_state* st, unsigned int* hist,
                                                    unsigned int* counter, int32_t* flags) {
   constexpr int KB = KeyBits<MODE>::value;
-  __shared__ unsigned int sh[256];
+  __shared__ unsigned int sh[BINS];
+  __shared__ unsigned int warp_tot[HIST_THREADS / 32];
   __shared__ bool is_last;
-  sh[threadIdx.x] = 0;
+  for (int b = threadIdx.x; b < BINS; b += HIST_THREADS) sh[b] = 0;
   __syncthreads();
   const unsigned long long prefix = st->prefix;
-  const int shift = KB - 8 * (pass + 1);
+  const int shift = pass_shift(KB, pass);
+  const unsigned dmask = (1u << pass_width(KB, pass)) - 1u;
+  const int hi_shift = shift + pass_width(KB, pass);  // bits above this digit
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   bool saw_nonfinite = false;
@@ -114,52 +133,73 @@ __global__ void __launch_bounds__(256) select_hist(SelParams P, int pass, mst_se
     const bool c = cand_key<MODE>(P, w, lane, key, nf);
     saw_nonfinite |= (c && nf);
     // entries whose higher digits differ from the prefix are out of the race
-    const bool live = c && (pass == 0 || (key >> (shift + 8)) == prefix);
-    const unsigned digit = live ? (unsigned)((key >> shift) & 0xFFu) : 256u;
+    const bool live = c && (pass == 0 || (key >> hi_shift) == prefix);
+    const unsigned digit = live ? (unsigned)((key >> shift) & dmask) : (unsigned)BINS;
     const unsigned peers = __match_any_sync(0xffffffffu, digit);
     if (live && lane == (__ffs(peers) - 1)) atomicAdd(&sh[digit], (unsigned)__popc(peers));
   }
   if (pass == 0 && saw_nonfinite) atomicOr(&flags[0], MST_FLAG_NONFINITE);
   __syncthreads();
-  if (sh[threadIdx.x]) atomicAdd(&hist[threadIdx.x], sh[threadIdx.x]);
+  for (int b = threadIdx.x; b < BINS; b += HIST_THREADS)
+    if (sh[b]) atomicAdd(&hist[b], sh[b]);
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) is_last = (atomicAdd(counter, 1u) == gridDim.x - 1);
   __syncthreads();
   if (!is_last) return;
-  // last block: every other block's histogram contribution is visible
+  // last block to finish: every other block's contribution is visible; pick the digit that holds the k-th key
   __threadfence();
-  sh[threadIdx.x] = atomicAdd(&hist[threadIdx.x], 0u);
+  unsigned int mine[BINS_PER_THREAD];
+  unsigned int tsum = 0;
+#pragma unroll
+  for (int j = 0; j < BINS_PER_THREAD; ++j) {
+    const int b = threadIdx.x * BINS_PER_THREAD + j;
+    mine[j] = atomicAdd(&hist[b], 0u);
+    hist[b] = 0;  // ready for the next pass
+    tsum += mine[j];
+  }
+  // exclusive prefix of the per-thread sums over the block
+  unsigned int incl = tsum;
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) warp_tot[threadIdx.x >> 5] = incl;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    long long k = st->k, cum = 0;
-    int bin = -1;
-    for (int b = 0; b < 256; ++b) {
-      if (cum + (long long)sh[b] >= k) { bin = b; break; }
-      cum += sh[b];
+  unsigned int before = incl - tsum;
+  for (int wv = 0; wv < (int)(threadIdx.x >> 5); ++wv) before += warp_tot[wv];
+  const long long k = st->k;
+  __syncthreads();  // everyone has read st->k before the owner rewrites it
+  const bool owner = (long long)before < k && k <= (long long)before + (long long)tsum;
+  if (owner) {
+    long long cum = before;
+    int bin = 0;
+#pragma unroll
+    for (int j = 0; j < BINS_PER_THREAD; ++j) {
+      if (cum + (long long)mine[j] >= k) { bin = j; break; }
+      cum += mine[j];
     }
-    if (bin < 0) {  // fewer candidates than requested: the host-side counts rule this out
-      atomicOr(&flags[0], MST_FLAG_CORRUPT);
-      bin = 255;
-      cum = 0;
-      k = 0;
-    }
-    const unsigned long long np = (prefix << 8) | (unsigned long long)bin;
+    const unsigned long long np = (prefix << pass_width(KB, pass)) | (unsigned long long)(threadIdx.x * BINS_PER_THREAD + bin);
     st->prefix = np;
     st->k = k - cum;
     if (shift == 0) {
       st->tau = np;
       st->rem = k - cum;
+      st->need_rank = ((long long)mine[bin] > k - cum) ? 1 : 0;  // ties at the threshold beyond what is taken
     }
+  }
+  if (threadIdx.x == HIST_THREADS - 1) {
+    const long long total = (long long)before + (long long)tsum;
+    if (total < k) atomicOr(&flags[0], MST_FLAG_CORRUPT);  // fewer candidates than requested: ruled out by the host counts
     *counter = 0;
   }
-  hist[threadIdx.x] = 0;
 }
 
-// cnt[w] = number of candidates in word w whose key equals tau
+// cnt[w] = number of candidates in word w whose key equals tau (skipped when no tie has to be ranked)
 template <int MODE>
 __global__ void __launch_bounds__(256) select_count_equal(SelParams P, const mst_select_state* st,
                                                           int32_t* __restrict__ cnt) {
+  if (!st->need_rank) return;
   const unsigned long long tau = st->tau;
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -176,6 +216,7 @@ __global__ void __launch_bounds__(256) select_mark(SelParams P, const mst_select
                                                    const int32_t* __restrict__ eq_scan, uint32_t* __restrict__ out) {
   const unsigned long long tau = st->tau;
   const long long rem = st->rem;
+  const bool need_rank = st->need_rank != 0;
   const int lane = threadIdx.x & 31;
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (w >= P.nwords) return;
@@ -184,7 +225,8 @@ __global__ void __launch_bounds__(256) select_mark(SelParams P, const mst_select
   const bool c = cand_key<MODE>(P, w, lane, key, nf);
   const bool iseq = c && key == tau;
   const unsigned eq = __ballot_sync(0xffffffffu, iseq);
-  const long long rank = (long long)eq_scan[w] + __popc(eq & lanemask_lt());
+  // without ties beyond the quota every entry equal to tau is taken; otherwise the first `rem` in index order
+  const long long rank = need_rank ? (long long)eq_scan[w] + __popc(eq & lanemask_lt()) : -1;
   const bool take = c && (key < tau || (iseq && rank < rem));
   const unsigned bits = __ballot_sync(0xffffffffu, take);
   if (lane == 0) out[w] = bits;
@@ -201,16 +243,15 @@ mst_status_t run_select(mst_layer* L, const SelParams& P, int64_t k, uint32_t* o
     MST_CUDA_TRY(cudaMemsetAsync(out_bits, 0, sizeof(uint32_t) * L->nwords, s));
     return MST_OK;
   }
-  constexpr int passes = KeyBits<MODE>::value / 8;
+  constexpr int passes = num_passes(KeyBits<MODE>::value);
   select_init<<<1, 256, 0, s>>>(L->sel, (long long)k, L->hist, L->counter);
-  const int64_t warps_needed = L->nwords;
-  int64_t blocks = (warps_needed * 32 + 255) / 256;
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  int64_t blocks = (L->nwords * 32 + HIST_THREADS - 1) / HIST_THREADS;
+  if (blocks > 74) blocks = 74;  // few blocks: each ends with one global add per non-empty bin
   for (int p = 0; p < passes; ++p)
-    select_hist<MODE><<<(unsigned)blocks, 256, 0, s>>>(P, p, L->sel, L->hist, L->counter, L->flags);
+    select_hist<MODE><<<(unsigned)blocks, HIST_THREADS, 0, s>>>(P, p, L->sel, L->hist, L->counter, L->flags);
   const unsigned wgrid = (unsigned)((L->nwords * 32 + 255) / 256);
   select_count_equal<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_cnt);
-  MST_TRY(mst_scan_i32(L->word_cnt, L->word_scan, L->nwords, L->block_sums, s));
+  MST_TRY(mst_scan_i32_if(L->word_cnt, L->word_scan, L->nwords, L->block_sums, &L->sel->need_rank, s));
   select_mark<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_scan, out_bits);
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
