@@ -27,7 +27,7 @@ struct mst_select_state {
   unsigned long long tau;     // final threshold key
   long long rem;              // entries equal to tau to take, in index order
   int need_rank;              // 1 when more entries equal tau than are taken (their index order then decides)
-  int pad;
+  int pad;                    // "done": set when an early pass already fixed the threshold (later passes return at once)
 };
 
 struct mst_layer {

@@ -53,7 +53,8 @@ struct KeyBits {
 template <int MODE>
 __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane, unsigned long long& key,
                                          bool& nonfinite) {
-  const int o = (int)(w / P.wpr), c = (int)(w % P.wpr) * 32 + lane;
+  const unsigned wu = (unsigned)w, wpr = (unsigned)P.wpr;   // nwords < 2^31
+  const int o = (int)(wu / wpr), c = (int)(wu - (unsigned)o * wpr) * 32 + lane;
   nonfinite = false;
   key = 0;
   if (MODE == MODE_PRUNE) {
@@ -106,6 +107,7 @@ __global__ void select_init(mst_select_state* st, long long k, unsigned int* his
     st->tau = 0;
     st->rem = 0;
     st->need_rank = 0;
+    st->pad = 0;   // 'done' flag: later passes return at once
     *counter = 0;
   }
   for (int b = threadIdx.x; b < BINS; b += blockDim.x) hist[b] = 0;
@@ -118,6 +120,7 @@ __global__ void __launch_bounds__(HIST_THREADS) select_hist(SelParams P, int pas
   __shared__ unsigned int sh[BINS];
   __shared__ unsigned int warp_tot[HIST_THREADS / 32];
   __shared__ bool is_last;
+  if (st->pad) return;  // an earlier pass already fixed the threshold
   for (int b = threadIdx.x; b < BINS; b += HIST_THREADS) sh[b] = 0;
   __syncthreads();
   const unsigned long long prefix = st->prefix;
@@ -127,16 +130,27 @@ __global__ void __launch_bounds__(HIST_THREADS) select_hist(SelParams P, int pas
   const int lane = threadIdx.x & 31;
   const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   bool saw_nonfinite = false;
-  for (int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < P.nwords; w += warps) {
-    unsigned long long key;
-    bool nf;
-    const bool c = cand_key<MODE>(P, w, lane, key, nf);
-    saw_nonfinite |= (c && nf);
-    // entries whose higher digits differ from the prefix are out of the race
-    const bool live = c && (pass == 0 || (key >> hi_shift) == prefix);
-    const unsigned digit = live ? (unsigned)((key >> shift) & dmask) : (unsigned)BINS;
-    const unsigned peers = __match_any_sync(0xffffffffu, digit);
-    if (live && lane == (__ffs(peers) - 1)) atomicAdd(&sh[digit], (unsigned)__popc(peers));
+  // four words per trip so that their dependent loads (mask word -> position -> value) overlap
+  constexpr int BATCH = 4;
+  for (int64_t w0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w0 < P.nwords; w0 += warps * BATCH) {
+    unsigned digit[BATCH];
+    bool live[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const int64_t w = w0 + (int64_t)j * warps;
+      unsigned long long key = 0;
+      bool nf = false;
+      const bool c = w < P.nwords && cand_key<MODE>(P, w, lane, key, nf);
+      saw_nonfinite |= (c && nf);
+      // entries whose higher digits differ from the prefix are out of the race
+      live[j] = c && (pass == 0 || (key >> hi_shift) == prefix);
+      digit[j] = live[j] ? (unsigned)((key >> shift) & dmask) : (unsigned)BINS;
+    }
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const unsigned peers = __match_any_sync(0xffffffffu, digit[j]);
+      if (live[j] && lane == (__ffs(peers) - 1)) atomicAdd(&sh[digit[j]], (unsigned)__popc(peers));
+    }
   }
   if (pass == 0 && saw_nonfinite) atomicOr(&flags[0], MST_FLAG_NONFINITE);
   __syncthreads();
@@ -186,6 +200,12 @@ __global__ void __launch_bounds__(HIST_THREADS) select_hist(SelParams P, int pas
       st->tau = np;
       st->rem = k - cum;
       st->need_rank = ((long long)mine[bin] > k - cum) ? 1 : 0;  // ties at the threshold beyond what is taken
+    } else if ((long long)mine[bin] == k - cum) {
+      // every key that shares this prefix is taken: the lower digits cannot matter, stop here
+      st->tau = (np << shift) | ((1ULL << shift) - 1ULL);
+      st->rem = k - cum;
+      st->need_rank = 0;
+      st->pad = 1;
     }
   }
   if (threadIdx.x == HIST_THREADS - 1) {
@@ -246,7 +266,7 @@ mst_status_t run_select(mst_layer* L, const SelParams& P, int64_t k, uint32_t* o
   constexpr int passes = num_passes(KeyBits<MODE>::value);
   select_init<<<1, 256, 0, s>>>(L->sel, (long long)k, L->hist, L->counter);
   int64_t blocks = (L->nwords * 32 + HIST_THREADS - 1) / HIST_THREADS;
-  if (blocks > 74) blocks = 74;  // few blocks: each ends with one global add per non-empty bin
+  if (blocks > 2 * 148) blocks = 2 * 148;  // all SMs fully occupied; each block ends with one global add per non-empty bin
   for (int p = 0; p < passes; ++p)
     select_hist<MODE><<<(unsigned)blocks, HIST_THREADS, 0, s>>>(P, p, L->sel, L->hist, L->counter, L->flags);
   const unsigned wgrid = (unsigned)((L->nwords * 32 + 255) / 256);
