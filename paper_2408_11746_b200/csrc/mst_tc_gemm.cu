@@ -18,6 +18,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "mst_internal.cuh"
 
 namespace {
@@ -139,6 +141,66 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// One 128 x BN accumulator (tensor-memory lanes = rows) -> global memory, 32 columns at a time.
+// q = lane quarter this warp may read, m0/n0 = first row / column of this block's tile.
+__device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_base, int acc, int q, int lane, int64_t m0,
+                                              int n0, int split) {
+  const int64_t m = (int64_t)m0 + q * 32 + lane;
+  const bool row_ok = m < P.M;
+#pragma unroll 1
+  for (int c = 0; c < BN / 32; ++c) {
+    const int n = n0 + c * 32;
+    if (n >= P.N) break;  // uniform
+    uint32_t r[32];
+    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+    if (!row_ok) continue;
+    if (P.epilogue == MST_TC_OUT_BF16) {
+      uint16_t* dst = reinterpret_cast<uint16_t*>(P.out) + m * P.ldc + n;
+      if (n + 32 <= P.N && ((P.ldc & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.out) & 15u) == 0)) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint4 o;
+          o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+          o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+          o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+          o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+          reinterpret_cast<uint4*>(dst)[v] = o;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (n + j < P.N) dst[j] = (uint16_t)(pack_bf16(__uint_as_float(r[j]), 0.f) & 0xFFFFu);
+      }
+    } else if (P.epilogue == MST_TC_OUT_F32) {
+      float* base = P.splits > 1 ? P.partial + (int64_t)split * P.M * P.N + m * P.N : reinterpret_cast<float*>(P.out) + m * P.ldc;
+      float* dst = base + n;
+      const int64_t ld = P.splits > 1 ? P.N : P.ldc;
+      if (n + 32 <= P.N && ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(base) & 15u) == 0)) {
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+          reinterpret_cast<uint4*>(dst)[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (n + j < P.N) dst[j] = __uint_as_float(r[j]);
+      }
+    } else {
+      // sampled: the 32 columns of this chunk are one mask word of row m
+      const int64_t wi = m * P.wpr + (n >> 5);
+      const uint32_t word = P.bits[wi];
+      float* dst = (P.splits > 1 ? P.partial + (int64_t)split * P.nnz : reinterpret_cast<float*>(P.out)) + P.wscan[wi];
+      int rank = 0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if ((word >> j) & 1u) {
+          dst[rank] = __uint_as_float(r[j]);
+          ++rank;
+        }
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params P) {
@@ -253,60 +315,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = (t / P.n_tiles) * BM, n0 = (t % P.n_tiles) * BN;
       if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
       tc_fence_after();
-      const int64_t m = (int64_t)m0 + q * 32 + lane;
-      const bool row_ok = m < P.M;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int n = n0 + c * 32;
-        if (n >= P.N) break;  // uniform
-        uint32_t r[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
-        if (!row_ok) continue;
-        if (P.epilogue == MST_TC_OUT_BF16) {
-          uint16_t* dst = reinterpret_cast<uint16_t*>(P.out) + m * P.ldc + n;
-          if (n + 32 <= P.N && ((P.ldc & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.out) & 15u) == 0)) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint4 o;
-              o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
-              o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
-              o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
-              o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-              reinterpret_cast<uint4*>(dst)[v] = o;
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n + j < P.N) dst[j] = (uint16_t)(pack_bf16(__uint_as_float(r[j]), 0.f) & 0xFFFFu);
-          }
-        } else if (P.epilogue == MST_TC_OUT_F32) {
-          float* base = P.splits > 1 ? P.partial + (int64_t)split * P.M * P.N + m * P.N : reinterpret_cast<float*>(P.out) + m * P.ldc;
-          float* dst = base + n;
-          const int64_t ld = P.splits > 1 ? P.N : P.ldc;
-          if (n + 32 <= P.N && ((ld & 3) == 0) && ((reinterpret_cast<uintptr_t>(base) & 15u) == 0)) {
-#pragma unroll
-            for (int v = 0; v < 8; ++v)
-              reinterpret_cast<uint4*>(dst)[v] = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n + j < P.N) dst[j] = __uint_as_float(r[j]);
-          }
-        } else {
-          // sampled: the 32 columns of this chunk are one mask word of row m
-          const int64_t wi = m * P.wpr + (n >> 5);
-          const uint32_t word = P.bits[wi];
-          float* dst = (P.splits > 1 ? P.partial + (int64_t)split * P.nnz : reinterpret_cast<float*>(P.out)) + P.wscan[wi];
-          int rank = 0;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if ((word >> j) & 1u) {
-              dst[rank] = __uint_as_float(r[j]);
-              ++rank;
-            }
-          }
-        }
-      }
+      epilogue_tile(P, tmem_base, acc, q, lane, m0, n0, split);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
@@ -324,6 +333,199 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------------- CTA-pair kernel
+// Same roles, but two blocks of a cluster (an SM pair) share one 256 x 256 output tile: each block loads its own 128
+// rows of A and its own half (128 of 256 columns) of B, the even block issues tcgen05.mma.cta_group::2 (M = 256) that
+// reads both blocks' shared memory and writes both blocks' tensor memory.  Per block this halves the shared-memory
+// traffic for B, which is what bounds the single-block kernel.  Barrier protocol:
+//   full[s]   (even block)  two arrivals (one per block's producer, each announcing its own bytes) + TMA bytes of both
+//   empty[s]  (each block)  one arrival, multicast by the even block's tcgen05.commit
+//   tfull[a]  (each block)  one arrival, multicast by tcgen05.commit after the tile's last MMA
+//   tempty[a] (even block)  eight arrivals: the four epilogue warps of both blocks
+constexpr int P_STAGES = 6;
+constexpr int PB_BYTES = (BN / 2) * BK * 2;        // this block's half of B: 16 KiB
+constexpr int P_STAGE_BYTES = A_BYTES + PB_BYTES;  // 32 KiB
+constexpr size_t P_SMEM_BYTES = (size_t)P_STAGES * P_STAGE_BYTES + 1024 + 256;
+// shared::cluster address of the same shared-memory location in the even block (rank 0) of the pair
+__device__ __forceinline__ uint32_t in_even_block(uint32_t local_addr) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(0u));
+  return r;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(tm), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"((uint16_t)3)
+               : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params P) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  const uint32_t bar_base = tiles_base + P_STAGES * P_STAGE_BYTES;
+  const uint32_t full0 = bar_base, empty0 = bar_base + 8 * P_STAGES, tfull0 = bar_base + 16 * P_STAGES,
+                 tempty0 = tfull0 + 16;
+  __shared__ uint32_t tmem_base_holder;
+  __shared__ int abort_sh;
+  volatile int* abort_flag = &abort_sh;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = even block (issues the MMAs), 1 = its peer
+  if (threadIdx.x == 0) {
+    abort_sh = 0;
+    for (int s = 0; s < P_STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 2);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull0 + 8 * a, 1);
+      mbar_init(tempty0 + 8 * a, 8);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // both blocks' barriers are initialised before any remote arrival or copy completion
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_holder;
+
+  const int m_pairs = (P.m_tiles + 1) / 2;
+  const int tiles = m_pairs * P.n_tiles;
+  const int64_t works = (int64_t)tiles * P.splits;
+  const int64_t pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer (both blocks)
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      for (int64_t w = pair; w < works && !*abort_flag; w += npairs) {
+        const int split = (int)(w / tiles), t = (int)(w % tiles);
+        const int m0 = (t / P.n_tiles) * (2 * BM) + (int)rank * BM;       // this block's rows
+        const int n0 = (t % P.n_tiles) * BN + (int)rank * (BN / 2);       // this block's half of B
+        const int kb0 = (int)((int64_t)split * P.kblocks / P.splits), kb1 = (int)((int64_t)(split + 1) * P.kblocks / P.splits);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
+          const uint32_t fb = in_even_block(full0 + 8 * s);  // the even block's barrier collects both blocks' bytes
+          const uint32_t sa = tiles_base + s * P_STAGE_BYTES, sb = sa + A_BYTES;
+          mbar_expect_tx_cluster(fb, P_STAGE_BYTES);
+          if (P.a_mn) {
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(sa + j * BOX_BYTES, &tmA, m0 + j * 64, kb * BK, fb);
+          } else {
+            tma_load_2d_pair(sa, &tmA, kb * BK, m0, fb);
+          }
+          if (P.b_mn) {
+            for (int j = 0; j < BN / 128; ++j) tma_load_2d_pair(sb + j * BOX_BYTES, &tmB, n0 + j * 64, kb * BK, fb);
+          } else {
+            tma_load_2d_pair(sb, &tmB, kb * BK, n0, fb);
+          }
+          if (++s == P_STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (even block only)
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.a_mn ? 1 : 0) << 15) |
+                             ((uint32_t)(P.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) |
+                             ((uint32_t)((2 * BM) >> 4) << 24);
+      int s = 0, acc = 0;
+      uint32_t ph = 0, acc_ph = 0;
+      for (int64_t w = pair; w < works && !*abort_flag; w += npairs) {
+        const int split = (int)(w / tiles);
+        const int kb0 = (int)((int64_t)split * P.kblocks / P.splits), kb1 = (int)((int64_t)(split + 1) * P.kblocks / P.splits);
+        if (!mbar_wait(tempty0 + 8 * acc, acc_ph ^ 1u, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        bool ok = true;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + s * P_STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t ad = P.a_mn ? smem_desc(sa + k * (UMMA_K * 128), BOX_BYTES, 1024)
+                                       : smem_desc(sa + k * (UMMA_K * 2), 16, 1024);
+            const uint64_t bd = P.b_mn ? smem_desc(sb + k * (UMMA_K * 128), BOX_BYTES, 1024)
+                                       : smem_desc(sb + k * (UMMA_K * 2), 16, 1024);
+            tc_mma_pair(d_tmem, ad, bd, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit_pair(empty0 + 8 * s);  // frees this stage in both blocks
+          if (++s == P_STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull0 + 8 * acc);  // both blocks' halves of the accumulator are complete
+        if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (both blocks, own 128 rows)
+    const int q = warp & 3;
+    int acc = 0;
+    uint32_t acc_ph = 0;
+    for (int64_t w = pair; w < works; w += npairs) {
+      const int split = (int)(w / tiles), t = (int)(w % tiles);
+      const int m0 = (t / P.n_tiles) * (2 * BM) + (int)rank * BM, n0 = (t % P.n_tiles) * BN;
+      if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
+      tc_fence_after();
+      epilogue_tile(P, tmem_base, acc, q, lane, m0, n0, split);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(in_even_block(tempty0 + 8 * acc));
+      if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (*abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer may still be signalling this block's barriers or reading its shared memory
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
@@ -414,9 +616,13 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   if (a.M <= 0 || a.N <= 0 || a.K <= 0) return MST_ERR_INVALID_ARG;
   if (!mst_tc_gemm_usable(a.A, a.lda, a.B, a.ldb)) return MST_ERR_SHAPE;
   CUtensorMap tmA, tmB;
+  // Block pairs (256-row tiles) pay off once there are at least two row tiles; MST_TC_PAIR=0/1 overrides.
+  bool pair = a.M > BM;
+  if (const char* e = getenv("MST_TC_PAIR")) pair = (e[0] == '1');
   // K-major: [rows x K], box 64 (K) x tile rows.  MN-major: [K x rows], box 64 (rows) x BK.
   const bool okA = a.a_mn_major ? make_map(&tmA, a.A, a.K, a.M, a.lda, BK) : make_map(&tmA, a.A, a.M, a.K, a.lda, BM);
-  const bool okB = a.b_mn_major ? make_map(&tmB, a.B, a.K, a.N, a.ldb, BK) : make_map(&tmB, a.B, a.N, a.K, a.ldb, BN);
+  const int b_rows = pair ? BN / 2 : BN;
+  const bool okB = a.b_mn_major ? make_map(&tmB, a.B, a.K, a.N, a.ldb, BK) : make_map(&tmB, a.B, a.N, a.K, a.ldb, b_rows);
   if (!okA || !okB) return MST_ERR_SHAPE;
   Params P;
   P.M = a.M;
@@ -438,10 +644,18 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   P.wpr = a.wpr;
   P.nnz = a.nnz;
   if (P.splits > 1 && !a.partial) return MST_ERR_INVALID_ARG;
-  MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
-  const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
-  const int grid = (int)(works < sm_count() ? works : sm_count());
-  tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, P);
+  if (pair) {
+    MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES));
+    const int64_t works = (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles * P.splits;
+    const int64_t max_pairs = sm_count() / 2;
+    const int grid = 2 * (int)(works < max_pairs ? works : max_pairs);
+    tc_gemm_pair_kernel<<<grid, NUM_THREADS, P_SMEM_BYTES, s>>>(tmA, tmB, P);
+  } else {
+    MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
+    const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
+    const int grid = (int)(works < sm_count() ? works : sm_count());
+    tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, P);
+  }
   MST_CUDA_TRY(cudaGetLastError());
   if (P.splits > 1) {
     const int64_t n = a.epilogue == MST_TC_OUT_F32 ? a.M * a.N : a.nnz;
