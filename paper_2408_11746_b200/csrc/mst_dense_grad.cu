@@ -83,13 +83,7 @@ extern "C" mst_status_t mst_dense_grad(const void* dY, int64_t lddy, const void*
     a.M = out_features; a.N = in_features; a.K = T;
     a.epilogue = MST_TC_OUT_F32;
     a.out = G; a.ldc = in_features;
-    const int64_t tiles = ((int64_t)(out_features + 127) / 128) * ((in_features + 255) / 256);
-    a.splits = mst_tc_pick_splits(tiles, (T + 63) / 64);
-    if (a.splits > 1) {
-      void* ws = nullptr;
-      MST_TRY(mst_workspace(sizeof(float) * (size_t)a.splits * out_features * in_features, &ws));
-      a.partial = (float*)ws;
-    }
+    a.splits = 0;
     return mst_tc_gemm(a, s);
   }
   dim3 grid((unsigned)((in_features + TN - 1) / TN), (unsigned)((out_features + TM - 1) / TM));

@@ -203,13 +203,7 @@ mst_status_t mst_launch_sddmm(const mst_layer* L, const void* dY, int64_t lddy, 
     a.epilogue = MST_TC_OUT_SAMPLED;
     a.out = dW;
     a.bits = L->bits[c]; a.wscan = L->wscan[c]; a.wpr = L->wpr; a.nnz = L->nnz;
-    const int64_t tiles = ((int64_t)(L->O + 127) / 128) * ((L->I + 255) / 256);
-    a.splits = mst_tc_pick_splits(tiles, (T + 63) / 64);
-    if (a.splits > 1) {
-      void* ws = nullptr;
-      MST_TRY(mst_workspace(sizeof(float) * (size_t)a.splits * L->nnz, &ws));
-      a.partial = (float*)ws;
-    }
+    a.splits = 0;
     return mst_tc_gemm(a, s);
   }
   if (L->dtype == MST_F32) return launch<float>(L, dY, lddy, X, ldx, T, dW, s);

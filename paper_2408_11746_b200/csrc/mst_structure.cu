@@ -230,23 +230,38 @@ __global__ void fill_csc(const uint32_t* __restrict__ bitsT, const int32_t* __re
   }
 }
 
-// ---- dense bf16 image of W.M (or its transpose) for the tensor-core path: one warp per mask word ------------------
-// Writes every element (value or +0), so no separate clear is needed; stores are contiguous along the row.
+// ---- dense bf16 image of W.M (or its transpose) for the tensor-core path ----------------------------------------------
+// One thread per 8 consecutive columns: the stored values of those columns are consecutive in CSR (or CSC) order, so
+// the thread reads them in one run and writes one 16-byte vector (value or +0 per column).  Every element is written,
+// no separate clear.  Needs C % 8 == 0 (the tensor-core path requires it anyway).
 __global__ void densify_from_bits(const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan, int R, int C,
                                   int wpr, const uint16_t* __restrict__ vals, const int32_t* __restrict__ perm,
                                   uint16_t* __restrict__ dense) {
-  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  if (w >= (int64_t)R * wpr) return;
-  const int r = (int)(w / wpr), c = (int)(w % wpr) * 32 + lane;
-  if (c >= C) return;
-  const uint32_t b = bits[w];
-  uint16_t v = 0;
-  if ((b >> lane) & 1u) {
-    const int32_t pos = wscan[w] + __popc(b & lanemask_lt());
-    v = vals[perm ? perm[pos] : pos];
+  const unsigned g = blockIdx.x * blockDim.x + threadIdx.x;  // group of 8 columns
+  const unsigned gpr = (unsigned)C >> 3;                     // groups per row
+  if (g >= (unsigned)R * gpr) return;
+  const unsigned r = g / gpr, c8 = g - r * gpr;
+  const unsigned w = r * (unsigned)wpr + (c8 >> 2);
+  const uint32_t word = bits[w];
+  const unsigned sh = (c8 & 3u) * 8u;
+  uint32_t m = (word >> sh) & 0xFFu;
+  uint16_t out[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (m) {
+    int32_t pos = wscan[w] + __popc(word & ((1u << sh) - 1u));
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      if ((m >> j) & 1u) {
+        out[j] = vals[perm ? perm[pos] : pos];
+        ++pos;
+      }
+    }
   }
-  dense[(int64_t)r * C + c] = v;
+  uint4 v;
+  v.x = (uint32_t)out[0] | ((uint32_t)out[1] << 16);
+  v.y = (uint32_t)out[2] | ((uint32_t)out[3] << 16);
+  v.z = (uint32_t)out[4] | ((uint32_t)out[5] << 16);
+  v.w = (uint32_t)out[6] | ((uint32_t)out[7] << 16);
+  *reinterpret_cast<uint4*>(dense + (size_t)r * C + (size_t)c8 * 8) = v;
 }
 
 // ---- export / validate ---------------------------------------------------------------------------
@@ -364,12 +379,13 @@ mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s) {
 
 mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s) {
   const int c = L->cur;
+  const int64_t groups = L->N / 8;  // callers guarantee O % 8 == 0 and I % 8 == 0
   if (!transpose)
-    densify_from_bits<<<blocks_for(L->nwords * 32, 256), 256, 0, s>>>(L->bits[c], L->wscan[c], L->O, L->I, L->wpr,
-                                                                      (const uint16_t*)L->vals[c], nullptr, L->dense_w);
+    densify_from_bits<<<blocks_for(groups, 256), 256, 0, s>>>(L->bits[c], L->wscan[c], L->O, L->I, L->wpr,
+                                                             (const uint16_t*)L->vals[c], nullptr, L->dense_w);
   else
-    densify_from_bits<<<blocks_for(L->nwordsT * 32, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->I, L->O, L->wpc,
-                                                                       (const uint16_t*)L->vals[c], L->perm, L->dense_wt);
+    densify_from_bits<<<blocks_for(groups, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->I, L->O, L->wpc,
+                                                             (const uint16_t*)L->vals[c], L->perm, L->dense_wt);
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

@@ -580,13 +580,25 @@ int sm_count() {
 
 }  // namespace
 
-int mst_tc_pick_splits(int64_t tiles, int64_t kblocks) {
-  const int sms = sm_count();
-  if (tiles * 4 >= sms * 3) return 1;  // one wave is already at least three quarters full
-  int64_t sp = sms / tiles;
-  if (sp > kblocks) sp = kblocks;
-  if (sp > 16) sp = 16;
-  return sp < 1 ? 1 : (int)sp;
+// Number of K ranges for a contraction whose output has few tiles: minimise a simple time model
+//   waves * (k-blocks per range * t_kblock + t_tile) + traffic of the partial sums
+// over 1..16 ranges.  `works1` = tile jobs with one range, `slots` = jobs that run at once (blocks or block pairs),
+// `out_bytes` = bytes one range writes as partial sums (and the reduction reads back).
+int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double out_bytes) {
+  const double t_kblock = 0.32e-6, t_tile = 1.5e-6, bw = 4.0e12, t_reduce_launch = 3.0e-6;
+  int best = 1;
+  double best_t = 1e30;
+  for (int sp = 1; sp <= 16 && sp <= kblocks; ++sp) {
+    const int64_t waves = (works1 * sp + slots - 1) / slots;
+    const double kb = (double)((kblocks + sp - 1) / sp);
+    double t = (double)waves * (kb * t_kblock + t_tile);
+    if (sp > 1) t += t_reduce_launch + (double)sp * out_bytes * 2.0 / bw;
+    if (t < best_t * 0.97) {  // prefer fewer ranges unless the gain is clear
+      best_t = t;
+      best = sp;
+    }
+  }
+  return best;
 }
 
 mst_status_t mst_workspace(size_t bytes, void** ptr) {
@@ -628,9 +640,7 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   P.M = a.M;
   P.N = a.N;
   P.kblocks = (int)((a.K + BK - 1) / BK);
-  P.splits = a.splits < 1 ? 1 : a.splits;
-  if (P.splits > P.kblocks) P.splits = P.kblocks;
-  if (a.epilogue == MST_TC_OUT_BF16) P.splits = 1;
+  P.splits = 1;
   P.m_tiles = (int)((a.M + BM - 1) / BM);
   P.n_tiles = (int)((a.N + BN - 1) / BN);
   P.a_mn = a.a_mn_major;
@@ -638,12 +648,25 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   P.epilogue = a.epilogue;
   P.out = a.out;
   P.ldc = a.ldc;
-  P.partial = a.partial;
+  P.partial = nullptr;
   P.bits = a.bits;
   P.wscan = a.wscan;
   P.wpr = a.wpr;
   P.nnz = a.nnz;
-  if (P.splits > 1 && !a.partial) return MST_ERR_INVALID_ARG;
+  if (a.epilogue != MST_TC_OUT_BF16) {
+    // few output tiles: cut the contraction range so that all SMs work; partial sums go to the shared scratch buffer
+    const int64_t works1 = pair ? (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles : (int64_t)P.m_tiles * P.n_tiles;
+    const int64_t slots = pair ? sm_count() / 2 : sm_count();
+    const double out_bytes = a.epilogue == MST_TC_OUT_F32 ? 4.0 * (double)a.M * (double)a.N : 4.0 * (double)a.nnz;
+    P.splits = a.splits > 0 ? a.splits : mst_tc_pick_splits(works1, slots, P.kblocks, out_bytes);
+    if (P.splits > P.kblocks) P.splits = P.kblocks;
+    if (P.splits > 1) {
+      const size_t per = a.epilogue == MST_TC_OUT_F32 ? (size_t)a.M * a.N : (size_t)a.nnz;
+      void* ws = nullptr;
+      MST_TRY(mst_workspace(sizeof(float) * per * P.splits, &ws));
+      P.partial = (float*)ws;
+    }
+  }
   if (pair) {
     MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES));
     const int64_t works = (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles * P.splits;
@@ -659,7 +682,7 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   MST_CUDA_TRY(cudaGetLastError());
   if (P.splits > 1) {
     const int64_t n = a.epilogue == MST_TC_OUT_F32 ? a.M * a.N : a.nnz;
-    if (n > 0) tc_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(a.partial, P.splits, n, (float*)a.out);
+    if (n > 0) tc_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(P.partial, P.splits, n, (float*)a.out);
     MST_CUDA_TRY(cudaGetLastError());
   }
   return MST_OK;

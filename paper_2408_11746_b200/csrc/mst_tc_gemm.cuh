@@ -29,8 +29,8 @@ struct mst_tc_gemm_args {
   int epilogue;
   void* out;
   int64_t ldc;
-  int splits;            // K is cut into `splits` contiguous ranges (F32 / SAMPLED epilogues only)
-  float* partial;        // [splits][M*N] (F32) or [splits][nnz] (SAMPLED) when splits > 1
+  int splits;            // 0 = choose; otherwise K is cut into this many contiguous ranges (F32 / SAMPLED epilogues);
+                         // partial sums live in the process-wide scratch buffer and are added in a fixed order
   const uint32_t* bits;  // SAMPLED: mask words, wpr per row
   const int32_t* wscan;  // SAMPLED: exclusive popcount scan of the words
   int wpr;
@@ -42,8 +42,7 @@ struct mst_tc_gemm_args {
 mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s);
 bool mst_tc_gemm_usable(const void* A, int64_t lda, const void* B, int64_t ldb);
 
-// How many K ranges to cut a contraction into so that `tiles` output tiles fill the GPU in one wave.
-int mst_tc_pick_splits(int64_t tiles, int64_t kblocks);
+int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double out_bytes);
 
 // Process-wide scratch buffer for handle-less entry points (grows on demand; growing synchronises the device).
 // Calls that use it must not overlap on the GPU.

@@ -1,0 +1,145 @@
+"""Full-size workloads (the five configurations) through the C ABI in the launch configuration the benchmark uses.
+
+At these sizes the oracle computes sampled outputs one by one (fwd_at / bwd_x_at / grad_at); the topology update is
+compared bit-exactly on whole layers (the oracle's sort of a few million keys takes about a second).
+"""
+import numpy as np
+import pytest
+
+import mst_inputs
+import oracle
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+if torch.cuda.is_available():
+    import paper_2408_11746_b200 as mst
+    from gpu_util import TOL, dev, export_csr, host, make_layer, mdtype, rel_err, tdtype, to_dev, value_bits
+
+N_SAMPLES = 3000
+
+
+def _sampled_products_ok(p, L, rng, mask=None, Wm=None):
+    """fwd / bwd_x / sddmm / dense_grad at full size, checked at random output positions."""
+    T, O, I = p.tokens, p.out_features, p.in_features
+    mask = p.mask if mask is None else mask
+    Wm = np.where(mask == 1, p.W, np.float32(0)) if Wm is None else Wm
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    Y = torch.empty((T, O), dtype=tdtype(p), device=dev())
+    dX = torch.empty((T, I), dtype=tdtype(p), device=dev())
+    nnz = L.nnz
+    dW = torch.empty((max(nnz, 1),), dtype=torch.float32, device=dev())
+    G = torch.empty((O, I), dtype=torch.float32, device=dev())
+    L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW); L.dense_grad(dY, X, T, G)
+    torch.cuda.synchronize()
+    tol = TOL[p.dtype]
+    t = rng.integers(0, T, N_SAMPLES); o = rng.integers(0, O, N_SAMPLES); i = rng.integers(0, I, N_SAMPLES)
+    ti, oi, ii = torch.from_numpy(t).to(dev()), torch.from_numpy(o).to(dev()), torch.from_numpy(i).to(dev())
+    assert rel_err(host(Y[ti, oi]), oracle.fwd_at(p.X, Wm, mask, t, o)) <= tol
+    assert rel_err(host(dX[ti, ii]), oracle.bwd_x_at(p.dY, Wm, mask, t, i)) <= tol
+    assert rel_err(host(G[oi, ii]), oracle.grad_at(p.dY, p.X, o, i)) <= tol
+    if nnz:
+        rows, cols = np.nonzero(mask)
+        k = rng.integers(0, nnz, N_SAMPLES)
+        ref = oracle.grad_at(p.dY, p.X, rows[k], cols[k])
+        assert rel_err(host(dW[torch.from_numpy(k).to(dev())]), ref) <= tol
+    return G
+
+
+def _update_and_compare(L, p, W, M, G_host, zeta, R, seed, step):
+    O, I = M.shape
+    Gd = torch.from_numpy(G_host).to(dev())
+    st = mst.mst_topology_update(L.handle, zeta, -1, R, seed, step, False, Gd)
+    n_prune, _, n_rand, n_grad = oracle.mg_counts(zeta, int(M.sum()), -1, O * I, R)
+    assert (st.n_prune, st.n_rand, st.n_grad) == (n_prune, n_rand, n_grad)
+    Wn, Mn, *_ = oracle.mg_update(W, M, G_host, n_prune, n_grad, n_rand, seed, step, p.layer_id)
+    rp, ci, vb = export_csr(L, p.dtype)
+    rp_r, ci_r, v_r = oracle.to_csr(Wn, Mn)
+    np.testing.assert_array_equal(rp, rp_r)
+    np.testing.assert_array_equal(ci, ci_r)
+    np.testing.assert_array_equal(vb, value_bits(v_r, p.dtype))
+    assert st.nnz_after == int(M.sum())
+    return Wn, Mn
+
+
+def test_config1_fp32_single_layer_full_check():
+    (p,) = mst_inputs.config1()
+    L = make_layer(p)
+    assert L.nnz == 589824
+    T, O, I = p.tokens, p.out_features, p.in_features
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    Y = torch.empty((T, O), device=dev()); dX = torch.empty((T, I), device=dev())
+    dW = torch.empty((L.nnz,), device=dev()); G = torch.empty((O, I), device=dev())
+    L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW); L.dense_grad(dY, X, T, G)
+    torch.cuda.synchronize()
+    Wm = np.where(p.mask == 1, p.W, np.float32(0))
+    Gr = oracle.dense_grad(p.dY, p.X)
+    rows, cols = np.nonzero(p.mask)
+    assert rel_err(host(Y), oracle.fwd(p.X, Wm, p.mask)) <= 1e-5
+    assert rel_err(host(dX), oracle.bwd_x(p.dY, Wm, p.mask)) <= 1e-5
+    assert rel_err(host(dW), Gr[rows, cols]) <= 1e-5
+    assert rel_err(host(G), Gr) <= 1e-5
+    # one update, zeta = 0.3, R = 0.25, on the oracle's dense gradient rounded to fp32
+    _update_and_compare(L, p, Wm.astype(np.float32), p.mask.copy(), Gr.astype(np.float32), 0.3, 0.25, 0x4D5354, 0)
+    L.validate()
+    L.close()
+
+
+def test_config2_gpt2_small_block_bf16():
+    rng = np.random.default_rng(2)
+    for p in mst_inputs.config2():
+        L = make_layer(p)
+        assert L.nnz == mst_inputs.exact_nnz(p.out_features, p.in_features, 0.25)
+        _sampled_products_ok(p, L, rng)
+        L.close()
+    assert mst.mst_device_error_flags() == 0
+
+
+@pytest.mark.parametrize("block", [0, 7])
+def test_config3_zipf_rows_update_every_step(block):
+    rng = np.random.default_rng(3 + block)
+    for p in mst_inputs.config3(blocks=1, first_block=block):
+        L = make_layer(p)
+        d = p.nnz / p.mask.size
+        assert 0.03 - 1e-6 <= d <= 0.10 + 1e-6 and int(p.mask.sum(1).max()) == p.in_features   # saturated heavy rows
+        G = _sampled_products_ok(p, L, rng)
+        W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+        M = p.mask.copy()
+        Gh = host(G)
+        for step in range(3):          # from the second step on the just-grown zeros tie at |w| = 0
+            W, M = _update_and_compare(L, p, W, M, Gh, 0.1, 0.25, 0x4D5354 + 3, step)
+        L.validate()
+        # the products still agree on the evolved structure
+        _sampled_products_ok(p, L, rng, mask=M, Wm=W)
+        L.close()
+    assert mst.mst_device_error_flags() == 0
+
+
+def test_config4_gpt2_medium_block_with_regrowth():
+    rng = np.random.default_rng(4)
+    for p in mst_inputs.config4(blocks=1):
+        L = make_layer(p)
+        G = _sampled_products_ok(p, L, rng)
+        W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+        Gh = host(G)
+        for R in (0.0, 0.25):          # pure gradient growth, then the mixed rule, each from the packed state
+            L2 = make_layer(p)
+            _update_and_compare(L2, p, W, p.mask.copy(), Gh, 0.3, R, 0x4D5354 + 4, 0)
+            L2.close()
+        L.close()
+    assert mst.mst_device_error_flags() == 0
+
+
+def test_config5_density_sweep_gpt2_large_shapes():
+    rng = np.random.default_rng(5)
+    base = mst_inputs.config5(1.0)
+    for p in base:
+        O, I = p.out_features, p.in_features
+        for d in mst_inputs.CONFIG5_DENSITIES:
+            nnz = mst_inputs.exact_nnz(O, I, d)
+            mask = np.ones((O, I), dtype=np.uint8) if d == 1.0 else mst_inputs.uniform_mask(O, I, nnz, 50 + int(d * 100), p.layer_id)
+            L = mst.Layer(p.layer_id, O, I, mst.MST_BF16)
+            L.pack(to_dev(p, "W"), torch.from_numpy(mask).to(dev()))
+            assert L.nnz == nnz
+            _sampled_products_ok(p, L, rng, mask=mask)
+            L.close()
+    assert mst.mst_device_error_flags() == 0
