@@ -1,0 +1,89 @@
+// Device-side building blocks on the 32-bit mask words (shared by the stand-alone structure kernels and by the
+// fused topology-update kernel).  In every function one warp handles one word and `lane` is the bit inside it.
+#pragma once
+#include <stdint.h>
+
+__device__ __forceinline__ unsigned mst_lanemask_lt() {
+  unsigned m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// CSR entries of mask word w.  Source of a value: dense W (pack) or the previous structure (update: an entry present
+// before and after keeps its value, a new entry starts at +0).
+template <typename V>
+__device__ __forceinline__ void mst_fill_csr_word(int64_t w, int lane, const uint32_t* __restrict__ bits,
+                                                  const int32_t* __restrict__ wscan, int O, int I, int wpr,
+                                                  uint16_t* __restrict__ col_idx, V* __restrict__ vals,
+                                                  int32_t* __restrict__ row_ptr, const V* __restrict__ dense_W,
+                                                  int64_t ldw, const uint32_t* __restrict__ old_bits,
+                                                  const int32_t* __restrict__ old_wscan, const V* __restrict__ old_vals) {
+  const int64_t nwords = (int64_t)O * wpr;
+  const unsigned wu = (unsigned)w;
+  const int o = (int)(wu / (unsigned)wpr), wc = (int)(wu - (unsigned)o * (unsigned)wpr);
+  const uint32_t b = bits[w];
+  const int32_t base = wscan[w];
+  if (wc == 0 && lane == 0) {
+    row_ptr[o] = base;
+    if (o == O - 1) row_ptr[O] = wscan[nwords];
+  }
+  if ((b >> lane) & 1u) {
+    const int32_t pos = base + __popc(b & mst_lanemask_lt());
+    const int c = wc * 32 + lane;
+    col_idx[pos] = (uint16_t)c;
+    V v;
+    if (dense_W) {
+      v = dense_W[(int64_t)o * ldw + c];
+    } else {
+      const uint32_t ob = old_bits[w];
+      if ((ob >> lane) & 1u) {
+        v = old_vals[old_wscan[w] + __popc(ob & mst_lanemask_lt())];
+      } else {
+        v = V(0);
+      }
+    }
+    vals[pos] = v;
+  }
+}
+
+// 32 x 32 bit tile (wr, wc) of the mask -> the same tile of the transposed mask.
+__device__ __forceinline__ void mst_transpose_tile(int64_t tile, int lane, const uint32_t* __restrict__ bits, int O, int I,
+                                                   int wpr, int wpc, uint32_t* __restrict__ bitsT) {
+  const unsigned tu = (unsigned)tile;
+  const int wr = (int)(tu / (unsigned)wpr), wc = (int)(tu - (unsigned)wr * (unsigned)wpr);
+  const int o = wr * 32 + lane;
+  const uint32_t word = o < O ? bits[(int64_t)o * wpr + wc] : 0u;
+  uint32_t mine = 0;
+#pragma unroll
+  for (int c = 0; c < 32; ++c) {
+    const uint32_t t = __ballot_sync(0xffffffffu, (word >> c) & 1u);
+    if (c == lane) mine = t;
+  }
+  const int i = wc * 32 + lane;
+  if (i < I) bitsT[(int64_t)i * wpc + wr] = mine;
+}
+
+// CSC entries of transposed mask word w: row index and the CSR position of the same entry.
+__device__ __forceinline__ void mst_fill_csc_word(int64_t w, int lane, const uint32_t* __restrict__ bitsT,
+                                                  const int32_t* __restrict__ wscanT, int O, int I, int wpr, int wpc,
+                                                  const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan,
+                                                  uint16_t* __restrict__ row_idx, int32_t* __restrict__ perm,
+                                                  int32_t* __restrict__ col_ptr) {
+  const int64_t nwordsT = (int64_t)I * wpc;
+  const unsigned wu = (unsigned)w;
+  const int i = (int)(wu / (unsigned)wpc), wr = (int)(wu - (unsigned)i * (unsigned)wpc);
+  const uint32_t b = bitsT[w];
+  const int32_t base = wscanT[w];
+  if (wr == 0 && lane == 0) {
+    col_ptr[i] = base;
+    if (i == I - 1) col_ptr[I] = wscanT[nwordsT];
+  }
+  if ((b >> lane) & 1u) {
+    const int o = wr * 32 + lane;
+    const int32_t posT = base + __popc(b & mst_lanemask_lt());
+    const int64_t wf = (int64_t)o * wpr + (i >> 5);
+    const uint32_t fb = bits[wf];
+    row_idx[posT] = (uint16_t)o;
+    perm[posT] = wscan[wf] + __popc(fb & ((1u << (i & 31)) - 1u));
+  }
+}

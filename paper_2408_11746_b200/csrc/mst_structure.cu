@@ -6,6 +6,7 @@
 // The same holds for the CSC view on the transposed bit mask.  Everything below is integer work,
 // stream-ordered, with no inter-block waiting (the scan is three plain kernels).
 #include "mst_internal.cuh"
+#include "mst_bits.cuh"
 
 #include <cuda_bf16.h>
 
@@ -159,75 +160,25 @@ __global__ void fill_csr(const uint32_t* __restrict__ bits, const int32_t* __res
                          const V* __restrict__ dense_W, int64_t ldw, const uint32_t* __restrict__ old_bits,
                          const int32_t* __restrict__ old_wscan, const V* __restrict__ old_vals) {
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  const int64_t nwords = (int64_t)O * wpr;
-  if (w >= nwords) return;
-  const int o = (int)(w / wpr), wc = (int)(w % wpr);
-  const uint32_t b = bits[w];
-  const int32_t base = wscan[w];
-  if (wc == 0 && lane == 0) {
-    row_ptr[o] = base;
-    if (o == O - 1) row_ptr[O] = wscan[nwords];
-  }
-  if ((b >> lane) & 1u) {
-    const int32_t pos = base + __popc(b & lanemask_lt());
-    const int c = wc * 32 + lane;
-    col_idx[pos] = (uint16_t)c;
-    V v;
-    if (dense_W) {
-      v = dense_W[(int64_t)o * ldw + c];
-    } else {
-      const uint32_t ob = old_bits[w];
-      if ((ob >> lane) & 1u) {
-        v = old_vals[old_wscan[w] + __popc(ob & lanemask_lt())];
-      } else {
-        v = V(0);
-      }
-    }
-    vals[pos] = v;
-  }
+  if (w >= (int64_t)O * wpr) return;
+  mst_fill_csr_word<V>(w, threadIdx.x & 31, bits, wscan, O, I, wpr, col_idx, vals, row_ptr, dense_W, ldw, old_bits,
+                       old_wscan, old_vals);
 }
 
 // ---- bit transpose: one warp per 32x32 bit tile -------------------------------------------------
 __global__ void transpose_bits(const uint32_t* __restrict__ bits, int O, int I, int wpr, int wpc,
                                uint32_t* __restrict__ bitsT) {
   const int64_t tile = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
   if (tile >= (int64_t)wpc * wpr) return;
-  const int wr = (int)(tile / wpr), wc = (int)(tile % wpr);
-  const int o = wr * 32 + lane;
-  const uint32_t word = o < O ? bits[(int64_t)o * wpr + wc] : 0u;
-  uint32_t mine = 0;
-  for (int c = 0; c < 32; ++c) {
-    const uint32_t t = __ballot_sync(0xffffffffu, (word >> c) & 1u);
-    if (c == lane) mine = t;
-  }
-  const int i = wc * 32 + lane;
-  if (i < I) bitsT[(int64_t)i * wpc + wr] = mine;
+  mst_transpose_tile(tile, threadIdx.x & 31, bits, O, I, wpr, wpc, bitsT);
 }
 
 __global__ void fill_csc(const uint32_t* __restrict__ bitsT, const int32_t* __restrict__ wscanT, int O, int I, int wpr,
                          int wpc, const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan,
                          uint16_t* __restrict__ row_idx, int32_t* __restrict__ perm, int32_t* __restrict__ col_ptr) {
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int lane = threadIdx.x & 31;
-  const int64_t nwordsT = (int64_t)I * wpc;
-  if (w >= nwordsT) return;
-  const int i = (int)(w / wpc), wr = (int)(w % wpc);
-  const uint32_t b = bitsT[w];
-  const int32_t base = wscanT[w];
-  if (wr == 0 && lane == 0) {
-    col_ptr[i] = base;
-    if (i == I - 1) col_ptr[I] = wscanT[nwordsT];
-  }
-  if ((b >> lane) & 1u) {
-    const int o = wr * 32 + lane;
-    const int32_t posT = base + __popc(b & lanemask_lt());
-    const int64_t wf = (int64_t)o * wpr + (i >> 5);
-    const uint32_t fb = bits[wf];
-    row_idx[posT] = (uint16_t)o;
-    perm[posT] = wscan[wf] + __popc(fb & ((1u << (i & 31)) - 1u));
-  }
+  if (w >= (int64_t)I * wpc) return;
+  mst_fill_csc_word(w, threadIdx.x & 31, bitsT, wscanT, O, I, wpr, wpc, bits, wscan, row_idx, perm, col_ptr);
 }
 
 // ---- dense bf16 image of W.M (or its transpose) for the tensor-core path ----------------------------------------------
