@@ -275,7 +275,7 @@ inline unsigned blocks_for(int64_t n, int per_block) { return (unsigned)((n + pe
 
 }  // namespace
 
-int64_t mst_scan_block_sums_len(int64_t n) { return (n + SCAN_TILE - 1) / SCAN_TILE + 1; }
+int64_t mst_scan_block_sums_len(int64_t n) { return (n + SCAN_TILE - 1) / SCAN_TILE + 1 + 1024; }
 
 mst_status_t mst_scan_i32_if(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, const int* enabled,
                              cudaStream_t s) {

@@ -11,6 +11,11 @@
 // Work layout: one warp per 32-bit mask word, lane = column inside the word, so reads of G and of the value array are
 // coalesced.  The last block to finish a histogram pass picks the digit (completion counter, no waiting).  The tie
 // ranking (count, scan) is skipped on the device when the threshold key has no surplus ties.
+#include <cooperative_groups.h>
+
+#include <cstdlib>
+
+#include "mst_bits.cuh"
 #include "mst_internal.cuh"
 
 namespace {
@@ -277,6 +282,302 @@ mst_status_t run_select(mst_layer* L, const SelParams& P, int64_t k, uint32_t* o
   return MST_OK;
 }
 
+// ------------------------------------------------------------------------------------------------ fused update
+// The whole update as ONE cooperative kernel: the phases above (histogram passes, digit picks, tie ranking, marking,
+// mask rewrite, scans, CSR and CSC fill) separated by grid-wide barriers instead of kernel boundaries.  Every block
+// owns one contiguous slice of the mask words for all word-wise phases, so that only the histogram -> pick steps, the
+// scans and the transpose need a barrier.  Every block computes each digit pick itself from the global histogram
+// (three rotating histogram buffers: the one for pass p+2 is cleared after the barrier of pass p).
+namespace cg = cooperative_groups;
+
+constexpr int FUSED_THREADS = 512;
+constexpr int FUSED_WARPS = FUSED_THREADS / 32;
+constexpr int FUSED_BPT = BINS / FUSED_THREADS;  // histogram bins per thread in the pick
+
+struct FusedParams {
+  SelParams sel;
+  long long n_prune, n_grad, n_rand;
+  uint32_t *pruned_bits, *grad_bits, *rand_bits, *new_bits;
+  int32_t *cnt, *scan, *bsums;
+  unsigned int* hist;  // [3][BINS], all zero at launch
+  int32_t* flags;
+  int32_t *new_wscan, *new_row_ptr;
+  uint16_t* new_col;
+  void* new_vals;
+  uint32_t* bitsT;
+  int32_t *wscanT, *col_ptr;
+  uint16_t* row_idx;
+  int32_t* perm;
+  int wpc;
+  int64_t nwordsT;
+};
+
+struct FusedShared {
+  unsigned int hist[BINS];
+  unsigned int warp_tot[FUSED_WARPS];
+  int red[FUSED_WARPS];
+  unsigned long long prefix, tau;
+  long long k, rem;
+  int need_rank, done, found;
+};
+
+__device__ __forceinline__ int fused_block_sum(int v, FusedShared& sh) {
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();  // sh.red free
+  if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = 0;
+#pragma unroll
+  for (int w = 0; w < FUSED_WARPS; ++w) r += sh.red[w];
+  return r;
+}
+
+// exclusive prefix of v over the block (thread order); total = sum over the block
+__device__ __forceinline__ int fused_block_excl_scan(int v, int& total, FusedShared& sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int x = v;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();
+  if (lane == 31) sh.red[warp] = x;
+  __syncthreads();
+  int before = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < FUSED_WARPS; ++w) {
+    const int t = sh.red[w];
+    if (w < warp) before += t;
+    tot += t;
+  }
+  total = tot;
+  return before + x - v;
+}
+
+// out[0..n] = exclusive scan of cnt[0..n); each block scans its slice [lo, hi).  One grid barrier inside.
+__device__ void fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int64_t lo, int64_t hi, int32_t* bsums,
+                                cg::grid_group& grid, FusedShared& sh) {
+  int v = 0;
+  for (int64_t i = lo + threadIdx.x; i < hi; i += FUSED_THREADS) v += cnt[i];
+  const int bs = fused_block_sum(v, sh);
+  if (threadIdx.x == 0) bsums[blockIdx.x] = bs;
+  grid.sync();
+  int off = 0, tot = 0;
+  for (int j = threadIdx.x; j < (int)gridDim.x; j += FUSED_THREADS) {
+    const int x = __ldcg(bsums + j);
+    tot += x;
+    if (j < (int)blockIdx.x) off += x;
+  }
+  off = fused_block_sum(off, sh);
+  tot = fused_block_sum(tot, sh);
+  int carry = off;
+  for (int64_t base = lo; base < hi; base += FUSED_THREADS) {
+    const int64_t i = base + threadIdx.x;
+    const int x = i < hi ? cnt[i] : 0;
+    int tile_total;
+    const int ex = fused_block_excl_scan(x, tile_total, sh);
+    if (i < hi) out[i] = carry + ex;
+    carry += tile_total;
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) out[n] = tot;
+  __syncthreads();
+}
+
+// One selection inside the fused kernel.  gpass counts the histogram passes executed so far (buffer rotation).
+template <int MODE>
+__device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* out_bits, int64_t lo, int64_t hi,
+                             int& gpass, cg::grid_group& grid, FusedShared& sh) {
+  constexpr int KB = KeyBits<MODE>::value;
+  constexpr int passes = num_passes(KB);
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (k_total <= 0) {  // uniform over the grid
+    for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) out_bits[w] = 0;
+    __syncthreads();
+    return;
+  }
+  if (threadIdx.x == 0) {
+    sh.prefix = 0;
+    sh.k = k_total;
+    sh.tau = 0;
+    sh.rem = 0;
+    sh.need_rank = 0;
+    sh.done = 0;
+  }
+  __syncthreads();
+  for (int pass = 0; pass < passes; ++pass) {
+    if (sh.done) break;  // same decision in every block
+    const int shift = pass_shift(KB, pass), width = pass_width(KB, pass);
+    const unsigned dmask = (1u << width) - 1u;
+    const int hi_shift = shift + width;
+    const unsigned long long prefix = sh.prefix;
+    const long long k = sh.k;
+    unsigned int* gh = F.hist + (gpass % 3) * BINS;
+    for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    bool saw_nonfinite = false;
+    constexpr int BATCH = 4;
+    for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * BATCH) {
+      unsigned digit[BATCH];
+      bool live[BATCH];
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) {
+        const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
+        unsigned long long key = 0;
+        bool nf = false;
+        const bool c = w < hi && cand_key<MODE>(P, w, lane, key, nf);
+        saw_nonfinite |= (c && nf);
+        live[j] = c && (pass == 0 || (key >> hi_shift) == prefix);
+        digit[j] = live[j] ? (unsigned)((key >> shift) & dmask) : (unsigned)BINS;
+      }
+#pragma unroll
+      for (int j = 0; j < BATCH; ++j) {
+        const unsigned peers = __match_any_sync(0xffffffffu, digit[j]);
+        if (live[j] && lane == (__ffs(peers) - 1)) atomicAdd(&sh.hist[digit[j]], (unsigned)__popc(peers));
+      }
+    }
+    if (pass == 0 && saw_nonfinite) atomicOr(&F.flags[0], MST_FLAG_NONFINITE);
+    __syncthreads();
+    for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS)
+      if (sh.hist[b]) atomicAdd(&gh[b], sh.hist[b]);
+    grid.sync();
+    // every block picks the digit from the complete histogram
+    unsigned int mine[FUSED_BPT];
+    unsigned int tsum = 0;
+#pragma unroll
+    for (int j = 0; j < FUSED_BPT; ++j) {
+      mine[j] = __ldcg(gh + threadIdx.x * FUSED_BPT + j);
+      tsum += mine[j];
+    }
+    if (blockIdx.x == 0) {  // clear the buffer of pass gpass + 2 (last read before this barrier)
+      unsigned int* gz = F.hist + ((gpass + 2) % 3) * BINS;
+      for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) gz[b] = 0;
+    }
+    unsigned int incl = tsum;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int y = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += y;
+    }
+    if (threadIdx.x == 0) sh.found = 0;
+    if (lane == 31) sh.warp_tot[warp] = incl;
+    __syncthreads();
+    unsigned int before = incl - tsum;
+    for (int wv = 0; wv < warp; ++wv) before += sh.warp_tot[wv];
+    const bool owner = (long long)before < k && k <= (long long)before + (long long)tsum;
+    if (owner) {
+      long long cum = before;
+      int bin = 0;
+      unsigned int bcount = 0;
+      for (int j = 0; j < FUSED_BPT; ++j) {
+        if (cum + (long long)mine[j] >= k) { bin = j; bcount = mine[j]; break; }
+        cum += mine[j];
+      }
+      const unsigned long long np = (prefix << width) | (unsigned long long)(threadIdx.x * FUSED_BPT + bin);
+      sh.prefix = np;
+      sh.k = k - cum;
+      sh.found = 1;
+      if (shift == 0) {
+        sh.tau = np;
+        sh.rem = k - cum;
+        sh.need_rank = ((long long)bcount > k - cum) ? 1 : 0;
+        sh.done = 1;
+      } else if ((long long)bcount == k - cum) {
+        sh.tau = (np << shift) | ((1ULL << shift) - 1ULL);
+        sh.rem = k - cum;
+        sh.need_rank = 0;
+        sh.done = 1;
+      }
+    }
+    __syncthreads();
+    if (!sh.found) {  // fewer candidates than requested (ruled out by the host counts): take everything
+      if (threadIdx.x == 0) {
+        sh.tau = ~0ULL;
+        sh.rem = 0x7FFFFFFFFFFFFFFFLL;
+        sh.need_rank = 0;
+        sh.done = 1;
+        if (blockIdx.x == 0) atomicOr(&F.flags[0], MST_FLAG_CORRUPT);
+      }
+      __syncthreads();
+    }
+    ++gpass;
+  }
+  const unsigned long long tau = sh.tau;
+  const long long rem = sh.rem;
+  const bool need_rank = sh.need_rank != 0;
+  if (need_rank) {  // rank the entries equal to tau in index order
+    for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
+      unsigned long long key;
+      bool nf;
+      const bool c = cand_key<MODE>(P, w, lane, key, nf);
+      const unsigned eq = __ballot_sync(0xffffffffu, c && key == tau);
+      if (lane == 0) F.cnt[w] = __popc(eq);
+    }
+    __syncthreads();
+    fused_grid_scan(F.cnt, F.scan, P.nwords, lo, hi, F.bsums, grid, sh);
+  }
+  for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
+    unsigned long long key;
+    bool nf;
+    const bool c = cand_key<MODE>(P, w, lane, key, nf);
+    const bool iseq = c && key == tau;
+    const unsigned eq = __ballot_sync(0xffffffffu, iseq);
+    const long long rank = need_rank ? (long long)F.scan[w] + __popc(eq & lanemask_lt()) : -1;
+    const bool take = c && (key < tau || (iseq && rank < rem));
+    const unsigned bits = __ballot_sync(0xffffffffu, take);
+    if (lane == 0) out_bits[w] = bits;
+  }
+  __syncthreads();
+}
+
+template <typename V>
+__global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const FusedParams F) {
+  cg::grid_group grid = cg::this_grid();
+  __shared__ FusedShared sh;
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t per = (P.nwords + gridDim.x - 1) / gridDim.x;
+  const int64_t lo = per * blockIdx.x < P.nwords ? per * blockIdx.x : P.nwords;
+  const int64_t hi = lo + per < P.nwords ? lo + per : P.nwords;
+  const int64_t perT = (F.nwordsT + gridDim.x - 1) / gridDim.x;
+  const int64_t loT = perT * blockIdx.x < F.nwordsT ? perT * blockIdx.x : F.nwordsT;
+  const int64_t hiT = loT + perT < F.nwordsT ? loT + perT : F.nwordsT;
+
+  int gpass = 0;
+  fused_select<MODE_PRUNE>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh);
+  fused_select<MODE_GRAD>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh);
+  fused_select<MODE_RAND>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh);
+
+  // mask rewrite: new = (old & ~pruned) | grad | rand, and its popcounts
+  for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
+    const uint32_t b = (P.old_bits[w] & ~F.pruned_bits[w]) | F.grad_bits[w] | F.rand_bits[w];
+    F.new_bits[w] = b;
+    F.cnt[w] = __popc(b);
+  }
+  __syncthreads();
+  fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, grid, sh);
+  grid.sync();  // new mask and its scan are complete everywhere
+  for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
+    mst_fill_csr_word<V>(w, lane, F.new_bits, F.new_wscan, P.O, P.I, P.wpr, F.new_col, (V*)F.new_vals, F.new_row_ptr,
+                         (const V*)nullptr, 0, P.old_bits, P.old_wscan, (const V*)P.vals);
+    const unsigned wu = (unsigned)w;
+    if (lane == 0 && wu % (unsigned)P.wpr == 0)
+      atomicMax(&F.flags[1], F.new_wscan[w + P.wpr] - F.new_wscan[w]);  // row population
+  }
+  {
+    const int64_t tiles = (int64_t)F.wpc * P.wpr;
+    for (int64_t t = (int64_t)blockIdx.x * FUSED_WARPS + warp; t < tiles; t += (int64_t)gridDim.x * FUSED_WARPS)
+      mst_transpose_tile(t, lane, F.new_bits, P.O, P.I, P.wpr, F.wpc, F.bitsT);
+  }
+  grid.sync();  // transposed mask complete
+  for (int64_t w = loT + threadIdx.x; w < hiT; w += FUSED_THREADS) F.cnt[w] = __popc(F.bitsT[w]);
+  __syncthreads();
+  fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, grid, sh);
+  grid.sync();  // col_ptr[I] needs the scan's last element, written by block 0
+  for (int64_t w = loT + warp; w < hiT; w += FUSED_WARPS)
+    mst_fill_csc_word(w, lane, F.bitsT, F.wscanT, P.O, P.I, P.wpr, F.wpc, F.new_bits, F.new_wscan, F.row_idx, F.perm,
+                      F.col_ptr);
+}
+
 inline unsigned long long host_mix(unsigned long long z) {
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
   z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
@@ -342,19 +643,52 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     P.stream = host_mix((b ^ (unsigned long long)(int64_t)L->layer_id) + SM64_GAMMA);
   }
 
-  MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
-  MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
-  MST_TRY(run_select<MODE_RAND>(L, P, n_rand, L->rand_bits, s));
-
-  MST_TRY(mst_combine_update_bits(L, n, s));
-  MST_TRY(mst_rebuild_from_bits(L, n, nullptr, 0, c, s));
+  bool fused = true;
+  if (const char* e = getenv("MST_UPDATE_FUSED")) fused = (e[0] != '0');
+  int grid_blocks = 0;
+  if (fused) {
+    int dev = 0, coop = 0, sms = 0, occ = 0;
+    const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, FUSED_THREADS, 0) != cudaSuccess || !coop || occ < 1)
+      fused = false;
+    else {
+      if (occ > 2) occ = 2;
+      grid_blocks = sms * occ;
+      const int64_t useful = (L->nwords + FUSED_WARPS - 1) / FUSED_WARPS;  // at least one word per warp
+      if (grid_blocks > useful) grid_blocks = (int)(useful < 1 ? 1 : useful);
+      if ((int64_t)grid_blocks > mst_scan_block_sums_len(L->nwords > L->nwordsT ? L->nwords : L->nwordsT)) fused = false;
+    }
+  }
+  if (fused) {
+    MST_CUDA_TRY(cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * BINS, s));
+    FusedParams F;
+    F.sel = P;
+    F.n_prune = n_prune; F.n_grad = n_grad; F.n_rand = n_rand;
+    F.pruned_bits = L->pruned_bits; F.grad_bits = L->grad_bits; F.rand_bits = L->rand_bits; F.new_bits = L->bits[n];
+    F.cnt = L->word_cnt; F.scan = L->word_scan; F.bsums = L->block_sums;
+    F.hist = L->hist; F.flags = L->flags;
+    F.new_wscan = L->wscan[n]; F.new_row_ptr = L->row_ptr[n]; F.new_col = L->col_idx[n]; F.new_vals = L->vals[n];
+    F.bitsT = L->bitsT; F.wscanT = L->wscanT; F.col_ptr = L->col_ptr; F.row_idx = L->row_idx; F.perm = L->perm;
+    F.wpc = L->wpc; F.nwordsT = L->nwordsT;
+    void* args[] = {&F};
+    const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
+    MST_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3(grid_blocks), dim3(FUSED_THREADS), args, 0, s));
+  } else {
+    MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
+    MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
+    MST_TRY(run_select<MODE_RAND>(L, P, n_rand, L->rand_bits, s));
+    MST_TRY(mst_combine_update_bits(L, n, s));
+    MST_TRY(mst_rebuild_from_bits(L, n, nullptr, 0, c, s));
+  }
   L->cur = n;
   const int64_t nnz_before = L->nnz;
   L->nnz = target;
-  MST_TRY(mst_build_csc(L, s));
+  if (!fused) MST_TRY(mst_build_csc(L, s));
 
   if (stats) {
-    max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
+    if (!fused) max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
     int32_t f[4] = {0, 0, 0, 0};
     int32_t total = 0;
     MST_CUDA_TRY(cudaMemcpyAsync(f, L->flags, sizeof(f), cudaMemcpyDeviceToHost, s));

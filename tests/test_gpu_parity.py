@@ -162,7 +162,10 @@ def _update_both(L, p, W, M, G, zeta, target, R, seed, step, allow=False):
     (256, 512, "bf16", 0.05, "zipf", 0.1, 0.25, False), (64, 96, "f32", 0.3, "uniform", 0.3, 0.0, False),
     (64, 96, "bf16", 0.3, "uniform", 0.3, 1.0, False), (96, 160, "bf16", 0.25, "uniform", 0.5, 0.25, True),
     (33, 31, "f32", 0.5, "uniform", 1.0, 0.5, False)])
-def test_update_is_bit_exact_over_consecutive_steps(O, I, dtype, density, kind, zeta, R, allow):
+@pytest.mark.parametrize("fused", ["1", "0"])
+def test_update_is_bit_exact_over_consecutive_steps(O, I, dtype, density, kind, zeta, R, allow, fused, monkeypatch):
+    # both implementations of the update: the single cooperative kernel and the kernel-per-phase sequence
+    monkeypatch.setenv("MST_UPDATE_FUSED", fused)
     p = _problem(O, I, 4, dtype, density, 300 + O + I, kind)
     L = make_layer(p)
     W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
