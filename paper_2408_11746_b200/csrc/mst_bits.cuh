@@ -87,3 +87,94 @@ __device__ __forceinline__ void mst_fill_csc_word(int64_t w, int lane, const uin
     perm[posT] = wscan[wf] + __popc(fb & ((1u << (i & 31)) - 1u));
   }
 }
+
+// ---- batched forms for kernels where a warp walks many words: B words per trip, loads grouped by dependency level so
+// ---- that they overlap (first the mask words and their scans, then the values they point to, then the stores).
+template <typename V, int B>
+__device__ __forceinline__ void mst_fill_csr_words(int64_t w0, int64_t stride, int64_t w_end, int lane,
+                                                   const uint32_t* bits, const int32_t* wscan, int O, int wpr,
+                                                   uint16_t* col_idx, V* vals, int32_t* row_ptr,
+                                                   const uint32_t* old_bits, const int32_t* old_wscan, const V* old_vals,
+                                                   int32_t* max_row) {
+  const int64_t nwords = (int64_t)O * wpr;
+  uint32_t b[B], ob[B];
+  int32_t base[B], obase[B];
+#pragma unroll
+  for (int j = 0; j < B; ++j) {
+    const int64_t w = w0 + j * stride;
+    const bool ok = w < w_end;
+    b[j] = ok ? bits[w] : 0u;
+    base[j] = ok ? wscan[w] : 0;
+    ob[j] = ok ? old_bits[w] : 0u;
+    obase[j] = ok ? old_wscan[w] : 0;
+  }
+  V v[B];
+#pragma unroll
+  for (int j = 0; j < B; ++j) {
+    v[j] = V(0);
+    if (((b[j] & ob[j]) >> lane) & 1u) v[j] = old_vals[obase[j] + __popc(ob[j] & mst_lanemask_lt())];
+  }
+#pragma unroll
+  for (int j = 0; j < B; ++j) {
+    const int64_t w = w0 + j * stride;
+    if (w >= w_end) continue;
+    const unsigned wu = (unsigned)w;
+    const int o = (int)(wu / (unsigned)wpr), wc = (int)(wu - (unsigned)o * (unsigned)wpr);
+    if (wc == 0 && lane == 0) {
+      row_ptr[o] = base[j];
+      const int32_t next = wscan[w + wpr];  // first word of the next row, or the total
+      if (o == O - 1) row_ptr[O] = wscan[nwords];
+      if (max_row) atomicMax(max_row, next - base[j]);
+    }
+    if ((b[j] >> lane) & 1u) {
+      const int32_t pos = base[j] + __popc(b[j] & mst_lanemask_lt());
+      col_idx[pos] = (uint16_t)(wc * 32 + lane);
+      vals[pos] = v[j];
+    }
+  }
+}
+
+template <int B>
+__device__ __forceinline__ void mst_fill_csc_words(int64_t w0, int64_t stride, int64_t w_end, int lane,
+                                                   const uint32_t* bitsT, const int32_t* wscanT, int I, int wpr, int wpc,
+                                                   const uint32_t* bits, const int32_t* wscan, uint16_t* row_idx,
+                                                   int32_t* perm, int32_t* col_ptr) {
+  const int64_t nwordsT = (int64_t)I * wpc;
+  uint32_t b[B], fb[B];
+  int32_t base[B], fs[B];
+  int ii[B], wrr[B];
+#pragma unroll
+  for (int j = 0; j < B; ++j) {
+    const int64_t w = w0 + j * stride;
+    const bool ok = w < w_end;
+    b[j] = ok ? bitsT[w] : 0u;
+    base[j] = ok ? wscanT[w] : 0;
+    const unsigned wu = (unsigned)w;
+    ii[j] = (int)(wu / (unsigned)wpc);
+    wrr[j] = (int)(wu - (unsigned)ii[j] * (unsigned)wpc);
+  }
+#pragma unroll
+  for (int j = 0; j < B; ++j) {
+    fb[j] = 0;
+    fs[j] = 0;
+    if ((b[j] >> lane) & 1u) {
+      const int64_t wf = (int64_t)(wrr[j] * 32 + lane) * wpr + (ii[j] >> 5);
+      fb[j] = bits[wf];
+      fs[j] = wscan[wf];
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < B; ++j) {
+    const int64_t w = w0 + j * stride;
+    if (w >= w_end) continue;
+    if (wrr[j] == 0 && lane == 0) {
+      col_ptr[ii[j]] = base[j];
+      if (ii[j] == I - 1) col_ptr[I] = wscanT[nwordsT];
+    }
+    if ((b[j] >> lane) & 1u) {
+      const int32_t posT = base[j] + __popc(b[j] & mst_lanemask_lt());
+      row_idx[posT] = (uint16_t)(wrr[j] * 32 + lane);
+      perm[posT] = fs[j] + __popc(fb[j] & ((1u << (ii[j] & 31)) - 1u));
+    }
+  }
+}

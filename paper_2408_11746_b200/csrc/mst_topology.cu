@@ -416,7 +416,7 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
     __syncthreads();
     bool saw_nonfinite = false;
-    constexpr int BATCH = 4;
+    constexpr int BATCH = 8;
     for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * BATCH) {
       unsigned digit[BATCH];
       bool live[BATCH];
@@ -515,16 +515,28 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     __syncthreads();
     fused_grid_scan(F.cnt, F.scan, P.nwords, lo, hi, F.bsums, grid, sh);
   }
-  for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
-    unsigned long long key;
-    bool nf;
-    const bool c = cand_key<MODE>(P, w, lane, key, nf);
-    const bool iseq = c && key == tau;
-    const unsigned eq = __ballot_sync(0xffffffffu, iseq);
-    const long long rank = need_rank ? (long long)F.scan[w] + __popc(eq & lanemask_lt()) : -1;
-    const bool take = c && (key < tau || (iseq && rank < rem));
-    const unsigned bits = __ballot_sync(0xffffffffu, take);
-    if (lane == 0) out_bits[w] = bits;
+  constexpr int MB = 4;
+  for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * MB) {
+    bool c[MB], iseq[MB];
+    unsigned long long key[MB];
+#pragma unroll
+    for (int j = 0; j < MB; ++j) {
+      const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
+      bool nf = false;
+      key[j] = 0;
+      c[j] = w < hi && cand_key<MODE>(P, w, lane, key[j], nf);
+      iseq[j] = c[j] && key[j] == tau;
+    }
+#pragma unroll
+    for (int j = 0; j < MB; ++j) {
+      const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
+      if (w >= hi) continue;  // uniform over the warp
+      const unsigned eq = __ballot_sync(0xffffffffu, iseq[j]);
+      const long long rank = need_rank ? (long long)F.scan[w] + __popc(eq & lanemask_lt()) : -1;
+      const bool take = c[j] && (key[j] < tau || (iseq[j] && rank < rem));
+      const unsigned bits = __ballot_sync(0xffffffffu, take);
+      if (lane == 0) out_bits[w] = bits;
+    }
   }
   __syncthreads();
 }
@@ -556,13 +568,9 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   __syncthreads();
   fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, grid, sh);
   grid.sync();  // new mask and its scan are complete everywhere
-  for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
-    mst_fill_csr_word<V>(w, lane, F.new_bits, F.new_wscan, P.O, P.I, P.wpr, F.new_col, (V*)F.new_vals, F.new_row_ptr,
-                         (const V*)nullptr, 0, P.old_bits, P.old_wscan, (const V*)P.vals);
-    const unsigned wu = (unsigned)w;
-    if (lane == 0 && wu % (unsigned)P.wpr == 0)
-      atomicMax(&F.flags[1], F.new_wscan[w + P.wpr] - F.new_wscan[w]);  // row population
-  }
+  for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * 4)
+    mst_fill_csr_words<V, 4>(w0, FUSED_WARPS, hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col, (V*)F.new_vals,
+                             F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals, &F.flags[1]);
   {
     const int64_t tiles = (int64_t)F.wpc * P.wpr;
     for (int64_t t = (int64_t)blockIdx.x * FUSED_WARPS + warp; t < tiles; t += (int64_t)gridDim.x * FUSED_WARPS)
@@ -573,9 +581,9 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   __syncthreads();
   fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, grid, sh);
   grid.sync();  // col_ptr[I] needs the scan's last element, written by block 0
-  for (int64_t w = loT + warp; w < hiT; w += FUSED_WARPS)
-    mst_fill_csc_word(w, lane, F.bitsT, F.wscanT, P.O, P.I, P.wpr, F.wpc, F.new_bits, F.new_wscan, F.row_idx, F.perm,
-                      F.col_ptr);
+  for (int64_t w0 = loT + warp; w0 < hiT; w0 += FUSED_WARPS * 4)
+    mst_fill_csc_words<4>(w0, FUSED_WARPS, hiT, lane, F.bitsT, F.wscanT, P.I, P.wpr, F.wpc, F.new_bits, F.new_wscan,
+                          F.row_idx, F.perm, F.col_ptr);
 }
 
 inline unsigned long long host_mix(unsigned long long z) {
