@@ -138,8 +138,7 @@ template <int B>
 __device__ __forceinline__ void mst_fill_csc_words(int64_t w0, int64_t stride, int64_t w_end, int lane,
                                                    const uint32_t* bitsT, const int32_t* wscanT, int I, int wpr, int wpc,
                                                    const uint32_t* bits, const int32_t* wscan, uint16_t* row_idx,
-                                                   int32_t* perm, int32_t* col_ptr) {
-  const int64_t nwordsT = (int64_t)I * wpc;
+                                                   int32_t* perm, int32_t* col_ptr, int32_t total) {
   uint32_t b[B], fb[B];
   int32_t base[B], fs[B];
   int ii[B], wrr[B];
@@ -169,7 +168,7 @@ __device__ __forceinline__ void mst_fill_csc_words(int64_t w0, int64_t stride, i
     if (w >= w_end) continue;
     if (wrr[j] == 0 && lane == 0) {
       col_ptr[ii[j]] = base[j];
-      if (ii[j] == I - 1) col_ptr[I] = wscanT[nwordsT];
+      if (ii[j] == I - 1) col_ptr[I] = total;  // the scan's last element, known to every block
     }
     if ((b[j] >> lane) & 1u) {
       const int32_t posT = base[j] + __popc(b[j] & mst_lanemask_lt());

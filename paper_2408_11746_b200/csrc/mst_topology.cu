@@ -355,7 +355,7 @@ __device__ __forceinline__ int fused_block_excl_scan(int v, int& total, FusedSha
 }
 
 // out[0..n] = exclusive scan of cnt[0..n); each block scans its slice [lo, hi).  One grid barrier inside.
-__device__ void fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int64_t lo, int64_t hi, int32_t* bsums,
+__device__ int fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int64_t lo, int64_t hi, int32_t* bsums,
                                 cg::grid_group& grid, FusedShared& sh) {
   int v = 0;
   for (int64_t i = lo + threadIdx.x; i < hi; i += FUSED_THREADS) v += cnt[i];
@@ -381,6 +381,7 @@ __device__ void fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int
   }
   if (blockIdx.x == 0 && threadIdx.x == 0) out[n] = tot;
   __syncthreads();
+  return tot;
 }
 
 // One selection inside the fused kernel.  gpass counts the histogram passes executed so far (buffer rotation).
@@ -567,23 +568,22 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   }
   __syncthreads();
   fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, grid, sh);
-  grid.sync();  // new mask and its scan are complete everywhere
-  for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * 4)
-    mst_fill_csr_words<V, 4>(w0, FUSED_WARPS, hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col, (V*)F.new_vals,
-                             F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals, &F.flags[1]);
+  // the barrier inside the scan came after every block wrote its part of the new mask: transpose it now
   {
     const int64_t tiles = (int64_t)F.wpc * P.wpr;
     for (int64_t t = (int64_t)blockIdx.x * FUSED_WARPS + warp; t < tiles; t += (int64_t)gridDim.x * FUSED_WARPS)
       mst_transpose_tile(t, lane, F.new_bits, P.O, P.I, P.wpr, F.wpc, F.bitsT);
   }
-  grid.sync();  // transposed mask complete
+  grid.sync();  // transposed mask and the scan of the new mask are complete everywhere
+  for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * 4)
+    mst_fill_csr_words<V, 4>(w0, FUSED_WARPS, hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col, (V*)F.new_vals,
+                             F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals, &F.flags[1]);
   for (int64_t w = loT + threadIdx.x; w < hiT; w += FUSED_THREADS) F.cnt[w] = __popc(F.bitsT[w]);
   __syncthreads();
-  fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, grid, sh);
-  grid.sync();  // col_ptr[I] needs the scan's last element, written by block 0
+  const int totT = fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, grid, sh);
   for (int64_t w0 = loT + warp; w0 < hiT; w0 += FUSED_WARPS * 4)
     mst_fill_csc_words<4>(w0, FUSED_WARPS, hiT, lane, F.bitsT, F.wscanT, P.I, P.wpr, F.wpc, F.new_bits, F.new_wscan,
-                          F.row_idx, F.perm, F.col_ptr);
+                          F.row_idx, F.perm, F.col_ptr, totT);
 }
 
 inline unsigned long long host_mix(unsigned long long z) {
