@@ -139,6 +139,90 @@ def cpu_baseline(tokens: int):
             "sample": "first %d of 8192 tokens of every layer, whole path once (%.1f s)" % (tokens, dt)}
 
 
+# ------------------------------------------------------------------------------------------ density sweep report
+def run_sweep(args) -> None:
+    """Forward + input gradient + weight gradient per (layer, density): time of the CUDA-core sparse kernels, of the
+    dense-tile tensor-core kernels and of the automatic choice, useful TFLOP/s, fraction of the roofline
+    max(useful flops / pipe peak, compulsory bytes / HBM bandwidth), and torch.matmul (cuBLAS bf16) on the same
+    shapes as the density-crossover reference.  Inputs are rotated over enough buffer sets to exceed L2."""
+    import torch
+    import paper_2408_11746_b200 as mst
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = measured_peaks()
+    width = mst_inputs.GPT2_WIDTH[args.sweep]
+    T = 8192 if args.sweep == "small" else 16384
+    densities = (1.0, 0.5, 0.25, 0.1, 0.05, 0.02)
+    reps = max(args.steps, 10)
+
+    def time_ms(fns):
+        """median time of each callable in fns, interleaved, CUDA events on the current stream"""
+        for f in fns:
+            for _ in range(3):
+                f()
+        torch.cuda.synchronize()
+        out = []
+        for f in fns:
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+            for a, b in ev:
+                a.record(); f(); b.record()
+            torch.cuda.synchronize()
+            ts = sorted(a.elapsed_time(b) for a, b in ev)
+            out.append(ts[len(ts) // 2])
+        return out
+
+    for li, (name, O, I) in enumerate(mst_inputs.block_shapes(width)):
+        nset = max(2, int(300e6 // (2 * T * (O + I) * 2)) + 1)      # buffer sets so that one round exceeds L2 twice over
+        Xs = [torch.randn(T, I, device=dev, dtype=torch.bfloat16) for _ in range(nset)]
+        dYs = [(torch.randn(T, O, device=dev, dtype=torch.bfloat16) * 1e-2) for _ in range(nset)]
+        Y = torch.empty(T, O, device=dev, dtype=torch.bfloat16)
+        dX = torch.empty(T, I, device=dev, dtype=torch.bfloat16)
+        Wd = (torch.randn(O, I, device=dev) * 0.02).to(torch.bfloat16)
+        ctr = [0]
+
+        def nxt():
+            ctr[0] = (ctr[0] + 1) % nset
+            return Xs[ctr[0]], dYs[ctr[0]]
+
+        def dense_all():
+            X, dY = nxt()
+            torch.matmul(X, Wd.t(), out=Y); torch.matmul(dY, Wd, out=dX); torch.matmul(dY.t(), X)
+        (t_dense,) = time_ms([dense_all])
+        for d in densities:
+            nnz = mst_inputs.exact_nnz(O, I, d)
+            mask = torch.from_numpy(mst_inputs.uniform_mask(O, I, nnz, mst_inputs.BASE_SEED + 5, li)).to(dev)
+            L = mst.Layer(li, O, I, mst.MST_BF16)
+            L.pack(Wd, mask)
+            dW = torch.empty(max(nnz, 1), device=dev, dtype=torch.float32)
+
+            def all3():
+                X, dY = nxt()
+                L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW)
+            res = {}
+            for pname, pid in (("cuda_core", mst.MST_PATH_CUDA_CORE), ("tensor_core", mst.MST_PATH_TENSOR_CORE),
+                               ("auto", mst.MST_PATH_AUTO)):
+                if pname == "cuda_core" and d > 0.3:
+                    continue                      # minutes of FMA work at these sizes; the crossover is far below
+                L.set_path(pid)
+                (res[pname],) = time_ms([all3])
+            L.close()
+            useful = 6.0 * T * nnz
+            byts = 3 * 2 * T * (O + I) + nnz * (3 * 4 + 4 + 4) + 12 * (O + 1)
+            t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
+            auto_pipe = "tensor"
+            pipe_peak = peaks["bf16_tflops_sustained"] if auto_pipe == "tensor" else FMA_PEAK_TFLOPS
+            t_roof = max(t_hbm, useful / (pipe_peak * 1e12))
+            print(json.dumps({
+                "layer": name, "O": O, "I": I, "T": T, "density": d, "nnz": nnz,
+                "ms": {k: round(v, 4) for k, v in res.items()}, "dense_cublas_ms": round(t_dense, 4),
+                "useful_tflops_auto": round(useful / (res["auto"] * 1e-3) / 1e12, 2),
+                "compulsory_gbs_auto": round(byts / (res["auto"] * 1e-3) / 1e9, 1),
+                "roofline": {"bound": "hbm" if t_hbm >= useful / (pipe_peak * 1e12) else auto_pipe,
+                             "frac": round(t_roof / (res["auto"] * 1e-3), 4), "pipe": auto_pipe},
+                "speedup_vs_dense_cublas": round(t_dense / res["auto"], 3)}), flush=True)
+
+
+
 # ------------------------------------------------------------------------------------------ our arm
 def main() -> None:
     ap = argparse.ArgumentParser()
@@ -149,10 +233,16 @@ def main() -> None:
     ap.add_argument("--ref-tokens", type=int, default=48, help="tokens per layer in one reference-arm step")
     ap.add_argument("--cpu-tokens", type=int, default=3072, help="tokens per layer in the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default=None, choices=["medium", "large", "small"],
+                    help="density sweep report on one block's FC shapes (not the bench line): one JSON object per "
+                         "(layer, density) with both kernel families and a dense cuBLAS GEMM beside them")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
 
     import torch
@@ -261,7 +351,7 @@ def main() -> None:
     def algorithmic(name, s):
         """(useful flops, compulsory bytes, pipe) of one call on layer slot s."""
         x, y, idx = T * s.I * es, T * s.O * es, s.nnz * (es + 2) + 4 * (s.O + 1)
-        pipe = "tensor" if s.nnz >= 0.04 * s.O * s.I else "alu"
+        pipe = "tensor"          # bf16 layers run on the dense-tile tensor-core kernels at every density
         if name == "spmm_fwd": return 2.0 * T * s.nnz, x + y + idx, pipe
         if name == "spmm_bwd_x": return 2.0 * T * s.nnz, x + y + idx + 4 * s.nnz, pipe
         if name == "sddmm_dw": return 2.0 * T * s.nnz, x + y + s.nnz * 2 + 4 * (s.O + 1) + 4 * s.nnz, pipe
@@ -300,7 +390,7 @@ def main() -> None:
     dom_family = max(fam_ms, key=fam_ms.get)
     dom = max((n for n in KERNELS if family[n] == dom_family), key=lambda n: per[n]["ms_per_step"])
     roof = dict(rooflines[dom])
-    tensor_path = all(s.nnz >= 0.04 * s.O * s.I for s in slots)
+    tensor_path = True
     roof["kernel"] = ("tc_gemm_pair_kernel" if tensor_path else "spmm/sddmm CUDA-core kernels") + " as " + dom \
         if dom_family == "contraction" else "mg_update_fused_kernel"
     roof["family_ms_per_step"] = fam_ms
