@@ -31,6 +31,8 @@ struct SelParams {
   const uint32_t* pruned_bits;
   const uint32_t* grad_bits;
   int O, I, wpr, allow;
+  int aligned;   // I % 32 == 0
+  int low_zero;  // low key bits known to be zero in the prune keys (16 for bf16 values)
   int64_t nwords;
   unsigned long long stream;
 };
@@ -58,8 +60,17 @@ struct KeyBits {
 template <int MODE>
 __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane, unsigned long long& key,
                                          bool& nonfinite) {
-  const unsigned wu = (unsigned)w, wpr = (unsigned)P.wpr;   // nwords < 2^31
-  const int o = (int)(wu / wpr), c = (int)(wu - (unsigned)o * wpr) * 32 + lane;
+  // flat index of this bit; when I is a multiple of 32 the mask words tile the flat index space exactly
+  long long f;
+  bool col_ok = true;
+  if (P.aligned) {
+    f = (long long)w * 32 + lane;
+  } else {
+    const unsigned wu = (unsigned)w, wpr = (unsigned)P.wpr;  // nwords < 2^31
+    const int o = (int)(wu / wpr), c = (int)(wu - (unsigned)o * wpr) * 32 + lane;
+    col_ok = c < P.I;
+    f = (long long)o * P.I + c;
+  }
   nonfinite = false;
   key = 0;
   if (MODE == MODE_PRUNE) {
@@ -77,16 +88,15 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
   } else if (MODE == MODE_GRAD) {
     uint32_t word = ~P.old_bits[w];
     if (P.allow) word |= P.pruned_bits[w];
-    if (c >= P.I || !((word >> lane) & 1u)) return false;
-    const uint32_t k = __float_as_uint(P.G[(int64_t)o * P.I + c]) & 0x7FFFFFFFu;
+    if (!col_ok || !((word >> lane) & 1u)) return false;
+    const uint32_t k = __float_as_uint(P.G[f]) & 0x7FFFFFFFu;
     nonfinite = k >= 0x7F800000u;
     key = 0xFFFFFFFFu - k;  // largest magnitude first
     return true;
   } else {
     const uint32_t word = ~P.old_bits[w] & ~P.grad_bits[w];
-    if (c >= P.I || !((word >> lane) & 1u)) return false;
-    const unsigned long long f = (unsigned long long)o * (unsigned long long)P.I + (unsigned long long)c;
-    key = sm64_mix(P.stream + SM64_GAMMA * (f + 1ULL));
+    if (!col_ok || !((word >> lane) & 1u)) return false;
+    key = sm64_mix(P.stream + SM64_GAMMA * ((unsigned long long)f + 1ULL));
     return true;
   }
 }
@@ -487,6 +497,12 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
         sh.rem = k - cum;
         sh.need_rank = 0;
         sh.done = 1;
+      } else if (MODE == MODE_PRUNE && shift <= P.low_zero) {
+        // the undecided low bits are zero in every key: the bucket is one run of equal keys
+        sh.tau = np << shift;
+        sh.rem = k - cum;
+        sh.need_rank = 1;
+        sh.done = 1;
       }
     }
     __syncthreads();
@@ -644,6 +660,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   P.I = L->I;
   P.wpr = L->wpr;
   P.allow = rule->allow_regrow_pruned ? 1 : 0;
+  P.aligned = (L->I % 32 == 0) ? 1 : 0;
+  P.low_zero = L->dtype == MST_BF16 ? 16 : 0;
   P.nwords = L->nwords;
   {  // state of the random-growth generator for (seed, step, layer): three chained SplitMix64 first outputs
     const unsigned long long a = host_mix(rule->seed + SM64_GAMMA);
