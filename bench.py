@@ -81,6 +81,22 @@ class ClockSampler:
                 "power_w_max": max(float(r[2]) for r in rows)}
 
 
+# ------------------------------------------------------------------------------------------ replicas (N > 1)
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: every replica runs the same independent workload, the job is as slow as the slowest."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(useful_flops_per_step: float, steps: int, world: int, ms: float) -> float:
+    """Whole-job useful TFLOP/s: `world` independent replicas each did `steps` steps in `ms` (max over ranks)."""
+    return useful_flops_per_step * steps * world / (ms * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 def run_reference(args) -> None:
     """Time the CPU checker, as it stands, on a bounded sample of the workload (rank 0 only)."""
@@ -332,13 +348,9 @@ def main() -> None:
     barrier()
     w1 = time.time()
     clocks = sampler.stop(w0, w1)
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
     useful = 6.0 * T * sum(s.nnz for s in slots)          # per step, per replica
-    value = useful * args.steps * world / (ms * 1e-3) / 1e12
+    value = aggregate_value(useful, args.steps, world, ms)
 
     # ---- per-kernel summary and the roofline of the dominant kernel
     per = {}
@@ -419,14 +431,10 @@ def main() -> None:
         e2e_step(1 + k)
     b = ev()
     barrier()
-    e2e_ms = a.elapsed_time(b)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(a.elapsed_time(b), dist, dev)
     h2d = sum(T * (s.I + s.O) * es for s in slots)
     d2h = sum(T * (s.I + s.O) * es + 4 * s.nnz for s in slots)
-    e2e = {"value": useful * e2e_steps * world / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    e2e = {"value": aggregate_value(useful, e2e_steps, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps}
 
     launches_per_layer = 9            # densify+contraction (fwd), same (bwd_x), contraction+reduce (sddmm, dense_grad), fused update
