@@ -135,6 +135,14 @@ mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy
 mst_status_t mst_dense_grad(const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T, int32_t out_features,
                             int32_t in_features, mst_dtype_t dtype, float* G, mst_stream_t stream);
 
+/* Weight gradient on the mask read out of a dense gradient: dW[k] = G[o_k, i_k] (CSR order).  On steps that compute
+ * the dense gradient anyway (every topology-update step: Algorithm 1 needs |grad L| on the empty slots and the
+ * optimizer needs it on the active ones) the separate SDDMM contraction is redundant.
+ * mst_dense_grad_dw = mst_dense_grad followed by this sampling: both G [O x I] and dW_vals [nnz] are written. */
+mst_status_t mst_sddmm_from_dense(const mst_layer_t* layer, const float* G_dense, float* dW_vals, mst_stream_t stream);
+mst_status_t mst_dense_grad_dw(const mst_layer_t* layer, const void* dY, int64_t lddy, const void* X, int64_t ldx,
+                               int64_t T, float* G_dense, float* dW_vals, mst_stream_t stream);
+
 /* Counts of one update (Algorithm 1, count lines), as the library computes them on the host:
  *   n_prune = clamp(floor(prune_frac * nnz), max(0, nnz - target), min(nnz, N - target)),
  *   n_grow = n_prune + target - nnz, n_rand = floor(n_grow * R), n_grad = n_grow - n_rand.

@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
-           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad",
+           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_status_string"]
 
@@ -65,6 +65,8 @@ _sig = {
     "mst_spmm_bwd_x": [_vp, _vp, _i64, _i64, _vp, _i64, _vp],
     "mst_sddmm_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp],
     "mst_dense_grad": [_vp, _i64, _vp, _i64, _i64, _i32, _i32, ctypes.c_int, _vp, _vp],
+    "mst_sddmm_from_dense": [_vp, _vp, _vp, _vp],
+    "mst_dense_grad_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp, _vp],
     "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
     "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
@@ -171,6 +173,15 @@ def mst_dense_grad(dY, lddy: int, X, ldx: int, T: int, out_features: int, in_fea
                                _stream(stream)), "mst_dense_grad")
 
 
+def mst_sddmm_from_dense(layer: int, G_dense, dW_vals, stream=None) -> None:
+    _check(_lib.mst_sddmm_from_dense(layer, _ptr(G_dense), _ptr(dW_vals), _stream(stream)), "mst_sddmm_from_dense")
+
+
+def mst_dense_grad_dw(layer: int, dY, lddy: int, X, ldx: int, T: int, G_dense, dW_vals, stream=None) -> None:
+    _check(_lib.mst_dense_grad_dw(layer, _ptr(dY), lddy, _ptr(X), ldx, T, _ptr(G_dense), _ptr(dW_vals),
+                                  _stream(stream)), "mst_dense_grad_dw")
+
+
 def mst_update_counts(prune_frac: float, nnz: int, target_nnz: int, numel: int, random_ratio: float):
     """(n_prune, n_grow, n_rand, n_grad)."""
     out = (_i64 * 4)()
@@ -255,6 +266,9 @@ class Layer:
     def dense_grad(self, dY, X, T: int, G, stream=None) -> None:
         mst_dense_grad(dY, self.out_features, X, self.in_features, T, self.out_features, self.in_features, self.dtype,
                        G, stream)
+
+    def dense_grad_dw(self, dY, X, T: int, G, dW_vals, stream=None) -> None:
+        mst_dense_grad_dw(self.handle, dY, self.out_features, X, self.in_features, T, G, dW_vals, stream)
 
     def update(self, prune_frac: float, **kw):
         return mst_topology_update(self.handle, prune_frac, **kw)

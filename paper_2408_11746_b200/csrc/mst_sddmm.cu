@@ -8,6 +8,7 @@
 // sum of entry j in lane j, which adds it to that entry's fp32 accumulator in shared memory.  The upstream-gradient
 // operands of a row stay in registers while consecutive entries share the row.  Every entry is owned by exactly one
 // warp and one lane, the token order is fixed: no atomics, deterministic.
+#include "mst_bits.cuh"
 #include "mst_internal.cuh"
 #include "mst_tc_gemm.cuh"
 
@@ -167,6 +168,19 @@ sddmm_window_kernel(const int32_t* __restrict__ row_ptr, const uint16_t* __restr
   }
 }
 
+// dW on the mask read out of a dense gradient: one warp per mask word, lane = column.
+__global__ void sample_dense_kernel(const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan, int O, int I,
+                                    int wpr, const float* __restrict__ G, float* __restrict__ dW) {
+  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= (int64_t)O * wpr) return;
+  const uint32_t b = bits[w];
+  if (!((b >> lane) & 1u)) return;
+  const unsigned wu = (unsigned)w;
+  const int o = (int)(wu / (unsigned)wpr), c = (int)(wu - (unsigned)o * (unsigned)wpr) * 32 + lane;
+  dW[wscan[w] + __popc(b & mst_lanemask_lt())] = G[(int64_t)o * I + c];
+}
+
 template <typename T>
 mst_status_t launch(const mst_layer* L, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T_total,
                     float* dW, cudaStream_t s) {
@@ -216,4 +230,25 @@ extern "C" mst_status_t mst_sddmm_dw(const mst_layer_t* L, const void* dY, int64
   if (L->nnz < 0) return MST_ERR_NOT_PACKED;
   if (lddy < L->O || ldx < L->I) return MST_ERR_SHAPE;
   return mst_launch_sddmm(L, dY, lddy, X, ldx, T, dW_vals, (cudaStream_t)stream);
+}
+
+extern "C" mst_status_t mst_sddmm_from_dense(const mst_layer_t* L, const float* G_dense, float* dW_vals,
+                                             mst_stream_t stream) {
+  if (!L || !G_dense || !dW_vals) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  if (L->nnz == 0) return MST_OK;
+  const int c = L->cur;
+  const int64_t threads = L->nwords * 32;
+  sample_dense_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      L->bits[c], L->wscan[c], L->O, L->I, L->wpr, G_dense, dW_vals);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_dense_grad_dw(const mst_layer_t* L, const void* dY, int64_t lddy, const void* X, int64_t ldx,
+                                          int64_t T, float* G_dense, float* dW_vals, mst_stream_t stream) {
+  if (!L || !G_dense || !dW_vals) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  MST_TRY(mst_dense_grad(dY, lddy, X, ldx, T, L->O, L->I, L->dtype, G_dense, stream));
+  return mst_sddmm_from_dense(L, G_dense, dW_vals, stream);
 }

@@ -265,3 +265,20 @@ def test_dense_grad_tensor_core_path(O, I, T):
     Gr = oracle.dense_grad(p.dY, p.X)
     assert rel_err(host(G), Gr) <= 1e-5          # exact bf16 products, fp32 accumulation
     np.testing.assert_array_equal(host(G).view(np.uint32), host(G2).view(np.uint32))     # deterministic
+
+
+@pytest.mark.parametrize("O,I,T,dtype", [(300, 520, 1000, "bf16"), (130, 257, 200, "f32"), (512, 512, 2048, "bf16")])
+def test_dense_grad_dw_gives_both_gradients(O, I, T, dtype):
+    p = _problem(O, I, T, dtype, 0.15, 6000 + O + I)
+    L = make_layer(p)
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    G = torch.full((O, I), float("nan"), dtype=torch.float32, device=dev())
+    dW = torch.full((p.nnz,), float("nan"), dtype=torch.float32, device=dev())
+    L.dense_grad_dw(dY, X, T, G, dW)
+    torch.cuda.synchronize()
+    Gr = oracle.dense_grad(p.dY, p.X)
+    rows, cols = np.nonzero(p.mask)
+    assert rel_err(host(G), Gr) <= TOL[dtype]
+    assert rel_err(host(dW), Gr[rows, cols]) <= TOL[dtype]
+    np.testing.assert_array_equal(host(dW), host(G)[rows, cols])        # exactly the sampled entries of G
+    L.close()
