@@ -192,6 +192,29 @@ mst_status_t mst_mask_to_csr_noalloc(int32_t out_features, int32_t in_features, 
                                      int64_t ldw, const uint8_t* mask, int64_t nnz_capacity, int32_t* row_ptr,
                                      int32_t* col_idx, void* vals, mst_stream_t stream);
 
+/* ---- Sparsity-Variation driver (host scalars; Sec. 3.1 equations for S_t, Sec. 3.2 for zeta_t and the Erdos-Renyi
+ * split; Table "Private hyperparameters of MST": S_M = 0.96, N = 5, Delta_W = Delta_R = 2000, T_U = 100000,
+ * zeta_1 = 0.3).  The printed equations are garbled; the reading is the cited cubic schedule, stepwise per stage:
+ *   warm-up      t in [0, N*delta_w):           S_t = S_M * (1 - (1 - k/N)^3),  k = floor(t / delta_w)
+ *   ultra-sparse t in [T_W, T_W + t_ultra):     S_t = S_M
+ *   restoration  t' = t - T_W - T_U in [0, N*delta_r):  S_t = S_M * (1 - k/N)^3,  k = floor(t' / delta_r); then 0.
+ * zeta_t = zeta_i / 2 * (1 + cos(pi (t - T_{i-1}) / (T_i - T_{i-1}))) on [T_{i-1}, T_i), T_0 = 0, T_1 = T_W + T_U,
+ * T_{i+1} = T_i + delta_r; zeta_i = zeta_1 * decay^(i-1) (the paper gives only zeta_1; decay = 1: no decay).
+ * mst_er_densities: d_l = eps (I_l + O_l) / (I_l O_l), eps such that sum d_l O_l I_l = global_density * sum O_l I_l;
+ * layers that would exceed 1 become dense and eps is re-solved. */
+typedef struct {
+  double max_sparsity; /* S_M */
+  int32_t n_stages;    /* N */
+  int64_t delta_w;     /* pruning frequency, steps per warm-up stage */
+  int64_t t_ultra;     /* T_U */
+  int64_t delta_r;     /* growing frequency, steps per restoration stage */
+} mst_sv_schedule_t;
+mst_status_t mst_sv_sparsity(const mst_sv_schedule_t* schedule, int64_t step, double* sparsity);
+mst_status_t mst_sv_update_fraction(const mst_sv_schedule_t* schedule, int64_t step, double zeta1, double decay,
+                                    double* zeta);
+mst_status_t mst_er_densities(int32_t n_layers, const int32_t* out_features, const int32_t* in_features,
+                              double global_density, double* densities);
+
 /* Sticky error bits of kernels that run without a layer handle (bit 0: a bounded wait inside the tensor-core
  * contraction expired and the block gave up; its output is then undefined).  Synchronises the device. */
 mst_status_t mst_device_error_flags(int32_t* flags);

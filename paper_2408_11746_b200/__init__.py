@@ -26,7 +26,8 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_mask_to_csr_noalloc",
-           "mst_device_error_flags", "mst_status_string"]
+           "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
+           "mst_status_string"]
 
 
 class MstError(RuntimeError):
@@ -38,6 +39,15 @@ class MstError(RuntimeError):
 class RegrowRule(ctypes.Structure):
     _fields_ = [("target_nnz", ctypes.c_int64), ("random_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
                 ("step", ctypes.c_uint64), ("allow_regrow_pruned", ctypes.c_int32)]
+
+
+class SvSchedule(ctypes.Structure):
+    """S_M, N, Delta_W, T_U, Delta_R of the Sparsity-Variation schedule (paper defaults)."""
+    _fields_ = [("max_sparsity", ctypes.c_double), ("n_stages", ctypes.c_int32), ("delta_w", ctypes.c_int64),
+                ("t_ultra", ctypes.c_int64), ("delta_r", ctypes.c_int64)]
+
+    def __init__(self, max_sparsity=0.96, n_stages=5, delta_w=2000, t_ultra=100000, delta_r=2000):
+        super().__init__(max_sparsity, n_stages, delta_w, t_ultra, delta_r)
 
 
 class UpdateStats(ctypes.Structure):
@@ -71,6 +81,9 @@ _sig = {
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
     "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
     "mst_device_error_flags": [ctypes.POINTER(_i32)],
+    "mst_sv_sparsity": [ctypes.POINTER(SvSchedule), _i64, ctypes.POINTER(_f64)],
+    "mst_sv_update_fraction": [ctypes.POINTER(SvSchedule), _i64, _f64, _f64, ctypes.POINTER(_f64)],
+    "mst_er_densities": [_i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32), _f64, ctypes.POINTER(_f64)],
     "mst_mask_to_csr_noalloc": [_i32, _i32, ctypes.c_int, _vp, _i64, _vp, _i64, _vp, _vp, _vp, _vp],
 }
 for _n, _a in _sig.items():
@@ -203,6 +216,29 @@ def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, ran
 def mst_layer_step_host(layer: int, X_host, dY_host, T: int, Y_host, dX_host, dW_vals_host, stream=None) -> None:
     _check(_lib.mst_layer_step_host(layer, _ptr(X_host), _ptr(dY_host), T, _ptr(Y_host), _ptr(dX_host),
                                     _ptr(dW_vals_host), _stream(stream)), "mst_layer_step_host")
+
+
+def mst_sv_sparsity(schedule: SvSchedule, step: int) -> float:
+    out = _f64()
+    _check(_lib.mst_sv_sparsity(ctypes.byref(schedule), step, ctypes.byref(out)), "mst_sv_sparsity")
+    return out.value
+
+
+def mst_sv_update_fraction(schedule: SvSchedule, step: int, zeta1: float = 0.3, decay: float = 1.0) -> float:
+    out = _f64()
+    _check(_lib.mst_sv_update_fraction(ctypes.byref(schedule), step, zeta1, decay, ctypes.byref(out)),
+           "mst_sv_update_fraction")
+    return out.value
+
+
+def mst_er_densities(shapes, global_density: float):
+    """shapes: [(out_features, in_features), ...] -> per-layer densities."""
+    n = len(shapes)
+    O = (_i32 * n)(*[int(o) for o, _ in shapes])
+    I = (_i32 * n)(*[int(i) for _, i in shapes])
+    d = (_f64 * n)()
+    _check(_lib.mst_er_densities(n, O, I, global_density, d), "mst_er_densities")
+    return [float(x) for x in d]
 
 
 def mst_device_error_flags() -> int:
