@@ -53,13 +53,17 @@ typedef enum {
  *   seed, step          the random-growth ranking is a pure function of (seed, step, layer_id, flat index):
  *                       candidates are ranked by SplitMix64 outputs (smaller first, ties by flat index)
  *   allow_regrow_pruned 0: links pruned in this update are not candidates for growth (default reading);
- *                       1: gradient growth may also pick just-pruned links (such a link keeps its value) */
+ *                       1: gradient growth may also pick just-pruned links (such a link keeps its value)
+ *   prune_grad_weight   lambda >= 0 of the MEST pruning criterion |theta| + lambda |grad| (scheme table); 0 = prune by
+ *                       |theta| alone (Mixed-Growing, SET, RigL).  With lambda != 0 the key is formed in fp32, one
+ *                       rounding per operation, and G_dense is needed even when nothing grows by gradient */
 typedef struct {
   int64_t target_nnz;
   double random_ratio;
   uint64_t seed;
   uint64_t step;
   int32_t allow_regrow_pruned;
+  float prune_grad_weight;
 } mst_regrow_rule_t;
 
 typedef struct {

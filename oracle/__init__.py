@@ -63,7 +63,7 @@ def lib():
             L.mst_oracle_mg_counts.argtypes = [ctypes.c_double, _i64, _i64, _i64, ctypes.c_double, _ip]
             L.mst_oracle_mg_counts.restype = ctypes.c_int
             L.mst_oracle_mg_update.argtypes = [_i64, _i64, _fp, _bp, _fp, _i64, _i64, _i64, _u64, _u64, _i64,
-                                               ctypes.c_int, _ip, _ip, _ip]
+                                               ctypes.c_int, _ip, _ip, _ip, ctypes.c_float]
             L.mst_oracle_mg_update.restype = ctypes.c_int
             _lib = L
     return _lib
@@ -190,7 +190,7 @@ class NonFinite(ValueError):
 
 
 def mg_update(W, M, G: Optional[np.ndarray], n_prune: int, n_grad: int, n_rand: int, seed: int, step: int,
-              layer_id: int, allow_regrow_pruned: bool = False):
+              layer_id: int, allow_regrow_pruned: bool = False, prune_grad_weight: float = 0.0):
     """One Mixed-Growing update.  Returns (W_new f32 [O,I], M_new u8 [O,I], I_prune, I_grad, I_rand)."""
     W = np.array(W, dtype=np.float32, order="C", copy=True)
     M = np.array(M, dtype=np.uint8, order="C", copy=True)
@@ -206,7 +206,7 @@ def mg_update(W, M, G: Optional[np.ndarray], n_prune: int, n_grad: int, n_rand: 
     ir = np.zeros(max(n_rand, 1), dtype=np.int64)
     rc = lib().mst_oracle_mg_update(O, I, _p(W, _fp), _p(M, _bp), Gp, int(n_prune), int(n_grad), int(n_rand),
                                     int(seed), int(step), int(layer_id), int(bool(allow_regrow_pruned)),
-                                    _p(ip, _ip), _p(ig, _ip), _p(ir, _ip))
+                                    _p(ip, _ip), _p(ig, _ip), _p(ir, _ip), float(prune_grad_weight))
     if rc == 1:
         raise NonFinite("non-finite |w| or |g| in a selection key")
     if rc != 0:

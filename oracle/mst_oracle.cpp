@@ -172,7 +172,7 @@ static inline uint32_t abs_bits(float v) {
 int mst_oracle_mg_update(int64_t O, int64_t I, float* W, uint8_t* M, const float* G,
                          int64_t n_prune, int64_t n_grad, int64_t n_rand,
                          uint64_t seed, uint64_t step, int64_t layer_id, int allow_regrow_pruned,
-                         int64_t* I_prune, int64_t* I_grad, int64_t* I_rand) {
+                         int64_t* I_prune, int64_t* I_grad, int64_t* I_rand, float prune_grad_weight) {
   const int64_t N = O * I;
   typedef std::pair<uint64_t, int64_t> KI;
   std::vector<uint8_t> old_mask(M, M + N);
@@ -181,7 +181,15 @@ int mst_oracle_mg_update(int64_t O, int64_t I, float* W, uint8_t* M, const float
   std::vector<KI> act;
   for (int64_t f = 0; f < N; ++f)
     if (old_mask[f]) {
-      const uint32_t k = abs_bits(W[f]);
+      // prune key: |theta| (Mixed-Growing, SET, RigL) or |theta| + lambda |grad| (the MEST column of the scheme
+      // table), the latter formed in float32 with one rounding per operation
+      uint32_t k = abs_bits(W[f]);
+      if (prune_grad_weight != 0.0f) {
+        if (!G) return 2;
+        volatile float prod = prune_grad_weight * std::fabs(G[f]);
+        volatile float sum = std::fabs(W[f]) + prod;
+        k = abs_bits(sum);
+      }
       if (n_prune > 0 && k >= 0x7F800000u) return 1;   // keys are only examined when something is selected
       act.push_back(KI(k, f));
     }

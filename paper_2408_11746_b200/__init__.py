@@ -38,7 +38,8 @@ class MstError(RuntimeError):
 
 class RegrowRule(ctypes.Structure):
     _fields_ = [("target_nnz", ctypes.c_int64), ("random_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
-                ("step", ctypes.c_uint64), ("allow_regrow_pruned", ctypes.c_int32)]
+                ("step", ctypes.c_uint64), ("allow_regrow_pruned", ctypes.c_int32),
+                ("prune_grad_weight", ctypes.c_float)]
 
 
 class SvSchedule(ctypes.Structure):
@@ -204,8 +205,10 @@ def mst_update_counts(prune_frac: float, nnz: int, target_nnz: int, numel: int, 
 
 def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, random_ratio: float = 0.25,
                         seed: int = 0, step: int = 0, allow_regrow_pruned: bool = False, G_dense=None,
+                        prune_grad_weight: float = 0.0,
                         want_stats: bool = True, stream=None) -> Optional[UpdateStats]:
-    rule = RegrowRule(int(target_nnz), float(random_ratio), int(seed), int(step), int(bool(allow_regrow_pruned)))
+    rule = RegrowRule(int(target_nnz), float(random_ratio), int(seed), int(step), int(bool(allow_regrow_pruned)),
+                      float(prune_grad_weight))
     stats = UpdateStats() if want_stats else None
     _check(_lib.mst_topology_update(layer, float(prune_frac), ctypes.byref(rule), _ptr(G_dense),
                                     ctypes.byref(stats) if want_stats else None, _stream(stream)),

@@ -33,6 +33,7 @@ struct SelParams {
   int O, I, wpr, allow;
   int aligned;   // I % 32 == 0
   int low_zero;  // low key bits known to be zero in the prune keys (16 for bf16 values)
+  float lambda;  // MEST prune key |w| + lambda |g| when non-zero
   int64_t nwords;
   unsigned long long stream;
 };
@@ -82,6 +83,10 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
       k = ((uint32_t)(((const uint16_t*)P.vals)[pos] & 0x7FFFu)) << 16;
     else
       k = ((const uint32_t*)P.vals)[pos] & 0x7FFFFFFFu;
+    if (P.lambda != 0.f) {  // MEST criterion, fp32 with one rounding per operation (never contracted to an FMA)
+      const float g = fabsf(P.G[f]);
+      k = __float_as_uint(__fadd_rn(__uint_as_float(k), __fmul_rn(P.lambda, g))) & 0x7FFFFFFFu;
+    }
     nonfinite = k >= 0x7F800000u;
     key = k;
     return true;
@@ -643,7 +648,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   const int64_t n_prune = cnt[0], n_rand = cnt[2], n_grad = cnt[3];
   const int64_t target = rule->target_nnz < 0 ? L->nnz : rule->target_nnz;
   if (target > L->cap) return MST_ERR_CAPACITY;
-  if (n_grad > 0 && !G_dense) return MST_ERR_INVALID_ARG;
+  if (!(rule->prune_grad_weight >= 0.f)) return MST_ERR_INVALID_ARG;
+  if ((n_grad > 0 || (rule->prune_grad_weight != 0.f && n_prune > 0)) && !G_dense) return MST_ERR_INVALID_ARG;
 
   const int c = L->cur, n = c ^ 1;
   MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t) * 4, s));
@@ -661,7 +667,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   P.wpr = L->wpr;
   P.allow = rule->allow_regrow_pruned ? 1 : 0;
   P.aligned = (L->I % 32 == 0) ? 1 : 0;
-  P.low_zero = L->dtype == MST_BF16 ? 16 : 0;
+  P.lambda = rule->prune_grad_weight;
+  P.low_zero = (L->dtype == MST_BF16 && P.lambda == 0.f) ? 16 : 0;
   P.nwords = L->nwords;
   {  // state of the random-growth generator for (seed, step, layer): three chained SplitMix64 first outputs
     const unsigned long long a = host_mix(rule->seed + SM64_GAMMA);

@@ -282,3 +282,27 @@ def test_dense_grad_dw_gives_both_gradients(O, I, T, dtype):
     assert rel_err(host(dW), Gr[rows, cols]) <= TOL[dtype]
     np.testing.assert_array_equal(host(dW), host(G)[rows, cols])        # exactly the sampled entries of G
     L.close()
+
+
+@pytest.mark.parametrize("dtype,fused", [("bf16", "1"), ("f32", "1"), ("bf16", "0")])
+def test_mest_prune_criterion_is_bit_exact(dtype, fused, monkeypatch):
+    # prune key |theta| + lambda |grad| (scheme table, MEST column), formed in fp32 on both sides
+    monkeypatch.setenv("MST_UPDATE_FUSED", fused)
+    O, I = 96, 160
+    p = _problem(O, I, 4, dtype, 0.3, 7100)
+    L = make_layer(p)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    M = p.mask.copy()
+    rng = np.random.default_rng(3)
+    for step in range(3):
+        G = (rng.standard_normal((O, I)) * 0.05).astype(np.float32)
+        st = mst.mst_topology_update(L.handle, 0.3, -1, 0.25, 5, step, False, torch.from_numpy(G).to(dev()),
+                                     prune_grad_weight=0.5)
+        c = oracle.mg_counts(0.3, int(M.sum()), -1, O * I, 0.25)
+        W, M, *_ = oracle.mg_update(W, M, G, c[0], c[3], c[2], 5, step, p.layer_id, False, 0.5)
+        rp, ci, vb = export_csr(L, dtype)
+        rp_r, ci_r, v_r = oracle.to_csr(W, M)
+        np.testing.assert_array_equal(rp, rp_r)
+        np.testing.assert_array_equal(ci, ci_r)
+        np.testing.assert_array_equal(vb, value_bits(v_r, dtype))
+    L.close()

@@ -224,3 +224,27 @@ def test_to_csr_roundtrip():
         D[o, cols] = v[rp[o]:rp[o + 1]]; Mb[o, cols] = 1
     np.testing.assert_array_equal(Mb, M); np.testing.assert_array_equal(D, W)
     np.testing.assert_array_equal(rp, np.concatenate([[0], np.cumsum(M.sum(1))]))
+
+
+def test_mest_prune_key():
+    # Scheme table, MEST column: prune by min(|theta| + lambda |grad|).  Independent float32 reference with numpy.
+    rng = np.random.default_rng(61)
+    W, M, G = _case(rng, 14, 40, 0.4)
+    nnz = int(M.sum())
+    lam = np.float32(0.37)
+    n_prune = nnz // 3
+    _, Mn, ip, _, _ = oracle.mg_update(W, M, G, n_prune, 0, 0, 0, 0, 0, False, float(lam))
+    act = np.nonzero(M.reshape(-1))[0]
+    key = (np.abs(W.reshape(-1)[act]).astype(np.float32) + (lam * np.abs(G.reshape(-1)[act]).astype(np.float32)).astype(np.float32)).astype(np.float32)
+    order = np.lexsort((act, key.view(np.uint32)))
+    np.testing.assert_array_equal(ip, act[order[:n_prune]])
+    # lambda = 0 is the magnitude rule; a huge lambda orders by |grad|
+    _, _, ip0, _, _ = oracle.mg_update(W, M, G, n_prune, 0, 0, 0, 0, 0, False, 0.0)
+    _, _, ipm, _, _ = oracle.mg_update(W, M, None, n_prune, 0, 0, 0, 0, 0)
+    np.testing.assert_array_equal(ip0, ipm)
+    _, _, ipl, _, _ = oracle.mg_update(W, M, G, n_prune, 0, 0, 0, 0, 0, False, 1e6)
+    g = np.abs(G.reshape(-1))
+    surv = np.setdiff1d(act, ipl)
+    assert g[ipl].max() <= g[surv].min() + 1e-6
+    with pytest.raises(ValueError):
+        oracle.mg_update(W, M, None, n_prune, 0, 0, 0, 0, 0, False, 0.5)      # the criterion needs the gradient
