@@ -59,8 +59,8 @@ struct KeyBits {
 
 // candidate test and key of bit `lane` of word w.  nonfinite is set when a magnitude key is Inf/NaN.
 template <int MODE>
-__device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane, unsigned long long& key,
-                                         bool& nonfinite) {
+__device__ __forceinline__ bool cand_key_w(const SelParams& P, int64_t w, int lane, uint32_t old_word, int32_t old_base,
+                                           uint32_t grad_word, unsigned long long& key, bool& nonfinite) {
   // flat index of this bit; when I is a multiple of 32 the mask words tile the flat index space exactly
   long long f;
   bool col_ok = true;
@@ -75,9 +75,9 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
   nonfinite = false;
   key = 0;
   if (MODE == MODE_PRUNE) {
-    const uint32_t word = P.old_bits[w];
+    const uint32_t word = old_word;
     if (!((word >> lane) & 1u)) return false;
-    const int32_t pos = P.old_wscan[w] + __popc(word & lanemask_lt());
+    const int32_t pos = old_base + __popc(word & lanemask_lt());
     uint32_t k;
     if (P.bf16)
       k = ((uint32_t)(((const uint16_t*)P.vals)[pos] & 0x7FFFu)) << 16;
@@ -91,7 +91,7 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
     key = k;
     return true;
   } else if (MODE == MODE_GRAD) {
-    uint32_t word = ~P.old_bits[w];
+    uint32_t word = ~old_word;
     if (P.allow) word |= P.pruned_bits[w];
     if (!col_ok || !((word >> lane) & 1u)) return false;
     const uint32_t k = __float_as_uint(P.G[f]) & 0x7FFFFFFFu;
@@ -99,11 +99,21 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
     key = 0xFFFFFFFFu - k;  // largest magnitude first
     return true;
   } else {
-    const uint32_t word = ~P.old_bits[w] & ~P.grad_bits[w];
+    const uint32_t word = ~old_word & ~grad_word;
     if (!col_ok || !((word >> lane) & 1u)) return false;
     key = sm64_mix(P.stream + SM64_GAMMA * ((unsigned long long)f + 1ULL));
     return true;
   }
+}
+
+// same, with the mask words fetched from global memory
+template <int MODE>
+__device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane, unsigned long long& key,
+                                         bool& nonfinite) {
+  const uint32_t ow = P.old_bits[w];
+  const int32_t ob = MODE == MODE_PRUNE ? P.old_wscan[w] : 0;
+  const uint32_t gw = MODE == MODE_RAND ? P.grad_bits[w] : 0u;
+  return cand_key_w<MODE>(P, w, lane, ow, ob, gw, key, nonfinite);
 }
 
 constexpr int RADIX_BITS = 11;
@@ -402,13 +412,17 @@ __device__ int fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int6
 // One selection inside the fused kernel.  gpass counts the histogram passes executed so far (buffer rotation).
 template <int MODE>
 __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* out_bits, int64_t lo, int64_t hi,
-                             int& gpass, cg::grid_group& grid, FusedShared& sh) {
+                             int& gpass, cg::grid_group& grid, FusedShared& sh, const uint32_t* s_old,
+                             const int32_t* s_base, uint32_t* s_grad) {
   constexpr int KB = KeyBits<MODE>::value;
   constexpr int passes = num_passes(KB);
   const SelParams& P = F.sel;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (k_total <= 0) {  // uniform over the grid
-    for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) out_bits[w] = 0;
+    for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
+      out_bits[w] = 0;
+      if (MODE == MODE_GRAD) s_grad[w - lo] = 0;
+    }
     __syncthreads();
     return;
   }
@@ -441,7 +455,8 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
         const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
         unsigned long long key = 0;
         bool nf = false;
-        const bool c = w < hi && cand_key<MODE>(P, w, lane, key, nf);
+        const int64_t li = w < hi ? w - lo : 0;
+        const bool c = w < hi && cand_key_w<MODE>(P, w, lane, s_old[li], s_base[li], s_grad[li], key, nf);
         saw_nonfinite |= (c && nf);
         live[j] = c && (pass == 0 || (key >> hi_shift) == prefix);
         digit[j] = live[j] ? (unsigned)((key >> shift) & dmask) : (unsigned)BINS;
@@ -530,7 +545,7 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
       unsigned long long key;
       bool nf;
-      const bool c = cand_key<MODE>(P, w, lane, key, nf);
+      const bool c = cand_key_w<MODE>(P, w, lane, s_old[w - lo], s_base[w - lo], s_grad[w - lo], key, nf);
       const unsigned eq = __ballot_sync(0xffffffffu, c && key == tau);
       if (lane == 0) F.cnt[w] = __popc(eq);
     }
@@ -546,7 +561,8 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
       const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
       bool nf = false;
       key[j] = 0;
-      c[j] = w < hi && cand_key<MODE>(P, w, lane, key[j], nf);
+      const int64_t li = w < hi ? w - lo : 0;
+      c[j] = w < hi && cand_key_w<MODE>(P, w, lane, s_old[li], s_base[li], s_grad[li], key[j], nf);
       iseq[j] = c[j] && key[j] == tau;
     }
 #pragma unroll
@@ -557,7 +573,10 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
       const long long rank = need_rank ? (long long)F.scan[w] + __popc(eq & lanemask_lt()) : -1;
       const bool take = c[j] && (key[j] < tau || (iseq[j] && rank < rem));
       const unsigned bits = __ballot_sync(0xffffffffu, take);
-      if (lane == 0) out_bits[w] = bits;
+      if (lane == 0) {
+        out_bits[w] = bits;
+        if (MODE == MODE_GRAD) s_grad[w - lo] = bits;  // the random selection of this block reads it from here
+      }
     }
   }
   __syncthreads();
@@ -576,10 +595,22 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   const int64_t loT = perT * blockIdx.x < F.nwordsT ? perT * blockIdx.x : F.nwordsT;
   const int64_t hiT = loT + perT < F.nwordsT ? loT + perT : F.nwordsT;
 
+  // this block's slice of the old mask and of its scan stays in shared memory for every selection pass
+  extern __shared__ uint32_t s_dyn[];
+  uint32_t* s_old = s_dyn;
+  int32_t* s_base = reinterpret_cast<int32_t*>(s_dyn + per);
+  uint32_t* s_grad = s_dyn + 2 * per;
+  for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
+    s_old[w - lo] = P.old_bits[w];
+    s_base[w - lo] = P.old_wscan[w];
+    s_grad[w - lo] = 0;
+  }
+  __syncthreads();
+
   int gpass = 0;
-  fused_select<MODE_PRUNE>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh);
-  fused_select<MODE_GRAD>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh);
-  fused_select<MODE_RAND>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh);
+  fused_select<MODE_PRUNE>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+  fused_select<MODE_GRAD>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+  fused_select<MODE_RAND>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
 
   // mask rewrite: new = (old & ~pruned) | grad | rand, and its popcounts
   for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
@@ -679,6 +710,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   bool fused = true;
   if (const char* e = getenv("MST_UPDATE_FUSED")) fused = (e[0] != '0');
   int grid_blocks = 0;
+  size_t fused_smem = 0;
   if (fused) {
     int dev = 0, coop = 0, sms = 0, occ = 0;
     const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
@@ -692,6 +724,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
       const int64_t useful = (L->nwords + FUSED_WARPS - 1) / FUSED_WARPS;  // at least one word per warp
       if (grid_blocks > useful) grid_blocks = (int)(useful < 1 ? 1 : useful);
       if ((int64_t)grid_blocks > mst_scan_block_sums_len(L->nwords > L->nwordsT ? L->nwords : L->nwordsT)) fused = false;
+      fused_smem = (size_t)((L->nwords + grid_blocks - 1) / grid_blocks) * 12;  // slice of mask, scan and grad words
+      if (fused_smem > 36 * 1024) fused = false;  // very large layers: kernel-per-phase path
     }
   }
   if (fused) {
@@ -707,7 +741,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     F.wpc = L->wpc; F.nwordsT = L->nwordsT;
     void* args[] = {&F};
     const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
-    MST_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3(grid_blocks), dim3(FUSED_THREADS), args, 0, s));
+    MST_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3(grid_blocks), dim3(FUSED_THREADS), args, fused_smem, s));
   } else {
     MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
     MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
