@@ -406,6 +406,14 @@ def main() -> None:
     roof["kernel"] = ("tc_gemm_pair_kernel" if tensor_path else "spmm/sddmm CUDA-core kernels") + " as " + dom \
         if dom_family == "contraction" else "mg_update_fused_kernel"
     roof["family_ms_per_step"] = fam_ms
+    # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of this call kind on layer fc1 (O=3072, I=768), from the
+    # ncu capture summarised in profiles/tc_gemm_pair_and_fused_update_gpt2small_block_d0.25.md (cold caches; output
+    # rows still sitting in L2 at kernel end are not counted).  Algorithmic bytes of the same launch beside it.
+    NCU_TRAFFIC_FC1 = {"spmm_fwd": 19.39e6, "spmm_bwd_x": 57.57e6, "sddmm_dw": 66.77e6, "dense_grad": 66.66e6}
+    if dom in NCU_TRAFFIC_FC1 and tensor_path:
+        fc1 = next(s for s in slots if s.O == 3072 and s.I == 768)
+        roof["traffic"] = NCU_TRAFFIC_FC1[dom]
+        roof["traffic_launch"] = "fc1 (O=3072, I=768): algorithmic %.2f MB" % (algorithmic(dom, fc1)[1] / 1e6)
     if dom_family == "contraction" and tensor_path:
         # what the tensor pipe itself sustains: executed dense flops of this call kind over its time
         dense_fl = sum(2.0 * T * s.O * s.I for s, _, _ in timers[dom])
