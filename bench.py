@@ -427,10 +427,13 @@ def main() -> None:
 
     # ---- end to end: host buffers in, host results out, through the C ABI
     def e2e_step(k):
+        # all four layers are issued before any wait: a layer's host copies overlap the other layers' kernels
         for s in slots:
-            mst.mst_layer_step_host(s.L.handle, s.Xh, s.dYh, T, s.Yh, s.dXh, s.dWh)
+            mst.mst_layer_step_host_async(s.L.handle, s.Xh, s.dYh, T, s.Yh, s.dXh, s.dWh)
             s.L.dense_grad(s.dY, s.X, T, s.G)
             s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=2, step=k, G_dense=s.G, want_stats=False)
+        for s in slots:
+            mst.mst_layer_step_host_wait(s.L.handle)
     e2e_step(0)
     barrier()
     e2e_steps = max(2, min(args.steps, 5))

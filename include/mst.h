@@ -223,6 +223,15 @@ mst_status_t mst_er_densities(int32_t n_layers, const int32_t* out_features, con
  * contraction expired and the block gave up; its output is then undefined).  Synchronises the device. */
 mst_status_t mst_device_error_flags(int32_t* flags);
 
+/* The same step without the final wait: inputs are copied on a copy-in stream owned by the layer, the three products
+ * run on `stream`, results are copied back on a copy-out stream owned by the layer.  Calls for several layers issued
+ * one after the other overlap one layer's copies with another layer's kernels (host buffers must be pinned for that).
+ * mst_layer_step_host_wait blocks until the layer's results are in host memory.  A layer's next async step waits for
+ * its previous one by itself. */
+mst_status_t mst_layer_step_host_async(mst_layer_t* layer, const void* X_host, const void* dY_host, int64_t T,
+                                       void* Y_host, void* dX_host, float* dW_vals_host, mst_stream_t stream);
+mst_status_t mst_layer_step_host_wait(mst_layer_t* layer);
+
 const char* mst_status_string(mst_status_t status);
 
 #ifdef __cplusplus

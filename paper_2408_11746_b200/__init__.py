@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
-           "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_mask_to_csr_noalloc",
+           "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
            "mst_status_string"]
 
@@ -81,6 +81,8 @@ _sig = {
     "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
     "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
+    "mst_layer_step_host_async": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
+    "mst_layer_step_host_wait": [_vp],
     "mst_device_error_flags": [ctypes.POINTER(_i32)],
     "mst_sv_sparsity": [ctypes.POINTER(SvSchedule), _i64, ctypes.POINTER(_f64)],
     "mst_sv_update_fraction": [ctypes.POINTER(SvSchedule), _i64, _f64, _f64, ctypes.POINTER(_f64)],
@@ -242,6 +244,15 @@ def mst_er_densities(shapes, global_density: float):
     d = (_f64 * n)()
     _check(_lib.mst_er_densities(n, O, I, global_density, d), "mst_er_densities")
     return [float(x) for x in d]
+
+
+def mst_layer_step_host_async(layer: int, X_host, dY_host, T: int, Y_host, dX_host, dW_vals_host, stream=None) -> None:
+    _check(_lib.mst_layer_step_host_async(layer, _ptr(X_host), _ptr(dY_host), T, _ptr(Y_host), _ptr(dX_host),
+                                          _ptr(dW_vals_host), _stream(stream)), "mst_layer_step_host_async")
+
+
+def mst_layer_step_host_wait(layer: int) -> None:
+    _check(_lib.mst_layer_step_host_wait(layer), "mst_layer_step_host_wait")
 
 
 def mst_device_error_flags() -> int:

@@ -133,12 +133,22 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->stg_x = L->stg_dy = L->stg_y = L->stg_dx = nullptr;
   L->stg_dw = nullptr;
   L->stg_tokens = 0;
+  L->async_ready = 0;
   *out = L;
   return MST_OK;
 }
 
 extern "C" mst_status_t mst_layer_destroy(mst_layer_t* L) {
   if (!L) return MST_OK;
+  if (L->async_ready) {
+    cudaStreamSynchronize(L->s_in);
+    cudaStreamSynchronize(L->s_out);
+    cudaStreamDestroy(L->s_in);
+    cudaStreamDestroy(L->s_out);
+    cudaEventDestroy(L->ev_in);
+    cudaEventDestroy(L->ev_compute);
+    cudaEventDestroy(L->ev_out);
+  }
   free_staging(L);
   cudaFree(L->bits[0]);  // base of the single allocation
   delete L;
@@ -175,14 +185,24 @@ extern "C" mst_status_t mst_values(mst_layer_t* L, void** vals, int64_t* nnz) {
   return MST_OK;
 }
 
-extern "C" mst_status_t mst_layer_step_host(mst_layer_t* L, const void* X_host, const void* dY_host, int64_t T,
-                                            void* Y_host, void* dX_host, float* dW_host, mst_stream_t stream) {
+extern "C" mst_status_t mst_layer_step_host_async(mst_layer_t* L, const void* X_host, const void* dY_host, int64_t T,
+                                                  void* Y_host, void* dX_host, float* dW_host, mst_stream_t stream) {
   if (!L || T < 0 || (T > 0 && (!X_host || !dY_host))) return MST_ERR_INVALID_ARG;
   if (L->nnz < 0) return MST_ERR_NOT_PACKED;
   cudaStream_t s = (cudaStream_t)stream;
   const size_t es = mst_elem_size(L->dtype);
+  if (!L->async_ready) {
+    MST_CUDA_TRY(cudaStreamCreateWithFlags(&L->s_in, cudaStreamNonBlocking));
+    MST_CUDA_TRY(cudaStreamCreateWithFlags(&L->s_out, cudaStreamNonBlocking));
+    MST_CUDA_TRY(cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming));
+    MST_CUDA_TRY(cudaEventCreateWithFlags(&L->ev_compute, cudaEventDisableTiming));
+    MST_CUDA_TRY(cudaEventCreateWithFlags(&L->ev_out, cudaEventDisableTiming));
+    L->async_ready = 1;
+  }
   if (T > L->stg_tokens || !L->stg_dw) {
     MST_CUDA_TRY(cudaStreamSynchronize(s));
+    MST_CUDA_TRY(cudaStreamSynchronize(L->s_in));
+    MST_CUDA_TRY(cudaStreamSynchronize(L->s_out));
     free_staging(L);
     const int64_t Ta = T > 0 ? T : 1;
     MST_CUDA_TRY(cudaMalloc(&L->stg_x, es * Ta * L->I));
@@ -192,17 +212,39 @@ extern "C" mst_status_t mst_layer_step_host(mst_layer_t* L, const void* X_host, 
     MST_CUDA_TRY(cudaMalloc((void**)&L->stg_dw, sizeof(float) * L->cap));
     L->stg_tokens = Ta;
   }
+  // inputs travel on the layer's copy-in stream once the previous step has finished with the staging buffers
+  MST_CUDA_TRY(cudaStreamWaitEvent(L->s_in, L->ev_out, 0));
   if (T > 0) {
-    MST_CUDA_TRY(cudaMemcpyAsync(L->stg_x, X_host, es * T * L->I, cudaMemcpyHostToDevice, s));
-    MST_CUDA_TRY(cudaMemcpyAsync(L->stg_dy, dY_host, es * T * L->O, cudaMemcpyHostToDevice, s));
+    MST_CUDA_TRY(cudaMemcpyAsync(L->stg_x, X_host, es * T * L->I, cudaMemcpyHostToDevice, L->s_in));
+    MST_CUDA_TRY(cudaMemcpyAsync(L->stg_dy, dY_host, es * T * L->O, cudaMemcpyHostToDevice, L->s_in));
   }
+  MST_CUDA_TRY(cudaEventRecord(L->ev_in, L->s_in));
+  MST_CUDA_TRY(cudaStreamWaitEvent(s, L->ev_in, 0));
   MST_TRY(mst_launch_spmm(L, false, L->stg_x, L->I, T, L->stg_y, L->O, s));
   MST_TRY(mst_launch_spmm(L, true, L->stg_dy, L->O, T, L->stg_dx, L->I, s));
   MST_TRY(mst_launch_sddmm(L, L->stg_dy, L->O, L->stg_x, L->I, T, L->stg_dw, s));
-  if (T > 0 && Y_host) MST_CUDA_TRY(cudaMemcpyAsync(Y_host, L->stg_y, es * T * L->O, cudaMemcpyDeviceToHost, s));
-  if (T > 0 && dX_host) MST_CUDA_TRY(cudaMemcpyAsync(dX_host, L->stg_dx, es * T * L->I, cudaMemcpyDeviceToHost, s));
+  MST_CUDA_TRY(cudaEventRecord(L->ev_compute, s));
+  // results travel back on the copy-out stream while the caller's stream goes on with the next layer
+  MST_CUDA_TRY(cudaStreamWaitEvent(L->s_out, L->ev_compute, 0));
+  if (T > 0 && Y_host) MST_CUDA_TRY(cudaMemcpyAsync(Y_host, L->stg_y, es * T * L->O, cudaMemcpyDeviceToHost, L->s_out));
+  if (T > 0 && dX_host) MST_CUDA_TRY(cudaMemcpyAsync(dX_host, L->stg_dx, es * T * L->I, cudaMemcpyDeviceToHost, L->s_out));
   if (dW_host && L->nnz > 0)
-    MST_CUDA_TRY(cudaMemcpyAsync(dW_host, L->stg_dw, sizeof(float) * L->nnz, cudaMemcpyDeviceToHost, s));
-  MST_CUDA_TRY(cudaStreamSynchronize(s));
+    MST_CUDA_TRY(cudaMemcpyAsync(dW_host, L->stg_dw, sizeof(float) * L->nnz, cudaMemcpyDeviceToHost, L->s_out));
+  MST_CUDA_TRY(cudaEventRecord(L->ev_out, L->s_out));
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_layer_step_host_wait(mst_layer_t* L) {
+  if (!L) return MST_ERR_INVALID_ARG;
+  if (!L->async_ready) return MST_OK;
+  MST_CUDA_TRY(cudaEventSynchronize(L->ev_out));
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_layer_step_host(mst_layer_t* L, const void* X_host, const void* dY_host, int64_t T,
+                                            void* Y_host, void* dX_host, float* dW_host, mst_stream_t stream) {
+  MST_TRY(mst_layer_step_host_async(L, X_host, dY_host, T, Y_host, dX_host, dW_host, stream));
+  MST_TRY(mst_layer_step_host_wait(L));
+  MST_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
   return MST_OK;
 }

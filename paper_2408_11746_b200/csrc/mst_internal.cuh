@@ -76,6 +76,10 @@ struct mst_layer {
   void *stg_x, *stg_dy, *stg_y, *stg_dx;
   float* stg_dw;
   int64_t stg_tokens;
+  // copy streams and events of the asynchronous host step (created on first use)
+  cudaStream_t s_in, s_out;
+  cudaEvent_t ev_in, ev_compute, ev_out;
+  int async_ready;
 };
 
 static inline size_t mst_elem_size(mst_dtype_t d) { return d == MST_F32 ? 4 : 2; }

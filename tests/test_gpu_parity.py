@@ -306,3 +306,28 @@ def test_mest_prune_criterion_is_bit_exact(dtype, fused, monkeypatch):
         np.testing.assert_array_equal(ci, ci_r)
         np.testing.assert_array_equal(vb, value_bits(v_r, dtype))
     L.close()
+
+
+def test_async_host_step_overlaps_layers_and_matches():
+    probs = [_problem(160, 200, 300, "bf16", 0.2, 8100), _problem(96, 256, 300, "bf16", 0.1, 8200)]
+    layers, bufs, want = [], [], []
+    for p in probs:
+        L = make_layer(p)
+        want.append(_run_products(p, L)[:3])
+        T, O, I = p.tokens, p.out_features, p.in_features
+        b = dict(X=torch.from_numpy(p.X_bits.view(np.int16)).pin_memory(), dY=torch.from_numpy(p.dY_bits.view(np.int16)).pin_memory(),
+                 Y=torch.empty((T, O), dtype=torch.int16).pin_memory(), dX=torch.empty((T, I), dtype=torch.int16).pin_memory(),
+                 dW=torch.empty((p.nnz,), dtype=torch.float32).pin_memory())
+        layers.append(L); bufs.append(b)
+    for rep in range(2):                       # the second round reuses the staging buffers of the first
+        for p, L, b in zip(probs, layers, bufs):
+            b["Y"].zero_(); b["dX"].zero_(); b["dW"].zero_()
+            mst.mst_layer_step_host_async(L.handle, b["X"], b["dY"], p.tokens, b["Y"], b["dX"], b["dW"])
+        for L in layers:
+            mst.mst_layer_step_host_wait(L.handle)
+        for (Y, dX, dW), b in zip(want, bufs):
+            np.testing.assert_array_equal(mst_inputs.bf16_bits_to_f32(b["Y"].numpy().view(np.uint16)), Y)
+            np.testing.assert_array_equal(mst_inputs.bf16_bits_to_f32(b["dX"].numpy().view(np.uint16)), dX)
+            np.testing.assert_array_equal(b["dW"].numpy(), dW)
+    for L in layers:
+        L.close()
