@@ -331,3 +331,31 @@ def test_async_host_step_overlaps_layers_and_matches():
             np.testing.assert_array_equal(b["dW"].numpy(), dW)
     for L in layers:
         L.close()
+
+
+@pytest.mark.parametrize("T", [0, 1, 127, 129])
+def test_token_count_edges_on_the_tensor_path(T):
+    O, I = 256, 192
+    p = _problem(O, I, max(T, 1), "bf16", 0.2, 9000 + T)
+    L = make_layer(p)
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    Y = torch.full((max(T, 1), O), 7.0, dtype=torch.bfloat16, device=dev())
+    dX = torch.full((max(T, 1), I), 7.0, dtype=torch.bfloat16, device=dev())
+    dW = torch.full((p.nnz,), 7.0, dtype=torch.float32, device=dev())
+    G = torch.full((O, I), 7.0, dtype=torch.float32, device=dev())
+    L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW); L.dense_grad(dY, X, T, G)
+    torch.cuda.synchronize()
+    if T == 0:                                  # nothing to contract: gradients are zero, activations untouched
+        assert float(dW.abs().max()) == 0.0 and float(G.abs().max()) == 0.0
+        assert float(Y.float().min()) == 7.0 and float(dX.float().min()) == 7.0
+    else:
+        Wm = np.where(p.mask == 1, p.W, np.float32(0))
+        Xs, dYs = p.X[:T], p.dY[:T]
+        assert rel_err(host(Y)[:T], oracle.fwd(Xs, Wm, p.mask)) <= TOL["bf16"]
+        assert rel_err(host(dX)[:T], oracle.bwd_x(dYs, Wm, p.mask)) <= TOL["bf16"]
+        Gr = oracle.dense_grad(dYs, Xs)
+        rows, cols = np.nonzero(p.mask)
+        assert rel_err(host(dW), Gr[rows, cols]) <= TOL["bf16"]
+        assert rel_err(host(G), Gr) <= TOL["bf16"]
+    assert mst.mst_device_error_flags() == 0
+    L.close()
