@@ -143,3 +143,18 @@ def test_config5_density_sweep_gpt2_large_shapes():
             _sampled_products_ok(p, L, rng, mask=mask)
             L.close()
     assert mst.mst_device_error_flags() == 0
+
+
+def test_lm_head_shape_large_out_features():
+    # the output layer of GPT-2 small (768 -> 50304) is sparsified too in the paper's FLOP model: a very wide O
+    rng = np.random.default_rng(6)
+    O, I, T = 50304, 768, 2048
+    p = mst_inputs.uniform_layer("lm_head", 0, O, I, T, "bf16", 0.1, 4242)
+    L = make_layer(p)
+    assert L.nnz == mst_inputs.exact_nnz(O, I, 0.1)
+    L.validate()
+    G = _sampled_products_ok(p, L, rng)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    _update_and_compare(L, p, W, p.mask.copy(), host(G), 0.3, 0.25, 11, 0)
+    L.close()
+    assert mst.mst_device_error_flags() == 0
