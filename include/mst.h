@@ -127,6 +127,21 @@ mst_status_t mst_spmm_fwd(const mst_layer_t* layer, const void* X, int64_t ldx, 
 mst_status_t mst_spmm_bwd_x(const mst_layer_t* layer, const void* dY, int64_t lddy, int64_t T, void* dX, int64_t lddx,
                             mst_stream_t stream);
 
+/* First layer of the MLP with its activation fused behind the product: H = GELU(X (W.M)^T), GELU(y) = y Phi(y)
+ * with Phi the standard normal distribution function (App. "Hyperparameters": activation GELU, no bias; the MLP
+ * term FLOPs_MLP of the FLOP model is fc1 -> GELU -> fc2).  X device [T x ldx]; H device [T x ldh], layer dtype.
+ * Y_pre (device [T x ldpre], layer dtype) receives the pre-activation X (W.M)^T for the backward pass; NULL to
+ * skip it.  On the tensor path GELU is taken on the fp32 accumulator, before the rounding to bf16. */
+mst_status_t mst_spmm_fwd_gelu(const mst_layer_t* layer, const void* X, int64_t ldx, int64_t T, void* Y_pre,
+                               int64_t ldpre, void* H, int64_t ldh, mst_stream_t stream);
+
+/* Input gradient of the second MLP layer carried through the activation in one pass:
+ * dPre[t,i] = (sum_{o:(o,i) in M} dY[t,o] W[o,i]) * GELU'(Y_pre[t,i]),  GELU'(y) = Phi(y) + y phi(y)
+ * (same passages; chain rule through H = GELU(Y_pre)).  `layer` is the layer that consumed H (fc2), so Y_pre and
+ * dPre have in_features columns: Y_pre device [T x ldpre] (read only), dPre device [T x lddpre], layer dtype. */
+mst_status_t mst_spmm_bwd_x_gelu(const mst_layer_t* layer, const void* dY, int64_t lddy, int64_t T, const void* Y_pre,
+                                 int64_t ldpre, void* dPre, int64_t lddpre, mst_stream_t stream);
+
 /* Weight gradient on the mask only, dW[k] = sum_t dY[t,o_k] X[t,i_k] for the k-th active entry in CSR order
  * (same passage).  dW_vals device float [nnz]. */
 mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,

@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
-           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
+           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
            "mst_status_string"]
@@ -74,6 +74,8 @@ _sig = {
     "mst_validate": [_vp, _vp],
     "mst_spmm_fwd": [_vp, _vp, _i64, _i64, _vp, _i64, _vp],
     "mst_spmm_bwd_x": [_vp, _vp, _i64, _i64, _vp, _i64, _vp],
+    "mst_spmm_fwd_gelu": [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp],
+    "mst_spmm_bwd_x_gelu": [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp],
     "mst_sddmm_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp],
     "mst_dense_grad": [_vp, _i64, _vp, _i64, _i64, _i32, _i32, ctypes.c_int, _vp, _vp],
     "mst_sddmm_from_dense": [_vp, _vp, _vp, _vp],
@@ -177,6 +179,16 @@ def mst_spmm_fwd(layer: int, X, ldx: int, T: int, Y, ldy: int, stream=None) -> N
 
 def mst_spmm_bwd_x(layer: int, dY, lddy: int, T: int, dX, lddx: int, stream=None) -> None:
     _check(_lib.mst_spmm_bwd_x(layer, _ptr(dY), lddy, T, _ptr(dX), lddx, _stream(stream)), "mst_spmm_bwd_x")
+
+
+def mst_spmm_fwd_gelu(layer: int, X, ldx: int, T: int, Y_pre, ldpre: int, H, ldh: int, stream=None) -> None:
+    _check(_lib.mst_spmm_fwd_gelu(layer, _ptr(X), ldx, T, _ptr(Y_pre), ldpre, _ptr(H), ldh,
+                                  _stream(stream)), "mst_spmm_fwd_gelu")
+
+
+def mst_spmm_bwd_x_gelu(layer: int, dY, lddy: int, T: int, Y_pre, ldpre: int, dPre, lddpre: int, stream=None) -> None:
+    _check(_lib.mst_spmm_bwd_x_gelu(layer, _ptr(dY), lddy, T, _ptr(Y_pre), ldpre, _ptr(dPre), lddpre, _stream(stream)),
+           "mst_spmm_bwd_x_gelu")
 
 
 def mst_sddmm_dw(layer: int, dY, lddy: int, X, ldx: int, T: int, dW_vals, stream=None) -> None:
@@ -309,6 +321,12 @@ class Layer:
 
     def bwd_x(self, dY, dX, T: int, stream=None) -> None:
         mst_spmm_bwd_x(self.handle, dY, self.out_features, T, dX, self.in_features, stream)
+
+    def fwd_gelu(self, X, H, T: int, Y_pre=None, stream=None) -> None:
+        mst_spmm_fwd_gelu(self.handle, X, self.in_features, T, Y_pre, self.out_features, H, self.out_features, stream)
+
+    def bwd_x_gelu(self, dY, Y_pre, dPre, T: int, stream=None) -> None:
+        mst_spmm_bwd_x_gelu(self.handle, dY, self.out_features, T, Y_pre, self.in_features, dPre, self.in_features, stream)
 
     def sddmm(self, dY, X, T: int, dW_vals, stream=None) -> None:
         mst_sddmm_dw(self.handle, dY, self.out_features, X, self.in_features, T, dW_vals, stream)

@@ -97,7 +97,8 @@ mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s);
 bool mst_use_tensor_path(const mst_layer* L);
 
 // kernels' launchers
+// act / pre / ldpre: element-wise step fused behind the product (see mst_tc_gemm.cuh); act = 0 for the plain product
 mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in, int64_t ldin, int64_t T, void* out,
-                             int64_t ldout, cudaStream_t s);
+                             int64_t ldout, cudaStream_t s, int act = 0, void* pre = nullptr, int64_t ldpre = 0);
 mst_status_t mst_launch_sddmm(const mst_layer* L, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,
                               float* dW, cudaStream_t s);

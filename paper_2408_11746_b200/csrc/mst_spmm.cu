@@ -191,16 +191,45 @@ mst_status_t launch(const int32_t* ptr, const uint16_t* idx, const void* vals, c
   return MST_OK;
 }
 
+// Element-wise pass behind the CUDA-core product (the tensor path fuses it into its epilogue instead).
+//   GELU:      out = gelu(src) where src = pre if given else out
+//   GELU_GRAD: out = out * gelu'(pre)
+template <typename T>
+__global__ void act_rows_kernel(T* __restrict__ out, int64_t ldout, const T* __restrict__ pre, int64_t ldpre, int64_t rows,
+                                int cols, int act) {
+  const int64_t n = rows * cols;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t t = e / cols;
+    const int c = (int)(e - t * cols);
+    T* o = out + t * ldout + c;
+    if (act == MST_ACT_GELU) {
+      store_out(o, mst_gelu(to_float(*(pre ? pre + t * ldpre + c : o))));
+    } else {
+      store_out(o, to_float(*o) * mst_gelu_grad(to_float(pre[t * ldpre + c])));
+    }
+  }
+}
+
+template <typename T>
+mst_status_t launch_act(void* out, int64_t ldout, const void* pre, int64_t ldpre, int64_t rows, int cols, int act,
+                        cudaStream_t s) {
+  const int64_t n = rows * cols;
+  const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 16);
+  act_rows_kernel<T><<<blocks, 256, 0, s>>>((T*)out, ldout, (const T*)pre, ldpre, rows, cols, act);
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+
 }  // namespace
 
 mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in, int64_t ldin, int64_t T, void* out,
-                             int64_t ldout, cudaStream_t s) {
+                             int64_t ldout, cudaStream_t s, int act, void* pre, int64_t ldpre) {
   if (T == 0) return MST_OK;
   const int c = L->cur;
+  const int rows = transpose ? L->I : L->O, cols = transpose ? L->O : L->I;
   // Dense-tile tensor-core path: expand W.M (or its transpose) to a dense bf16 image, then out = in * image^T.
   if (mst_use_tensor_path(L) && (ldout % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0)) {
     const uint16_t* image = transpose ? L->dense_wt : L->dense_w;
-    const int rows = transpose ? L->I : L->O, cols = transpose ? L->O : L->I;
     if (mst_tc_gemm_usable(in, ldin, image, cols)) {
       MST_TRY(mst_densify(L, transpose, s));
       mst_tc_gemm_args a = {};
@@ -209,17 +238,26 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
       a.M = T; a.N = rows; a.K = cols;
       a.epilogue = MST_TC_OUT_BF16;
       a.out = out; a.ldc = ldout; a.splits = 1;
+      a.act = act; a.pre = pre; a.ldpre = ldpre;
       return mst_tc_gemm(a, s);
     }
   }
+  // CUDA cores: the product lands in the pre-activation buffer when the caller keeps one, else in the output
+  void* prod = (act == MST_ACT_GELU && pre) ? pre : out;
+  const int64_t ldprod = (act == MST_ACT_GELU && pre) ? ldpre : ldout;
+  mst_status_t st;
   if (!transpose) {
-    if (L->dtype == MST_F32)
-      return launch<float, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, out, ldout, T, L->O, L->I, s);
-    return launch<uint16_t, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, out, ldout, T, L->O, L->I, s);
+    st = L->dtype == MST_F32
+             ? launch<float, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, s)
+             : launch<uint16_t, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, s);
+  } else {
+    st = L->dtype == MST_F32
+             ? launch<float, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, s)
+             : launch<uint16_t, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, s);
   }
-  if (L->dtype == MST_F32)
-    return launch<float, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, out, ldout, T, L->I, L->O, s);
-  return launch<uint16_t, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, out, ldout, T, L->I, L->O, s);
+  if (st != MST_OK || act == MST_ACT_NONE) return st;
+  return L->dtype == MST_F32 ? launch_act<float>(out, ldout, pre, ldpre, T, rows, act, s)
+                             : launch_act<uint16_t>(out, ldout, pre, ldpre, T, rows, act, s);
 }
 
 extern "C" mst_status_t mst_spmm_fwd(const mst_layer_t* L, const void* X, int64_t ldx, int64_t T, void* Y, int64_t ldy,
@@ -236,4 +274,22 @@ extern "C" mst_status_t mst_spmm_bwd_x(const mst_layer_t* L, const void* dY, int
   if (L->nnz < 0) return MST_ERR_NOT_PACKED;
   if (lddy < L->O || lddx < L->I) return MST_ERR_SHAPE;
   return mst_launch_spmm(L, true, dY, lddy, T, dX, lddx, (cudaStream_t)stream);
+}
+
+extern "C" mst_status_t mst_spmm_fwd_gelu(const mst_layer_t* L, const void* X, int64_t ldx, int64_t T, void* Y_pre,
+                                          int64_t ldpre, void* H, int64_t ldh, mst_stream_t stream) {
+  if (!L || T < 0 || (T > 0 && (!X || !H))) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  if (ldx < L->I || ldh < L->O || (Y_pre && ldpre < L->O)) return MST_ERR_SHAPE;
+  return mst_launch_spmm(L, false, X, ldx, T, H, ldh, (cudaStream_t)stream, MST_ACT_GELU, Y_pre, ldpre);
+}
+
+extern "C" mst_status_t mst_spmm_bwd_x_gelu(const mst_layer_t* L, const void* dY, int64_t lddy, int64_t T,
+                                            const void* Y_pre, int64_t ldpre, void* dPre, int64_t lddpre,
+                                            mst_stream_t stream) {
+  if (!L || T < 0 || (T > 0 && (!dY || !Y_pre || !dPre))) return MST_ERR_INVALID_ARG;
+  if (L->nnz < 0) return MST_ERR_NOT_PACKED;
+  if (lddy < L->O || lddpre < L->I || ldpre < L->I) return MST_ERR_SHAPE;
+  return mst_launch_spmm(L, true, dY, lddy, T, dPre, lddpre, (cudaStream_t)stream, MST_ACT_GELU_GRAD,
+                         const_cast<void*>(Y_pre), ldpre);
 }

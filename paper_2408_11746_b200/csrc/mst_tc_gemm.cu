@@ -50,6 +50,9 @@ struct Params {
   const int32_t* wscan;
   int wpr;
   int64_t nnz;
+  int act;
+  void* pre;
+  int64_t ldpre;
 };
 
 // ------------------------------------------------------------------------------------------- PTX wrappers
@@ -155,6 +158,50 @@ __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_bas
     tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
     if (!row_ok) continue;
     if (P.epilogue == MST_TC_OUT_BF16) {
+      if (P.act) {
+        uint16_t* pre = reinterpret_cast<uint16_t*>(P.pre) + m * P.ldpre + n;
+        const bool pre_vec = n + 32 <= P.N && ((P.ldpre & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.pre) & 15u) == 0);
+        if (P.act == MST_ACT_GELU) {
+          if (P.pre) {  // keep the pre-activation for the backward pass
+            if (pre_vec) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                uint4 o;
+                o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+                o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+                o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+                o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                reinterpret_cast<uint4*>(pre)[v] = o;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (n + j < P.N) pre[j] = (uint16_t)(pack_bf16(__uint_as_float(r[j]), 0.f) & 0xFFFFu);
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(mst_gelu(__uint_as_float(r[j])));
+        } else {  // multiply by the derivative at the stored pre-activation
+          if (pre_vec) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              const uint4 p4 = reinterpret_cast<const uint4*>(pre)[v];
+              const uint32_t pw[4] = {p4.x, p4.y, p4.z, p4.w};
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const float lo = __uint_as_float(pw[h] << 16), hi = __uint_as_float(pw[h] & 0xFFFF0000u);
+                r[8 * v + 2 * h] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h]) * mst_gelu_grad(lo));
+                r[8 * v + 2 * h + 1] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h + 1]) * mst_gelu_grad(hi));
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n + j < P.N)
+                r[j] = __float_as_uint(__uint_as_float(r[j]) * mst_gelu_grad(__uint_as_float((uint32_t)pre[j] << 16)));
+          }
+        }
+      }
       uint16_t* dst = reinterpret_cast<uint16_t*>(P.out) + m * P.ldc + n;
       if (n + 32 <= P.N && ((P.ldc & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.out) & 15u) == 0)) {
 #pragma unroll
@@ -653,6 +700,10 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   P.wscan = a.wscan;
   P.wpr = a.wpr;
   P.nnz = a.nnz;
+  P.act = a.epilogue == MST_TC_OUT_BF16 ? a.act : 0;
+  P.pre = a.pre;
+  P.ldpre = a.ldpre;
+  if (P.act == MST_ACT_GELU_GRAD && !P.pre) return MST_ERR_INVALID_ARG;
   if (a.epilogue != MST_TC_OUT_BF16) {
     // few output tiles: cut the contraction range so that all SMs work; partial sums go to the shared scratch buffer
     const int64_t works1 = pair ? (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles : (int64_t)P.m_tiles * P.n_tiles;

@@ -18,6 +18,16 @@
 //                       out[wscan[w] + rank] for mask word w = m*wpr + n/32 (needs N-tile offsets multiple of 32)
 enum { MST_TC_OUT_BF16 = 0, MST_TC_OUT_F32 = 1, MST_TC_OUT_SAMPLED = 2 };
 
+// Element-wise step fused into the bf16 epilogue (GPT-2 MLP: fc1 -> GELU -> fc2, erf form):
+//   GELU       out = gelu(acc), optionally pre = acc
+//   GELU_GRAD  out = acc * gelu'(pre)
+enum { MST_ACT_NONE = 0, MST_ACT_GELU = 1, MST_ACT_GELU_GRAD = 2 };
+
+__host__ __device__ inline float mst_gelu(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+__host__ __device__ inline float mst_gelu_grad(float x) {
+  return 0.5f * (1.0f + erff(x * 0.70710678118654752f)) + x * 0.39894228040143268f * expf(-0.5f * x * x);
+}
+
 struct mst_tc_gemm_args {
   const void* A;
   int64_t lda;
@@ -35,6 +45,10 @@ struct mst_tc_gemm_args {
   const int32_t* wscan;  // SAMPLED: exclusive popcount scan of the words
   int wpr;
   int64_t nnz;           // SAMPLED: number of stored entries (partial stride)
+  int act;               // BF16 epilogue only: MST_ACT_NONE / MST_ACT_GELU / MST_ACT_GELU_GRAD
+  void* pre;             // GELU: optional bf16 output for the pre-activation (may be NULL);
+                         // GELU_GRAD: bf16 input holding the pre-activation the derivative is taken at
+  int64_t ldpre;
 };
 
 // Returns MST_ERR_SHAPE when the operands cannot be described to the TMA unit (leading dimension or base address
