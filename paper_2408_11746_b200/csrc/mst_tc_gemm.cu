@@ -6,8 +6,9 @@
 //   warp 1     one lane issues tcgen05.mma (M=128, N=256, K=16 per instruction) from shared-memory descriptors
 //              into one of two 128x256 fp32 accumulators in tensor memory, tcgen05.commit releases the smem stage
 //              ("empty") and, after the last K block, hands the accumulator to the epilogue ("tmem_full");
-//   warps 2-5  epilogue: tcgen05.ld 32 columns at a time (one row per thread), convert / sample / store, then
-//              release the accumulator ("tmem_empty") so the next tile's MMAs overlap this tile's stores.
+//   warps 2-9  epilogue, two warps per tensor-memory lane quarter taking alternate 32-column chunks: tcgen05.ld
+//              (one row per thread), convert / activate / sample / store, then release the accumulator
+//              ("tmem_empty") so the next tile's MMAs overlap this tile's stores.
 // Operands may be K-major ([rows x K] row-major) or MN-major ([K x rows] row-major, as dY and X are for
 // G = dY^T X): the tile is fetched with 64-element-wide boxes either way and described to the tensor core with the
 // matching canonical layout (K-major: 8-row groups 1024 B apart; MN-major: 64-wide blocks one box apart).
@@ -29,7 +30,8 @@ constexpr int A_BYTES = BM * BK * 2;  // 16 KiB
 constexpr int B_BYTES = BN * BK * 2;  // 32 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int BOX_BYTES = 64 * BK * 2;  // one 64-wide MN-major box: 8 KiB
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 8;  // two per tensor-memory lane quarter, alternating 32-column chunks
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
@@ -144,23 +146,57 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Phi(x) and exp(-x^2/2) for the fused activation.  The complementary error function is the five-term rational
+// approximation of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7, far under the bf16 rounding of the
+// result); it shares its exponential with the normal density, and Phi of a negative argument is formed without
+// cancellation.  It costs about a third of erff's instructions; the epilogue is still the slower side of the
+// overlap when an activation is fused (two special-function operations per element).
+__device__ __forceinline__ void phi_fast(float x, float& cdf, float& e) {
+  const float z = fabsf(x) * 0.70710678118654752f;
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
+  e = __expf(-0.5f * x * x);
+  float poly = fmaf(t, 1.061405429f, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  const float q = 0.5f * poly * t * e;  // Phi(-|x|)
+  cdf = x >= 0.0f ? 1.0f - q : q;
+}
+__device__ __forceinline__ float gelu_fast(float x) {
+  float cdf, e;
+  phi_fast(x, cdf, e);
+  return x * cdf;
+}
+__device__ __forceinline__ float gelu_grad_fast(float x) {
+  float cdf, e;
+  phi_fast(x, cdf, e);
+  return fmaf(x * 0.39894228040143268f, e, cdf);
+}
+
 // One 128 x BN accumulator (tensor-memory lanes = rows) -> global memory, 32 columns at a time.
 // q = lane quarter this warp may read, m0/n0 = first row / column of this block's tile.
-__device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_base, int acc, int q, int lane, int64_t m0,
-                                              int n0, int split) {
+// c0 = first chunk this warp takes; the warps of one lane quarter interleave their chunks.
+__device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_base, int acc, int q, int c0, int lane,
+                                              int64_t m0, int n0, int split) {
   const int64_t m = (int64_t)m0 + q * 32 + lane;
   const bool row_ok = m < P.M;
 #pragma unroll 1
-  for (int c = 0; c < BN / 32; ++c) {
+  for (int c = c0; c < BN / 32; c += EPI_WARPS / 4) {
     const int n = n0 + c * 32;
     if (n >= P.N) break;  // uniform
     uint32_t r[32];
+    // derivative mode: the stored pre-activation of this chunk is fetched ahead of the tensor-memory read
+    uint16_t* pre = reinterpret_cast<uint16_t*>(P.pre) + m * P.ldpre + n;
+    const bool pre_vec = n + 32 <= P.N && ((P.ldpre & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.pre) & 15u) == 0);
+    uint4 p4[4];
+    if (P.act == MST_ACT_GELU_GRAD && pre_vec && row_ok) {
+#pragma unroll
+      for (int v = 0; v < 4; ++v) p4[v] = __ldg(reinterpret_cast<const uint4*>(pre) + v);
+    }
     tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
     if (!row_ok) continue;
     if (P.epilogue == MST_TC_OUT_BF16) {
       if (P.act) {
-        uint16_t* pre = reinterpret_cast<uint16_t*>(P.pre) + m * P.ldpre + n;
-        const bool pre_vec = n + 32 <= P.N && ((P.ldpre & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.pre) & 15u) == 0);
         if (P.act == MST_ACT_GELU) {
           if (P.pre) {  // keep the pre-activation for the backward pass
             if (pre_vec) {
@@ -180,25 +216,24 @@ __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_bas
             }
           }
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(mst_gelu(__uint_as_float(r[j])));
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(gelu_fast(__uint_as_float(r[j])));
         } else {  // multiply by the derivative at the stored pre-activation
           if (pre_vec) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
-              const uint4 p4 = reinterpret_cast<const uint4*>(pre)[v];
-              const uint32_t pw[4] = {p4.x, p4.y, p4.z, p4.w};
+              const uint32_t pw[4] = {p4[v].x, p4[v].y, p4[v].z, p4[v].w};
 #pragma unroll
               for (int h = 0; h < 4; ++h) {
                 const float lo = __uint_as_float(pw[h] << 16), hi = __uint_as_float(pw[h] & 0xFFFF0000u);
-                r[8 * v + 2 * h] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h]) * mst_gelu_grad(lo));
-                r[8 * v + 2 * h + 1] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h + 1]) * mst_gelu_grad(hi));
+                r[8 * v + 2 * h] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h]) * gelu_grad_fast(lo));
+                r[8 * v + 2 * h + 1] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h + 1]) * gelu_grad_fast(hi));
               }
             }
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
               if (n + j < P.N)
-                r[j] = __float_as_uint(__uint_as_float(r[j]) * mst_gelu_grad(__uint_as_float((uint32_t)pre[j] << 16)));
+                r[j] = __float_as_uint(__uint_as_float(r[j]) * gelu_grad_fast(__uint_as_float((uint32_t)pre[j] << 16)));
           }
         }
       }
@@ -271,7 +306,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull0 + 8 * a, 1);
-      mbar_init(tempty0 + 8 * a, 4);
+      mbar_init(tempty0 + 8 * a, EPI_WARPS);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -323,6 +358,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 256, operand majors
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.a_mn ? 1 : 0) << 15) |
                              ((uint32_t)(P.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // The issue loop is one thread's serial instruction stream; everything that does not depend on the stage is
+      // formed once here.  K-major: 16 K-elements = 32 bytes further along the swizzled row; MN-major: 16 rows of
+      // 128 bytes.
+      const uint64_t adesc0 = smem_desc(tiles_base, P.a_mn ? BOX_BYTES : 16, 1024);
+      const uint64_t bdesc0 = smem_desc(tiles_base + A_BYTES, P.b_mn ? BOX_BYTES : 16, 1024);
+      const uint32_t a_kstep = (uint32_t)(P.a_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      const uint32_t b_kstep = (uint32_t)(P.b_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       for (int64_t w = blockIdx.x; w < works && !*abort_flag; w += gridDim.x) {
@@ -335,15 +377,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = tiles_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          // descriptors of this stage: the start-address field moves by 16-byte units, nothing else changes
+          const uint64_t ad = adesc0 + (uint64_t)(uint32_t)(s * (STAGE_BYTES >> 4));
+          const uint64_t bd = bdesc0 + (uint64_t)(uint32_t)(s * (STAGE_BYTES >> 4));
+          tc_mma(d_tmem, ad, bd, idesc, kb > kb0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t ad = P.a_mn ? smem_desc(sa + k * (UMMA_K * 128), BOX_BYTES, 1024)
-                                       : smem_desc(sa + k * (UMMA_K * 2), 16, 1024);
-            const uint64_t bd = P.b_mn ? smem_desc(sb + k * (UMMA_K * 128), BOX_BYTES, 1024)
-                                       : smem_desc(sb + k * (UMMA_K * 2), 16, 1024);
-            tc_mma(d_tmem, ad, bd, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-          }
+          for (int k = 1; k < BK / UMMA_K; ++k) tc_mma(d_tmem, ad + (uint64_t)(k * a_kstep), bd + (uint64_t)(k * b_kstep), idesc, 1u);
           tc_commit(empty0 + 8 * s);  // the smem stage is free once these MMAs have read it
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -353,7 +392,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
     int acc = 0;
     uint32_t acc_ph = 0;
@@ -362,7 +401,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = (t / P.n_tiles) * BM, n0 = (t % P.n_tiles) * BN;
       if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile(P, tmem_base, acc, q, lane, m0, n0, split);
+      epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
@@ -391,7 +430,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 //   full[s]   (even block)  two arrivals (one per block's producer, each announcing its own bytes) + TMA bytes of both
 //   empty[s]  (each block)  one arrival, multicast by the even block's tcgen05.commit
 //   tfull[a]  (each block)  one arrival, multicast by tcgen05.commit after the tile's last MMA
-//   tempty[a] (even block)  eight arrivals: the four epilogue warps of both blocks
+//   tempty[a] (even block)  sixteen arrivals: the eight epilogue warps of both blocks
 constexpr int P_STAGES = 6;
 constexpr int PB_BYTES = (BN / 2) * BK * 2;        // this block's half of B: 16 KiB
 constexpr int P_STAGE_BYTES = A_BYTES + PB_BYTES;  // 32 KiB
@@ -460,7 +499,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull0 + 8 * a, 1);
-      mbar_init(tempty0 + 8 * a, 8);
+      mbar_init(tempty0 + 8 * a, 2 * EPI_WARPS);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -516,6 +555,10 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.a_mn ? 1 : 0) << 15) |
                              ((uint32_t)(P.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) |
                              ((uint32_t)((2 * BM) >> 4) << 24);
+      const uint64_t adesc0 = smem_desc(tiles_base, P.a_mn ? BOX_BYTES : 16, 1024);
+      const uint64_t bdesc0 = smem_desc(tiles_base + A_BYTES, P.b_mn ? BOX_BYTES : 16, 1024);
+      const uint32_t a_kstep = (uint32_t)(P.a_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+      const uint32_t b_kstep = (uint32_t)(P.b_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       for (int64_t w = pair; w < works && !*abort_flag; w += npairs) {
@@ -528,15 +571,12 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = tiles_base + s * P_STAGE_BYTES, sb = sa + A_BYTES;
+          // descriptors of this stage: the start-address field moves by 16-byte units, nothing else changes
+          const uint64_t ad = adesc0 + (uint64_t)(uint32_t)(s * (P_STAGE_BYTES >> 4));
+          const uint64_t bd = bdesc0 + (uint64_t)(uint32_t)(s * (P_STAGE_BYTES >> 4));
+          tc_mma_pair(d_tmem, ad, bd, idesc, kb > kb0 ? 1u : 0u);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t ad = P.a_mn ? smem_desc(sa + k * (UMMA_K * 128), BOX_BYTES, 1024)
-                                       : smem_desc(sa + k * (UMMA_K * 2), 16, 1024);
-            const uint64_t bd = P.b_mn ? smem_desc(sb + k * (UMMA_K * 128), BOX_BYTES, 1024)
-                                       : smem_desc(sb + k * (UMMA_K * 2), 16, 1024);
-            tc_mma_pair(d_tmem, ad, bd, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-          }
+          for (int k = 1; k < BK / UMMA_K; ++k) tc_mma_pair(d_tmem, ad + (uint64_t)(k * a_kstep), bd + (uint64_t)(k * b_kstep), idesc, 1u);
           tc_commit_pair(empty0 + 8 * s);  // frees this stage in both blocks
           if (++s == P_STAGES) { s = 0; ph ^= 1u; }
         }
@@ -555,7 +595,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int m0 = (t / P.n_tiles) * (2 * BM) + (int)rank * BM, n0 = (t % P.n_tiles) * BN;
       if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile(P, tmem_base, acc, q, lane, m0, n0, split);
+      epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(in_even_block(tempty0 + 8 * acc));
