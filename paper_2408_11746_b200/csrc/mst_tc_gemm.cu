@@ -34,7 +34,8 @@ constexpr int EPI_WARPS = 8;  // two per tensor-memory lane quarter, alternating
 constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr uint32_t SPIN_LIMIT = 20u * 1000u * 1000u;
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int OUT_BOX_BYTES = 32 * 128;  // one epilogue warp's staging box: 32 rows x 128 bytes
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + EPI_WARPS * OUT_BOX_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 
 __device__ int g_tc_error = 0;  // sticky: 1 = a bounded wait expired
 
@@ -55,6 +56,7 @@ struct Params {
   int act;
   void* pre;
   int64_t ldpre;
+  int tma_out;  // rows leave through shared memory and TMA stores (tensor map tmC) instead of per-thread stores
 };
 
 // ------------------------------------------------------------------------------------------- PTX wrappers
@@ -100,6 +102,22 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       "l"(tm), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+
+// Bulk tensor stores (shared -> global) and their per-thread group bookkeeping.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(x),
+               "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(tm), "r"(src),
+               "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -149,12 +167,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Phi(x) and exp(-x^2/2) for the fused activation.  The complementary error function is the five-term rational
 // approximation of Abramowitz & Stegun 7.1.26 (absolute error below 1.5e-7, far under the bf16 rounding of the
 // result); it shares its exponential with the normal density, and Phi of a negative argument is formed without
-// cancellation.  It costs about a third of erff's instructions; the epilogue is still the slower side of the
-// overlap when an activation is fused (two special-function operations per element).
+// cancellation.  It costs about a third of erff's instructions (flush-to-zero reciprocal and exp2, whose default
+// forms carry denormal handling); the epilogue is still the slower side of the overlap when an activation is fused.
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void phi_fast(float x, float& cdf, float& e) {
   const float z = fabsf(x) * 0.70710678118654752f;
-  const float t = __fdividef(1.0f, fmaf(0.3275911f, z, 1.0f));
-  e = __expf(-0.5f * x * x);
+  const float t = rcp_approx(fmaf(0.3275911f, z, 1.0f));
+  e = ex2_approx(x * x * -0.72134752044448170f);  // exp(-x^2 / 2)
   float poly = fmaf(t, 1.061405429f, -1.453152027f);
   poly = fmaf(poly, t, 1.421413741f);
   poly = fmaf(poly, t, -0.284496736f);
@@ -173,8 +201,53 @@ __device__ __forceinline__ float gelu_grad_fast(float x) {
   return fmaf(x * 0.39894228040143268f, e, cdf);
 }
 
-// One 128 x BN accumulator (tensor-memory lanes = rows) -> global memory, 32 columns at a time.
-// q = lane quarter this warp may read, m0/n0 = first row / column of this block's tile.
+// Activation step of one 32-column chunk held in registers (row m, columns n..n+31).  GELU: r <- gelu(r), the
+// pre-activation going to P.pre when given; GELU_GRAD: r <- r * gelu'(pre), pre already fetched into p4 when pre_vec.
+__device__ __forceinline__ void act_chunk(const Params& P, uint32_t (&r)[32], uint16_t* pre, bool pre_vec, const uint4 (&p4)[4],
+                                          int n) {
+  if (P.act == MST_ACT_GELU) {
+    if (P.pre) {  // keep the pre-activation for the backward pass
+      if (pre_vec) {
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          uint4 o;
+          o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
+          o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+          o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+          o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+          reinterpret_cast<uint4*>(pre)[v] = o;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (n + j < P.N) pre[j] = (uint16_t)(pack_bf16(__uint_as_float(r[j]), 0.f) & 0xFFFFu);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(gelu_fast(__uint_as_float(r[j])));
+  } else {  // multiply by the derivative at the stored pre-activation
+    if (pre_vec) {
+#pragma unroll
+      for (int v = 0; v < 4; ++v) {
+        const uint32_t pw[4] = {p4[v].x, p4[v].y, p4[v].z, p4[v].w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+          const float lo = __uint_as_float(pw[h] << 16), hi = __uint_as_float(pw[h] & 0xFFFF0000u);
+          r[8 * v + 2 * h] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h]) * gelu_grad_fast(lo));
+          r[8 * v + 2 * h + 1] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h + 1]) * gelu_grad_fast(hi));
+        }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (n + j < P.N)
+          r[j] = __float_as_uint(__uint_as_float(r[j]) * gelu_grad_fast(__uint_as_float((uint32_t)pre[j] << 16)));
+    }
+  }
+}
+
+// One 128 x BN accumulator (tensor-memory lanes = rows) -> global memory, 32 columns at a time, each thread storing
+// its own row.  q = lane quarter this warp may read, m0/n0 = first row / column of this block's tile.
 // c0 = first chunk this warp takes; the warps of one lane quarter interleave their chunks.
 __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_base, int acc, int q, int c0, int lane,
                                               int64_t m0, int n0, int split) {
@@ -196,47 +269,7 @@ __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_bas
     tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
     if (!row_ok) continue;
     if (P.epilogue == MST_TC_OUT_BF16) {
-      if (P.act) {
-        if (P.act == MST_ACT_GELU) {
-          if (P.pre) {  // keep the pre-activation for the backward pass
-            if (pre_vec) {
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                uint4 o;
-                o.x = pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]));
-                o.y = pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
-                o.z = pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
-                o.w = pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
-                reinterpret_cast<uint4*>(pre)[v] = o;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (n + j < P.N) pre[j] = (uint16_t)(pack_bf16(__uint_as_float(r[j]), 0.f) & 0xFFFFu);
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(gelu_fast(__uint_as_float(r[j])));
-        } else {  // multiply by the derivative at the stored pre-activation
-          if (pre_vec) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              const uint32_t pw[4] = {p4[v].x, p4[v].y, p4[v].z, p4[v].w};
-#pragma unroll
-              for (int h = 0; h < 4; ++h) {
-                const float lo = __uint_as_float(pw[h] << 16), hi = __uint_as_float(pw[h] & 0xFFFF0000u);
-                r[8 * v + 2 * h] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h]) * gelu_grad_fast(lo));
-                r[8 * v + 2 * h + 1] = __float_as_uint(__uint_as_float(r[8 * v + 2 * h + 1]) * gelu_grad_fast(hi));
-              }
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n + j < P.N)
-                r[j] = __float_as_uint(__uint_as_float(r[j]) * gelu_grad_fast(__uint_as_float((uint32_t)pre[j] << 16)));
-          }
-        }
-      }
+      if (P.act) act_chunk(P, r, pre, pre_vec, p4, n);
       uint16_t* dst = reinterpret_cast<uint16_t*>(P.out) + m * P.ldc + n;
       if (n + 32 <= P.N && ((P.ldc & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.out) & 15u) == 0)) {
 #pragma unroll
@@ -283,13 +316,93 @@ __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_bas
   }
 }
 
+// The same accumulator leaving through shared memory: each warp owns a 32-row x 128-byte staging box (128-byte
+// swizzle: 16-byte piece j of row r sits at piece j ^ (r & 7), so the 32 row-owning lanes write without bank
+// conflicts), fills it from its registers and one lane hands it to the TMA unit, which writes whole lines and clips
+// rows >= M and columns >= N.  bf16: 64 columns per box (two tensor-memory reads); fp32: 32 columns per box, the
+// K-range index as third coordinate.  Per-thread stores of a row-per-lane layout touch 32 lines per instruction and
+// were measured to slow the concurrent main loop by about 15 %.
+__device__ __forceinline__ void epilogue_tile_tma(const Params& P, const CUtensorMap* tmC, uint32_t stage, uint32_t tmem_base,
+                                                  int acc, int q, int c0, int lane, int64_t m0, int n0, int split) {
+  const int64_t row0 = (int64_t)m0 + q * 32;
+  const int64_t m = row0 + lane;
+  const bool row_ok = m < P.M;
+  const uint32_t my_row = stage + (uint32_t)lane * 128u;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  if (P.epilogue == MST_TC_OUT_BF16) {
+#pragma unroll 1
+    for (int g = c0; g < BN / 64; g += EPI_WARPS / 4) {
+      const int n = n0 + g * 64;
+      if (n >= P.N) break;  // uniform
+      if (lane == 0) bulk_wait_read();  // the box's previous contents have left shared memory
+      __syncwarp();
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int nn = n + h * 32;
+        if (nn >= P.N) break;  // uniform; the TMA store clips these columns
+        uint32_t r[32];
+        uint16_t* pre = reinterpret_cast<uint16_t*>(P.pre) + m * P.ldpre + nn;
+        const bool pre_vec = nn + 32 <= P.N && ((P.ldpre & 7) == 0) && ((reinterpret_cast<uintptr_t>(P.pre) & 15u) == 0);
+        uint4 p4[4];
+        if (P.act == MST_ACT_GELU_GRAD && pre_vec && row_ok) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) p4[v] = __ldg(reinterpret_cast<const uint4*>(pre) + v);
+        }
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + g * 64 + h * 32), r);
+        if (P.act && row_ok) act_chunk(P, r, pre, pre_vec, p4, nn);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const uint32_t piece = (uint32_t)(h * 4 + v) ^ sw;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + piece * 16u),
+                       "r"(pack_bf16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]))),
+                       "r"(pack_bf16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]))),
+                       "r"(pack_bf16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]))),
+                       "r"(pack_bf16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7])))
+                       : "memory");
+        }
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0 && row0 < P.M) {
+        tma_store_2d(tmC, stage, n, (int)row0);
+        bulk_commit();
+      }
+    }
+  } else {
+#pragma unroll 1
+    for (int c = c0; c < BN / 32; c += EPI_WARPS / 4) {
+      const int n = n0 + c * 32;
+      if (n >= P.N) break;  // uniform
+      if (lane == 0) bulk_wait_read();
+      __syncwarp();
+      uint32_t r[32];
+      tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+#pragma unroll
+      for (int v = 0; v < 8; ++v) {
+        const uint32_t piece = (uint32_t)v ^ sw;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + piece * 16u), "r"(r[4 * v]), "r"(r[4 * v + 1]),
+                     "r"(r[4 * v + 2]), "r"(r[4 * v + 3])
+                     : "memory");
+      }
+      fence_async_smem();
+      __syncwarp();
+      if (lane == 0 && row0 < P.M) {
+        tma_store_3d(tmC, stage, n, (int)row0, split);
+        bulk_commit();
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------- kernel
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params P) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, const Params P) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
-  const uint32_t bar_base = tiles_base + STAGES * STAGE_BYTES;
+  const uint32_t out_base = tiles_base + STAGES * STAGE_BYTES;  // epilogue staging boxes (1024-byte aligned)
+  const uint32_t bar_base = out_base + EPI_WARPS * OUT_BOX_BYTES;
   // barrier slots (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
   const uint32_t full0 = bar_base, empty0 = bar_base + 8 * STAGES, tfull0 = bar_base + 16 * STAGES,
                  tempty0 = tfull0 + 16;
@@ -394,6 +507,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..9)
     const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+    const bool use_tma = P.tma_out && P.epilogue != MST_TC_OUT_SAMPLED;
     int acc = 0;
     uint32_t acc_ph = 0;
     for (int64_t w = blockIdx.x; w < works; w += gridDim.x) {
@@ -401,12 +515,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = (t / P.n_tiles) * BM, n0 = (t % P.n_tiles) * BN;
       if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
+      if (use_tma)
+        epilogue_tile_tma(P, &tmC, out_base + (uint32_t)(warp - 2) * OUT_BOX_BYTES, tmem_base, acc, q, (warp - 2) >> 2, lane, m0,
+                          n0, split);
+      else
+        epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
+    if (use_tma && lane == 0) bulk_wait_all();  // this warp's stores have landed before shared memory is given back
   }
 
   // ------------------------------------------------------------------ teardown
@@ -434,7 +553,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 constexpr int P_STAGES = 6;
 constexpr int PB_BYTES = (BN / 2) * BK * 2;        // this block's half of B: 16 KiB
 constexpr int P_STAGE_BYTES = A_BYTES + PB_BYTES;  // 32 KiB
-constexpr size_t P_SMEM_BYTES = (size_t)P_STAGES * P_STAGE_BYTES + 1024 + 256;
+constexpr size_t P_SMEM_BYTES = (size_t)P_STAGES * P_STAGE_BYTES + EPI_WARPS * OUT_BOX_BYTES + 1024 + 256;
 // shared::cluster address of the same shared-memory location in the even block (rank 0) of the pair
 __device__ __forceinline__ uint32_t in_even_block(uint32_t local_addr) {
   uint32_t r;
@@ -478,11 +597,13 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
-tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params P) {
+tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmC, const Params P) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
-  const uint32_t bar_base = tiles_base + P_STAGES * P_STAGE_BYTES;
+  const uint32_t out_base = tiles_base + P_STAGES * P_STAGE_BYTES;
+  const uint32_t bar_base = out_base + EPI_WARPS * OUT_BOX_BYTES;
   const uint32_t full0 = bar_base, empty0 = bar_base + 8 * P_STAGES, tfull0 = bar_base + 16 * P_STAGES,
                  tempty0 = tfull0 + 16;
   __shared__ uint32_t tmem_base_holder;
@@ -588,6 +709,7 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else {
     // ------------------------------------------------------------------ epilogue (both blocks, own 128 rows)
     const int q = warp & 3;
+    const bool use_tma = P.tma_out && P.epilogue != MST_TC_OUT_SAMPLED;
     int acc = 0;
     uint32_t acc_ph = 0;
     for (int64_t w = pair; w < works; w += npairs) {
@@ -595,12 +717,17 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int m0 = (t / P.n_tiles) * (2 * BM) + (int)rank * BM, n0 = (t % P.n_tiles) * BN;
       if (!mbar_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
       tc_fence_after();
-      epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
+      if (use_tma)
+        epilogue_tile_tma(P, &tmC, out_base + (uint32_t)(warp - 2) * OUT_BOX_BYTES, tmem_base, acc, q, (warp - 2) >> 2, lane, m0,
+                          n0, split);
+      else
+        epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(in_even_block(tempty0 + 8 * acc));
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
+    if (use_tma && lane == 0) bulk_wait_all();  // this warp's stores have landed before shared memory is given back
   }
 
   // ------------------------------------------------------------------ teardown
@@ -653,6 +780,29 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Output maps for the staged epilogue.  bf16 [M x N] (ld elements between rows), box 64 columns x 32 rows;
+// fp32 [splits x M x N], box 32 columns x 32 rows x 1.  Both boxes are 128 bytes wide (128-byte swizzle).
+bool make_out_map_bf16(CUtensorMap* tm, void* base, int64_t M, int64_t N, int64_t ld) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || (ld % 8) != 0 || (reinterpret_cast<uintptr_t>(base) & 15u) != 0) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  cuuint32_t box[2] = {64u, 32u};
+  cuuint32_t estr[2] = {1u, 1u};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+bool make_out_map_f32(CUtensorMap* tm, void* base, int64_t M, int64_t N, int64_t ld, int64_t slab_elems, int splits) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || (ld % 4) != 0 || (slab_elems % 4) != 0 || (reinterpret_cast<uintptr_t>(base) & 15u) != 0) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)splits};
+  cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)slab_elems * 4};
+  cuuint32_t box[3] = {32u, 32u, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int sm_count() {
@@ -758,17 +908,31 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
       P.partial = (float*)ws;
     }
   }
+  // staged epilogue when the output can be described to the TMA unit (MST_TC_TMA_OUT=0 keeps per-thread stores)
+  CUtensorMap tmC = tmA;
+  P.tma_out = 0;
+  if (a.epilogue == MST_TC_OUT_BF16) {
+    P.tma_out = make_out_map_bf16(&tmC, a.out, a.M, a.N, a.ldc) ? 1 : 0;
+  } else if (a.epilogue == MST_TC_OUT_F32) {
+    P.tma_out = (P.splits > 1 ? make_out_map_f32(&tmC, P.partial, a.M, a.N, a.N, a.M * a.N, P.splits)
+                              : make_out_map_f32(&tmC, a.out, a.M, a.N, a.ldc, a.M * a.ldc, 1))
+                    ? 1
+                    : 0;
+  }
+  if (const char* e = getenv("MST_TC_TMA_OUT")) {
+    if (e[0] == '0') P.tma_out = 0;
+  }
   if (pair) {
     MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES));
     const int64_t works = (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles * P.splits;
     const int64_t max_pairs = sm_count() / 2;
     const int grid = 2 * (int)(works < max_pairs ? works : max_pairs);
-    tc_gemm_pair_kernel<<<grid, NUM_THREADS, P_SMEM_BYTES, s>>>(tmA, tmB, P);
+    tc_gemm_pair_kernel<<<grid, NUM_THREADS, P_SMEM_BYTES, s>>>(tmA, tmB, tmC, P);
   } else {
     MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
     const int grid = (int)(works < sm_count() ? works : sm_count());
-    tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, P);
+    tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmC, P);
   }
   MST_CUDA_TRY(cudaGetLastError());
   if (P.splits > 1) {

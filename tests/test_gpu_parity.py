@@ -359,3 +359,34 @@ def test_token_count_edges_on_the_tensor_path(T):
         assert rel_err(host(G), Gr) <= TOL["bf16"]
     assert mst.mst_device_error_flags() == 0
     L.close()
+
+
+@pytest.mark.parametrize("O,I,T", [(520, 328, 900), (136, 264, 72), (768, 3072, 1000), (100, 64, 33)])
+def test_staged_and_direct_stores_agree(O, I, T, monkeypatch):
+    # the contraction's rows leave either through shared memory and TMA stores (default) or by per-thread stores;
+    # both must write the same bits, and neither may touch the padding columns or rows past the tail
+    p = _problem(O, I, T, "bf16", 0.2, 8100 + O + I + T)
+    L = make_layer(p)
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    outs = []
+    for mode in ("1", "0"):
+        monkeypatch.setenv("MST_TC_TMA_OUT", mode)
+        Y = torch.full((T + 3, O + 8), float("nan"), dtype=torch.bfloat16, device=dev())
+        dX = torch.full((T + 3, I + 8), float("nan"), dtype=torch.bfloat16, device=dev())
+        G = torch.full((O + 2, I + 4), float("nan"), dtype=torch.float32, device=dev())
+        mst.mst_spmm_fwd(L.handle, X, I, T, Y, O + 8)
+        mst.mst_spmm_bwd_x(L.handle, dY, O, T, dX, I + 8)
+        mst.mst_dense_grad(dY, O, X, I, T, O, I, mst.MST_BF16, G)     # G is the first O*I elements of the buffer
+        torch.cuda.synchronize()
+        assert torch.isnan(Y[:, O:]).all() and torch.isnan(Y[T:]).all() and not torch.isnan(Y[:T, :O]).any()
+        assert torch.isnan(dX[:, I:]).all() and torch.isnan(dX[T:]).all() and not torch.isnan(dX[:T, :I]).any()
+        Gflat = G.view(-1)[: O * I]
+        assert not torch.isnan(Gflat).any() and torch.isnan(G.view(-1)[O * I:]).all()
+        outs.append((Y[:T, :O].clone(), dX[:T, :I].clone(), Gflat.clone()))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    Wm = np.where(p.mask == 1, p.W, np.float32(0))
+    assert rel_err(host(outs[0][0]), oracle.fwd(p.X, Wm, p.mask)) <= TOL["bf16"]
+    assert rel_err(host(outs[0][2]).reshape(O, I), oracle.dense_grad(p.dY, p.X)) <= 1e-5
+    assert mst.mst_device_error_flags() == 0
+    L.close()
