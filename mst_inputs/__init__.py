@@ -238,3 +238,33 @@ def config5(density: float, tokens: int = 16384) -> List[LayerProblem]:
     """One GPT-2-large block's four FC shapes at one point of the density sweep."""
     return [uniform_layer(n, i, o, k, tokens, "bf16", density, BASE_SEED + 5)
             for i, (n, o, k) in enumerate(block_shapes(1280))]
+
+
+# --------------------------------------------------------------------------
+# attention inputs
+# --------------------------------------------------------------------------
+@dataclass
+class AttentionProblem:
+    """Fused qkv activations of a GPT-2 attention layer: ``qkv`` is [batch * seq, 3 * heads * head_dim] (the output
+    of the qkv projection: queries, keys, values side by side, heads contiguous inside each), stored-precision bf16
+    values as float32 plus their bit patterns."""
+    batch: int
+    seq: int
+    heads: int
+    head_dim: int
+    qkv: np.ndarray
+    qkv_bits: np.ndarray
+
+    def split(self):
+        """(Q, K, V) as float32 [batch, heads, seq, head_dim] views of the stored values."""
+        c = self.heads * self.head_dim
+        x = self.qkv.reshape(self.batch, self.seq, 3, self.heads, self.head_dim)
+        return tuple(np.ascontiguousarray(x[:, :, k].transpose(0, 2, 1, 3)) for k in range(3))
+
+
+def attention_problem(batch: int, seq: int, heads: int = 12, head_dim: int = 64, seed: int = BASE_SEED + 7,
+                      std: float = 1.0) -> AttentionProblem:
+    """N(0, std^2) queries, keys and values (unit variance gives scaled scores of unit variance), rounded to bf16."""
+    x = normal((batch * seq, 3 * heads * head_dim), std, seed, 0x617474)
+    bits = f32_to_bf16_bits(x)
+    return AttentionProblem(batch, seq, heads, head_dim, bf16_bits_to_f32(bits), bits)
