@@ -142,6 +142,20 @@ mst_status_t mst_spmm_fwd_gelu(const mst_layer_t* layer, const void* X, int64_t 
 mst_status_t mst_spmm_bwd_x_gelu(const mst_layer_t* layer, const void* dY, int64_t lddy, int64_t T, const void* Y_pre,
                                  int64_t ldpre, void* dPre, int64_t lddpre, mst_stream_t stream);
 
+/* Unfactorized strided sparse self-attention, forward (Sec. 3.3):
+ *   Out[i] = sum_{j in S_i} softmax_j(q_i . k_j / sqrt(d)) v_j,   S_i = { j <= i : i - j < l  or  (i - j) mod l == 0 },
+ * the same S_i in every head (the set formula is printed with an intersection; text, figure and the FLOP ratios of
+ * the appendix table fix the union).  Q, K, V: device bf16, token-major, `ld` elements between consecutive tokens,
+ * head h in columns h*head_dim .. (so the three column slices of a fused qkv activation can be passed as they are);
+ * token b*seq_len + i is position i of sequence b.  Out: device bf16 [batch*seq_len x ldo], same column layout.
+ * lse (device float [batch, heads, seq_len], may be NULL) receives log sum_j exp(q_i . k_j / sqrt(d)) for a backward
+ * pass.  Supported: head_dim = 64, seq_len a multiple of 128, stride l = 128 or 256, seq_len / l <= 16, ld and ldo
+ * multiples of 8, 16-byte aligned pointers; anything else MST_ERR_SHAPE.  Scores and sums are fp32, the softmax
+ * weights are rounded to bf16 before they multiply the values. */
+mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, const void* V, int64_t ld, int32_t batch,
+                                       int32_t seq_len, int32_t heads, int32_t head_dim, int32_t stride, void* Out,
+                                       int64_t ldo, float* lse, mst_stream_t stream);
+
 /* Weight gradient on the mask only, dW[k] = sum_t dY[t,o_k] X[t,i_k] for the k-th active entry in CSR order
  * (same passage).  dW_vals device float [nnz]. */
 mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,

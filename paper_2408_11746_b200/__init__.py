@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
-           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
+           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_strided_attention_fwd", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
            "mst_status_string"]
@@ -76,6 +76,7 @@ _sig = {
     "mst_spmm_bwd_x": [_vp, _vp, _i64, _i64, _vp, _i64, _vp],
     "mst_spmm_fwd_gelu": [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp],
     "mst_spmm_bwd_x_gelu": [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp],
+    "mst_strided_attention_fwd": [_vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _vp, _i64, _vp, _vp],
     "mst_sddmm_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp],
     "mst_dense_grad": [_vp, _i64, _vp, _i64, _i64, _i32, _i32, ctypes.c_int, _vp, _vp],
     "mst_sddmm_from_dense": [_vp, _vp, _vp, _vp],
@@ -189,6 +190,12 @@ def mst_spmm_fwd_gelu(layer: int, X, ldx: int, T: int, Y_pre, ldpre: int, H, ldh
 def mst_spmm_bwd_x_gelu(layer: int, dY, lddy: int, T: int, Y_pre, ldpre: int, dPre, lddpre: int, stream=None) -> None:
     _check(_lib.mst_spmm_bwd_x_gelu(layer, _ptr(dY), lddy, T, _ptr(Y_pre), ldpre, _ptr(dPre), lddpre, _stream(stream)),
            "mst_spmm_bwd_x_gelu")
+
+
+def mst_strided_attention_fwd(Q, K, V, ld: int, batch: int, seq_len: int, heads: int, head_dim: int, stride: int, Out,
+                              ldo: int, lse=None, stream=None) -> None:
+    _check(_lib.mst_strided_attention_fwd(_ptr(Q), _ptr(K), _ptr(V), ld, batch, seq_len, heads, head_dim, stride,
+                                          _ptr(Out), ldo, _ptr(lse), _stream(stream)), "mst_strided_attention_fwd")
 
 
 def mst_sddmm_dw(layer: int, dY, lddy: int, X, ldx: int, T: int, dW_vals, stream=None) -> None:

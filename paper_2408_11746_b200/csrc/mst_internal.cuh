@@ -96,6 +96,9 @@ mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
 mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s);
 bool mst_use_tensor_path(const mst_layer* L);
 
+// sticky error word of the attention kernel's bounded waits (mst_attention.cu)
+mst_status_t mst_attention_error_flags(int32_t* flags);
+
 // kernels' launchers
 // act / pre / ldpre: element-wise step fused behind the product (see mst_tc_gemm.cuh); act = 0 for the plain product
 mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in, int64_t ldin, int64_t T, void* out,
