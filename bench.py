@@ -97,6 +97,57 @@ def aggregate_value(useful_flops_per_step: float, steps: int, world: int, ms: fl
     return useful_flops_per_step * steps * world / (ms * 1e-3) / 1e12
 
 
+# ------------------------------------------------------------------------------------------ attention report
+def run_attention(args) -> None:
+    """Strided sparse attention forward on the attention input of a 16384-token GPT-2-small batch."""
+    import torch
+    import paper_2408_11746_b200 as mst
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    B, n, H, d = 16, 1024, 12, 64
+    C = H * d
+    p = mst_inputs.attention_problem(B, n, H, d)
+    qkv = torch.from_numpy(p.qkv_bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    out = torch.empty((B * n, C), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((B, H, n), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    base = qkv.data_ptr()
+
+    def timed(f, reps=10, inner=4):
+        for _ in range(3):
+            f()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(inner):
+                f()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / inner)
+        return float(np.median(ts)) * 1e-3
+
+    x = qkv.view(B, n, 3, H, d)
+    q, k, v = (x[:, :, j].transpose(1, 2) for j in range(3))
+    t_dense = timed(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True))
+    for stride in (256, 128):
+        t = timed(lambda: mst.mst_strided_attention_fwd(base, base + 2 * C, base + 4 * C, 3 * C, B, n, H, d, stride, out,
+                                                        C, lse))
+        kept = sum(min(i, stride - 1) + 1 + i // stride for i in range(n))        # |S_i| summed over positions
+        useful = 4.0 * d * kept * B * H                                            # scores + weighted sum, kept pairs
+        executed = 4.0 * d * n * (stride + 128) * B * H                            # the two tile products as issued
+        bytes_alg = 4.0 * B * n * C * 2 + 4.0 * B * H * n
+        print(json.dumps({
+            "report": "strided_attention_fwd", "stride": stride, "batch": B, "seq_len": n, "heads": H, "head_dim": d,
+            "us": t * 1e6, "useful_tflops": useful / t / 1e12, "executed_tflops": executed / t / 1e12,
+            "kept_fraction": kept / float(n * n),
+            "roofline": {"bound": "hbm", "achieved": bytes_alg / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": bytes_alg / t / 1e9 / peaks["hbm_gbs"]},
+            "torch_dense_causal_us": t_dense * 1e6}))
+    assert mst.mst_device_error_flags() == 0
+
+
 # ------------------------------------------------------------------------------------------ reference arm
 def run_reference(args) -> None:
     """Time the CPU checker, as it stands, on a bounded sample of the workload (rank 0 only)."""
@@ -252,8 +303,14 @@ def main() -> None:
     ap.add_argument("--sweep", default=None, choices=["medium", "large", "small"],
                     help="density sweep report on one block's FC shapes (not the bench line): one JSON object per "
                          "(layer, density) with both kernel families and a dense cuBLAS GEMM beside them")
+    ap.add_argument("--attention", action="store_true",
+                    help="report on the strided sparse attention forward (not the bench line): one JSON object per "
+                         "stride at 16 x 1024 tokens, 12 heads of 64, with torch's dense causal attention beside it")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.attention:
+        run_attention(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return

@@ -149,7 +149,7 @@ mst_status_t mst_spmm_bwd_x_gelu(const mst_layer_t* layer, const void* dY, int64
  * head h in columns h*head_dim .. (so the three column slices of a fused qkv activation can be passed as they are);
  * token b*seq_len + i is position i of sequence b.  Out: device bf16 [batch*seq_len x ldo], same column layout.
  * lse (device float [batch, heads, seq_len], may be NULL) receives log sum_j exp(q_i . k_j / sqrt(d)) for a backward
- * pass.  Supported: head_dim = 64, seq_len a multiple of 128, stride l = 128 or 256, seq_len / l <= 16, ld and ldo
+ * pass.  Supported: head_dim = 64, seq_len a multiple of 128, stride l = 128 or 256, seq_len <= 8 l, ld and ldo
  * multiples of 8, 16-byte aligned pointers; anything else MST_ERR_SHAPE.  Scores and sums are fp32, the softmax
  * weights are rounded to bf16 before they multiply the values. */
 mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, const void* V, int64_t ld, int32_t batch,

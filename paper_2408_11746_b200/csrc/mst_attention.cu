@@ -1,15 +1,19 @@
 // Strided sparse self-attention, forward (Sec. 3.3: position i attends to j <= i with i - j < l, and to every l-th
 // earlier position j = i - l, i - 2l, ...; every head uses the same pattern).
 //
-// One block per (batch, head, 128 queries).  The window part is two dense tensor-core products on a [128 x (l+128)]
-// score tile: the keys q0 - l .. q0 + 127 cover the window of every query of the block, so no loop over key blocks
-// and no running softmax is needed:
-//   control warp   TMA loads Q, the l/128 + 1 key blocks and value blocks; tcgen05.mma S = Q K^T (fp32, tensor
-//                  memory); after the softmax warps have written P, tcgen05.mma O = P V;
-//   4 softmax warps (thread = query row = tensor-memory lane): scores of the strided positions on CUDA cores
-//                  (at most n/l - 1 dot products of 64), row maximum and sum over tensor memory, P in bf16 into
-//                  shared memory in the K-major 128-byte-swizzled operand layout, then O / sum plus the strided
-//                  positions' values, written as bf16.
+// A tile is (batch, head, 128 queries).  Its window part is two dense tensor-core products on a [128 x (l+128)]
+// score tile: the keys q0 - l .. q0 + 127 cover the window of every query of the tile, so there is no loop over key
+// blocks and no running softmax.  One persistent block per SM walks over the tiles, its warps specialised:
+//   warp 0     TMA producer: Q and the l/128 + 1 key blocks as soon as the previous tile's S = Q K^T has completed,
+//              the value blocks as soon as the previous tile's O = P V has completed (single buffers, loads of tile
+//              t+1 fly during the softmax of tile t);
+//   warp 1     one lane issues tcgen05.mma: O(t) = P V once P(t) is written, then S(t+1) = Q K^T (fp32, tensor memory);
+//   warps 2-9  softmax, two warps per tensor-memory lane quarter (thread = query row, the pair splitting the visible
+//              32-key chunks by parity and the output columns in halves): scores of the strided positions on CUDA
+//              cores, row maximum, P = exp(s - max) in bf16 into shared memory
+//              in the K-major 128-byte-swizzled operand layout, row sum, and after the second product O / sum plus
+//              the strided positions' values, written as bf16.  Chunks no row of the warp can see are skipped, chunks
+//              every row sees in full skip the mask arithmetic.
 // Keys before the start of the sequence (q0 < l) are fetched from the rows in front of it (another sequence of the
 // batch, or the TMA unit's zero fill before row 0) and masked by position, never by value.
 // Every mbarrier wait is bounded (abort flag + sticky error word), as in the contraction kernel.
@@ -27,13 +31,17 @@ namespace {
 using namespace mst_ptx;
 
 constexpr int D = 64;          // head dimension
-constexpr int BQ = 128;        // queries per block = tensor-memory lanes
+constexpr int BQ = 128;        // queries per tile = tensor-memory lanes
 constexpr int KB = 128;        // keys per key block
 constexpr int TILE_BYTES = 128 * D * 2;  // one [128 x 64] bf16 tile, 16 KiB
-constexpr int ATT_THREADS = 160;         // 4 softmax warps + 1 control warp
+constexpr int SM_WARPS = 8;              // softmax warps
+constexpr int FAR_WARPS = 4;               // warps for the attended positions outside the tile
+constexpr int ATT_THREADS = 64 + 32 * SM_WARPS + 32 * FAR_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int O_COL = 448;     // output accumulator: tensor-memory columns 448..511
-constexpr int MAX_EXTRA = 15;  // strided positions per query: seq / l - 1
+constexpr int FAR_COL = 384;   // far positions' weighted value sums: columns 384..447
+constexpr int MAX_FAR = 6;       // attended positions outside the tile, i - 2l, i - 3l, ...: seq / l - 2
+constexpr int RED_BYTES = 2 * BQ * 4 + 2 * BQ * 4;  // partial row sums of a pair's two warps; far positions' (max, sum)
 
 __device__ int g_attn_error = 0;
 
@@ -43,8 +51,10 @@ struct AttnParams {
   uint16_t* out;
   int64_t ldo;
   float* lse;       // [batch, heads, seq] or NULL
-  int seq, heads, stride;
+  int seq, heads, stride, batch;
   int nkb;          // key blocks per tile: stride / 128 + 1
+  int qblocks;      // seq / 128
+  int tiles;        // batch * heads * qblocks
 };
 
 __device__ __forceinline__ bool att_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
@@ -68,35 +78,93 @@ __device__ __forceinline__ float dot8(const uint4& a, const uint4& b, float acc)
   return acc;
 }
 
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+// The two warps of a lane quarter meet on an mbarrier of two arrivals (a bounded wait, unlike a named barrier, so an
+// aborting block cannot leave a warp behind); shared-memory writes made before it are visible after it.
+__device__ __forceinline__ bool pair_meet(uint32_t bar, uint32_t parity, int lane, volatile int* abort_flag) {
+  __syncwarp();
+  if (lane == 0) mbar_arrive(bar);
+  return att_wait(bar, parity, abort_flag);
+}
+
+// tile index -> (sequence, head, first query); late query blocks first: they carry the most strided positions
+__device__ __forceinline__ void tile_coords(const AttnParams& P, int t, int& b, int& h, int& q0) {
+  const int qb = P.qblocks - 1 - t / (P.batch * P.heads);
+  const int bh = t % (P.batch * P.heads);
+  b = bh / P.heads;
+  h = bh % P.heads;
+  q0 = qb * BQ;
+}
+
+// Scores (unscaled) of this warp's 32 rows of tile t against the positions i - 2l, i - 3l, ...:
+// se[k] = q_i . k_{i-(k+2)l} for the row i = q0 + qtr*32 + lane.  The warp reads the rows together, eight lanes per
+// 128-byte row (four rows per instruction, whole lines), reduces over the eight lanes and hands each row's result to
+// the lane that owns the row; one row per lane would touch 32 lines per load instruction.
+__device__ __forceinline__ void far_scores(const AttnParams& P, int t, int qtr, int lane, int l, float (&se)[MAX_FAR]) {
+  int b, h, q0;
+  tile_coords(P, t, b, h, q0);
+  const int i_lo = q0 + qtr * 32;
+  const int n_far_max = (i_lo + 31) / l - 1 < MAX_FAR ? (i_lo + 31) / l - 1 : MAX_FAR;   // uniform over the warp
+  if (n_far_max <= 0) return;
+  const int grp = lane >> 3, piece = lane & 7;
+  const int64_t tok0 = (int64_t)b * P.seq + i_lo;
+  uint4 qv[8];
+#pragma unroll
+  for (int rr = 0; rr < 8; ++rr)
+    qv[rr] = __ldg(reinterpret_cast<const uint4*>(P.Q + (tok0 + rr * 4 + grp) * P.ld + h * D) + piece);
+#pragma unroll
+  for (int k = 0; k < MAX_FAR; ++k) {
+    if (k < n_far_max) {
+      // rows of the 32-row group all have the same number of far positions (i_lo and l are multiples of 32)
+      float mine = 0.f;
+#pragma unroll
+      for (int rr = 0; rr < 8; ++rr) {
+        const uint4 kv =
+            __ldg(reinterpret_cast<const uint4*>(P.K + (tok0 + rr * 4 + grp - (int64_t)(k + 2) * l) * P.ld + h * D) + piece);
+        float a = dot8(qv[rr], kv, 0.f);
+        a += __shfl_xor_sync(0xffffffffu, a, 1);
+        a += __shfl_xor_sync(0xffffffffu, a, 2);
+        a += __shfl_xor_sync(0xffffffffu, a, 4);
+        const float got = __shfl_sync(0xffffffffu, a, (lane & 3) * 8);   // row rr*4 + (lane & 3)
+        if ((lane >> 2) == rr) mine = got;
+      }
+      se[k] = mine;
+    }
+  }
+}
+
+__global__ void __maxnreg__(128)
 strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                              const __grid_constant__ CUtensorMap tmV, const AttnParams P) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int nkb = P.nkb;
   const uint32_t q_s = base, k_s = q_s + TILE_BYTES, v_s = k_s + nkb * TILE_BYTES, p_s = v_s + nkb * TILE_BYTES;
-  const uint32_t bar0 = p_s + 2 * nkb * TILE_BYTES;
+  const uint32_t red_s = p_s + 2 * nkb * TILE_BYTES;
+  const uint32_t bar0 = red_s + RED_BYTES;
   const uint32_t bar_qk = bar0, bar_v = bar0 + 8, bar_s = bar0 + 16, bar_p = bar0 + 24, bar_o = bar0 + 32;
+  const uint32_t bar_pair0 = bar0 + 40;  // one per lane quarter
+  const uint32_t bar_far_full = bar0 + 72, bar_far_empty = bar0 + 80;
+  float* red = reinterpret_cast<float*>(smem_raw + (red_s - smem_u32(smem_raw)));  // [2 halves][128 rows]
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_sh;
   volatile int* abort_flag = &abort_sh;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int q0 = blockIdx.x * BQ, h = blockIdx.y, b = blockIdx.z;
   const int l = P.stride;
-  const int jb = q0 - l;                               // first key of the tile (may be negative)
-  const int64_t row_base = (int64_t)b * P.seq;         // first token of this sequence
 
   if (threadIdx.x == 0) {
     abort_sh = 0;
     mbar_init(bar_qk, 1);
     mbar_init(bar_v, 1);
     mbar_init(bar_s, 1);
-    mbar_init(bar_p, 4);
+    mbar_init(bar_p, SM_WARPS);
     mbar_init(bar_o, 1);
+    for (int qq = 0; qq < 4; ++qq) mbar_init(bar_pair0 + 8 * qq, 2);
+    mbar_init(bar_far_full, FAR_WARPS);
+    mbar_init(bar_far_empty, SM_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 4) {
+  if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
                  "r"(TMEM_COLS)
                  : "memory");
@@ -107,167 +175,286 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
 
-  if (warp == 4) {
-    // ------------------------------------------------------------------ control: loads and the two products
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      const int col = h * D;
-      mbar_expect_tx(bar_qk, (uint32_t)((1 + nkb) * TILE_BYTES));
-      tma_load_2d(q_s, &tmQ, col, (int)(row_base + q0), bar_qk);
-      for (int kb = 0; kb < nkb; ++kb) tma_load_2d(k_s + kb * TILE_BYTES, &tmK, col, (int)(row_base + jb + kb * KB), bar_qk);
-      mbar_expect_tx(bar_v, (uint32_t)(nkb * TILE_BYTES));
-      for (int kb = 0; kb < nkb; ++kb) tma_load_2d(v_s + kb * TILE_BYTES, &tmV, col, (int)(row_base + jb + kb * KB), bar_v);
-
-      bool ok = att_wait(bar_qk, 0, abort_flag);
-      if (ok) {
+      uint32_t it = 0;
+      for (int t = blockIdx.x; t < P.tiles && !*abort_flag; t += gridDim.x, ++it) {
+        int b, h, q0;
+        tile_coords(P, t, b, h, q0);
+        const int col = h * D;
+        const int row_q = b * P.seq + q0, row_k = row_q - l;
+        // Q and K are free once the previous tile's first product has completed, V once its second has
+        if (it > 0 && !att_wait(bar_s, (it - 1) & 1u, abort_flag)) break;
+        mbar_expect_tx(bar_qk, (uint32_t)((1 + nkb) * TILE_BYTES));
+        tma_load_2d(q_s, &tmQ, col, row_q, bar_qk);
+        for (int kb = 0; kb < nkb; ++kb) tma_load_2d(k_s + kb * TILE_BYTES, &tmK, col, row_k + kb * KB, bar_qk);
+        if (it > 0 && !att_wait(bar_o, (it - 1) & 1u, abort_flag)) break;
+        mbar_expect_tx(bar_v, (uint32_t)(nkb * TILE_BYTES));
+        for (int kb = 0; kb < nkb; ++kb) tma_load_2d(v_s + kb * TILE_BYTES, &tmV, col, row_k + kb * KB, bar_v);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      // S[:, kb*128 .. +128) = Q K_kb^T : M = 128, N = 128, both operands K-major, four K steps of 16
+      const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KB >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
+      // O = P V : M = 128, N = 64, P K-major (64-key blocks of 16 KiB), V as stored (keys x 64: MN-major)
+      const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) |
+                              ((uint32_t)(BQ >> 4) << 24);
+      const uint64_t qd = smem_desc(q_s, 16, 1024), kd0 = smem_desc(k_s, 16, 1024);
+      const uint64_t pd0 = smem_desc(p_s, 16, 1024), vd0 = smem_desc(v_s, 8192, 1024);
+      const int ksteps = nkb * KB / 16;
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < P.tiles && ok && !*abort_flag; t += gridDim.x, ++it) {
+        const uint32_t ph = it & 1u;
+        // first product of this tile: S is free (the previous tile's P has been written, so S has been read)
+        ok = att_wait(bar_qk, ph, abort_flag);
+        if (!ok) break;
         tc_fence_after();
-        // S[:, kb*128 .. +128) = Q K_kb^T : M = 128, N = 128, both operands K-major, four K steps of 16
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KB >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
-        const uint64_t qd = smem_desc(q_s, 16, 1024);
         for (int kb = 0; kb < nkb; ++kb) {
-          const uint64_t kd = smem_desc(k_s + kb * TILE_BYTES, 16, 1024);
+          const uint64_t kd = kd0 + (uint64_t)(uint32_t)(kb * (TILE_BYTES >> 4));
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
-            tc_mma(tmem_base + (uint32_t)(kb * KB), qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc, ks > 0 ? 1u : 0u);
+            tc_mma(tmem_base + (uint32_t)(kb * KB), qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc1, ks > 0 ? 1u : 0u);
         }
         tc_commit(bar_s);
-        ok = att_wait(bar_v, 0, abort_flag) && att_wait(bar_p, 0, abort_flag);
-      }
-      if (ok) {
+        // second product once P is in shared memory and V has landed
+        ok = att_wait(bar_v, ph, abort_flag) && att_wait(bar_p, ph, abort_flag);
+        if (!ok) break;
         tc_fence_after();
-        // O = P V : M = 128, N = 64, P K-major (64-key blocks of 16 KiB), V as stored (keys x 64: MN-major)
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) |
-                               ((uint32_t)(BQ >> 4) << 24);
-        const int ksteps = nkb * KB / 16;
         for (int ks = 0; ks < ksteps; ++ks) {
-          const uint64_t pd = smem_desc(p_s + (uint32_t)(ks >> 2) * TILE_BYTES + (uint32_t)(ks & 3) * 32u, 16, 1024);
-          const uint64_t vd = smem_desc(v_s + (uint32_t)ks * (16u * 128u), 8192, 1024);
-          tc_mma(tmem_base + (uint32_t)O_COL, pd, vd, idesc, ks > 0 ? 1u : 0u);
+          const uint64_t pd = pd0 + (uint64_t)(uint32_t)((ks >> 2) * (TILE_BYTES >> 4) + (ks & 3) * 2);
+          const uint64_t vd = vd0 + (uint64_t)(uint32_t)(ks * ((16 * 128) >> 4));
+          tc_mma(tmem_base + (uint32_t)O_COL, pd, vd, idesc2, ks > 0 ? 1u : 0u);
         }
         tc_commit(bar_o);
       }
     }
-  } else {
-    // ------------------------------------------------------------------ softmax: thread = query row
-    const int r = warp * 32 + lane;
-    const int i = q0 + r;                               // position in the sequence
-    const int64_t tok = row_base + i;
-    const float c = 0.125f * 1.4426950408889634f;       // log2(e) / sqrt(64)
-    const int n_ext = i / l < MAX_EXTRA ? i / l : MAX_EXTRA;
-    const uint4* qrow = reinterpret_cast<const uint4*>(P.Q + tok * P.ld + h * D);
-    float s_ext[MAX_EXTRA];
-#pragma unroll 1
-    for (int k = 0; k < n_ext; ++k) {
-      const uint4* krow = reinterpret_cast<const uint4*>(P.K + (tok - (int64_t)(k + 1) * l) * P.ld + h * D);
-      float acc = 0.f;
-#pragma unroll
-      for (int v = 0; v < 8; ++v) acc = dot8(__ldg(qrow + v), __ldg(krow + v), acc);
-      s_ext[k] = acc;
-    }
-    float m = -INFINITY;
-#pragma unroll 1
-    for (int k = 0; k < n_ext; ++k) m = fmaxf(m, s_ext[k]);
-
-    // chunks of 32 keys that hold a visible key for some row of this warp
-    const int i_lo = q0 + warp * 32, i_hi = i_lo + 31;
+  } else if (warp < 2 + SM_WARPS) {
+    // ------------------------------------------------------------------ softmax: thread = query row, two warps per row
+    const int q = warp & 3;                 // tensor-memory lane quarter
+    const int half = (warp - 2) >> 2;       // which warp of the pair
+    const int r = q * 32 + lane;
+    const float c = 0.125f * 1.4426950408889634f;  // log2(e) / sqrt(64)
+    const uint32_t sw = (uint32_t)(r & 7);
     const int nchunks = nkb * 4;
-    bool ok = att_wait(bar_s, 0, abort_flag);
-    tc_fence_after();
-    if (ok) {
-      // pass 1: row maximum
-#pragma unroll 1
-      for (int ch = 0; ch < nchunks; ++ch) {
-        const int j0 = jb + ch * 32;
-        if (j0 > i_hi || j0 + 31 <= i_lo - l || j0 + 31 < 0) continue;  // uniform over the warp: nothing visible
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(ch * 32), v);
+    float* red_sum = red;                   // [2][128]
+    // The position i - l is row r of the tile's first key block, so its score sits in S and its value in the V tile:
+    // the window mask simply reaches one key further (distance <= l).  Positions i - 2l, i - 3l, ... lie outside
+    // the tile: the far warps form their softmax partials (maximum, sum, weighted value sum) a tile ahead and the
+    // epilogue below merges them with the window's.
+    const float* far_stat = red + 2 * BQ;   // [128][2]: maximum (unscaled score), sum
+    int t = blockIdx.x;
+    uint32_t it = 0;
+    for (; t < P.tiles; t += gridDim.x, ++it) {
+      const uint32_t ph = it & 1u;
+      int b, h, q0;
+      tile_coords(P, t, b, h, q0);
+      const int i = q0 + r;                 // position in the sequence
+      const int jb = q0 - l;                // first key of the tile (may be negative)
+      const int64_t tok = (int64_t)b * P.seq + i;
+      const bool has_far = i / l >= 2;      // uniform over the warp (32 rows between multiples of 128)
+      float m = -INFINITY;
+      const int i_lo = q0 + q * 32, i_hi = i_lo + 31;
+
+      if (!att_wait(bar_s, ph, abort_flag)) break;
+      tc_fence_after();
+      // The chunks (32 keys) some row of this warp can see are a contiguous range: from the window start of the
+      // warp's first row (or key 0) to the diagonal of its last row.
+      const int ch_lo = (jb < 0 && -jb / 32 > q) ? -jb / 32 : q;
+      const int ch_hi = l / 32 + q;
+      const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+      // pass 1: row maximum.  Both warps of the pair scan every visible chunk (cheaper than meeting to exchange it);
+      // the load of the next chunk is in flight while this one is reduced.
+      {
+        auto reduce_max = [&](const uint32_t (&v)[32], int ch) {
+          const int j0 = jb + ch * 32;
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          if (j0 >= 0 && j0 + 31 <= i_lo && i_hi - j0 <= l) {            // every row sees the whole chunk
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int j = j0 + e;
-          const bool vis = j >= 0 && j <= i && i - j < l;
-          m = fmaxf(m, vis ? __uint_as_float(v[e]) : -INFINITY);
+            for (int e = 0; e < 32; ++e) m4[e & 3] = fmaxf(m4[e & 3], __uint_as_float(v[e]));
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const int j = j0 + e;
+              const bool vis = j >= 0 && j <= i && i - j <= l;
+              m4[e & 3] = fmaxf(m4[e & 3], vis ? __uint_as_float(v[e]) : -INFINITY);
+            }
+          }
+          m = fmaxf(fmaxf(m, fmaxf(m4[0], m4[1])), fmaxf(m4[2], m4[3]));
+        };
+        uint32_t va[32], vb[32];
+        int ch = ch_lo;
+        tmem_ld32_nowait(t_row + (uint32_t)(ch * 32), va);
+#pragma unroll 1
+        while (true) {
+          tmem_ld_wait(va);
+          if (ch + 1 <= ch_hi) tmem_ld32_nowait(t_row + (uint32_t)((ch + 1) * 32), vb);
+          reduce_max(va, ch);
+          if (++ch > ch_hi) break;
+          tmem_ld_wait(vb);
+          if (ch + 1 <= ch_hi) tmem_ld32_nowait(t_row + (uint32_t)((ch + 1) * 32), va);
+          reduce_max(vb, ch);
+          if (++ch > ch_hi) break;
         }
       }
-      // pass 2: P = exp(s - m) in bf16 into the operand layout, row sum in fp32
-      float sum = 0.f;
-      const float mc = m * c;
+      // pass 2 over this warp's chunks (those of its parity): P = exp(s - m) in bf16 into the operand layout,
+      // partial row sum in fp32; chunks of its parity outside the visible range are zero-filled
+      float s4[4] = {0.f, 0.f, 0.f, 0.f};
+      const float mc = m * c;               // finite: key i itself is visible
+      {
+        auto p_addr = [&](int ch, int g) {
+          return p_s + (uint32_t)(ch >> 1) * TILE_BYTES + (uint32_t)r * 128u + (((uint32_t)((ch & 1) * 4 + g) ^ sw) << 4);
+        };
 #pragma unroll 1
-      for (int ch = 0; ch < nchunks; ++ch) {
-        const int j0 = jb + ch * 32;
-        const uint32_t prow = p_s + (uint32_t)(ch >> 1) * TILE_BYTES + (uint32_t)r * 128u;
-        const uint32_t piece0 = (uint32_t)(ch & 1) * 4u;
-        const uint32_t sw = (uint32_t)(r & 7);
-        if (j0 > i_hi || j0 + 31 <= i_lo - l || j0 + 31 < 0) {
+        for (int ch = half; ch < nchunks; ch += 2) {
+          if (ch >= ch_lo && ch <= ch_hi) continue;
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(prow + (((piece0 + q) ^ sw) << 4)), "r"(0u) : "memory");
-          continue;
+          for (int g = 0; g < 4; ++g)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(p_addr(ch, g)), "r"(0u) : "memory");
         }
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(ch * 32), v);
-        float p[32];
+        auto exp_store = [&](const uint32_t (&v)[32], int ch) {
+          const int j0 = jb + ch * 32;
+          float p[32];
+          if (j0 >= 0 && j0 + 31 <= i_lo && i_hi - j0 <= l) {            // every row sees the whole chunk
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int j = j0 + e;
-          const bool vis = j >= 0 && j <= i && i - j < l;
-          p[e] = vis ? ex2_ftz(fmaf(__uint_as_float(v[e]), c, -mc)) : 0.f;
-          sum += p[e];
-        }
+            for (int e = 0; e < 32; ++e) p[e] = ex2_ftz(fmaf(__uint_as_float(v[e]), c, -mc));
+          } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(prow + (((piece0 + q) ^ sw) << 4)),
-                       "r"(pack_bf16(p[8 * q + 0], p[8 * q + 1])), "r"(pack_bf16(p[8 * q + 2], p[8 * q + 3])),
-                       "r"(pack_bf16(p[8 * q + 4], p[8 * q + 5])), "r"(pack_bf16(p[8 * q + 6], p[8 * q + 7]))
-                       : "memory");
-      }
-      // strided positions' weights (kept in fp32, applied on CUDA cores below)
+            for (int e = 0; e < 32; ++e) {
+              const int j = j0 + e;
+              const bool vis = j >= 0 && j <= i && i - j <= l;
+              p[e] = vis ? ex2_ftz(fmaf(__uint_as_float(v[e]), c, -mc)) : 0.f;
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 32; ++e) s4[e & 3] += p[e];
+          uint32_t w[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) w[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+#pragma unroll
+          for (int g = 0; g < 4; ++g)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_addr(ch, g)), "r"(w[4 * g]), "r"(w[4 * g + 1]),
+                         "r"(w[4 * g + 2]), "r"(w[4 * g + 3])
+                         : "memory");
+        };
 #pragma unroll 1
-      for (int k = 0; k < n_ext; ++k) {
-        s_ext[k] = ex2_ftz(fmaf(s_ext[k], c, -mc));
-        sum += s_ext[k];
+        for (int ch = ch_lo + ((ch_lo ^ half) & 1); ch <= ch_hi; ch += 2) {   // visible chunks of this warp's parity
+          uint32_t v[32];
+          tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+          exp_store(v, ch);
+        }
       }
-      fence_async_smem();  // P is read by the tensor core through the async proxy
+      float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      red_sum[half * BQ + r] = sum;
+      fence_async_smem();   // P is read by the tensor core through the async proxy
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_p);
 
-      if (P.lse) P.lse[((int64_t)b * P.heads + h) * P.seq + i] = m * 0.125f + __logf(sum);
-
-      ok = att_wait(bar_o, 0, abort_flag);
+      if (!pair_meet(bar_pair0 + 8 * q, ph, lane, abort_flag)) break;   // one meeting per tile
+      sum += red_sum[(half ^ 1) * BQ + r];
+      if (!att_wait(bar_o, ph, abort_flag)) break;
+      if (!att_wait(bar_far_full, ph, abort_flag)) break;
       tc_fence_after();
-      if (ok) {
+      {
+        // this warp's half of the output columns; merge the far positions' partial softmax
+        uint32_t v[32];
+        tmem_ld32(t_row + (uint32_t)(O_COL + half * 32), v);
+        float o[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(v[e]);
+        float mm = m;
+        if (has_far) {
+          const float m_e = far_stat[2 * r], sum_e = far_stat[2 * r + 1];
+          tmem_ld32(t_row + (uint32_t)(FAR_COL + half * 32), v);
+          mm = fmaxf(m, m_e);
+          const float a_w = ex2_ftz((m - mm) * c), a_e = ex2_ftz((m_e - mm) * c);
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = fmaf(a_w, o[e], a_e * __uint_as_float(v[e]));
+          sum = fmaf(a_w, sum, a_e * sum_e);
+        }
+        if (P.lse && half == 0) P.lse[((int64_t)b * P.heads + h) * P.seq + i] = mm * 0.125f + __logf(sum);
         const float inv = 1.0f / sum;
-        uint16_t* orow = P.out + tok * P.ldo + h * D;
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-          uint32_t v[32];
-          tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(O_COL + half * 32), v);
-          float o[32];
+        uint16_t* orow = P.out + tok * P.ldo + h * D + half * 32;
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(v[e]);
-#pragma unroll 1
-          for (int k = 0; k < n_ext; ++k) {
-            const uint4* vrow = reinterpret_cast<const uint4*>(P.V + (tok - (int64_t)(k + 1) * l) * P.ld + h * D) + half * 4;
-            const float pk = s_ext[k];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const uint4 x = __ldg(vrow + q);
-              o[8 * q + 0] = fmaf(pk, bf_lo(x.x), o[8 * q + 0]); o[8 * q + 1] = fmaf(pk, bf_hi(x.x), o[8 * q + 1]);
-              o[8 * q + 2] = fmaf(pk, bf_lo(x.y), o[8 * q + 2]); o[8 * q + 3] = fmaf(pk, bf_hi(x.y), o[8 * q + 3]);
-              o[8 * q + 4] = fmaf(pk, bf_lo(x.z), o[8 * q + 4]); o[8 * q + 5] = fmaf(pk, bf_hi(x.z), o[8 * q + 5]);
-              o[8 * q + 6] = fmaf(pk, bf_lo(x.w), o[8 * q + 6]); o[8 * q + 7] = fmaf(pk, bf_hi(x.w), o[8 * q + 7]);
-            }
-          }
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            uint4 w;
-            w.x = pack_bf16(o[8 * q + 0] * inv, o[8 * q + 1] * inv);
-            w.y = pack_bf16(o[8 * q + 2] * inv, o[8 * q + 3] * inv);
-            w.z = pack_bf16(o[8 * q + 4] * inv, o[8 * q + 5] * inv);
-            w.w = pack_bf16(o[8 * q + 6] * inv, o[8 * q + 7] * inv);
-            reinterpret_cast<uint4*>(orow)[half * 4 + q] = w;
-          }
+        for (int g = 0; g < 4; ++g) {
+          uint4 w;
+          w.x = pack_bf16(o[8 * g + 0] * inv, o[8 * g + 1] * inv);
+          w.y = pack_bf16(o[8 * g + 2] * inv, o[8 * g + 3] * inv);
+          w.z = pack_bf16(o[8 * g + 4] * inv, o[8 * g + 5] * inv);
+          w.w = pack_bf16(o[8 * g + 6] * inv, o[8 * g + 7] * inv);
+          reinterpret_cast<uint4*>(orow)[g] = w;
         }
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_far_empty);   // the far warps may overwrite their columns and statistics
+      tc_fence_before();   // the next tile's products overwrite S and O after this warp's next arrival on bar_p
+    }
+  } else {
+    // ------------------------------------------------------------------ far positions: i - 2l, i - 3l, ...
+    // A softmax of their own per row (maximum, sum, weighted value sum in fp32), formed while the other warps work on
+    // the previous tile, handed over through 64 spare tensor-memory columns and two floats of shared memory per row.
+    const int q = warp & 3;                 // lane quarter = the 32 rows this warp serves
+    const int r = q * 32 + lane;
+    const float c = 0.125f * 1.4426950408889634f;
+    float* far_stat = red + 2 * BQ;
+    const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
+    uint32_t it = 0;
+    for (int t = blockIdx.x; t < P.tiles; t += gridDim.x, ++it) {
+      int b, h, q0;
+      tile_coords(P, t, b, h, q0);
+      const int i = q0 + r;
+      const int n_far = i / l - 1 < MAX_FAR ? i / l - 1 : MAX_FAR;   // uniform over the warp; may be <= 0
+      float se[MAX_FAR];
+      float m_e = -INFINITY, sum_e = 0.f;
+      uint32_t oe[2][32];
+      if (n_far > 0) {
+        far_scores(P, t, q, lane, l, se);
+#pragma unroll
+        for (int k = 0; k < MAX_FAR; ++k) m_e = fmaxf(m_e, k < n_far ? se[k] : -INFINITY);
+        float acc[64];
+#pragma unroll
+        for (int e = 0; e < 64; ++e) acc[e] = 0.f;
+        const int64_t tok = (int64_t)b * P.seq + i;
+#pragma unroll 1
+        for (int k = 0; k < n_far; ++k) {
+          float sk = se[0];
+#pragma unroll
+          for (int kk = 1; kk < MAX_FAR; ++kk) sk = kk == k ? se[kk] : sk;
+          const float pk = ex2_ftz((sk - m_e) * c);
+          sum_e += pk;
+          const uint4* vrow = reinterpret_cast<const uint4*>(P.V + (tok - (int64_t)(k + 2) * l) * P.ld + h * D);
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            const uint4 x = __ldg(vrow + g);
+            acc[8 * g + 0] = fmaf(pk, bf_lo(x.x), acc[8 * g + 0]); acc[8 * g + 1] = fmaf(pk, bf_hi(x.x), acc[8 * g + 1]);
+            acc[8 * g + 2] = fmaf(pk, bf_lo(x.y), acc[8 * g + 2]); acc[8 * g + 3] = fmaf(pk, bf_hi(x.y), acc[8 * g + 3]);
+            acc[8 * g + 4] = fmaf(pk, bf_lo(x.z), acc[8 * g + 4]); acc[8 * g + 5] = fmaf(pk, bf_hi(x.z), acc[8 * g + 5]);
+            acc[8 * g + 6] = fmaf(pk, bf_lo(x.w), acc[8 * g + 6]); acc[8 * g + 7] = fmaf(pk, bf_hi(x.w), acc[8 * g + 7]);
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          oe[0][e] = __float_as_uint(acc[e]);
+          oe[1][e] = __float_as_uint(acc[32 + e]);
+        }
+      }
+      // the previous tile's epilogue has read the columns and the statistics
+      if (it > 0 && !att_wait(bar_far_empty, (it - 1) & 1u, abort_flag)) break;
+      tc_fence_after();
+      if (n_far > 0) {
+        tmem_st32(t_row + (uint32_t)FAR_COL, oe[0]);
+        tmem_st32(t_row + (uint32_t)(FAR_COL + 32), oe[1]);
+        far_stat[2 * r] = m_e;
+        far_stat[2 * r + 1] = sum_e;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_far_full);
     }
   }
 
@@ -277,7 +464,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
@@ -326,7 +513,7 @@ extern "C" mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, 
                                                   void* Out, int64_t ldo, float* lse, mst_stream_t stream) {
   if (!Q || !K || !V || !Out || batch < 0 || seq_len <= 0 || heads <= 0) return MST_ERR_INVALID_ARG;
   if (head_dim != D || seq_len % BQ != 0 || stride <= 0 || stride % KB != 0 || stride + KB > O_COL) return MST_ERR_SHAPE;
-  if (seq_len / stride - 1 > MAX_EXTRA) return MST_ERR_SHAPE;
+  if (seq_len / stride - 2 > MAX_FAR) return MST_ERR_SHAPE;
   const int64_t width = (int64_t)heads * D;
   if (ld < width || ldo < width || ld % 8 != 0 || ldo % 8 != 0) return MST_ERR_SHAPE;
   if (((reinterpret_cast<uintptr_t>(Q) | reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V) |
@@ -346,9 +533,17 @@ extern "C" mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, 
   P.lse = lse;
   P.seq = seq_len; P.heads = heads; P.stride = stride;
   P.nkb = stride / KB + 1;
-  const size_t smem = (size_t)(1 + 4 * P.nkb) * TILE_BYTES + 1024 + 64;
+  P.batch = batch;
+  P.qblocks = seq_len / BQ;
+  const int64_t tiles = (int64_t)batch * heads * P.qblocks;
+  if (tiles > 0x7FFFFFFF) return MST_ERR_SHAPE;
+  P.tiles = (int)tiles;
+  const size_t smem = (size_t)(1 + 4 * P.nkb) * TILE_BYTES + RED_BYTES + 1024 + 128;
   MST_CUDA_TRY(cudaFuncSetAttribute(strided_attention_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  dim3 grid((unsigned)(seq_len / BQ), (unsigned)heads, (unsigned)batch);
+  int dev = 0, sms = 0;
+  MST_CUDA_TRY(cudaGetDevice(&dev));
+  MST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int grid = (int)(tiles < sms ? tiles : sms);   // one persistent block per SM
   strided_attention_fwd_kernel<<<grid, ATT_THREADS, smem, (cudaStream_t)stream>>>(tmQ, tmK, tmV, P);
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;

@@ -3,12 +3,22 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdio>
+#include <cstdlib>
+
 #include "mst.h"
 
-#define MST_CUDA_TRY(expr)                       \
-  do {                                           \
-    cudaError_t e__ = (expr);                    \
-    if (e__ != cudaSuccess) return MST_ERR_CUDA; \
+// With MST_DEBUG set in the environment a failing CUDA call is named on stderr before MST_ERR_CUDA is returned.
+inline void mst_report_cuda_error(cudaError_t e, const char* what, const char* file, int line) {
+  if (getenv("MST_DEBUG")) fprintf(stderr, "libmst: %s failed at %s:%d: %s\n", what, file, line, cudaGetErrorString(e));
+}
+#define MST_CUDA_TRY(expr)                                        \
+  do {                                                            \
+    cudaError_t e__ = (expr);                                     \
+    if (e__ != cudaSuccess) {                                     \
+      mst_report_cuda_error(e__, #expr, __FILE__, __LINE__);      \
+      return MST_ERR_CUDA;                                        \
+    }                                                             \
   } while (0)
 
 #define MST_TRY(expr)                   \
