@@ -41,7 +41,7 @@ constexpr int TMEM_COLS = 512;
 constexpr int O_COL = 448;     // output accumulator: tensor-memory columns 448..511
 constexpr int FAR_COL = 384;   // far positions' weighted value sums: columns 384..447
 constexpr int MAX_FAR = 6;       // attended positions outside the tile, i - 2l, i - 3l, ...: seq / l - 2
-constexpr int RED_BYTES = 2 * BQ * 4 + 2 * BQ * 4;  // partial row sums of a pair's two warps; far positions' (max, sum)
+constexpr int RED_BYTES = 3 * 2 * BQ * 4;  // a pair's partial row sums, the far positions' (max, sum), a pair's partial maxima
 
 __device__ int g_attn_error = 0;
 
@@ -141,7 +141,8 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
   const uint32_t q_s = base, k_s = q_s + TILE_BYTES, v_s = k_s + nkb * TILE_BYTES, p_s = v_s + nkb * TILE_BYTES;
   const uint32_t red_s = p_s + 2 * nkb * TILE_BYTES;
   const uint32_t bar0 = red_s + RED_BYTES;
-  const uint32_t bar_qk = bar0, bar_v = bar0 + 8, bar_s = bar0 + 16, bar_p = bar0 + 24, bar_o = bar0 + 32;
+  const uint32_t bar_qk = bar0, bar_v = bar0 + 8, bar_s = bar0 + 16, bar_o = bar0 + 32;
+  const uint32_t bar_p0 = bar0 + 88;     // one per key block: P of that block is written (and S read) by all softmax warps
   const uint32_t bar_pair0 = bar0 + 40;  // one per lane quarter
   const uint32_t bar_far_full = bar0 + 72, bar_far_empty = bar0 + 80;
   float* red = reinterpret_cast<float*>(smem_raw + (red_s - smem_u32(smem_raw)));  // [2 halves][128 rows]
@@ -157,7 +158,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
     mbar_init(bar_qk, 1);
     mbar_init(bar_v, 1);
     mbar_init(bar_s, 1);
-    mbar_init(bar_p, SM_WARPS);
+    for (int kb = 0; kb < 3; ++kb) mbar_init(bar_p0 + 8 * kb, SM_WARPS);
     mbar_init(bar_o, 1);
     for (int qq = 0; qq < 4; ++qq) mbar_init(bar_pair0 + 8 * qq, 2);
     mbar_init(bar_far_full, FAR_WARPS);
@@ -204,7 +205,6 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
                               ((uint32_t)(BQ >> 4) << 24);
       const uint64_t qd = smem_desc(q_s, 16, 1024), kd0 = smem_desc(k_s, 16, 1024);
       const uint64_t pd0 = smem_desc(p_s, 16, 1024), vd0 = smem_desc(v_s, 8192, 1024);
-      const int ksteps = nkb * KB / 16;
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < P.tiles && ok && !*abort_flag; t += gridDim.x, ++it) {
@@ -220,15 +220,21 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
             tc_mma(tmem_base + (uint32_t)(kb * KB), qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc1, ks > 0 ? 1u : 0u);
         }
         tc_commit(bar_s);
-        // second product once P is in shared memory and V has landed
-        ok = att_wait(bar_v, ph, abort_flag) && att_wait(bar_p, ph, abort_flag);
-        if (!ok) break;
-        tc_fence_after();
-        for (int ks = 0; ks < ksteps; ++ks) {
-          const uint64_t pd = pd0 + (uint64_t)(uint32_t)((ks >> 2) * (TILE_BYTES >> 4) + (ks & 3) * 2);
-          const uint64_t vd = vd0 + (uint64_t)(uint32_t)(ks * ((16 * 128) >> 4));
-          tc_mma(tmem_base + (uint32_t)O_COL, pd, vd, idesc2, ks > 0 ? 1u : 0u);
+        // second product, key block by key block as the softmax warps finish writing P for it
+        ok = att_wait(bar_v, ph, abort_flag);
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+          ok = att_wait(bar_p0 + 8 * kb, ph, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k8 = 0; k8 < KB / 16; ++k8) {
+            const int ks = kb * (KB / 16) + k8;
+            const uint64_t pd = pd0 + (uint64_t)(uint32_t)((ks >> 2) * (TILE_BYTES >> 4) + (ks & 3) * 2);
+            const uint64_t vd = vd0 + (uint64_t)(uint32_t)(ks * ((16 * 128) >> 4));
+            tc_mma(tmem_base + (uint32_t)O_COL, pd, vd, idesc2, ks > 0 ? 1u : 0u);
+          }
         }
+        if (!ok) break;
         tc_commit(bar_o);
       }
     }
@@ -241,6 +247,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
     const uint32_t sw = (uint32_t)(r & 7);
     const int nchunks = nkb * 4;
     float* red_sum = red;                   // [2][128]
+    float* red_max = red + 4 * BQ;          // [2][128]
     // The position i - l is row r of the tile's first key block, so its score sits in S and its value in the V tile:
     // the window mask simply reaches one key further (distance <= l).  Positions i - 2l, i - 3l, ... lie outside
     // the tile: the far warps form their softmax partials (maximum, sum, weighted value sum) a tile ahead and the
@@ -266,8 +273,8 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
       const int ch_lo = (jb < 0 && -jb / 32 > q) ? -jb / 32 : q;
       const int ch_hi = l / 32 + q;
       const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
-      // pass 1: row maximum.  Both warps of the pair scan every visible chunk (cheaper than meeting to exchange it);
-      // the load of the next chunk is in flight while this one is reduced.
+      // pass 1: row maximum over this warp's chunks (those of its parity), the load of the next chunk in flight while
+      // this one is reduced; the pair then exchanges its maxima
       {
         auto reduce_max = [&](const uint32_t (&v)[32], int ch) {
           const int j0 = jb + ch * 32;
@@ -285,21 +292,28 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
           }
           m = fmaxf(fmaxf(m, fmaxf(m4[0], m4[1])), fmaxf(m4[2], m4[3]));
         };
-        uint32_t va[32], vb[32];
-        int ch = ch_lo;
-        tmem_ld32_nowait(t_row + (uint32_t)(ch * 32), va);
+        int ch = ch_lo + ((ch_lo ^ half) & 1);
+        if (ch <= ch_hi) {
+          uint32_t va[32], vb[32];
+          tmem_ld32_nowait(t_row + (uint32_t)(ch * 32), va);
 #pragma unroll 1
-        while (true) {
-          tmem_ld_wait(va);
-          if (ch + 1 <= ch_hi) tmem_ld32_nowait(t_row + (uint32_t)((ch + 1) * 32), vb);
-          reduce_max(va, ch);
-          if (++ch > ch_hi) break;
-          tmem_ld_wait(vb);
-          if (ch + 1 <= ch_hi) tmem_ld32_nowait(t_row + (uint32_t)((ch + 1) * 32), va);
-          reduce_max(vb, ch);
-          if (++ch > ch_hi) break;
+          while (true) {
+            tmem_ld_wait(va);
+            if (ch + 2 <= ch_hi) tmem_ld32_nowait(t_row + (uint32_t)((ch + 2) * 32), vb);
+            reduce_max(va, ch);
+            ch += 2;
+            if (ch > ch_hi) break;
+            tmem_ld_wait(vb);
+            if (ch + 2 <= ch_hi) tmem_ld32_nowait(t_row + (uint32_t)((ch + 2) * 32), va);
+            reduce_max(vb, ch);
+            ch += 2;
+            if (ch > ch_hi) break;
+          }
         }
       }
+      red_max[half * BQ + r] = m;
+      if (!pair_meet(bar_pair0 + 8 * q, 0, lane, abort_flag)) break;   // two meetings per tile: parities 0, 1
+      m = fmaxf(m, red_max[(half ^ 1) * BQ + r]);                      // finite: the pair has seen key i itself
       // pass 2 over this warp's chunks (those of its parity): P = exp(s - m) in bf16 into the operand layout,
       // partial row sum in fp32; chunks of its parity outside the visible range are zero-filled
       float s4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -340,21 +354,26 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
                          "r"(w[4 * g + 2]), "r"(w[4 * g + 3])
                          : "memory");
         };
+        // visible chunks of this warp's parity, key block by key block; each finished block is announced so that the
+        // second product can start on it while the later blocks are still exponentiated
 #pragma unroll 1
-        for (int ch = ch_lo + ((ch_lo ^ half) & 1); ch <= ch_hi; ch += 2) {   // visible chunks of this warp's parity
-          uint32_t v[32];
-          tmem_ld32(t_row + (uint32_t)(ch * 32), v);
-          exp_store(v, ch);
+        for (int kb = 0; kb < nkb; ++kb) {
+#pragma unroll 1
+          for (int ch = 4 * kb + half; ch < 4 * kb + 4; ch += 2) {
+            if (ch < ch_lo || ch > ch_hi) continue;
+            uint32_t v[32];
+            tmem_ld32(t_row + (uint32_t)(ch * 32), v);
+            exp_store(v, ch);
+          }
+          fence_async_smem();   // P is read by the tensor core through the async proxy
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_p0 + 8 * kb);
         }
       }
       float sum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
       red_sum[half * BQ + r] = sum;
-      fence_async_smem();   // P is read by the tensor core through the async proxy
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_p);
-
-      if (!pair_meet(bar_pair0 + 8 * q, ph, lane, abort_flag)) break;   // one meeting per tile
+      if (!pair_meet(bar_pair0 + 8 * q, 1, lane, abort_flag)) break;
       sum += red_sum[(half ^ 1) * BQ + r];
       if (!att_wait(bar_o, ph, abort_flag)) break;
       if (!att_wait(bar_far_full, ph, abort_flag)) break;
@@ -392,7 +411,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_far_empty);   // the far warps may overwrite their columns and statistics
-      tc_fence_before();   // the next tile's products overwrite S and O after this warp's next arrival on bar_p
+      tc_fence_before();   // the next tile's products overwrite S and O after this warp's next arrivals
     }
   } else {
     // ------------------------------------------------------------------ far positions: i - 2l, i - 3l, ...
