@@ -37,7 +37,8 @@ def _run(p, stride, want_lse=True, pad=0):
     (1, 1024, 2, 256, 0),      # the paper's setting: n = 1024, l = 256
     (3, 256, 2, 256, 8),       # stride = n: plain causal attention inside one window; padded leading dimensions
     (2, 128, 1, 128, 0),       # a single query block
-    (1, 1024, 1, 128, 0)])     # seven strided positions
+    (1, 1024, 1, 128, 0),      # seven strided positions
+    (1, 2048, 2, 256, 0)])     # the longest supported sequence for l = 256: six positions outside the tile
 def test_forward_matches_oracle(batch, seq, heads, stride, pad):
     p = mst_inputs.attention_problem(batch, seq, heads, 64, seed=900 + seq + stride)
     out, lse = _run(p, stride, pad=pad)
