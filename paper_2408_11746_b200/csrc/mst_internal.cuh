@@ -21,6 +21,41 @@ inline void mst_report_cuda_error(cudaError_t e, const char* what, const char* f
     }                                                             \
   } while (0)
 
+// Programmatic dependent launch.  A kernel started with mst_launch_overlapped may become resident and run its set-up
+// (barrier initialisation, tensor-memory allocation, descriptor fetch) while its predecessor in the stream drains; it
+// executes mst_grid_dependency_wait() before it reads or writes global memory (a no-op for a normal launch), and
+// mst_grid_launch_dependents() as early as it likes to let its own successor do the same.  MST_PDL=0 turns the
+// launch attribute off.
+#ifdef __CUDACC__
+__device__ __forceinline__ void mst_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void mst_grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+inline int mst_pdl_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("MST_PDL");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v;
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t mst_launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                         Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = mst_pdl_enabled();
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 #define MST_TRY(expr)                   \
   do {                                  \
     mst_status_t s__ = (expr);          \

@@ -188,6 +188,8 @@ __global__ void fill_csc(const uint32_t* __restrict__ bitsT, const int32_t* __re
 __global__ void densify_from_bits(const uint32_t* __restrict__ bits, const int32_t* __restrict__ wscan, int R, int C,
                                   int wpr, const uint16_t* __restrict__ vals, const int32_t* __restrict__ perm,
                                   uint16_t* __restrict__ dense) {
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();
   const unsigned g = blockIdx.x * blockDim.x + threadIdx.x;  // group of 8 columns
   const unsigned gpr = (unsigned)C >> 3;                     // groups per row
   if (g >= (unsigned)R * gpr) return;
@@ -332,11 +334,13 @@ mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s) {
   const int c = L->cur;
   const int64_t groups = L->N / 8;  // callers guarantee O % 8 == 0 and I % 8 == 0
   if (!transpose)
-    densify_from_bits<<<blocks_for(groups, 256), 256, 0, s>>>(L->bits[c], L->wscan[c], L->O, L->I, L->wpr,
-                                                             (const uint16_t*)L->vals[c], nullptr, L->dense_w);
+    MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
+                                       (const uint32_t*)L->bits[c], (const int32_t*)L->wscan[c], L->O, L->I, L->wpr,
+                                       (const uint16_t*)L->vals[c], (const int32_t*)nullptr, L->dense_w));
   else
-    densify_from_bits<<<blocks_for(groups, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->I, L->O, L->wpc,
-                                                             (const uint16_t*)L->vals[c], L->perm, L->dense_wt);
+    MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
+                                       (const uint32_t*)L->bitsT, (const int32_t*)L->wscanT, L->I, L->O, L->wpc,
+                                       (const uint16_t*)L->vals[c], (const int32_t*)L->perm, L->dense_wt));
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

@@ -334,6 +334,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();  // set-up above overlaps the predecessor's tail; global memory only from here on
 
   const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
   const int tiles = P.m_tiles * P.n_tiles;
@@ -536,6 +538,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   cluster_sync_all();  // both blocks' barriers are initialised before any remote arrival or copy completion
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_holder;
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();
 
   const int m_pairs = (P.m_tiles + 1) / 2;
   const int tiles = m_pairs * P.n_tiles;
@@ -646,6 +650,8 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 // out[i] = sum over splits of partial[s][i], fixed order
 __global__ void tc_reduce_kernel(const float* __restrict__ partial, int splits, int64_t n, float* __restrict__ out) {
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   float s = partial[i];
@@ -828,17 +834,19 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
     const int64_t works = (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles * P.splits;
     const int64_t max_pairs = sm_count() / 2;
     const int grid = 2 * (int)(works < max_pairs ? works : max_pairs);
-    tc_gemm_pair_kernel<<<grid, NUM_THREADS, P_SMEM_BYTES, s>>>(tmA, tmB, tmC, P);
+    MST_CUDA_TRY(mst_launch_overlapped(tc_gemm_pair_kernel, dim3(grid), dim3(NUM_THREADS), P_SMEM_BYTES, s, tmA, tmB, tmC, P));
   } else {
     MST_CUDA_TRY(cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES));
     const int64_t works = (int64_t)P.m_tiles * P.n_tiles * P.splits;
     const int grid = (int)(works < sm_count() ? works : sm_count());
-    tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, s>>>(tmA, tmB, tmC, P);
+    MST_CUDA_TRY(mst_launch_overlapped(tc_gemm_kernel, dim3(grid), dim3(NUM_THREADS), SMEM_BYTES, s, tmA, tmB, tmC, P));
   }
   MST_CUDA_TRY(cudaGetLastError());
   if (P.splits > 1) {
     const int64_t n = a.epilogue == MST_TC_OUT_F32 ? a.M * a.N : a.nnz;
-    if (n > 0) tc_reduce_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>(P.partial, P.splits, n, (float*)a.out);
+    if (n > 0)
+      MST_CUDA_TRY(mst_launch_overlapped(tc_reduce_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, s,
+                                         (const float*)P.partial, P.splits, n, (float*)a.out));
     MST_CUDA_TRY(cudaGetLastError());
   }
   return MST_OK;
