@@ -485,19 +485,24 @@ def main() -> None:
 
     # ---- end to end: host buffers in, host results out, through the C ABI
     def e2e_step(k):
-        # all four layers are issued before any wait: a layer's host copies overlap the other layers' kernels
+        # Every step copies its inputs in and its results out.  Nothing waits between layers or between steps: a layer's
+        # copies overlap the other layers' kernels, and a step's results leave while the next step's inputs arrive.
         for s in slots:
             mst.mst_layer_step_host_async(s.L.handle, s.Xh, s.dYh, T, s.Yh, s.dXh, s.dWh)
             s.L.dense_grad(s.dY, s.X, T, s.G)
             s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=2, step=k, G_dense=s.G, want_stats=False)
+
+    def e2e_wait():
         for s in slots:
             mst.mst_layer_step_host_wait(s.L.handle)
     e2e_step(0)
+    e2e_wait()
     barrier()
-    e2e_steps = max(2, min(args.steps, 5))
+    e2e_steps = max(2, min(args.steps, 10))
     a = ev()
     for k in range(e2e_steps):
         e2e_step(1 + k)
+    e2e_wait()               # the last step's results are in host memory
     b = ev()
     barrier()
     e2e_ms = max_over_ranks(a.elapsed_time(b), dist, dev)

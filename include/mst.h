@@ -255,8 +255,11 @@ mst_status_t mst_device_error_flags(int32_t* flags);
 /* The same step without the final wait: inputs are copied on a copy-in stream owned by the layer, the three products
  * run on `stream`, results are copied back on a copy-out stream owned by the layer.  Calls for several layers issued
  * one after the other overlap one layer's copies with another layer's kernels (host buffers must be pinned for that).
- * mst_layer_step_host_wait blocks until the layer's results are in host memory.  A layer's next async step waits for
- * its previous one by itself. */
+ * mst_layer_step_host_wait blocks until the results of the layer's latest async step (and of every earlier one) are
+ * in host memory.  Steps of one layer may be issued back to back without a wait: the next step's inputs are copied in
+ * once the previous step's kernels have read them, its kernels start once the previous results have left the device
+ * buffers; the host buffers of a step must stay untouched until a wait that covers it has returned.
+ * Bit 1 of mst_device_error_flags is the attention kernel's expired-wait flag. */
 mst_status_t mst_layer_step_host_async(mst_layer_t* layer, const void* X_host, const void* dY_host, int64_t T,
                                        void* Y_host, void* dX_host, float* dW_vals_host, mst_stream_t stream);
 mst_status_t mst_layer_step_host_wait(mst_layer_t* layer);

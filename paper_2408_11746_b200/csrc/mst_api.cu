@@ -212,14 +212,16 @@ extern "C" mst_status_t mst_layer_step_host_async(mst_layer_t* L, const void* X_
     MST_CUDA_TRY(cudaMalloc((void**)&L->stg_dw, sizeof(float) * L->cap));
     L->stg_tokens = Ta;
   }
-  // inputs travel on the layer's copy-in stream once the previous step has finished with the staging buffers
-  MST_CUDA_TRY(cudaStreamWaitEvent(L->s_in, L->ev_out, 0));
+  // Inputs travel on the layer's copy-in stream as soon as the previous step's kernels have read the input staging
+  // buffers; its results may still be on their way out (the two directions of the link work at the same time).
+  MST_CUDA_TRY(cudaStreamWaitEvent(L->s_in, L->ev_compute, 0));
   if (T > 0) {
     MST_CUDA_TRY(cudaMemcpyAsync(L->stg_x, X_host, es * T * L->I, cudaMemcpyHostToDevice, L->s_in));
     MST_CUDA_TRY(cudaMemcpyAsync(L->stg_dy, dY_host, es * T * L->O, cudaMemcpyHostToDevice, L->s_in));
   }
   MST_CUDA_TRY(cudaEventRecord(L->ev_in, L->s_in));
   MST_CUDA_TRY(cudaStreamWaitEvent(s, L->ev_in, 0));
+  MST_CUDA_TRY(cudaStreamWaitEvent(s, L->ev_out, 0));  // the previous step's results have left the output staging buffers
   MST_TRY(mst_launch_spmm(L, false, L->stg_x, L->I, T, L->stg_y, L->O, s));
   MST_TRY(mst_launch_spmm(L, true, L->stg_dy, L->O, T, L->stg_dx, L->I, s));
   MST_TRY(mst_launch_sddmm(L, L->stg_dy, L->O, L->stg_x, L->I, T, L->stg_dw, s));

@@ -333,6 +333,35 @@ def test_async_host_step_overlaps_layers_and_matches():
         L.close()
 
 
+def test_async_host_steps_back_to_back_without_waiting():
+    # three steps of one layer issued without a wait in between, each with its own inputs and result buffers: a
+    # step's inputs arrive while the previous step's results leave, and no staging buffer is reused too early
+    O, I, T = 512, 768, 2048          # large enough that the copies and the kernels really overlap
+    steps = []
+    L = None
+    for k in range(3):
+        p = _problem(O, I, T, "bf16", 0.2, 8300 + k)
+        if L is None:
+            p0, L = p, make_layer(p)
+        q = mst_inputs.make_layer(p0.name, p0.layer_id, O, I, T, "bf16", p0.mask, 8300 + k)   # same weights' mask, new X / dY
+        q.W, q.W_bits = p0.W, p0.W_bits
+        want = _run_products(q, L)[:3]
+        b = dict(X=torch.from_numpy(q.X_bits.view(np.int16)).pin_memory(), dY=torch.from_numpy(q.dY_bits.view(np.int16)).pin_memory(),
+                 Y=torch.zeros((T, O), dtype=torch.int16).pin_memory(), dX=torch.zeros((T, I), dtype=torch.int16).pin_memory(),
+                 dW=torch.zeros((p0.nnz,), dtype=torch.float32).pin_memory())
+        steps.append((want, b))
+    for _, b in steps:
+        mst.mst_layer_step_host_async(L.handle, b["X"], b["dY"], T, b["Y"], b["dX"], b["dW"])
+    mst.mst_layer_step_host_wait(L.handle)      # the latest step; the earlier ones precede it on the same streams
+    torch.cuda.synchronize()
+    for (Y, dX, dW), b in steps:
+        np.testing.assert_array_equal(mst_inputs.bf16_bits_to_f32(b["Y"].numpy().view(np.uint16)), Y)
+        np.testing.assert_array_equal(mst_inputs.bf16_bits_to_f32(b["dX"].numpy().view(np.uint16)), dX)
+        np.testing.assert_array_equal(b["dW"].numpy(), dW)
+    assert mst.mst_device_error_flags() == 0
+    L.close()
+
+
 @pytest.mark.parametrize("T", [0, 1, 127, 129])
 def test_token_count_edges_on_the_tensor_path(T):
     O, I = 256, 192
