@@ -249,7 +249,8 @@ mst_status_t mst_er_densities(int32_t n_layers, const int32_t* out_features, con
                               double global_density, double* densities);
 
 /* Sticky error bits of kernels that run without a layer handle (bit 0: a bounded wait inside the tensor-core
- * contraction expired and the block gave up; its output is then undefined).  Synchronises the device. */
+ * contraction expired and the block gave up; its output is then undefined; bit 1: the same in the attention
+ * kernel).  Synchronises the device. */
 mst_status_t mst_device_error_flags(int32_t* flags);
 
 /* The same step without the final wait: inputs are copied on a copy-in stream owned by the layer, the three products
@@ -258,8 +259,7 @@ mst_status_t mst_device_error_flags(int32_t* flags);
  * mst_layer_step_host_wait blocks until the results of the layer's latest async step (and of every earlier one) are
  * in host memory.  Steps of one layer may be issued back to back without a wait: the next step's inputs are copied in
  * once the previous step's kernels have read them, its kernels start once the previous results have left the device
- * buffers; the host buffers of a step must stay untouched until a wait that covers it has returned.
- * Bit 1 of mst_device_error_flags is the attention kernel's expired-wait flag. */
+ * buffers; the host buffers of a step must stay untouched until a wait that covers it has returned. */
 mst_status_t mst_layer_step_host_async(mst_layer_t* layer, const void* X_host, const void* dY_host, int64_t T,
                                        void* Y_host, void* dX_host, float* dW_vals_host, mst_stream_t stream);
 mst_status_t mst_layer_step_host_wait(mst_layer_t* layer);
