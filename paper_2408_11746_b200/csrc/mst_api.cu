@@ -93,7 +93,6 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   const size_t o_flags = cv.take(4 * 4);
   const size_t o_counter = cv.take(4);
   const size_t o_dense = dtype == MST_BF16 ? cv.take(2 * (size_t)N) : 0;
-  const size_t o_denseT = dtype == MST_BF16 ? cv.take(2 * (size_t)N) : 0;
 
   unsigned char* base = nullptr;
   if (cudaMalloc((void**)&base, cv.off) != cudaSuccess) {
@@ -128,7 +127,7 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->flags = (int32_t*)(base + o_flags);
   L->counter = (unsigned int*)(base + o_counter);
   L->dense_w = dtype == MST_BF16 ? (uint16_t*)(base + o_dense) : nullptr;
-  L->dense_wt = dtype == MST_BF16 ? (uint16_t*)(base + o_denseT) : nullptr;
+  L->csc_valid = 0;
   L->path = MST_PATH_AUTO;
   L->stg_x = L->stg_dy = L->stg_y = L->stg_dx = nullptr;
   L->stg_dw = nullptr;

@@ -93,7 +93,9 @@ struct mst_layer {
   uint16_t* col_idx[2];  // [cap]
   void* vals[2];         // [cap] layer dtype
 
-  // CSC view of the live structure
+  // CSC view of the live structure.  Built at pack; the fused update skips it for layers whose input gradient runs
+  // on the tensor path (which reads the dense image, not the CSC view) and it is then rebuilt on first use.
+  mutable int csc_valid;
   uint32_t* bitsT;       // [nwordsT]
   int32_t* wscanT;       // [nwordsT+1]
   int32_t* col_ptr;      // [I+1]
@@ -112,9 +114,9 @@ struct mst_layer {
   int32_t* flags;         // [4]: error bits, max row nnz, spare
   unsigned int* counter;  // [1] block-completion counter
 
-  // dense bf16 images of W.M for the tensor-core path (bf16 layers only): [O x I] and its transpose [I x O]
+  // dense bf16 image of W.M for the tensor-core path (bf16 layers only): [O x I]; the input gradient reads it as an
+  // MN-major operand, so no transposed copy is kept
   uint16_t* dense_w;
-  uint16_t* dense_wt;
   int path;  // mst_compute_path_t
 
   // host staging for mst_layer_step_host
@@ -137,8 +139,9 @@ mst_status_t mst_scan_i32_if(const int32_t* in, int32_t* out, int64_t n, int32_t
                              cudaStream_t s);
 mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set, cudaStream_t s);
 mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s);
+mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s);  // builds the CSC view if it is stale
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
-mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s);
+mst_status_t mst_densify(const mst_layer* L, cudaStream_t s);
 bool mst_use_tensor_path(const mst_layer* L);
 
 // sticky error word of the attention kernel's bounded waits (mst_attention.cu)

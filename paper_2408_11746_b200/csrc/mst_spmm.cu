@@ -227,14 +227,16 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
   if (T == 0) return MST_OK;
   const int c = L->cur;
   const int rows = transpose ? L->I : L->O, cols = transpose ? L->O : L->I;
-  // Dense-tile tensor-core path: expand W.M (or its transpose) to a dense bf16 image, then out = in * image^T.
+  // Dense-tile tensor-core path: expand W.M to a dense bf16 image [O x I].  Forward: out = in * image^T, the image a
+  // K-major operand.  Input gradient: out = in * image, the same image read as an MN-major operand ([K = O] rows of
+  // I contiguous columns), so no transposed copy and no CSC view are needed.
   if (mst_use_tensor_path(L) && (ldout % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0)) {
-    const uint16_t* image = transpose ? L->dense_wt : L->dense_w;
-    if (mst_tc_gemm_usable(in, ldin, image, cols)) {
-      MST_TRY(mst_densify(L, transpose, s));
+    const uint16_t* image = L->dense_w;
+    if (mst_tc_gemm_usable(in, ldin, image, L->I)) {
+      MST_TRY(mst_densify(L, s));
       mst_tc_gemm_args a = {};
       a.A = in; a.lda = ldin; a.a_mn_major = 0;
-      a.B = image; a.ldb = cols; a.b_mn_major = 0;
+      a.B = image; a.ldb = L->I; a.b_mn_major = transpose ? 1 : 0;
       a.M = T; a.N = rows; a.K = cols;
       a.epilogue = MST_TC_OUT_BF16;
       a.out = out; a.ldc = ldout; a.splits = 1;
@@ -251,6 +253,7 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
              ? launch<float, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, s)
              : launch<uint16_t, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, s);
   } else {
+    MST_TRY(mst_ensure_csc(L, s));
     st = L->dtype == MST_F32
              ? launch<float, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, s)
              : launch<uint16_t, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, s);

@@ -327,20 +327,23 @@ mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s) {
   fill_csc<<<blocks_for(L->nwordsT * 32, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->O, L->I, L->wpr, L->wpc, L->bits[c],
                                                             L->wscan[c], L->row_idx, L->perm, L->col_ptr);
   MST_CUDA_TRY(cudaGetLastError());
+  L->csc_valid = 1;
   return MST_OK;
 }
 
-mst_status_t mst_densify(const mst_layer* L, bool transpose, cudaStream_t s) {
+mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s) {
+  if (L->csc_valid) return MST_OK;
+  return mst_build_csc(const_cast<mst_layer*>(L), s);
+}
+
+mst_status_t mst_densify(const mst_layer* L, cudaStream_t s) {
   const int c = L->cur;
-  const int64_t groups = L->N / 8;  // callers guarantee O % 8 == 0 and I % 8 == 0
-  if (!transpose)
+  const int64_t groups = L->N / 8;  // callers guarantee I % 8 == 0
+  {
     MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
                                        (const uint32_t*)L->bits[c], (const int32_t*)L->wscan[c], L->O, L->I, L->wpr,
                                        (const uint16_t*)L->vals[c], (const int32_t*)nullptr, L->dense_w));
-  else
-    MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
-                                       (const uint32_t*)L->bitsT, (const int32_t*)L->wscanT, L->I, L->O, L->wpc,
-                                       (const uint16_t*)L->vals[c], (const int32_t*)L->perm, L->dense_wt));
+  }
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
@@ -394,6 +397,7 @@ extern "C" mst_status_t mst_export_csc(const mst_layer_t* L, int32_t* col_ptr, i
   if (!L) return MST_ERR_INVALID_ARG;
   if (L->nnz < 0) return MST_ERR_NOT_PACKED;
   cudaStream_t s = (cudaStream_t)stream;
+  MST_TRY(mst_ensure_csc(L, s));
   if (col_ptr)
     MST_CUDA_TRY(cudaMemcpyAsync(col_ptr, L->col_ptr, sizeof(int32_t) * (L->I + 1), cudaMemcpyDeviceToDevice, s));
   if (row_idx && L->nnz > 0) widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->row_idx, L->nnz, row_idx);
@@ -408,6 +412,7 @@ extern "C" mst_status_t mst_validate(const mst_layer_t* L, mst_stream_t stream) 
   if (L->nnz < 0) return MST_ERR_NOT_PACKED;
   cudaStream_t s = (cudaStream_t)stream;
   const int c = L->cur;
+  MST_TRY(mst_ensure_csc(L, s));
   validate_rows<<<blocks_for(L->O, 128), 128, 0, s>>>(L->row_ptr[c], L->col_idx[c], L->bits[c], L->O, L->I, L->wpr,
                                                      L->nnz, L->flags);
   validate_cols<<<blocks_for(L->I, 128), 128, 0, s>>>(L->col_ptr, L->row_idx, L->perm, L->row_ptr[c], L->col_idx[c],

@@ -335,6 +335,7 @@ struct FusedParams {
   int32_t* perm;
   int wpc;
   int64_t nwordsT;
+  int build_csc;  // 0: leave the CSC view stale (the layer's input gradient reads the dense image instead)
 };
 
 struct FusedShared {
@@ -404,7 +405,7 @@ __device__ int fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int6
     if (i < hi) out[i] = carry + ex;
     carry += tile_total;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) out[n] = tot;
+  if (threadIdx.x == 0) out[n] = tot;  // every block writes the same total: whoever reads it next in this block sees it
   __syncthreads();
   return tot;
 }
@@ -621,15 +622,16 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   __syncthreads();
   fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, grid, sh);
   // the barrier inside the scan came after every block wrote its part of the new mask: transpose it now
-  {
+  if (F.build_csc) {
     const int64_t tiles = (int64_t)F.wpc * P.wpr;
     for (int64_t t = (int64_t)blockIdx.x * FUSED_WARPS + warp; t < tiles; t += (int64_t)gridDim.x * FUSED_WARPS)
       mst_transpose_tile(t, lane, F.new_bits, P.O, P.I, P.wpr, F.wpc, F.bitsT);
+    grid.sync();  // the transposed mask is complete everywhere
   }
-  grid.sync();  // transposed mask and the scan of the new mask are complete everywhere
   for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * 4)
     mst_fill_csr_words<V, 4>(w0, FUSED_WARPS, hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col, (V*)F.new_vals,
                              F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals, &F.flags[1]);
+  if (!F.build_csc) return;  // uniform over the grid
   for (int64_t w = loT + threadIdx.x; w < hiT; w += FUSED_THREADS) F.cnt[w] = __popc(F.bitsT[w]);
   __syncthreads();
   const int totT = fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, grid, sh);
@@ -739,6 +741,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     F.new_wscan = L->wscan[n]; F.new_row_ptr = L->row_ptr[n]; F.new_col = L->col_idx[n]; F.new_vals = L->vals[n];
     F.bitsT = L->bitsT; F.wscanT = L->wscanT; F.col_ptr = L->col_ptr; F.row_idx = L->row_idx; F.perm = L->perm;
     F.wpc = L->wpc; F.nwordsT = L->nwordsT;
+    F.build_csc = mst_use_tensor_path(L) ? 0 : 1;
+    L->csc_valid = F.build_csc;
     void* args[] = {&F};
     const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
     MST_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3(grid_blocks), dim3(FUSED_THREADS), args, fused_smem, s));

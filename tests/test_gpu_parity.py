@@ -419,3 +419,32 @@ def test_staged_and_direct_stores_agree(O, I, T, monkeypatch):
     assert rel_err(host(outs[0][2]).reshape(O, I), oracle.dense_grad(p.dY, p.X)) <= 1e-5
     assert mst.mst_device_error_flags() == 0
     L.close()
+
+
+def test_csc_view_is_rebuilt_on_demand_after_an_update():
+    # the fused update leaves the CSC view stale for layers whose input gradient runs on the tensor path; the
+    # CUDA-core input gradient, the CSC export and the structure check rebuild it when they need it
+    p = _problem(256, 320, 200, "bf16", 0.2, 9400)
+    L = make_layer(p)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
+    Wn, Mn = _update_both(L, p, W, p.mask.copy(), G, 0.3, -1, 0.25, 5, 0)      # ends with validate
+    st = mst.mst_topology_update(L.handle, 0.2, -1, 0.5, 5, 1, False, torch.from_numpy(G).to(dev()))   # stale again
+    n_prune, _, n_rand, n_grad = oracle.mg_counts(0.2, int(Mn.sum()), -1, Mn.size, 0.5)
+    Wn, Mn, *_ = oracle.mg_update(Wn, Mn, G, n_prune, n_grad, n_rand, 5, 1, p.layer_id)
+    dXr = oracle.bwd_x(p.dY, Wn, Mn)
+    dY = to_dev(p, "dY")
+    for path in (mst.MST_PATH_TENSOR_CORE, mst.MST_PATH_CUDA_CORE):
+        L.set_path(path)
+        dX = torch.full((p.tokens, 320), float("nan"), dtype=torch.bfloat16, device=dev())
+        L.bwd_x(dY, dX, p.tokens)
+        torch.cuda.synchronize()
+        assert rel_err(host(dX), dXr) <= TOL["bf16"], path
+    cp, ri, pm = export_csc(L)
+    rp, ci, _ = export_csr(L, "bf16")
+    rows = np.repeat(np.arange(256), np.diff(rp))
+    order = np.lexsort((rows, ci))                   # CSC order: by column, then row
+    np.testing.assert_array_equal(ri, rows[order])
+    np.testing.assert_array_equal(pm, order)
+    np.testing.assert_array_equal(cp, np.concatenate([[0], np.cumsum(np.bincount(ci, minlength=320))]))
+    L.close()
