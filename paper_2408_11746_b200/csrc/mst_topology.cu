@@ -587,6 +587,8 @@ template <typename V>
 __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const FusedParams F) {
   cg::grid_group grid = cg::this_grid();
   __shared__ FusedShared sh;
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();
   const SelParams& P = F.sel;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t per = (P.nwords + gridDim.x - 1) / gridDim.x;
@@ -745,7 +747,20 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     L->csc_valid = F.build_csc;
     void* args[] = {&F};
     const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
-    MST_CUDA_TRY(cudaLaunchCooperativeKernel(fn, dim3(grid_blocks), dim3(FUSED_THREADS), args, fused_smem, s));
+    // cooperative launch that may also start while its predecessor drains (the kernel waits before its first access)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid_blocks);
+    cfg.blockDim = dim3(FUSED_THREADS);
+    cfg.dynamicSmemBytes = fused_smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = mst_pdl_enabled() ? 2 : 1;
+    MST_CUDA_TRY(cudaLaunchKernelExC(&cfg, fn, args));
   } else {
     MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
     MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
