@@ -56,6 +56,14 @@ template <int MODE>
 struct KeyBits {
   static constexpr int value = MODE == MODE_RAND ? 64 : 32;
 };
+template <int MODE>
+struct KeyWord {
+  typedef uint32_t type;
+};
+template <>
+struct KeyWord<MODE_RAND> {
+  typedef unsigned long long type;
+};
 
 // candidate test and key of bit `lane` of word w.  nonfinite is set when a magnitude key is Inf/NaN.
 template <int MODE>
@@ -416,6 +424,8 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
                              int& gpass, cg::grid_group& grid, FusedShared& sh, const uint32_t* s_old,
                              const int32_t* s_base, uint32_t* s_grad) {
   constexpr int KB = KeyBits<MODE>::value;
+  // magnitude keys are 32 bits wide: their passes compare and shift 32-bit words, only the hashes need 64
+  typedef typename KeyWord<MODE>::type K;
   constexpr int passes = num_passes(KB);
   const SelParams& P = F.sel;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -441,7 +451,7 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     const int shift = pass_shift(KB, pass), width = pass_width(KB, pass);
     const unsigned dmask = (1u << width) - 1u;
     const int hi_shift = shift + width;
-    const unsigned long long prefix = sh.prefix;
+    const K prefix = (K)sh.prefix;
     const long long k = sh.k;
     unsigned int* gh = F.hist + (gpass % 3) * BINS;
     for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
@@ -454,13 +464,14 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
 #pragma unroll
       for (int j = 0; j < BATCH; ++j) {
         const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
-        unsigned long long key = 0;
+        unsigned long long key64 = 0;
         bool nf = false;
         const int64_t li = w < hi ? w - lo : 0;
-        const bool c = w < hi && cand_key_w<MODE>(P, w, lane, s_old[li], s_base[li], s_grad[li], key, nf);
+        const bool c = w < hi && cand_key_w<MODE>(P, w, lane, s_old[li], s_base[li], s_grad[li], key64, nf);
+        const K key = (K)key64;
         saw_nonfinite |= (c && nf);
-        live[j] = c && (pass == 0 || (key >> hi_shift) == prefix);
-        digit[j] = live[j] ? (unsigned)((key >> shift) & dmask) : (unsigned)BINS;
+        live[j] = c && (pass == 0 || (K)(key >> hi_shift) == prefix);
+        digit[j] = live[j] ? (unsigned)((key >> shift) & (K)dmask) : (unsigned)BINS;
       }
 #pragma unroll
       for (int j = 0; j < BATCH; ++j) {
@@ -539,15 +550,15 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     }
     ++gpass;
   }
-  const unsigned long long tau = sh.tau;
+  const K tau = (K)sh.tau;
   const long long rem = sh.rem;
   const bool need_rank = sh.need_rank != 0;
   if (need_rank) {  // rank the entries equal to tau in index order
     for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
-      unsigned long long key;
+      unsigned long long key64;
       bool nf;
-      const bool c = cand_key_w<MODE>(P, w, lane, s_old[w - lo], s_base[w - lo], s_grad[w - lo], key, nf);
-      const unsigned eq = __ballot_sync(0xffffffffu, c && key == tau);
+      const bool c = cand_key_w<MODE>(P, w, lane, s_old[w - lo], s_base[w - lo], s_grad[w - lo], key64, nf);
+      const unsigned eq = __ballot_sync(0xffffffffu, c && (K)key64 == tau);
       if (lane == 0) F.cnt[w] = __popc(eq);
     }
     __syncthreads();
@@ -556,14 +567,15 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
   constexpr int MB = 4;
   for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * MB) {
     bool c[MB], iseq[MB];
-    unsigned long long key[MB];
+    K key[MB];
 #pragma unroll
     for (int j = 0; j < MB; ++j) {
       const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
       bool nf = false;
-      key[j] = 0;
+      unsigned long long key64 = 0;
       const int64_t li = w < hi ? w - lo : 0;
-      c[j] = w < hi && cand_key_w<MODE>(P, w, lane, s_old[li], s_base[li], s_grad[li], key[j], nf);
+      c[j] = w < hi && cand_key_w<MODE>(P, w, lane, s_old[li], s_base[li], s_grad[li], key64, nf);
+      key[j] = (K)key64;
       iseq[j] = c[j] && key[j] == tau;
     }
 #pragma unroll
