@@ -467,7 +467,7 @@ def main() -> None:
     # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of this call kind on layer fc1 (O=3072, I=768), from the
     # ncu capture summarised in profiles/tc_gemm_pair_and_fused_update_gpt2small_block_d0.25.md (cold caches; output
     # rows still sitting in L2 at kernel end are not counted).  Algorithmic bytes of the same launch beside it.
-    NCU_TRAFFIC_FC1 = {"spmm_fwd": 19.36e6, "spmm_bwd_x": 57.64e6, "sddmm_dw": 66.70e6, "dense_grad": 66.65e6}
+    NCU_TRAFFIC_FC1 = {"spmm_fwd": 19.34e6, "spmm_bwd_x": 57.84e6, "sddmm_dw": 66.49e6, "dense_grad": 66.52e6}
     if dom in NCU_TRAFFIC_FC1 and tensor_path:
         fc1 = next(s for s in slots if s.O == 3072 and s.I == 768)
         roof["traffic"] = NCU_TRAFFIC_FC1[dom]
