@@ -807,6 +807,10 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
     const int64_t slots = pair ? sm_count() / 2 : sm_count();
     const double out_bytes = a.epilogue == MST_TC_OUT_F32 ? 4.0 * (double)a.M * (double)a.N : 4.0 * (double)a.nnz;
     P.splits = a.splits > 0 ? a.splits : mst_tc_pick_splits(works1, slots, P.kblocks, out_bytes);
+    if (const char* e = getenv("MST_TC_SPLITS")) {  // measurement override
+      const int v = atoi(e);
+      if (v > 0) P.splits = v;
+    }
     if (P.splits > P.kblocks) P.splits = P.kblocks;
     if (P.splits > 1) {
       const size_t per = a.epilogue == MST_TC_OUT_F32 ? (size_t)a.M * a.N : (size_t)a.nnz;
