@@ -419,7 +419,13 @@ __device__ int fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int6
 }
 
 // One selection inside the fused kernel.  gpass counts the histogram passes executed so far (buffer rotation).
-template <int MODE>
+// Words per warp whose keys may stay in registers for a whole selection (CACHED): the warp's words are fixed
+// (lo + warp + j * FUSED_WARPS), so each lane loads the key of its bit of each word once and every later pass, the tie
+// count and the marking sweep work from registers instead of fetching G or the values again.  For the 64-bit hash keys
+// the high word is kept; the digits below bit 32 and ties on the high word recompute the hash.
+constexpr int KEYS_PER_LANE = 16;
+
+template <int MODE, bool CACHED>
 __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* out_bits, int64_t lo, int64_t hi,
                              int& gpass, cg::grid_group& grid, FusedShared& sh, const uint32_t* s_old,
                              const int32_t* s_base, uint32_t* s_grad) {
@@ -446,6 +452,33 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     sh.done = 0;
   }
   __syncthreads();
+  uint32_t kc[KEYS_PER_LANE];  // CACHED: key word of this lane's bit of word j; bit j of candm: it is a candidate
+  uint32_t candm = 0;
+  bool cache_nonfinite = false;
+  if (CACHED) {
+#pragma unroll
+    for (int j = 0; j < KEYS_PER_LANE; ++j) {
+      const int64_t w = lo + warp + (int64_t)j * FUSED_WARPS;
+      kc[j] = 0;
+      if (w < hi) {  // uniform over the warp
+        unsigned long long key64 = 0;
+        bool nf = false;
+        const bool c = cand_key_w<MODE>(P, w, lane, s_old[w - lo], s_base[w - lo], s_grad[w - lo], key64, nf);
+        kc[j] = MODE == MODE_RAND ? (uint32_t)(key64 >> 32) : (uint32_t)key64;
+        if (c) candm |= 1u << j;
+        cache_nonfinite |= (c && nf);
+      }
+    }
+  }
+  // full-width key of cached entry j (a candidate): only the hash keys hold more than the cached word
+  auto cached_full_key = [&](int j) -> K {
+    if (MODE != MODE_RAND) return (K)kc[j];
+    const int64_t w = lo + warp + (int64_t)j * FUSED_WARPS;
+    unsigned long long key64 = 0;
+    bool nf = false;
+    cand_key_w<MODE>(P, w, lane, s_old[w - lo], s_base[w - lo], s_grad[w - lo], key64, nf);
+    return (K)key64;
+  };
   for (int pass = 0; pass < passes; ++pass) {
     if (sh.done) break;  // same decision in every block
     const int shift = pass_shift(KB, pass), width = pass_width(KB, pass);
@@ -456,8 +489,24 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     unsigned int* gh = F.hist + (gpass % 3) * BINS;
     for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
     __syncthreads();
-    bool saw_nonfinite = false;
+    bool saw_nonfinite = cache_nonfinite;
     constexpr int BATCH = 8;
+    if (CACHED) {
+      const bool hi_word = MODE == MODE_RAND && shift >= 32;  // digit and prefix lie inside the cached high word
+#pragma unroll
+      for (int j = 0; j < KEYS_PER_LANE; ++j) {
+        if (lo + warp + (int64_t)j * FUSED_WARPS >= hi) break;  // uniform over the warp
+        const bool c = (candm >> j) & 1u;
+        K key = 0;
+        if (MODE != MODE_RAND) key = (K)kc[j];
+        else if (hi_word) key = (K)((unsigned long long)kc[j] << 32);
+        else if (c) key = cached_full_key(j);
+        const bool lv = c && (pass == 0 || (K)(key >> hi_shift) == prefix);
+        const unsigned dg = lv ? (unsigned)((key >> shift) & (K)dmask) : (unsigned)BINS;
+        const unsigned peers = __match_any_sync(0xffffffffu, dg);
+        if (lv && lane == (__ffs(peers) - 1)) atomicAdd(&sh.hist[dg], (unsigned)__popc(peers));
+      }
+    } else
     for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * BATCH) {
       unsigned digit[BATCH];
       bool live[BATCH];
@@ -554,6 +603,21 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
   const long long rem = sh.rem;
   const bool need_rank = sh.need_rank != 0;
   if (need_rank) {  // rank the entries equal to tau in index order
+    if (CACHED) {
+#pragma unroll
+      for (int j = 0; j < KEYS_PER_LANE; ++j) {
+        const int64_t w = lo + warp + (int64_t)j * FUSED_WARPS;
+        if (w >= hi) break;
+        const bool c = (candm >> j) & 1u;
+        bool e = false;
+        if (c) {
+          if (MODE != MODE_RAND) e = (K)kc[j] == tau;
+          else if ((K)kc[j] == (K)(tau >> (KB - 32))) e = cached_full_key(j) == tau;
+        }
+        const unsigned eq = __ballot_sync(0xffffffffu, e);
+        if (lane == 0) F.cnt[w] = __popc(eq);
+      }
+    } else
     for (int64_t w = lo + warp; w < hi; w += FUSED_WARPS) {
       unsigned long long key64;
       bool nf;
@@ -565,6 +629,37 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     fused_grid_scan(F.cnt, F.scan, P.nwords, lo, hi, F.bsums, grid, sh);
   }
   constexpr int MB = 4;
+  if (CACHED) {
+#pragma unroll
+    for (int j = 0; j < KEYS_PER_LANE; ++j) {
+      const int64_t w = lo + warp + (int64_t)j * FUSED_WARPS;
+      if (w >= hi) break;  // uniform over the warp
+      const bool c = (candm >> j) & 1u;
+      bool below = false, equal = false;
+      if (c) {
+        if (MODE != MODE_RAND) {
+          below = (K)kc[j] < tau;
+          equal = (K)kc[j] == tau;
+        } else {
+          const K th = (K)(tau >> (KB - 32));
+          if ((K)kc[j] < th) below = true;
+          else if ((K)kc[j] == th) {
+            const K key = cached_full_key(j);
+            below = key < tau;
+            equal = key == tau;
+          }
+        }
+      }
+      const unsigned eq = __ballot_sync(0xffffffffu, equal);
+      const long long rank = need_rank ? (long long)F.scan[w] + __popc(eq & lanemask_lt()) : -1;
+      const bool take = below || (equal && rank < rem);
+      const unsigned bits = __ballot_sync(0xffffffffu, take);
+      if (lane == 0) {
+        out_bits[w] = bits;
+        if (MODE == MODE_GRAD) s_grad[w - lo] = bits;
+      }
+    }
+  } else
   for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * MB) {
     bool c[MB], iseq[MB];
     K key[MB];
@@ -623,9 +718,15 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   __syncthreads();
 
   int gpass = 0;
-  fused_select<MODE_PRUNE>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
-  fused_select<MODE_GRAD>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
-  fused_select<MODE_RAND>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+  if (per <= (int64_t)FUSED_WARPS * KEYS_PER_LANE) {  // uniform over the grid: every warp's words fit its key registers
+    fused_select<MODE_PRUNE, true>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_GRAD, true>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_RAND, true>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+  } else {
+    fused_select<MODE_PRUNE, false>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_GRAD, false>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_RAND, false>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+  }
 
   // mask rewrite: new = (old & ~pruned) | grad | rand, and its popcounts
   for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
