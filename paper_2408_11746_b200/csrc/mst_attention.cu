@@ -39,7 +39,6 @@ constexpr int FAR_WARPS = 4;               // warps for the attended positions o
 constexpr int ATT_THREADS = 64 + 32 * SM_WARPS + 32 * FAR_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int O_COL = 448;     // output accumulator: tensor-memory columns 448..511
-constexpr int FAR_COL = 384;   // far positions' weighted value sums: columns 384..447
 constexpr int MAX_FAR = 6;       // attended positions outside the tile, i - 2l, i - 3l, ...: seq / l - 2
 constexpr int RED_BYTES = 3 * 2 * BQ * 4;  // a pair's partial row sums, the far positions' (max, sum), a pair's partial maxima
 
@@ -144,7 +143,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
   const uint32_t bar_qk = bar0, bar_v = bar0 + 8, bar_s = bar0 + 16, bar_o = bar0 + 32;
   const uint32_t bar_p0 = bar0 + 88;     // one per key block: P of that block is written (and S read) by all softmax warps
   const uint32_t bar_pair0 = bar0 + 40;  // one per lane quarter
-  const uint32_t bar_far_full = bar0 + 72, bar_far_empty = bar0 + 80;
+  const uint32_t bar_stat = bar0 + 72, bar_epi = bar0 + 80;  // window statistics published / epilogue of the tile done
   float* red = reinterpret_cast<float*>(smem_raw + (red_s - smem_u32(smem_raw)));  // [2 halves][128 rows]
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_sh;
@@ -161,8 +160,8 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
     for (int kb = 0; kb < 3; ++kb) mbar_init(bar_p0 + 8 * kb, SM_WARPS);
     mbar_init(bar_o, 1);
     for (int qq = 0; qq < 4; ++qq) mbar_init(bar_pair0 + 8 * qq, 2);
-    mbar_init(bar_far_full, FAR_WARPS);
-    mbar_init(bar_far_empty, SM_WARPS);
+    mbar_init(bar_stat, SM_WARPS / 2);
+    mbar_init(bar_epi, FAR_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -222,6 +221,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
         tc_commit(bar_s);
         // second product, key block by key block as the softmax warps finish writing P for it
         ok = att_wait(bar_v, ph, abort_flag);
+        if (ok && it > 0) ok = att_wait(bar_epi, (it - 1) & 1u, abort_flag);   // the previous tile's O has been read
         for (int kb = 0; kb < nkb && ok; ++kb) {
           ok = att_wait(bar_p0 + 8 * kb, ph, abort_flag);
           if (!ok) break;
@@ -252,7 +252,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
     // the window mask simply reaches one key further (distance <= l).  Positions i - 2l, i - 3l, ... lie outside
     // the tile: the far warps form their softmax partials (maximum, sum, weighted value sum) a tile ahead and the
     // epilogue below merges them with the window's.
-    const float* far_stat = red + 2 * BQ;   // [128][2]: maximum (unscaled score), sum
+    float* win_stat = red + 2 * BQ;         // [128][2]: the window's maximum (unscaled score) and sum, for the epilogue
     int t = blockIdx.x;
     uint32_t it = 0;
     for (; t < P.tiles; t += gridDim.x, ++it) {
@@ -262,7 +262,6 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
       const int i = q0 + r;                 // position in the sequence
       const int jb = q0 - l;                // first key of the tile (may be negative)
       const int64_t tok = (int64_t)b * P.seq + i;
-      const bool has_far = i / l >= 2;      // uniform over the warp (32 rows between multiples of 128)
       float m = -INFINITY;
       const int i_lo = q0 + q * 32, i_hi = i_lo + 31;
 
@@ -375,69 +374,44 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
       red_sum[half * BQ + r] = sum;
       if (!pair_meet(bar_pair0 + 8 * q, 1, lane, abort_flag)) break;
       sum += red_sum[(half ^ 1) * BQ + r];
-      if (!att_wait(bar_o, ph, abort_flag)) break;
-      if (!att_wait(bar_far_full, ph, abort_flag)) break;
-      tc_fence_after();
-      {
-        // this warp's half of the output columns; merge the far positions' partial softmax
-        uint32_t v[32];
-        tmem_ld32(t_row + (uint32_t)(O_COL + half * 32), v);
-        float o[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(v[e]);
-        float mm = m;
-        if (has_far) {
-          const float m_e = far_stat[2 * r], sum_e = far_stat[2 * r + 1];
-          tmem_ld32(t_row + (uint32_t)(FAR_COL + half * 32), v);
-          mm = fmaxf(m, m_e);
-          const float a_w = ex2_ftz((m - mm) * c), a_e = ex2_ftz((m_e - mm) * c);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = fmaf(a_w, o[e], a_e * __uint_as_float(v[e]));
-          sum = fmaf(a_w, sum, a_e * sum_e);
-        }
-        if (P.lse && half == 0) P.lse[((int64_t)b * P.heads + h) * P.seq + i] = mm * 0.125f + __logf(sum);
-        const float inv = 1.0f / sum;
-        uint16_t* orow = P.out + tok * P.ldo + h * D + half * 32;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint4 w;
-          w.x = pack_bf16(o[8 * g + 0] * inv, o[8 * g + 1] * inv);
-          w.y = pack_bf16(o[8 * g + 2] * inv, o[8 * g + 3] * inv);
-          w.z = pack_bf16(o[8 * g + 4] * inv, o[8 * g + 5] * inv);
-          w.w = pack_bf16(o[8 * g + 6] * inv, o[8 * g + 7] * inv);
-          reinterpret_cast<uint4*>(orow)[g] = w;
-        }
+      // The epilogue belongs to the far warps: they hold the far positions' partial sums in registers, read O from
+      // tensor memory when the second product has completed and write the rows.  The first warp of the pair hands them
+      // the window's maximum and sum; these warps go straight on to the next tile.
+      if (half == 0) {
+        if (it > 0 && !att_wait(bar_epi, (it - 1) & 1u, abort_flag)) break;   // the previous tile's pair has been read
+        win_stat[2 * r] = m;
+        win_stat[2 * r + 1] = sum;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_stat);
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_far_empty);   // the far warps may overwrite their columns and statistics
       tc_fence_before();   // the next tile's products overwrite S and O after this warp's next arrivals
     }
   } else {
     // ------------------------------------------------------------------ far positions: i - 2l, i - 3l, ...
-    // A softmax of their own per row (maximum, sum, weighted value sum in fp32), formed while the other warps work on
-    // the previous tile, handed over through 64 spare tensor-memory columns and two floats of shared memory per row.
+    // A softmax of their own per row (maximum, sum, weighted value sum in fp32, kept in registers), formed while the
+    // other warps work on the tile; then the tile's epilogue: O from tensor memory once the second product has
+    // completed, the window's maximum and sum from shared memory, the two partial softmaxes merged, rows written.
     const int q = warp & 3;                 // lane quarter = the 32 rows this warp serves
     const int r = q * 32 + lane;
     const float c = 0.125f * 1.4426950408889634f;
-    float* far_stat = red + 2 * BQ;
+    const float* win_stat = red + 2 * BQ;
     const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16);
     uint32_t it = 0;
     for (int t = blockIdx.x; t < P.tiles; t += gridDim.x, ++it) {
+      const uint32_t ph = it & 1u;
       int b, h, q0;
       tile_coords(P, t, b, h, q0);
       const int i = q0 + r;
       const int n_far = i / l - 1 < MAX_FAR ? i / l - 1 : MAX_FAR;   // uniform over the warp; may be <= 0
       float se[MAX_FAR];
       float m_e = -INFINITY, sum_e = 0.f;
-      uint32_t oe[2][32];
+      float acc[64];
+#pragma unroll
+      for (int e = 0; e < 64; ++e) acc[e] = 0.f;
       if (n_far > 0) {
         far_scores(P, t, q, lane, l, se);
 #pragma unroll
         for (int k = 0; k < MAX_FAR; ++k) m_e = fmaxf(m_e, k < n_far ? se[k] : -INFINITY);
-        float acc[64];
-#pragma unroll
-        for (int e = 0; e < 64; ++e) acc[e] = 0.f;
         const int64_t tok = (int64_t)b * P.seq + i;
 #pragma unroll 1
         for (int k = 0; k < n_far; ++k) {
@@ -456,24 +430,45 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
             acc[8 * g + 6] = fmaf(pk, bf_lo(x.w), acc[8 * g + 6]); acc[8 * g + 7] = fmaf(pk, bf_hi(x.w), acc[8 * g + 7]);
           }
         }
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          oe[0][e] = __float_as_uint(acc[e]);
-          oe[1][e] = __float_as_uint(acc[32 + e]);
-        }
       }
-      // the previous tile's epilogue has read the columns and the statistics
-      if (it > 0 && !att_wait(bar_far_empty, (it - 1) & 1u, abort_flag)) break;
+      // epilogue of the tile: O / sum merged with the far positions' partial softmax, written as bf16
+      if (!att_wait(bar_o, ph, abort_flag)) break;
+      if (!att_wait(bar_stat, ph, abort_flag)) break;
       tc_fence_after();
-      if (n_far > 0) {
-        tmem_st32(t_row + (uint32_t)FAR_COL, oe[0]);
-        tmem_st32(t_row + (uint32_t)(FAR_COL + 32), oe[1]);
-        far_stat[2 * r] = m_e;
-        far_stat[2 * r + 1] = sum_e;
+      {
+        const float m_w = win_stat[2 * r];
+        float sum = win_stat[2 * r + 1];
+        float mm = m_w, a_w = 1.f, a_e = 0.f;
+        if (n_far > 0) {
+          mm = fmaxf(m_w, m_e);
+          a_w = ex2_ftz((m_w - mm) * c);
+          a_e = ex2_ftz((m_e - mm) * c);
+          sum = fmaf(a_w, sum, a_e * sum_e);
+        }
+        if (P.lse) P.lse[((int64_t)b * P.heads + h) * P.seq + i] = mm * 0.125f + __logf(sum);
+        const float inv = 1.0f / sum;
+        uint16_t* orow = P.out + ((int64_t)b * P.seq + i) * P.ldo + h * D;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t v[32];
+          tmem_ld32(t_row + (uint32_t)(O_COL + hf * 32), v);
+          float o[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] = fmaf(a_w, __uint_as_float(v[e]), a_e * acc[hf * 32 + e]) * inv;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint4 w;
+            w.x = pack_bf16(o[8 * g + 0], o[8 * g + 1]);
+            w.y = pack_bf16(o[8 * g + 2], o[8 * g + 3]);
+            w.z = pack_bf16(o[8 * g + 4], o[8 * g + 5]);
+            w.w = pack_bf16(o[8 * g + 6], o[8 * g + 7]);
+            reinterpret_cast<uint4*>(orow)[hf * 4 + g] = w;
+          }
+        }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_far_full);
+      if (lane == 0) mbar_arrive(bar_epi);
     }
   }
 
