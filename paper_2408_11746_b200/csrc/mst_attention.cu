@@ -199,6 +199,7 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
     if (lane == 0) {
       // S[:, kb*128 .. +128) = Q K_kb^T : M = 128, N = 128, both operands K-major, four K steps of 16
       const uint32_t idesc1 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(KB >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
+      const uint32_t idesc1_wide = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)((2 * KB) >> 3) << 17) | ((uint32_t)(BQ >> 4) << 24);
       // O = P V : M = 128, N = 64, P K-major (64-key blocks of 16 KiB), V as stored (keys x 64: MN-major)
       const uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(D >> 3) << 17) |
                               ((uint32_t)(BQ >> 4) << 24);
@@ -212,11 +213,14 @@ strided_attention_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __gr
         ok = att_wait(bar_qk, ph, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        for (int kb = 0; kb < nkb; ++kb) {
+        // key blocks two at a time (N = 256: the blocks are contiguous in shared memory), a last odd one alone:
+        // each instruction carries a fixed cost, and the softmax warps wait for the whole of this product
+        for (int kb = 0; kb < nkb; kb += 2) {
           const uint64_t kd = kd0 + (uint64_t)(uint32_t)(kb * (TILE_BYTES >> 4));
+          const uint32_t idesc = kb + 1 < nkb ? idesc1_wide : idesc1;
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
-            tc_mma(tmem_base + (uint32_t)(kb * KB), qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc1, ks > 0 ? 1u : 0u);
+            tc_mma(tmem_base + (uint32_t)(kb * KB), qd + (uint64_t)(ks * 2), kd + (uint64_t)(ks * 2), idesc, ks > 0 ? 1u : 0u);
         }
         tc_commit(bar_s);
         // second product, key block by key block as the softmax warps finish writing P for it
