@@ -97,6 +97,62 @@ def aggregate_value(useful_flops_per_step: float, steps: int, world: int, ms: fl
     return useful_flops_per_step * steps * world / (ms * 1e-3) / 1e12
 
 
+# ------------------------------------------------------------------------------------------ MLP report
+def run_mlp(args) -> None:
+    """fc1 -> GELU -> fc2 of GPT-2 small at 16384 tokens: the fused calls beside the plain products."""
+    import torch
+    import paper_2408_11746_b200 as mst
+    dev = torch.device("cuda", 0)
+    T = 16384
+    ps = {p.name: p for p in mst_inputs.config2(tokens=T)}
+    p1, p2 = ps["fc1"], ps["fc2"]
+
+    def up_bits(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    layers = []
+    for p in (p1, p2):
+        L = mst.Layer(p.layer_id, p.out_features, p.in_features, mst.MST_BF16)
+        L.pack(up_bits(p.W_bits), torch.from_numpy(p.mask).to(dev))
+        layers.append(L)
+    L1, L2 = layers
+    X, dY = up_bits(p1.X_bits), up_bits(p2.dY_bits)
+    H = torch.empty((T, p1.out_features), dtype=torch.bfloat16, device=dev)
+    Ypre, dPre = torch.empty_like(H), torch.empty_like(H)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(f, reps=10, inner=8):
+        for _ in range(3):
+            f()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(inner):
+                f()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / inner)
+        return float(np.median(ts)) * 1e3
+
+    L1.fwd_gelu(X, H, T, Y_pre=Ypre)
+    out = {
+        "report": "mlp_pair", "tokens": T, "fc1": [p1.out_features, p1.in_features], "density": 0.25,
+        "fwd_us": timed(lambda: L1.fwd(X, H, T)),
+        "fwd_gelu_us": timed(lambda: L1.fwd_gelu(X, H, T)),
+        "fwd_gelu_keep_preactivation_us": timed(lambda: L1.fwd_gelu(X, H, T, Y_pre=Ypre)),
+        "bwd_x_us": timed(lambda: L2.bwd_x(dY, dPre, T)),
+        "bwd_x_gelu_us": timed(lambda: L2.bwd_x_gelu(dY, Ypre, dPre, T)),
+        "elementwise_gelu_us": timed(lambda: torch.nn.functional.gelu(Ypre)),
+        "elementwise_gelu_backward_us": timed(lambda: torch.ops.aten.gelu_backward(dPre, Ypre)),
+    }
+    assert mst.mst_device_error_flags() == 0
+    print(json.dumps(out))
+    for L in layers:
+        L.close()
+
+
 # ------------------------------------------------------------------------------------------ attention report
 def run_attention(args) -> None:
     """Strided sparse attention forward on the attention input of a 16384-token GPT-2-small batch."""
@@ -307,10 +363,16 @@ def main() -> None:
     ap.add_argument("--attention", action="store_true",
                     help="report on the strided sparse attention forward (not the bench line): one JSON object per "
                          "stride at 16 x 1024 tokens, 12 heads of 64, with torch's dense causal attention beside it")
+    ap.add_argument("--mlp", action="store_true",
+                    help="report on the MLP pair with the activation fused (not the bench line): fc1 forward with GELU, "
+                         "fc2 input gradient with GELU', against the plain products, GPT-2 small, 16384 tokens")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.attention:
         run_attention(args)
+        return
+    if args.mlp:
+        run_mlp(args)
         return
     if args.impl == "reference":
         run_reference(args)

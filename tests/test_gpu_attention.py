@@ -61,16 +61,17 @@ def test_larger_scores_and_run_to_run_identity():
     assert rel_err(a, ref) <= TOL["bf16"]
 
 
-def test_gpt2_small_full_size_sampled():
+@pytest.mark.parametrize("stride", [256, 128])
+def test_gpt2_small_full_size_sampled(stride):
     # 16 sequences of 1024 tokens, 12 heads: the attention input of the benchmark's 16384-token batch
-    rng = np.random.default_rng(12)
+    rng = np.random.default_rng(12 + stride)
     p = mst_inputs.attention_problem(16, 1024, 12, 64)
-    out, _ = _run(p, 256, want_lse=False)
+    out, _ = _run(p, stride, want_lse=False)
     Q, K, V = p.split()
     n = 400
     b = rng.integers(0, 16, n); h = rng.integers(0, 12, n); i = rng.integers(0, 1024, n)
     i[:8] = [0, 127, 128, 255, 256, 511, 768, 1023]
-    ref = att.strided_attention_at(Q, K, V, 256, b, h, i)
+    ref = att.strided_attention_at(Q, K, V, stride, b, h, i)
     assert rel_err(out[b, h, i], ref) <= TOL["bf16"]
 
 
