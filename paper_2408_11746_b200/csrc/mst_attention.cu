@@ -7,13 +7,18 @@
 //   warp 0     TMA producer: Q and the l/128 + 1 key blocks as soon as the previous tile's S = Q K^T has completed,
 //              the value blocks as soon as the previous tile's O = P V has completed (single buffers, loads of tile
 //              t+1 fly during the softmax of tile t);
-//   warp 1     one lane issues tcgen05.mma: O(t) = P V once P(t) is written, then S(t+1) = Q K^T (fp32, tensor memory);
+//   warp 1     one lane issues tcgen05.mma: S = Q K^T (fp32, tensor memory; two key blocks per instruction), then
+//              O = P V key block by key block as the softmax warps announce each block of P;
 //   warps 2-9  softmax, two warps per tensor-memory lane quarter (thread = query row, the pair splitting the visible
-//              32-key chunks by parity and the output columns in halves): scores of the strided positions on CUDA
-//              cores, row maximum, P = exp(s - max) in bf16 into shared memory
-//              in the K-major 128-byte-swizzled operand layout, row sum, and after the second product O / sum plus
-//              the strided positions' values, written as bf16.  Chunks no row of the warp can see are skipped, chunks
-//              every row sees in full skip the mask arithmetic.
+//              32-key chunks by parity): row maximum (exchanged inside the pair), P = exp(s - max) in bf16 into shared
+//              memory in the K-major 128-byte-swizzled operand layout, row sum; the pair's first warp publishes the
+//              window's maximum and sum and both go on to the next tile.  Chunks no row of the warp can see are
+//              skipped, chunks every row sees in full skip the mask arithmetic.  The position i - l is row r of the
+//              tile's first key block, so the mask simply reaches one key further (distance <= l);
+//   warps 10-13 the positions outside the tile, i - 2l, i - 3l, ... (at most n/l - 2 per query): a softmax of their
+//              own on CUDA cores (scores, maximum, sum, weighted value sum kept in registers), then the tile's
+//              epilogue: O from tensor memory once the second product has completed, the two partial softmaxes
+//              merged, rows written as bf16 (and the log-sum-exp when asked for).
 // Keys before the start of the sequence (q0 < l) are fetched from the rows in front of it (another sequence of the
 // batch, or the TMA unit's zero fill before row 0) and masked by position, never by value.
 // Every mbarrier wait is bounded (abort flag + sticky error word), as in the contraction kernel.
