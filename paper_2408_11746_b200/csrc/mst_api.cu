@@ -88,7 +88,7 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   const size_t o_cnt = cv.take(4 * (size_t)(wmax + 1));
   const size_t o_scan = cv.take(4 * (size_t)(wmax + 1));
   const size_t o_bsum = cv.take(4 * (size_t)(mst_scan_block_sums_len(wmax) + 1024));
-  const size_t o_hist = cv.take(4 * 2048 * 3);
+  const size_t o_hist = cv.take(4 * (size_t)MST_SELECT_BINS * 3);
   const size_t o_sel = cv.take(sizeof(mst_select_state));
   const size_t o_flags = cv.take(4 * 4);
   const size_t o_counter = cv.take(4);

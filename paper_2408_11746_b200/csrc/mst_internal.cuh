@@ -109,7 +109,7 @@ struct mst_layer {
   int32_t* word_cnt;      // [max(nwords, nwordsT)+1]
   int32_t* word_scan;     // [max(nwords, nwordsT)+1]
   int32_t* block_sums;    // scan partials
-  unsigned int* hist;     // [2048]
+  unsigned int* hist;     // [3][MST_SELECT_BINS]: rotating global histograms of the radix select
   mst_select_state* sel;  // [1]
   int32_t* flags;         // [4]: error bits, max row nnz, spare
   unsigned int* counter;  // [1] block-completion counter
@@ -146,6 +146,10 @@ bool mst_use_tensor_path(const mst_layer* L);
 
 // sticky error word of the attention kernel's bounded waits (mst_attention.cu)
 mst_status_t mst_attention_error_flags(int32_t* flags);
+
+// bins of one radix-select pass (digit width MST_SELECT_RADIX_BITS)
+constexpr int MST_SELECT_RADIX_BITS = 11;
+constexpr int MST_SELECT_BINS = 1 << MST_SELECT_RADIX_BITS;
 
 // kernels' launchers
 // act / pre / ldpre: element-wise step fused behind the product (see mst_tc_gemm.cuh); act = 0 for the plain product

@@ -124,8 +124,8 @@ __device__ __forceinline__ bool cand_key(const SelParams& P, int64_t w, int lane
   return cand_key_w<MODE>(P, w, lane, ow, ob, gw, key, nonfinite);
 }
 
-constexpr int RADIX_BITS = 11;
-constexpr int BINS = 1 << RADIX_BITS;  // 2048
+constexpr int RADIX_BITS = MST_SELECT_RADIX_BITS;
+constexpr int BINS = MST_SELECT_BINS;
 constexpr int HIST_THREADS = 1024;
 constexpr int BINS_PER_THREAD = BINS / HIST_THREADS;
 
