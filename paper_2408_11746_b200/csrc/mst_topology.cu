@@ -743,7 +743,9 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   }
   for (int64_t w0 = lo + warp; w0 < hi; w0 += FUSED_WARPS * 4)
     mst_fill_csr_words<V, 4>(w0, FUSED_WARPS, hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col, (V*)F.new_vals,
-                             F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals, &F.flags[1]);
+                             F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals,
+                             F.build_csc ? &F.flags[1] : nullptr);  // without the barrier above the next row's scan entry
+                                                                    // may belong to a block that has not written it yet
   if (!F.build_csc) return;  // uniform over the grid
   for (int64_t w = loT + threadIdx.x; w < hiT; w += FUSED_THREADS) F.cnt[w] = __popc(F.bitsT[w]);
   __syncthreads();
@@ -885,7 +887,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   if (!fused) MST_TRY(mst_build_csc(L, s));
 
   if (stats) {
-    if (!fused) max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
+    // the fused kernel records the longest row itself only when it also builds the CSC view
+    if (!fused || !L->csc_valid) max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
     int32_t f[4] = {0, 0, 0, 0};
     int32_t total = 0;
     MST_CUDA_TRY(cudaMemcpyAsync(f, L->flags, sizeof(f), cudaMemcpyDeviceToHost, s));
