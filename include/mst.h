@@ -17,8 +17,13 @@
  *     host memory (stats, nnz) synchronise that stream.
  *   - argument, shape, dtype, capacity and count errors are detected on the host before any
  *     launch.  Problems only the device can see (a non-finite selection key, a corrupt structure)
- *     set a sticky flag in handle-owned memory that mst_validate and mst_topology_update(stats)
- *     report.
+ *     set a flag in handle-owned memory that stays set until mst_validate or
+ *     mst_topology_update(stats != NULL) has returned it once; an update with stats == NULL
+ *     never clears it.
+ *   - calls that split their contraction range (mst_dense_grad, mst_dense_grad_dw, mst_sddmm_dw,
+ *     mst_layer_step_host[_async] on bf16 layers) keep partial sums in one scratch buffer per
+ *     device, allocated on first use and grown on demand: two such calls must not overlap on the
+ *     GPU (one stream, or ordered by events).
  */
 #ifndef MST_H_
 #define MST_H_
@@ -157,7 +162,7 @@ mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, const void*
                                        int64_t ldo, float* lse, mst_stream_t stream);
 
 /* Weight gradient on the mask only, dW[k] = sum_t dY[t,o_k] X[t,i_k] for the k-th active entry in CSR order
- * (same passage).  dW_vals device float [nnz]. */
+ * (same passage).  dW_vals device float [nnz].  May use the per-device split scratch (see the conventions above). */
 mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,
                           float* dW_vals, mst_stream_t stream);
 
@@ -189,7 +194,10 @@ mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_t target_nn
  * deterministic.
  *   prune_frac  zeta in [0,1]
  *   G_dense     device float [O x I] contiguous; may be NULL iff n_grad == 0
- *   stats       host, may be NULL; when given the call synchronises and reports device-side errors */
+ *   stats       host, may be NULL; when given the call synchronises and reports device-side errors.  An update that
+ *               is reported as failed (MST_ERR_NONFINITE, MST_ERR_CORRUPT) is NOT applied: mask, values and nnz stay
+ *               as they were.  With stats == NULL nothing is checked on the host: a non-finite key then leaves an
+ *               applied, undefined selection behind and the error flag set for the next reporting call. */
 mst_status_t mst_topology_update(mst_layer_t* layer, double prune_frac, const mst_regrow_rule_t* regrow_rule,
                                  const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream);
 

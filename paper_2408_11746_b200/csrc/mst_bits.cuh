@@ -122,9 +122,10 @@ __device__ __forceinline__ void mst_fill_csr_words(int64_t w0, int64_t stride, i
     const int o = (int)(wu / (unsigned)wpr), wc = (int)(wu - (unsigned)o * (unsigned)wpr);
     if (wc == 0 && lane == 0) {
       row_ptr[o] = base[j];
-      const int32_t next = wscan[w + wpr];  // first word of the next row, or the total
       if (o == O - 1) row_ptr[O] = wscan[nwords];
-      if (max_row) atomicMax(max_row, next - base[j]);
+      // the next row's first scan entry (or the total) may belong to another block: read only behind a grid barrier,
+      // which is what a non-null max_row promises
+      if (max_row) atomicMax(max_row, wscan[w + wpr] - base[j]);
     }
     if ((b[j] >> lane) & 1u) {
       const int32_t pos = base[j] + __popc(b[j] & mst_lanemask_lt());

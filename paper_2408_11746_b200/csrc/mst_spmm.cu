@@ -176,12 +176,9 @@ constexpr size_t spmm_smem() {
 template <typename T, bool PERM>
 mst_status_t launch(const int32_t* ptr, const uint16_t* idx, const void* vals, const int32_t* perm, const void* in,
                     int64_t ldin, void* out, int64_t ldout, int64_t T_total, int R_total, int C, cudaStream_t s) {
-  static bool configured = false;
   const size_t smem = spmm_smem<T>();
-  if (!configured) {
-    MST_CUDA_TRY(cudaFuncSetAttribute(spmm_panel_kernel<T, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    configured = true;
-  }
+  // per call: the attribute belongs to the current device's copy of the kernel
+  MST_CUDA_TRY(cudaFuncSetAttribute(spmm_panel_kernel<T, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   constexpr int VEC = Cfg<T>::VEC;
   const int vec_ok = (ldin % VEC == 0) && (C % VEC == 0) && ((reinterpret_cast<uintptr_t>(in) & 15u) == 0);
   dim3 grid((unsigned)((R_total + PANEL - 1) / PANEL), (unsigned)((T_total + TOK - 1) / TOK));

@@ -421,6 +421,7 @@ extern "C" mst_status_t mst_validate(const mst_layer_t* L, mst_stream_t stream) 
   int32_t f = 0;
   MST_CUDA_TRY(cudaMemcpyAsync(&f, L->flags, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
   MST_CUDA_TRY(cudaStreamSynchronize(s));
+  if (f) MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t), s));  // reported once, then cleared
   if (f & MST_FLAG_CORRUPT) return MST_ERR_CORRUPT;
   if (f & MST_FLAG_NONFINITE) return MST_ERR_NONFINITE;
   return MST_OK;

@@ -727,13 +727,14 @@ bool make_out_map_f32(CUtensorMap* tm, void* base, int64_t M, int64_t N, int64_t
 }
 
 int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  static int n[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return 148;
+  if (!n[dev]) {
+    if (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0) n[dev] = 148;
   }
-  return n;
+  return n[dev];
 }
 
 }  // namespace
@@ -759,21 +760,29 @@ int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double ou
   return best;
 }
 
+// Scratch for the partial sums of a K-range split: one buffer per device, grown on demand (growing waits for the
+// device and frees the old buffer).  Every call that splits its contraction range shares its device's buffer, so two
+// such calls must not overlap on the GPU (mst_dense_grad, mst_dense_grad_dw, mst_sddmm_dw and the host-step calls on
+// the tensor path): keep them on one stream or order them with events.
 mst_status_t mst_workspace(size_t bytes, void** ptr) {
-  static void* buf = nullptr;
-  static size_t cap = 0;
-  if (bytes > cap) {
-    if (buf) {
+  constexpr int MAX_DEVICES = 64;
+  static void* buf[MAX_DEVICES] = {};
+  static size_t cap[MAX_DEVICES] = {};
+  int dev = 0;
+  MST_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEVICES) return MST_ERR_CUDA;
+  if (bytes > cap[dev]) {
+    if (buf[dev]) {
       MST_CUDA_TRY(cudaDeviceSynchronize());
-      MST_CUDA_TRY(cudaFree(buf));
-      buf = nullptr;
-      cap = 0;
+      MST_CUDA_TRY(cudaFree(buf[dev]));
+      buf[dev] = nullptr;
+      cap[dev] = 0;
     }
     const size_t want = (bytes + ((size_t)1 << 20)) & ~(((size_t)1 << 20) - 1);
-    MST_CUDA_TRY(cudaMalloc(&buf, want));
-    cap = want;
+    MST_CUDA_TRY(cudaMalloc(&buf[dev], want));
+    cap[dev] = want;
   }
-  *ptr = buf;
+  *ptr = buf[dev];
   return MST_OK;
 }
 

@@ -388,8 +388,13 @@ __device__ __forceinline__ int fused_block_excl_scan(int v, int& total, FusedSha
 }
 
 // out[0..n] = exclusive scan of cnt[0..n); each block scans its slice [lo, hi).  One grid barrier inside.
+// The per-block partial sums of consecutive scans alternate between two areas of `bsums` (gscan counts the scans of
+// this launch): a block that has left scan k may already be writing its partial sum of scan k+1 while a slower block
+// still reads the partial sums of scan k, and an area is only rewritten two scans later, behind the next barrier.
 __device__ int fused_grid_scan(const int32_t* cnt, int32_t* out, int64_t n, int64_t lo, int64_t hi, int32_t* bsums,
-                                cg::grid_group& grid, FusedShared& sh) {
+                                int& gscan, cg::grid_group& grid, FusedShared& sh) {
+  bsums += (gscan & 1) * (int)gridDim.x;
+  ++gscan;
   int v = 0;
   for (int64_t i = lo + threadIdx.x; i < hi; i += FUSED_THREADS) v += cnt[i];
   const int bs = fused_block_sum(v, sh);
@@ -426,7 +431,7 @@ constexpr int KEYS_PER_LANE = 16;
 
 template <int MODE, bool CACHED>
 __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* out_bits, int64_t lo, int64_t hi,
-                             int& gpass, cg::grid_group& grid, FusedShared& sh, const uint32_t* s_old,
+                             int& gpass, int& gscan, cg::grid_group& grid, FusedShared& sh, const uint32_t* s_old,
                              const int32_t* s_base, uint32_t* s_grad) {
   constexpr int KB = KeyBits<MODE>::value;
   // magnitude keys are 32 bits wide: their passes compare and shift 32-bit words, only the hashes need 64
@@ -624,7 +629,7 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
       if (lane == 0) F.cnt[w] = __popc(eq);
     }
     __syncthreads();
-    fused_grid_scan(F.cnt, F.scan, P.nwords, lo, hi, F.bsums, grid, sh);
+    fused_grid_scan(F.cnt, F.scan, P.nwords, lo, hi, F.bsums, gscan, grid, sh);
   }
   constexpr int MB = 4;
   if (CACHED) {
@@ -715,15 +720,15 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   }
   __syncthreads();
 
-  int gpass = 0;
+  int gpass = 0, gscan = 0;
   if (per <= (int64_t)FUSED_WARPS * KEYS_PER_LANE) {  // uniform over the grid: every warp's words fit its key registers
-    fused_select<MODE_PRUNE, true>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
-    fused_select<MODE_GRAD, true>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
-    fused_select<MODE_RAND, true>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_PRUNE, true>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_GRAD, true>(F, F.n_grad, F.grad_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_RAND, true>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad);
   } else {
-    fused_select<MODE_PRUNE, false>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
-    fused_select<MODE_GRAD, false>(F, F.n_grad, F.grad_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
-    fused_select<MODE_RAND, false>(F, F.n_rand, F.rand_bits, lo, hi, gpass, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_PRUNE, false>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_GRAD, false>(F, F.n_grad, F.grad_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad);
+    fused_select<MODE_RAND, false>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad);
   }
 
   // mask rewrite: new = (old & ~pruned) | grad | rand, and its popcounts
@@ -733,7 +738,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
     F.cnt[w] = __popc(b);
   }
   __syncthreads();
-  fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, grid, sh);
+  fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, gscan, grid, sh);
   // the barrier inside the scan came after every block wrote its part of the new mask: transpose it now
   if (F.build_csc) {
     const int64_t tiles = (int64_t)F.wpc * P.wpr;
@@ -749,7 +754,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   if (!F.build_csc) return;  // uniform over the grid
   for (int64_t w = loT + threadIdx.x; w < hiT; w += FUSED_THREADS) F.cnt[w] = __popc(F.bitsT[w]);
   __syncthreads();
-  const int totT = fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, grid, sh);
+  const int totT = fused_grid_scan(F.cnt, F.wscanT, F.nwordsT, loT, hiT, F.bsums, gscan, grid, sh);
   for (int64_t w0 = loT + warp; w0 < hiT; w0 += FUSED_WARPS * 4)
     mst_fill_csc_words<4>(w0, FUSED_WARPS, hiT, lane, F.bitsT, F.wscanT, P.I, P.wpr, F.wpc, F.new_bits, F.new_wscan,
                           F.row_idx, F.perm, F.col_ptr, totT);
@@ -800,7 +805,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   if ((n_grad > 0 || (rule->prune_grad_weight != 0.f && n_prune > 0)) && !G_dense) return MST_ERR_INVALID_ARG;
 
   const int c = L->cur, n = c ^ 1;
-  MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t) * 4, s));
+  // flags[0] (error bits) stays set until a reporting call has returned it; only the per-update statistic is cleared
+  MST_CUDA_TRY(cudaMemsetAsync(L->flags + 1, 0, sizeof(int32_t) * 3, s));
 
   SelParams P;
   P.old_bits = L->bits[c];
@@ -840,7 +846,8 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
       grid_blocks = sms * occ;
       const int64_t useful = (L->nwords + FUSED_WARPS - 1) / FUSED_WARPS;  // at least one word per warp
       if (grid_blocks > useful) grid_blocks = (int)(useful < 1 ? 1 : useful);
-      if ((int64_t)grid_blocks > mst_scan_block_sums_len(L->nwords > L->nwordsT ? L->nwords : L->nwordsT)) fused = false;
+      // two alternating partial-sum areas of grid_blocks entries each (the buffer carries 1024 spare entries)
+      if (2 * (int64_t)grid_blocks > mst_scan_block_sums_len(L->nwords > L->nwordsT ? L->nwords : L->nwordsT) + 1024) fused = false;
       fused_smem = (size_t)((L->nwords + grid_blocks - 1) / grid_blocks) * 12;  // slice of mask, scan and grad words
       if (fused_smem > 36 * 1024) fused = false;  // very large layers: kernel-per-phase path
     }
@@ -881,11 +888,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     MST_TRY(mst_combine_update_bits(L, n, s));
     MST_TRY(mst_rebuild_from_bits(L, n, nullptr, 0, c, s));
   }
-  L->cur = n;
   const int64_t nnz_before = L->nnz;
-  L->nnz = target;
-  if (!fused) MST_TRY(mst_build_csc(L, s));
-
   if (stats) {
     // the fused kernel records the longest row itself only when it also builds the CSC view
     if (!fused || !L->csc_valid) max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
@@ -900,8 +903,18 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     stats->n_grad = n_grad;
     stats->n_rand = n_rand;
     stats->max_row_nnz = f[1];
-    if (f[0] & MST_FLAG_NONFINITE) return MST_ERR_NONFINITE;
-    if ((f[0] & MST_FLAG_CORRUPT) || total != target) return MST_ERR_CORRUPT;
+    const bool bad = (f[0] & (MST_FLAG_NONFINITE | MST_FLAG_CORRUPT)) || total != target;
+    if (bad) {
+      // A rejected update is not applied: the structure built in the other buffer set is dropped and the layer keeps
+      // its mask, values and nnz.  The CSC arrays may hold the rejected structure, so the view is rebuilt on next use.
+      L->csc_valid = 0;
+      MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t), s));  // reported: cleared
+      stats->nnz_after = nnz_before;
+      return (f[0] & MST_FLAG_NONFINITE) ? MST_ERR_NONFINITE : MST_ERR_CORRUPT;
+    }
   }
+  L->cur = n;
+  L->nnz = target;
+  if (!fused) MST_TRY(mst_build_csc(L, s));
   return MST_OK;
 }

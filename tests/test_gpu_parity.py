@@ -192,6 +192,50 @@ def test_update_changes_density_both_ways_and_reaches_dense_and_empty():
     L.close()
 
 
+def test_fused_update_tie_rank_scans_do_not_share_partial_sums():
+    """Two grid-wide scans with no barrier of their own between them (a tie-rank scan directly followed by the scan of
+    the new mask) must not share their per-block partial sums.  Pure-prune updates of a bf16 layer (prune keys tie all
+    the time) and R = 0 updates on a gradient with few distinct magnitudes, many iterations, bit-exact each time."""
+    O, I = 768, 768          # enough mask words for a full-size cooperative grid
+    p = _problem(O, I, 4, "bf16", 0.5, 901)
+    L = make_layer(p)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    W = mst_inputs.bf16_bits_to_f32((mst_inputs.f32_to_bf16_bits(W) & np.uint16(0xFF80)))   # 1 mantissa bit: heavy ties
+    Wd = torch.from_numpy(mst_inputs.f32_to_bf16_bits(W).view(np.int16)).to(dev()).view(torch.bfloat16)
+    L.pack(Wd, torch.from_numpy(p.mask).to(dev()))
+    M = p.mask.copy()
+    nnz = int(M.sum())
+    for step in range(12):   # warm-up style: prune only, the target shrinks every step
+        nnz = int(nnz * 0.93)
+        W, M = _update_both(L, p, W, M, None, 0.05, nnz, 0.0, 5, step)
+    rng = np.random.default_rng(17)
+    for step in range(12):   # R = 0 on a gradient with four distinct magnitudes
+        G = rng.choice(np.array([0.5, -0.5, 0.25, -1.0], dtype=np.float32), size=(O, I))
+        W, M = _update_both(L, p, W, M, G, 0.3, -1, 0.0, 5, 100 + step)
+    L.close()
+
+
+def test_rejected_update_leaves_the_layer_unchanged():
+    p = _problem(64, 96, 4, "bf16", 0.25, 77)
+    L = make_layer(p)
+    rp0, ci0, vb0 = export_csr(L, p.dtype)
+    G = torch.zeros(64, 96, device=dev())
+    o, i = np.argwhere(p.mask == 0)[5]
+    G[o, i] = float("inf")
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_topology_update(L.handle, 0.3, -1, 0.25, 0, 0, False, G)
+    assert e.value.status == 6
+    assert L.nnz == p.nnz
+    rp1, ci1, vb1 = export_csr(L, p.dtype)
+    np.testing.assert_array_equal(rp0, rp1)
+    np.testing.assert_array_equal(ci0, ci1)
+    np.testing.assert_array_equal(vb0, vb1)
+    L.validate()                                   # the flag was reported once and is clear again; CSC view rebuilt
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    _update_both(L, p, W, p.mask.copy(), np.ones((64, 96), np.float32), 0.3, -1, 0.25, 0, 1)   # a good update still works
+    L.close()
+
+
 def test_update_without_gradient_and_identity():
     p = _problem(64, 64, 4, "f32", 0.25, 66)
     L = make_layer(p)
