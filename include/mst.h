@@ -87,11 +87,18 @@ mst_status_t mst_layer_destroy(mst_layer_t* layer);
  *                         tensor cores (work proportional to O*I, about 18x the FMA pipe's rate); the weight gradient
  *                         is the dense contraction sampled on the mask in its epilogue.  Needs 16-byte-aligned rows
  *                         (leading dimensions multiple of 8), otherwise the CUDA-core kernels are used.
- *   MST_PATH_AUTO         (default) tensor cores for bf16 layers whenever the operands are aligned (on B200 they are
- *                         faster at every density down to at least 2 %), CUDA cores otherwise.
- * fp32 layers always use the CUDA-core kernels.  Results of the two paths agree within the stated tolerance, not
+ *   MST_PATH_SPARSE_TC    forward and input gradient on the 2:4 structured-sparse tensor-core instruction: W.M is
+ *                         split into the first two entries of every group of four consecutive contraction indices
+ *                         (run at twice the dense tensor rate) and the few third and fourth entries, which the
+ *                         kernel's epilogue adds from a feature-major copy of the activation columns they multiply.
+ *                         Exact for any mask; pays off while few groups hold more than two entries (density up to
+ *                         about 0.25).  Needs nnz <= O*I/4 and aligned operands, otherwise the dense tiles are used.
+ *                         The weight gradient stays the dense contraction sampled on the mask.
+ *   MST_PATH_AUTO         (default) bf16 layers with aligned operands: the structured-sparse instruction at densities
+ *                         where it was measured faster than dense tiles, dense tiles above; CUDA cores otherwise.
+ * fp32 layers always use the CUDA-core kernels.  Results of the paths agree within the stated tolerance, not
  * bit for bit (different summation order). */
-typedef enum { MST_PATH_AUTO = 0, MST_PATH_CUDA_CORE = 1, MST_PATH_TENSOR_CORE = 2 } mst_compute_path_t;
+typedef enum { MST_PATH_AUTO = 0, MST_PATH_CUDA_CORE = 1, MST_PATH_TENSOR_CORE = 2, MST_PATH_SPARSE_TC = 3 } mst_compute_path_t;
 mst_status_t mst_set_compute_path(mst_layer_t* layer, mst_compute_path_t path);
 
 /* Number of active entries (host value; known after mst_pack / mst_topology_update without a sync). */
@@ -258,7 +265,7 @@ mst_status_t mst_er_densities(int32_t n_layers, const int32_t* out_features, con
 
 /* Sticky error bits of kernels that run without a layer handle (bit 0: a bounded wait inside the tensor-core
  * contraction expired and the block gave up; its output is then undefined; bit 1: the same in the attention
- * kernel).  Synchronises the device. */
+ * kernel; bit 2: the same in the structured-sparse contraction).  Synchronises the device. */
 mst_status_t mst_device_error_flags(int32_t* flags);
 
 /* The same step without the final wait: inputs are copied on a copy-in stream owned by the layer, the three products

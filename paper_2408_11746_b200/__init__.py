@@ -18,7 +18,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libmst.so")
 
 MST_F32, MST_BF16 = 0, 1
-MST_PATH_AUTO, MST_PATH_CUDA_CORE, MST_PATH_TENSOR_CORE = 0, 1, 2
+MST_PATH_AUTO, MST_PATH_CUDA_CORE, MST_PATH_TENSOR_CORE, MST_PATH_SPARSE_TC = 0, 1, 2, 3
 MST_OK = 0
 STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "MST_ERR_DTYPE", 4: "MST_ERR_CAPACITY",
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",

@@ -65,6 +65,7 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->nwordsT = (int64_t)I * L->wpc;
   L->nnz = -1;
   L->cur = 0;
+  L->version = 0;
   const int64_t wmax = L->nwords > L->nwordsT ? L->nwords : L->nwordsT;
   const size_t es = mst_elem_size(dtype);
 
@@ -149,13 +150,14 @@ extern "C" mst_status_t mst_layer_destroy(mst_layer_t* L) {
     cudaEventDestroy(L->ev_out);
   }
   free_staging(L);
+  mst_sp24_free(L);
   cudaFree(L->bits[0]);  // base of the single allocation
   delete L;
   return MST_OK;
 }
 
 extern "C" mst_status_t mst_set_compute_path(mst_layer_t* L, mst_compute_path_t path) {
-  if (!L || path < MST_PATH_AUTO || path > MST_PATH_TENSOR_CORE) return MST_ERR_INVALID_ARG;
+  if (!L || path < MST_PATH_AUTO || path > MST_PATH_SPARSE_TC) return MST_ERR_INVALID_ARG;
   L->path = path;
   return MST_OK;
 }
@@ -167,6 +169,14 @@ extern "C" mst_status_t mst_set_compute_path(mst_layer_t* L, mst_compute_path_t 
 bool mst_use_tensor_path(const mst_layer* L) {
   if (L->dtype != MST_BF16 || L->path == MST_PATH_CUDA_CORE) return false;
   return true;
+}
+
+// Forward and input gradient on the structured-sparse instruction: on request, or under AUTO up to the density where
+// it was measured faster than dense tiles.
+bool mst_use_sparse_tc_path(const mst_layer* L) {
+  if (L->dtype != MST_BF16 || L->nnz < 0) return false;
+  if (L->path == MST_PATH_SPARSE_TC) return true;
+  return false;
 }
 
 extern "C" mst_status_t mst_layer_nnz(const mst_layer_t* L, int64_t* nnz) {

@@ -7,6 +7,7 @@
 #include <cstdlib>
 
 #include "mst.h"
+#include "mst_tc_sparse.cuh"
 
 // With MST_DEBUG set in the environment a failing CUDA call is named on stderr before MST_ERR_CUDA is returned.
 inline void mst_report_cuda_error(cudaError_t e, const char* what, const char* file, int line) {
@@ -85,6 +86,7 @@ struct mst_layer {
   int64_t nwordsT;    // I * wpc
   int64_t nnz;        // host copy, -1 = not packed
   int cur;            // which of the two buffer sets is live
+  int64_t version;    // bumped whenever the mask changes (pack, accepted topology update)
 
   // live structure is set [cur]; a topology update builds set [cur^1] and flips
   uint32_t* bits[2];     // [nwords]    bit (o, i) at word o*wpr + i/32, bit i%32
@@ -118,6 +120,9 @@ struct mst_layer {
   // MN-major operand, so no transposed copy is kept
   uint16_t* dense_w;
   int path;  // mst_compute_path_t
+  // 2:4 split of W.M (forward) and of its transpose (input gradient) for the structured-sparse tensor-core path;
+  // allocated on first use
+  mst_sp24 sp[2];
 
   // host staging for mst_layer_step_host
   void *stg_x, *stg_dy, *stg_y, *stg_dx;
@@ -143,6 +148,7 @@ mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s);  // builds the 
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
 mst_status_t mst_densify(const mst_layer* L, cudaStream_t s);
 bool mst_use_tensor_path(const mst_layer* L);
+bool mst_use_sparse_tc_path(const mst_layer* L);
 
 // sticky error word of the attention kernel's bounded waits (mst_attention.cu)
 mst_status_t mst_attention_error_flags(int32_t* flags);

@@ -227,6 +227,8 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
   // Dense-tile tensor-core path: expand W.M to a dense bf16 image [O x I].  Forward: out = in * image^T, the image a
   // K-major operand.  Input gradient: out = in * image, the same image read as an MN-major operand ([K = O] rows of
   // I contiguous columns), so no transposed copy and no CSC view are needed.
+  if (act == MST_ACT_NONE && mst_use_sparse_tc_path(L) && mst_sp24_usable(L, transpose ? 1 : 0, in, ldin, out, ldout))
+    return mst_sp24_product(const_cast<mst_layer*>(L), transpose ? 1 : 0, in, ldin, T, out, ldout, s);
   if (mst_use_tensor_path(L) && (ldout % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0)) {
     const uint16_t* image = L->dense_w;
     if (mst_tc_gemm_usable(in, ldin, image, L->I)) {

@@ -372,6 +372,7 @@ extern "C" mst_status_t mst_pack(mst_layer_t* L, const void* W_dense, int64_t ld
   if (total > L->cap) return MST_ERR_CAPACITY;
   MST_TRY(mst_rebuild_from_bits(L, set, W_dense, ldw, set, s));
   L->nnz = total;
+  ++L->version;
   MST_TRY(mst_build_csc(L, s));
   MST_CUDA_TRY(cudaStreamSynchronize(s));
   return MST_OK;

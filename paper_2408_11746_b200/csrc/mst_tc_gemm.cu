@@ -760,31 +760,34 @@ int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double ou
   return best;
 }
 
-// Scratch for the partial sums of a K-range split: one buffer per device, grown on demand (growing waits for the
-// device and frees the old buffer).  Every call that splits its contraction range shares its device's buffer, so two
-// such calls must not overlap on the GPU (mst_dense_grad, mst_dense_grad_dw, mst_sddmm_dw and the host-step calls on
-// the tensor path): keep them on one stream or order them with events.
-mst_status_t mst_workspace(size_t bytes, void** ptr) {
+// Per-device scratch buffers, grown on demand (growing waits for the device and frees the old buffer).
+//   MST_WS_SPLIT    partial sums of a K-range split.  Every call that splits its contraction range shares its device's
+//                   buffer, so two such calls must not overlap on the GPU (mst_dense_grad, mst_dense_grad_dw,
+//                   mst_sddmm_dw and the host-step calls on the tensor path): keep them on one stream or order them
+//                   with events.
+//   MST_WS_COLUMNS  feature-major copy of activation columns for the structured-sparse path (same rule).
+mst_status_t mst_workspace_kind(int kind, size_t bytes, void** ptr) {
   constexpr int MAX_DEVICES = 64;
-  static void* buf[MAX_DEVICES] = {};
-  static size_t cap[MAX_DEVICES] = {};
+  static void* buf[MST_WS_KINDS][MAX_DEVICES] = {};
+  static size_t cap[MST_WS_KINDS][MAX_DEVICES] = {};
   int dev = 0;
   MST_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= MAX_DEVICES) return MST_ERR_CUDA;
-  if (bytes > cap[dev]) {
-    if (buf[dev]) {
+  if (dev < 0 || dev >= MAX_DEVICES || kind < 0 || kind >= MST_WS_KINDS) return MST_ERR_CUDA;
+  if (bytes > cap[kind][dev]) {
+    if (buf[kind][dev]) {
       MST_CUDA_TRY(cudaDeviceSynchronize());
-      MST_CUDA_TRY(cudaFree(buf[dev]));
-      buf[dev] = nullptr;
-      cap[dev] = 0;
+      MST_CUDA_TRY(cudaFree(buf[kind][dev]));
+      buf[kind][dev] = nullptr;
+      cap[kind][dev] = 0;
     }
     const size_t want = (bytes + ((size_t)1 << 20)) & ~(((size_t)1 << 20) - 1);
-    MST_CUDA_TRY(cudaMalloc(&buf[dev], want));
-    cap[dev] = want;
+    MST_CUDA_TRY(cudaMalloc(&buf[kind][dev], want));
+    cap[kind][dev] = want;
   }
-  *ptr = buf[dev];
+  *ptr = buf[kind][dev];
   return MST_OK;
 }
+mst_status_t mst_workspace(size_t bytes, void** ptr) { return mst_workspace_kind(MST_WS_SPLIT, bytes, ptr); }
 
 bool mst_tc_gemm_usable(const void* A, int64_t lda, const void* B, int64_t ldb) {
   return (lda % 8 == 0) && (ldb % 8 == 0) && ((reinterpret_cast<uintptr_t>(A) & 15u) == 0) &&
@@ -889,6 +892,8 @@ extern "C" mst_status_t mst_device_error_flags(int32_t* flags) {
   MST_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)));
   int32_t att = 0;
   MST_TRY(mst_attention_error_flags(&att));
-  *flags = v | (att << 1);
+  int32_t sp = 0;
+  MST_TRY(mst_sp24_error_flags(&sp));
+  *flags = v | (att << 1) | (sp << 2);
   return MST_OK;
 }

@@ -61,3 +61,6 @@ int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double ou
 // Process-wide scratch buffer for handle-less entry points (grows on demand; growing synchronises the device).
 // Calls that use it must not overlap on the GPU.
 mst_status_t mst_workspace(size_t bytes, void** ptr);
+// The same per purpose: split partial sums, feature-major activation columns of the structured-sparse path.
+enum { MST_WS_SPLIT = 0, MST_WS_COLUMNS = 1, MST_WS_KINDS = 2 };
+mst_status_t mst_workspace_kind(int kind, size_t bytes, void** ptr);

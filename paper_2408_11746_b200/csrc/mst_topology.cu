@@ -915,6 +915,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   }
   L->cur = n;
   L->nnz = target;
+  ++L->version;
   if (!fused) MST_TRY(mst_build_csc(L, s));
   return MST_OK;
 }
