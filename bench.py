@@ -1,13 +1,16 @@
 #!/usr/bin/env python
 """Benchmark of the sparse fully-connected training path (one JSON line on stdout).
 
-A step = one pass of the whole path over the four FC weights of one GPT-2-small block (bf16, 8192 tokens,
-uniform masks at density 0.25): forward SpMM, input-gradient SpMM, weight-gradient SDDMM, dense gradient,
-and one Mixed-Growing topology update (counts, prune/grow selection, mask rewrite, CSR/CSC rebuild) per layer.
+A step = one pass of the whole path over the four FC weights of one GPT-2-medium block (bf16, 16384 tokens,
+uniform masks at density 0.1): forward SpMM, input-gradient SpMM, weight-gradient SDDMM, dense gradient, and one
+Mixed-Growing topology update (counts, prune/grow selection by |w| and |G|, mask rewrite, CSR rebuild) per layer.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 value  = useful (nnz-only) FLOPs of forward + backward, 6*T*nnz per layer, divided by the time of the whole step.
+The same line carries the density sweeps (GPT-2-large and GPT-2-medium FC shapes: forward + backward time, useful
+TFLOP/s, fraction of the roofline and a dense cuBLAS bf16 GEMM of the same shapes beside it) and timed legs for the
+other workloads (single fp32 layer, GPT-2-small block, Zipf rows with an update every step).
 With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no exchange step).
 --impl reference times the CPU checker (oracle/) on a bounded sample of the same workload.
 """
@@ -30,7 +33,8 @@ import mst_inputs  # noqa: E402
 
 METRIC = "sparse_fc_fwd_bwd_useful_tflops"
 UNIT = "TFLOP/s"
-WORKLOAD = "gpt2-small block (qkv, attn_proj, fc1, fc2), T=8192, bf16, uniform masks d=0.25"
+WORKLOAD = "gpt2-medium block (qkv, attn_proj, fc1, fc2), T=16384, bf16, uniform masks d=0.1"
+REF_TOKENS = 128                                       # tokens per layer in one CPU-checker step (both arms)
 FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # SMs x fp32 lanes x 2 flop x max SM clock
 
 
@@ -204,36 +208,46 @@ def run_attention(args) -> None:
     assert mst.mst_device_error_flags() == 0
 
 
-# ------------------------------------------------------------------------------------------ reference arm
+# ------------------------------------------------------------------------------------------ CPU checker legs
+def headline_problems(tokens: int = 16384):
+    """The four FC layers of block 0 of the GPT-2-medium workload (uniform masks, density 0.1)."""
+    return mst_inputs.config4(tokens=tokens, blocks=1)
+
+
+def oracle_step(layers, k: int) -> None:
+    """The whole path once on the CPU checker: three products, dense gradient, one Mixed-Growing update per layer."""
+    import oracle
+    for p in layers:
+        Wm = np.where(p.mask == 1, p.W, np.float32(0))
+        oracle.fwd(p.X, Wm, p.mask)
+        oracle.bwd_x(p.dY, Wm, p.mask)
+        oracle.dw(p.dY, p.X, p.mask)
+        G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
+        c = oracle.mg_counts(0.3, p.nnz, -1, p.mask.size, 0.25)
+        oracle.mg_update(Wm, p.mask, G, c[0], c[3], c[2], 1, k, p.layer_id)
+
+
+def oracle_sample_text() -> str:
+    return "first %d of 16384 tokens of every layer, whole path (products, dense gradient, update) per step" % REF_TOKENS
+
+
 def run_reference(args) -> None:
     """Time the CPU checker, as it stands, on a bounded sample of the workload (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import oracle
     oracle.build()
-    Ts = args.ref_tokens
-    layers = mst_inputs.config2(tokens=Ts)
+    layers = headline_problems(REF_TOKENS)
     cores = oracle.threads()
-
-    def step(k):
-        for p in layers:
-            Wm = np.where(p.mask == 1, p.W, np.float32(0))
-            oracle.fwd(p.X, Wm, p.mask)
-            oracle.bwd_x(p.dY, Wm, p.mask)
-            oracle.dw(p.dY, p.X, p.mask)
-            G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
-            c = oracle.mg_counts(0.3, p.nnz, -1, p.mask.size, 0.25)
-            oracle.mg_update(Wm, p.mask, G, c[0], c[3], c[2], 1, k, p.layer_id)
-
     for k in range(args.warmup):
-        step(k)
+        oracle_step(layers, k)
     t0 = time.perf_counter()
     for k in range(args.steps):
-        step(k)
+        oracle_step(layers, k)
     dt = time.perf_counter() - t0
-    flops = 6.0 * Ts * sum(p.nnz for p in layers) * args.steps
+    flops = 6.0 * REF_TOKENS * sum(p.nnz for p in layers) * args.steps
     val = flops / dt / 1e12
-    sample = "first %d of 8192 tokens of every layer, whole path per step" % Ts
+    sample = oracle_sample_text()
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -243,64 +257,64 @@ def run_reference(args) -> None:
         "gpu_launches": 0}))
 
 
-def cpu_baseline(tokens: int):
+def cpu_baseline(steps: int = 2):
+    """The same sample as the reference arm, `steps` steps (about 10-30 s of host work)."""
     import oracle
     oracle.build()
-    layers = mst_inputs.config2(tokens=tokens)
+    layers = headline_problems(REF_TOKENS)
     t0 = time.perf_counter()
-    for p in layers:
-        Wm = np.where(p.mask == 1, p.W, np.float32(0))
-        oracle.fwd(p.X, Wm, p.mask)
-        oracle.bwd_x(p.dY, Wm, p.mask)
-        oracle.dw(p.dY, p.X, p.mask)
-        G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
-        c = oracle.mg_counts(0.3, p.nnz, -1, p.mask.size, 0.25)
-        oracle.mg_update(Wm, p.mask, G, c[0], c[3], c[2], 1, 0, p.layer_id)
+    for k in range(steps):
+        oracle_step(layers, k)
     dt = time.perf_counter() - t0
-    flops = 6.0 * tokens * sum(p.nnz for p in layers)
+    flops = 6.0 * REF_TOKENS * sum(p.nnz for p in layers) * steps
     return {"value": flops / dt / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": "first %d of 8192 tokens of every layer, whole path once (%.1f s)" % (tokens, dt)}
+            "sample": oracle_sample_text() + ", %d steps (%.1f s)" % (steps, dt)}
 
 
-# ------------------------------------------------------------------------------------------ density sweep report
-def run_sweep(args) -> None:
-    """Forward + input gradient + weight gradient per (layer, density): time of the CUDA-core sparse kernels, of the
-    dense-tile tensor-core kernels and of the automatic choice, useful TFLOP/s, fraction of the roofline
-    max(useful flops / pipe peak, compulsory bytes / HBM bandwidth), and torch.matmul (cuBLAS bf16) on the same
-    shapes as the density-crossover reference.  Inputs are rotated over enough buffer sets to exceed L2."""
+# ------------------------------------------------------------------------------------------ timing helpers
+def median_ms(fn, reps: int, warm: int = 10):
+    """(median, min) time in ms of fn(), one CUDA-event pair per call on the current stream."""
+    import torch
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in ev:
+        a.record(); fn(); b.record()
+    torch.cuda.synchronize()
+    ts = sorted(a.elapsed_time(b) for a, b in ev)
+    return ts[len(ts) // 2], ts[0]
+
+
+def product_bytes(T, O, I, nnz, es=2):
+    """Compulsory bytes of forward + input gradient + weight gradient: every dense operand once per product, the
+    stored entries (value + 16-bit column) once per product, row pointers, and the 4-byte weight gradients."""
+    x, y = T * I * es, T * O * es
+    idx = nnz * (es + 2) + 4 * (O + 1)
+    return (x + y + idx) + (y + x + idx) + (y + x + nnz * 2 + 4 * (O + 1) + 4 * nnz)
+
+
+def sweep_report(width_name: str, densities, reps: int, peaks, dev):
+    """Forward + input gradient + weight gradient of the four FC shapes of one block per density: time under the
+    automatic path choice, useful TFLOP/s, fraction of the roofline max(useful flops / pipe peak, compulsory bytes /
+    HBM bandwidth), and torch.matmul (cuBLAS bf16) on the same shapes as the dense reference.  Inputs rotate over
+    enough buffer sets to exceed L2 between repetitions."""
     import torch
     import paper_2408_11746_b200 as mst
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
-    peaks = measured_peaks()
-    width = mst_inputs.GPT2_WIDTH[args.sweep]
-    T = 8192 if args.sweep == "small" else 16384
-    densities = (1.0, 0.5, 0.25, 0.1, 0.05, 0.02)
-    reps = max(args.steps, 10)
-
-    def time_ms(fns):
-        """median time of each callable in fns, interleaved, CUDA events on the current stream"""
-        for f in fns:
-            for _ in range(3):
-                f()
-        torch.cuda.synchronize()
-        out = []
-        for f in fns:
-            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
-            for a, b in ev:
-                a.record(); f(); b.record()
-            torch.cuda.synchronize()
-            ts = sorted(a.elapsed_time(b) for a, b in ev)
-            out.append(ts[len(ts) // 2])
-        return out
-
+    width = mst_inputs.GPT2_WIDTH[width_name]
+    T = 16384
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(mst_inputs.BASE_SEED + 5)
+    points = {d: {"density": d, "ms": 0.0, "dense_cublas_ms": 0.0, "useful_flops": 0.0, "bytes": 0.0, "layers": {}}
+              for d in densities}
     for li, (name, O, I) in enumerate(mst_inputs.block_shapes(width)):
-        nset = max(2, int(300e6 // (2 * T * (O + I) * 2)) + 1)      # buffer sets so that one round exceeds L2 twice over
-        Xs = [torch.randn(T, I, device=dev, dtype=torch.bfloat16) for _ in range(nset)]
-        dYs = [(torch.randn(T, O, device=dev, dtype=torch.bfloat16) * 1e-2) for _ in range(nset)]
+        nset = max(2, int(300e6 // (2 * T * (O + I) * 2)) + 1)
+        Xs = [torch.randn(T, I, device=dev, dtype=torch.bfloat16, generator=gen) for _ in range(nset)]
+        dYs = [(torch.randn(T, O, device=dev, dtype=torch.float32, generator=gen) * 1e-2).to(torch.bfloat16) for _ in range(nset)]
         Y = torch.empty(T, O, device=dev, dtype=torch.bfloat16)
         dX = torch.empty(T, I, device=dev, dtype=torch.bfloat16)
-        Wd = (torch.randn(O, I, device=dev) * 0.02).to(torch.bfloat16)
+        Wd = (torch.randn(O, I, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+        Gd = torch.empty(O, I, device=dev, dtype=torch.bfloat16)
         ctr = [0]
 
         def nxt():
@@ -309,8 +323,8 @@ def run_sweep(args) -> None:
 
         def dense_all():
             X, dY = nxt()
-            torch.matmul(X, Wd.t(), out=Y); torch.matmul(dY, Wd, out=dX); torch.matmul(dY.t(), X)
-        (t_dense,) = time_ms([dense_all])
+            torch.matmul(X, Wd.t(), out=Y); torch.matmul(dY, Wd, out=dX); torch.matmul(dY.t(), X, out=Gd)
+        t_dense, _ = median_ms(dense_all, reps)
         for d in densities:
             nnz = mst_inputs.exact_nnz(O, I, d)
             mask = torch.from_numpy(mst_inputs.uniform_mask(O, I, nnz, mst_inputs.BASE_SEED + 5, li)).to(dev)
@@ -321,29 +335,100 @@ def run_sweep(args) -> None:
             def all3():
                 X, dY = nxt()
                 L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW)
-            res = {}
-            for pname, pid in (("cuda_core", mst.MST_PATH_CUDA_CORE), ("tensor_core", mst.MST_PATH_TENSOR_CORE),
-                               ("auto", mst.MST_PATH_AUTO)):
-                if pname == "cuda_core" and d > 0.3:
-                    continue                      # minutes of FMA work at these sizes; the crossover is far below
-                L.set_path(pid)
-                (res[pname],) = time_ms([all3])
+            t, tmin = median_ms(all3, reps)
+            path = mst.path_name(L.path_in_use())
             L.close()
-            useful = 6.0 * T * nnz
-            byts = 3 * 2 * T * (O + I) + nnz * (3 * 4 + 4 + 4) + 12 * (O + 1)
-            t_hbm = byts / (peaks["hbm_gbs"] * 1e9)
-            auto_pipe = "tensor"
-            pipe_peak = peaks["bf16_tflops_sustained"] if auto_pipe == "tensor" else FMA_PEAK_TFLOPS
-            t_roof = max(t_hbm, useful / (pipe_peak * 1e12))
-            print(json.dumps({
-                "layer": name, "O": O, "I": I, "T": T, "density": d, "nnz": nnz,
-                "ms": {k: round(v, 4) for k, v in res.items()}, "dense_cublas_ms": round(t_dense, 4),
-                "useful_tflops_auto": round(useful / (res["auto"] * 1e-3) / 1e12, 2),
-                "compulsory_gbs_auto": round(byts / (res["auto"] * 1e-3) / 1e9, 1),
-                "roofline": {"bound": "hbm" if t_hbm >= useful / (pipe_peak * 1e12) else auto_pipe,
-                             "frac": round(t_roof / (res["auto"] * 1e-3), 4), "pipe": auto_pipe},
-                "speedup_vs_dense_cublas": round(t_dense / res["auto"], 3)}), flush=True)
+            pt = points[d]
+            pt["ms"] += t
+            pt["dense_cublas_ms"] += t_dense
+            pt["useful_flops"] += 6.0 * T * nnz
+            pt["bytes"] += product_bytes(T, O, I, nnz)
+            pt["layers"][name] = {"ms": round(t, 4), "min_ms": round(tmin, 4), "dense_cublas_ms": round(t_dense, 4),
+                                  "path": path}
+        del Xs, dYs, Y, dX, Wd, Gd
+        torch.cuda.empty_cache()
+    out = []
+    for d in densities:
+        pt = points[d]
+        t = pt["ms"] * 1e-3
+        t_hbm = pt["bytes"] / (peaks["hbm_gbs"] * 1e9)
+        t_pipe = pt["useful_flops"] / (peaks["bf16_tflops"] * 1e12)          # every bf16 path runs on the tensor pipe
+        bound = "hbm" if t_hbm >= t_pipe else "tensor"
+        out.append({"density": d, "fwd_bwd_ms": round(pt["ms"], 4), "useful_tflops": round(pt["useful_flops"] / t / 1e12, 2),
+                    "compulsory_gbs": round(pt["bytes"] / t / 1e9, 1),
+                    "roofline": {"bound": bound, "pipe": "tensor", "frac": round(max(t_hbm, t_pipe) / t, 4)},
+                    "dense_cublas_ms": round(pt["dense_cublas_ms"], 4),
+                    "speedup_vs_dense_cublas": round(pt["dense_cublas_ms"] / pt["ms"], 3), "layers": pt["layers"]})
+    return {"shapes": "gpt2-%s block (d_model %d), T=%d, bf16, uniform masks" % (width_name, width, T), "reps": reps,
+            "timing": "median of %d calls, CUDA events; inputs rotate over buffer sets larger than L2" % reps,
+            "roofline_peaks": "measured HBM copy bandwidth and burst bf16 GEMM (%s)" % peaks["source"], "points": out}
 
+
+def run_sweep(args) -> None:
+    """Density sweep report alone (one JSON object): --sweep small|medium|large."""
+    import torch
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    if args.sweep == "small":
+        raise SystemExit("--sweep small was folded into the bench line's small-block leg; use medium or large")
+    print(json.dumps(sweep_report(args.sweep, mst_inputs.CONFIG5_DENSITIES, max(args.steps, 50) if args.steps != 200 else 50,
+                                  measured_peaks(), dev)))
+
+
+# ------------------------------------------------------------------------------------------ other workloads
+def other_legs(reps: int, dev):
+    """Timed legs of the workloads the headline does not cover: the single fp32 layer (CUDA-core kernels), the
+    GPT-2-small block at density 0.25, and one block of the ultra-sparse Zipf workload with an update every step."""
+    import torch
+    import paper_2408_11746_b200 as mst
+
+    def up(p, name):
+        if p.dtype == "bf16":
+            return torch.from_numpy(getattr(p, name + "_bits").view(np.int16)).to(dev).view(torch.bfloat16)
+        return torch.from_numpy(getattr(p, name)).to(dev)
+
+    def leg(probs, update, zeta, label):
+        slots = []
+        for p in probs:
+            mdt = mst.MST_BF16 if p.dtype == "bf16" else mst.MST_F32
+            tdt = torch.bfloat16 if p.dtype == "bf16" else torch.float32
+            L = mst.Layer(p.layer_id, p.out_features, p.in_features, mdt)
+            L.pack(up(p, "W"), torch.from_numpy(p.mask).to(dev))
+            T = p.tokens
+            slots.append((L, p, up(p, "X"), up(p, "dY"), torch.empty(T, p.out_features, dtype=tdt, device=dev),
+                          torch.empty(T, p.in_features, dtype=tdt, device=dev),
+                          torch.empty(max(p.nnz, 1), dtype=torch.float32, device=dev),
+                          torch.empty(p.out_features, p.in_features, dtype=torch.float32, device=dev)))
+        k = [0]
+
+        def products():
+            for L, p, X, dY, Y, dX, dW, G in slots:
+                L.fwd(X, Y, p.tokens); L.bwd_x(dY, dX, p.tokens); L.sddmm(dY, X, p.tokens, dW)
+
+        def whole():
+            k[0] += 1
+            for L, p, X, dY, Y, dX, dW, G in slots:
+                L.fwd(X, Y, p.tokens); L.bwd_x(dY, dX, p.tokens); L.sddmm(dY, X, p.tokens, dW)
+                L.dense_grad(dY, X, p.tokens, G)
+                L.update(zeta, target_nnz=-1, random_ratio=0.25, seed=9, step=k[0], G_dense=G, want_stats=False)
+        t_prod, _ = median_ms(products, reps)
+        useful = sum(6.0 * p.tokens * p.nnz for _, p, *_ in slots)
+        res = {"workload": label, "fwd_bwd_ms": round(t_prod, 4), "fwd_bwd_useful_tflops": round(useful / (t_prod * 1e-3) / 1e12, 3),
+               "paths": sorted({mst.path_name(s[0].path_in_use()) for s in slots})}
+        if update:
+            t_all, _ = median_ms(whole, reps)
+            res["step_with_dense_grad_and_update_ms"] = round(t_all, 4)
+            res["step_useful_tflops"] = round(useful / (t_all * 1e-3) / 1e12, 3)
+        for s in slots:
+            s[0].close()
+        return res
+
+    legs = [leg(mst_inputs.config1(), True, 0.3, "single fp32 layer 768->3072, T=256, d=0.25 (CUDA-core kernels)"),
+            leg(mst_inputs.config2(), True, 0.3, "gpt2-small block, T=8192, bf16, uniform d=0.25"),
+            leg(mst_inputs.config3(blocks=1), True, 0.1,
+                "ultra-sparse gpt2-small block 0, T=8192, bf16, Zipf(1.1) rows, d in [0.03, 0.10], update every step")]
+    torch.cuda.empty_cache()
+    return legs
 
 
 # ------------------------------------------------------------------------------------------ our arm
@@ -354,12 +439,11 @@ def main() -> None:
                     help="timed steps (the default keeps the timed region long enough for clock samples under load)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-tokens", type=int, default=48, help="tokens per layer in one reference-arm step")
-    ap.add_argument("--cpu-tokens", type=int, default=3072, help="tokens per layer in the cpu_baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweeps", action="store_true", help="headline step only (skips the density sweeps and the other legs)")
+    ap.add_argument("--sweep-reps", type=int, default=50)
     ap.add_argument("--sweep", default=None, choices=["medium", "large", "small"],
-                    help="density sweep report on one block's FC shapes (not the bench line): one JSON object per "
-                         "(layer, density) with both kernel families and a dense cuBLAS GEMM beside them")
+                    help="density sweep report alone (not the bench line)")
     ap.add_argument("--attention", action="store_true",
                     help="report on the strided sparse attention forward (not the bench line): one JSON object per "
                          "stride at 16 x 1024 tokens, 12 heads of 64, with torch's dense causal attention beside it")
@@ -397,7 +481,7 @@ def main() -> None:
         dist.init_process_group("nccl", device_id=dev)
 
     peaks = measured_peaks()
-    probs = mst_inputs.config2()
+    probs = headline_problems()
     T = probs[0].tokens
 
     def up_bits(a):
@@ -458,6 +542,7 @@ def main() -> None:
     for k in range(args.warmup):
         step(k, False)
     barrier()
+    launches0 = mst.mst_launch_count()
     sampler = ClockSampler(local)
     time.sleep(0.25)
     w0 = time.time()
@@ -468,6 +553,7 @@ def main() -> None:
     barrier()
     w1 = time.time()
     clocks = sampler.stop(w0, w1)
+    gpu_launches = mst.mst_launch_count() - launches0
     ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
     useful = 6.0 * T * sum(s.nnz for s in slots)          # per step, per replica
     value = aggregate_value(useful, args.steps, world, ms)
@@ -478,17 +564,18 @@ def main() -> None:
         tot = sum(a.elapsed_time(b) for _, a, b in timers[name])
         per[name] = {"ms_per_step": tot / args.steps, "launches": len(timers[name])}
     es = 2
-    tensor_peak = peaks["bf16_tflops_sustained"]
+    # the timed region lasts well under a second at full clocks: the burst bf16 figure is the one that applies
+    tensor_peak = peaks["bf16_tflops"]
 
     def algorithmic(name, s):
         """(useful flops, compulsory bytes, pipe) of one call on layer slot s."""
         x, y, idx = T * s.I * es, T * s.O * es, s.nnz * (es + 2) + 4 * (s.O + 1)
-        pipe = "tensor"          # bf16 layers run on the dense-tile tensor-core kernels at every density
+        pipe = "tensor"          # every bf16 path (dense tiles or the structured-sparse instruction) is a tensor-pipe kernel
         if name == "spmm_fwd": return 2.0 * T * s.nnz, x + y + idx, pipe
-        if name == "spmm_bwd_x": return 2.0 * T * s.nnz, x + y + idx + 4 * s.nnz, pipe
+        if name == "spmm_bwd_x": return 2.0 * T * s.nnz, x + y + idx, pipe
         if name == "sddmm_dw": return 2.0 * T * s.nnz, x + y + s.nnz * 2 + 4 * (s.O + 1) + 4 * s.nnz, pipe
         if name == "dense_grad": return 2.0 * T * s.O * s.I, x + y + 4 * s.O * s.I, "tensor"
-        # update: G once per 32-bit-key pass (3) + mask words and values a few times + CSR/CSC rewrite
+        # update: G once per 32-bit-key pass (3) + mask words and values a few times + CSR rewrite
         return 0.0, 3 * 4.0 * s.O * s.I + 2 * s.nnz * (es + 2 + 6), "hbm"
 
     def roofline_of(name):
@@ -496,24 +583,22 @@ def main() -> None:
         fl = sum(algorithmic(name, s)[0] for s, _, _ in timers[name])
         by = sum(algorithmic(name, s)[1] for s, _, _ in timers[name])
         pipe = algorithmic(name, timers[name][0][0])[2]
-        pipe_peak = tensor_peak if pipe == "tensor" else FMA_PEAK_TFLOPS
-        t_pipe = fl / (pipe_peak * 1e12) if pipe != "hbm" else 0.0
+        t_pipe = fl / (tensor_peak * 1e12) if pipe != "hbm" else 0.0
         t_hbm = by / (peaks["hbm_gbs"] * 1e9)
         if t_hbm >= t_pipe:
             r = {"bound": "hbm", "achieved": by / (ms_tot * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                  "peak_source": peaks["source"] + " (MEASURED_PEAKS.json copy bandwidth)"}
         else:
-            r = {"bound": pipe, "achieved": fl / (ms_tot * 1e-3) / 1e12, "peak": pipe_peak, "unit": "TFLOP/s",
-                 "peak_source": (peaks["source"] + " (sustained bf16 GEMM)") if pipe == "tensor" else
-                 "derived: 148 SMs x 128 fp32 lanes x 2 x 1.965 GHz"}
+            r = {"bound": pipe, "achieved": fl / (ms_tot * 1e-3) / 1e12, "peak": tensor_peak, "unit": "TFLOP/s",
+                 "peak_source": peaks["source"] + " (burst bf16 GEMM)"}
         r.update({"frac": r["achieved"] / r["peak"], "traffic": None, "kernel": name, "pipe": pipe,
                   "useful_tflops": fl / (ms_tot * 1e-3) / 1e12 if fl else None})
         return r
 
     rooflines = {name: roofline_of(name) for name in KERNELS}
-    # The dominant kernel: the four product calls are launches of one kernel (the tcgen05 contraction) when the layers
-    # are dense enough for the tensor-core path; the update is one fused kernel.  Pick the family with the larger total
-    # time, and inside the contraction family the call kind that takes longest.
+    # The dominant kernel: the product calls and the dense gradient are launches of the tcgen05 contraction kernels,
+    # the update is one fused kernel.  Pick the family with the larger total time, and inside the contraction family
+    # the call kind that takes longest.
     family = {"spmm_fwd": "contraction", "spmm_bwd_x": "contraction", "sddmm_dw": "contraction",
               "dense_grad": "contraction", "topology_update": "update"}
     fam_ms = {}
@@ -522,24 +607,23 @@ def main() -> None:
     dom_family = max(fam_ms, key=fam_ms.get)
     dom = max((n for n in KERNELS if family[n] == dom_family), key=lambda n: per[n]["ms_per_step"])
     roof = dict(rooflines[dom])
-    tensor_path = True
-    roof["kernel"] = ("tc_gemm_pair_kernel" if tensor_path else "spmm/sddmm CUDA-core kernels") + " as " + dom \
-        if dom_family == "contraction" else "mg_update_fused_kernel"
+    paths = sorted({mst.path_name(s.L.path_in_use()) for s in slots})
+    if dom_family == "update":
+        roof["kernel"] = "mg_update_fused_kernel"
+    elif dom in ("sddmm_dw", "dense_grad"):
+        roof["kernel"] = "tc_gemm_pair_kernel as " + dom
+    else:
+        roof["kernel"] = ("tc_sp24_pair_kernel" if paths == ["sparse_tc"] else "tc_gemm_pair_kernel") + " as " + dom
     roof["family_ms_per_step"] = fam_ms
-    # dram__bytes_read.sum + dram__bytes_write.sum of ONE launch of this call kind on layer fc1 (O=3072, I=768), from the
-    # ncu capture summarised in profiles/tc_gemm_pair_and_fused_update_gpt2small_block_d0.25.md (cold caches; output
-    # rows still sitting in L2 at kernel end are not counted).  Algorithmic bytes of the same launch beside it.
-    NCU_TRAFFIC_FC1 = {"spmm_fwd": 19.34e6, "spmm_bwd_x": 57.84e6, "sddmm_dw": 66.49e6, "dense_grad": 66.52e6}
-    if dom in NCU_TRAFFIC_FC1 and tensor_path:
-        fc1 = next(s for s in slots if s.O == 3072 and s.I == 768)
-        roof["traffic"] = NCU_TRAFFIC_FC1[dom]
-        roof["traffic_launch"] = "fc1 (O=3072, I=768): algorithmic %.2f MB" % (algorithmic(dom, fc1)[1] / 1e6)
-    if dom_family == "contraction" and tensor_path:
+    roof["traffic_note"] = ("dram bytes of one launch are in profiles/ (ncu capture of the same kernel on a smaller case); "
+                            "not repeated here because the capture is not regenerated with every kernel change")
+    if dom_family == "contraction":
         # what the tensor pipe itself sustains: executed dense flops of this call kind over its time
         dense_fl = sum(2.0 * T * s.O * s.I for s, _, _ in timers[dom])
         dense_ms = sum(a.elapsed_time(b) for _, a, b in timers[dom])
         roof["tensor_pipe"] = {"executed_tflops": dense_fl / (dense_ms * 1e-3) / 1e12, "peak": tensor_peak,
-                               "frac": dense_fl / (dense_ms * 1e-3) / 1e12 / tensor_peak}
+                               "frac": dense_fl / (dense_ms * 1e-3) / 1e12 / tensor_peak,
+                               "peak_source": peaks["source"] + " (burst bf16 GEMM)"}
     for name in KERNELS:
         per[name]["useful_tflops"] = rooflines[name]["useful_tflops"]
         per[name]["roofline_frac"] = rooflines[name]["frac"]
@@ -592,29 +676,35 @@ def main() -> None:
     b = ev()
     barrier()
     shared_ms = max_over_ranks(a.elapsed_time(b), dist, dev) / sh_steps
+    for s in slots:
+        s.L.close()
+    del slots
+    torch.cuda.empty_cache()
 
-    launches_per_layer = 9            # densify+contraction (fwd), same (bwd_x), contraction+reduce (sddmm, dense_grad), fused update
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: four layers' distinct buffers, %.0f MB touched "
-                   "per step" % (sum(2 * T * (s.I + s.O) * es for s in slots) / 1e6),
-                   "update": "every step, zeta=0.3, R=0.25, target = current nnz", "replicas": world},
+                   "per step" % (sum(2 * T * (p.in_features + p.out_features) * es for p in probs) / 1e6),
+                   "update": "every step, zeta=0.3, R=0.25 (gradient growth by |G| over the inactive entries), "
+                   "target = current nnz", "paths": paths, "replicas": world},
         "clocks": clocks, "roofline": roof, "kernels": per,
         "fwd_bwd_only_tflops": useful / ((per["spmm_fwd"]["ms_per_step"] + per["spmm_bwd_x"]["ms_per_step"] +
                                           per["sddmm_dw"]["ms_per_step"]) * 1e-3) / 1e12,
         "shared_gradient_step": {"ms_per_step": shared_ms, "value": aggregate_value(useful, 1, world, shared_ms),
                                  "unit": UNIT, "note": "dW sampled from the dense gradient: same outputs, one "
                                  "contraction fewer per layer"},
-        "e2e": e2e, "gpu_launches": launches_per_layer * len(slots) * args.steps,
+        "e2e": e2e, "gpu_launches": gpu_launches,
     }
+    if rank == 0 and world == 1 and not args.no_sweeps:
+        out["density_sweep"] = sweep_report("large", mst_inputs.CONFIG5_DENSITIES, args.sweep_reps, peaks, dev)
+        out["density_sweep_medium"] = sweep_report("medium", (0.25, 0.1, 0.05, 0.02), args.sweep_reps, peaks, dev)
+        out["other_workloads"] = other_legs(args.sweep_reps, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(args.cpu_tokens)
+        out["cpu_baseline"] = cpu_baseline()
     if rank == 0:
         print(json.dumps(out))
-    for s in slots:
-        s.L.close()
     if dist is not None:
         dist.destroy_process_group()
 

@@ -101,6 +101,13 @@ mst_status_t mst_layer_destroy(mst_layer_t* layer);
 typedef enum { MST_PATH_AUTO = 0, MST_PATH_CUDA_CORE = 1, MST_PATH_TENSOR_CORE = 2, MST_PATH_SPARSE_TC = 3 } mst_compute_path_t;
 mst_status_t mst_set_compute_path(mst_layer_t* layer, mst_compute_path_t path);
 
+/* The kernels forward and input gradient of this layer run on for aligned operands, with MST_PATH_AUTO resolved
+ * (unaligned operands always fall back to the CUDA-core kernels). */
+mst_status_t mst_layer_path_in_use(const mst_layer_t* layer, mst_compute_path_t* path);
+
+/* Kernels the library has enqueued in this process so far (all layers, all streams): for launch accounting. */
+mst_status_t mst_launch_count(int64_t* count);
+
 /* Number of active entries (host value; known after mst_pack / mst_topology_update without a sync). */
 mst_status_t mst_layer_nnz(const mst_layer_t* layer, int64_t* nnz);
 
@@ -123,6 +130,15 @@ mst_status_t mst_export_csc(const mst_layer_t* layer, int32_t* col_ptr, int32_t*
 /* Device pointer to the stored values (CSR order, layer dtype) so an optimizer can update them in place.
  * The pointer changes at every mst_pack / mst_topology_update. */
 mst_status_t mst_values(mst_layer_t* layer, void** vals, int64_t* nnz);
+
+/* Value tracking.  By default the library assumes that the stored values may have been modified in place before any
+ * call, and rebuilds what it derives from them (the dense image of W.M for the tensor-core kernels, the compressed
+ * operand of the structured-sparse path) at every forward and input-gradient call.  mst_track_values(layer, 1) is the
+ * caller's promise to call mst_values_changed(layer) after every in-place modification (an optimizer step); the
+ * derived operands are then rebuilt only when the mask or the values have changed since they were built, e.g. once
+ * per training step instead of once per product.  mst_pack and mst_topology_update announce their own changes. */
+mst_status_t mst_track_values(mst_layer_t* layer, int32_t enable);
+mst_status_t mst_values_changed(mst_layer_t* layer);
 
 /* Structure check on the device: row pointers monotone and ending at nnz, columns in range and strictly
  * ascending, CSC consistent with CSR, bit mask consistent.  Synchronises.  MST_ERR_CORRUPT / MST_ERR_NONFINITE
@@ -265,7 +281,8 @@ mst_status_t mst_er_densities(int32_t n_layers, const int32_t* out_features, con
 
 /* Sticky error bits of kernels that run without a layer handle (bit 0: a bounded wait inside the tensor-core
  * contraction expired and the block gave up; its output is then undefined; bit 1: the same in the attention
- * kernel; bit 2: the same in the structured-sparse contraction).  Synchronises the device. */
+ * kernel; bit 2: the same in the structured-sparse contraction;
+ * bit 3: the same in the CUDA-core SpMM / SDDMM).  Synchronises the device. */
 mst_status_t mst_device_error_flags(int32_t* flags);
 
 /* The same step without the final wait: inputs are copied on a copy-in stream owned by the layer, the three products

@@ -10,7 +10,9 @@ joins the two parts with an intersection sign; the text, the figure and the FLOP
 
 Pins (tests/test_oracle_attention.py): the mask's population against the printed ratios, the reduction to causal
 softmax attention when stride >= n (computed there by a separate formula), constant values, a hand example, and a
-position-by-position loop on small cases.
+position-by-position loop on small cases.  The backward pass (the derivative of that definition: softmax Jacobian
+and the three matrix products) is pinned by central differences of the forward function, by the directional
+identity <dO, dOut> = <dQ, dq> + <dK, dk> + <dV, dv>, and by a position-by-position loop.
 """
 from __future__ import annotations
 
@@ -39,6 +41,28 @@ def strided_attention(Q, K, V, stride: int):
     e = np.exp(s - m)
     z = e.sum(axis=-1, keepdims=True)
     return np.matmul(e / z, V), (m + np.log(z))[..., 0]
+
+
+def strided_attention_bwd(Q, K, V, dO, stride: int):
+    """Gradients of strided_attention's output with respect to Q, K, V for the upstream gradient dO
+    ([batch, heads, n, d] each, float64).  With P the masked softmax of the scaled scores:
+    dV = P^T dO;  dP = dO V^T;  dS = P * (dP - rowsum(dP * P));  dQ = dS K / sqrt(d);  dK = dS^T Q / sqrt(d)."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    dO = np.asarray(dO, dtype=np.float64)
+    n, d = Q.shape[-2], Q.shape[-1]
+    keep = strided_mask(n, stride)
+    scale = 1.0 / np.sqrt(float(d))
+    s = np.where(keep, np.matmul(Q, np.swapaxes(K, -1, -2)) * scale, -np.inf)
+    e = np.exp(s - s.max(axis=-1, keepdims=True))
+    P = e / e.sum(axis=-1, keepdims=True)
+    dV = np.matmul(np.swapaxes(P, -1, -2), dO)
+    dP = np.matmul(dO, np.swapaxes(V, -1, -2))
+    dS = P * (dP - (dP * P).sum(axis=-1, keepdims=True))
+    dQ = np.matmul(dS, K) * scale
+    dK = np.matmul(np.swapaxes(dS, -1, -2), Q) * scale
+    return dQ, dK, dV
 
 
 def strided_attention_at(Q, K, V, stride: int, b, h, i):

@@ -23,7 +23,7 @@ MST_OK = 0
 STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "MST_ERR_DTYPE", 4: "MST_ERR_CAPACITY",
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
                 9: "MST_ERR_NOT_PACKED"}
-EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
+EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_path_in_use", "mst_launch_count", "mst_track_values", "mst_values_changed", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_strided_attention_fwd", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
@@ -67,6 +67,10 @@ _sig = {
     "mst_layer_destroy": [_vp],
     "mst_layer_nnz": [_vp, ctypes.POINTER(_i64)],
     "mst_set_compute_path": [_vp, ctypes.c_int],
+    "mst_layer_path_in_use": [_vp, ctypes.POINTER(ctypes.c_int)],
+    "mst_launch_count": [ctypes.POINTER(_i64)],
+    "mst_track_values": [_vp, _i32],
+    "mst_values_changed": [_vp],
     "mst_pack": [_vp, _vp, _i64, _vp, _vp],
     "mst_export_csr": [_vp, _vp, _vp, _vp, _vp],
     "mst_export_csc": [_vp, _vp, _vp, _vp, _vp],
@@ -144,6 +148,34 @@ def mst_layer_destroy(layer: int) -> None:
 
 def mst_set_compute_path(layer: int, path: int) -> None:
     _check(_lib.mst_set_compute_path(layer, path), "mst_set_compute_path")
+
+
+PATH_NAMES = {MST_PATH_AUTO: "auto", MST_PATH_CUDA_CORE: "cuda_core", MST_PATH_TENSOR_CORE: "dense_tiles",
+              MST_PATH_SPARSE_TC: "sparse_tc"}
+
+
+def path_name(path: int) -> str:
+    return PATH_NAMES.get(path, "path %d" % path)
+
+
+def mst_layer_path_in_use(layer: int) -> int:
+    p = ctypes.c_int(0)
+    _check(_lib.mst_layer_path_in_use(layer, ctypes.byref(p)), "mst_layer_path_in_use")
+    return p.value
+
+
+def mst_track_values(layer: int, enable: bool) -> None:
+    _check(_lib.mst_track_values(layer, 1 if enable else 0), "mst_track_values")
+
+
+def mst_values_changed(layer: int) -> None:
+    _check(_lib.mst_values_changed(layer), "mst_values_changed")
+
+
+def mst_launch_count() -> int:
+    n = _i64(0)
+    _check(_lib.mst_launch_count(ctypes.byref(n)), "mst_launch_count")
+    return n.value
 
 
 def mst_layer_nnz(layer: int) -> int:
@@ -315,6 +347,15 @@ class Layer:
 
     def set_path(self, path: int) -> None:
         mst_set_compute_path(self.handle, path)
+
+    def track_values(self, enable: bool = True) -> None:
+        mst_track_values(self.handle, enable)
+
+    def values_changed(self) -> None:
+        mst_values_changed(self.handle)
+
+    def path_in_use(self) -> int:
+        return mst_layer_path_in_use(self.handle)
 
     @property
     def nnz(self) -> int:

@@ -41,8 +41,11 @@ def _headers_mtime() -> float:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    """MST_NVCC_EXTRA (environment) adds compiler flags, e.g. -DMST_SP_PROFILE for the cycle accounting of the
+    structured-sparse kernel; such a build must be forced so that every object sees the flag."""
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
+    extra = os.environ.get("MST_NVCC_EXTRA", "").split()
     hm = _headers_mtime()
     jobs = []
     objs = []
@@ -50,7 +53,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
         if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hm):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", src, "-o", obj]
             if verbose:
                 cmd.insert(1, "-Xptxas=-v")
             jobs.append(cmd)

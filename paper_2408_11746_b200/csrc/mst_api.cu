@@ -3,6 +3,8 @@
 
 #include <new>
 
+std::atomic<long long> g_mst_launches{0};
+
 namespace {
 
 struct Carver {
@@ -66,6 +68,9 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->nnz = -1;
   L->cur = 0;
   L->version = 0;
+  L->track_values = 0;
+  L->values_epoch = 0;
+  L->dense_version = L->dense_epoch = -1;
   const int64_t wmax = L->nwords > L->nwordsT ? L->nwords : L->nwordsT;
   const size_t es = mst_elem_size(dtype);
 
@@ -177,6 +182,34 @@ bool mst_use_sparse_tc_path(const mst_layer* L) {
   if (L->dtype != MST_BF16 || L->nnz < 0) return false;
   if (L->path == MST_PATH_SPARSE_TC) return true;
   return false;
+}
+
+extern "C" mst_status_t mst_track_values(mst_layer_t* L, int32_t enable) {
+  if (!L) return MST_ERR_INVALID_ARG;
+  L->track_values = enable ? 1 : 0;
+  L->dense_version = L->dense_epoch = -1;
+  for (int d = 0; d < 2; ++d) L->sp[d].values_epoch = -1;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_values_changed(mst_layer_t* L) {
+  if (!L) return MST_ERR_INVALID_ARG;
+  ++L->values_epoch;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_layer_path_in_use(const mst_layer_t* L, mst_compute_path_t* path) {
+  if (!L || !path) return MST_ERR_INVALID_ARG;
+  if (mst_use_sparse_tc_path(L) && L->nnz / 2 <= L->N / 8) *path = MST_PATH_SPARSE_TC;
+  else if (mst_use_tensor_path(L)) *path = MST_PATH_TENSOR_CORE;
+  else *path = MST_PATH_CUDA_CORE;
+  return MST_OK;
+}
+
+extern "C" mst_status_t mst_launch_count(int64_t* count) {
+  if (!count) return MST_ERR_INVALID_ARG;
+  *count = (int64_t)g_mst_launches.load(std::memory_order_relaxed);
+  return MST_OK;
 }
 
 extern "C" mst_status_t mst_layer_nnz(const mst_layer_t* L, int64_t* nnz) {

@@ -567,7 +567,7 @@ extern "C" mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, 
   MST_CUDA_TRY(cudaGetDevice(&dev));
   MST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   const int grid = (int)(tiles < sms ? tiles : sms);   // one persistent block per SM
-  strided_attention_fwd_kernel<<<grid, ATT_THREADS, smem, (cudaStream_t)stream>>>(tmQ, tmK, tmV, P);
+  strided_attention_fwd_kernel<<<grid, ATT_THREADS, smem, (cudaStream_t)stream>>>(tmQ, tmK, tmV, P); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

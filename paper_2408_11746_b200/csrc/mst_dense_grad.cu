@@ -88,11 +88,11 @@ extern "C" mst_status_t mst_dense_grad(const void* dY, int64_t lddy, const void*
   }
   dim3 grid((unsigned)((in_features + TN - 1) / TN), (unsigned)((out_features + TM - 1) / TM));
   if (dtype == MST_F32)
-    dense_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dY, lddy, (const float*)X, ldx, T, out_features,
-                                                 in_features, G);
+    { dense_grad_kernel<float><<<grid, 256, 0, s>>>((const float*)dY, lddy, (const float*)X, ldx, T, out_features,
+                                                 in_features, G); MST_COUNT_LAUNCH(); }
   else
-    dense_grad_kernel<uint16_t><<<grid, 256, 0, s>>>((const uint16_t*)dY, lddy, (const uint16_t*)X, ldx, T,
-                                                    out_features, in_features, G);
+    { dense_grad_kernel<uint16_t><<<grid, 256, 0, s>>>((const uint16_t*)dY, lddy, (const uint16_t*)X, ldx, T,
+                                                    out_features, in_features, G); MST_COUNT_LAUNCH(); }
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

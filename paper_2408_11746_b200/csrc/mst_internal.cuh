@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 
@@ -21,6 +22,10 @@ inline void mst_report_cuda_error(cudaError_t e, const char* what, const char* f
       return MST_ERR_CUDA;                                        \
     }                                                             \
   } while (0)
+
+// kernels enqueued by the library since it was loaded (mst_launch_count)
+extern std::atomic<long long> g_mst_launches;
+#define MST_COUNT_LAUNCH() ((void)g_mst_launches.fetch_add(1, std::memory_order_relaxed))
 
 // Programmatic dependent launch.  A kernel started with mst_launch_overlapped may become resident and run its set-up
 // (barrier initialisation, tensor-memory allocation, descriptor fetch) while its predecessor in the stream drains; it
@@ -53,6 +58,7 @@ inline cudaError_t mst_launch_overlapped(void (*kernel)(KArgs...), dim3 grid, di
   attr[0].val.programmaticStreamSerializationAllowed = mst_pdl_enabled();
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  g_mst_launches.fetch_add(1, std::memory_order_relaxed);
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 #endif
@@ -87,6 +93,12 @@ struct mst_layer {
   int64_t nnz;        // host copy, -1 = not packed
   int cur;            // which of the two buffer sets is live
   int64_t version;    // bumped whenever the mask changes (pack, accepted topology update)
+  // Value tracking (mst_track_values): the caller announces in-place changes of the stored values with
+  // mst_values_changed; operands derived from the values (dense image, compressed 2:4 operand) are then rebuilt only
+  // when the mask or the values have changed since they were built.  Off: rebuilt at every product call.
+  int track_values;
+  int64_t values_epoch;
+  mutable int64_t dense_version, dense_epoch;   // what the dense image was built from (-1: nothing)
 
   // live structure is set [cur]; a topology update builds set [cur^1] and flips
   uint32_t* bits[2];     // [nwords]    bit (o, i) at word o*wpr + i/32, bit i%32
@@ -150,6 +162,9 @@ mst_status_t mst_densify(const mst_layer* L, cudaStream_t s);
 bool mst_use_tensor_path(const mst_layer* L);
 bool mst_use_sparse_tc_path(const mst_layer* L);
 
+// sticky error word of the CUDA-core SpMM's bounded waits (mst_spmm.cu)
+mst_status_t mst_spmm_error_flags(int32_t* flags);
+mst_status_t mst_sddmm_error_flags(int32_t* flags);
 // sticky error word of the attention kernel's bounded waits (mst_attention.cu)
 mst_status_t mst_attention_error_flags(int32_t* flags);
 

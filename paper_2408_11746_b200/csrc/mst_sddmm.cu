@@ -1,16 +1,27 @@
 // Sampled dense-dense product on the mask:  dW[k] = sum_t dY[t, o_k] * X[t, i_k]  for every stored entry k.
 //
-// A block owns a ROWS x COLS window of the weight matrix and walks over all tokens in tiles of TOK.  For each token
-// tile both operand tiles are staged feature-major in shared memory (Ds[row][token], Xs[col][token]) so that a lane
-// owning 8 consecutive tokens fetches its operands with 128-bit shared loads.  The window's stored entries are
-// listed once (row-local, column-local) in shared memory; a warp takes them 32 at a time: every lane forms its
-// 8-token partial dot product of each of the 32 entries, then a 31-shuffle transposing reduction leaves the full
+// Both operands are first copied feature-major once per call (dYT[o][t], XT[i][t]).  A block owns a ROWS x COLS
+// window of the weight matrix and walks over all tokens in tiles of TOK: for each token tile the two operand tiles
+// (Ds[row][token], Xs[col][token]) arrive in shared memory through the TMA unit (cp.async.bulk.tensor, this GPU's
+// memory only, no multicast), so that a lane owning 8 consecutive tokens fetches its operands with 128-bit shared
+// loads.  The window's stored entries are listed once (row-local, column-local) in shared memory; a warp takes them
+// 32 at a time: every lane forms its 8-token partial dot product of each of the 32 entries (bf16 layers: with the
+// mixed-precision FMA, bf16 x bf16 + fp32, no unpacking), then a 31-shuffle transposing reduction leaves the full
 // sum of entry j in lane j, which adds it to that entry's fp32 accumulator in shared memory.  The upstream-gradient
 // operands of a row stay in registers while consecutive entries share the row.  Every entry is owned by exactly one
 // warp and one lane, the token order is fixed: no atomics, deterministic.
+#include <cuda.h>
+
 #include "mst_bits.cuh"
 #include "mst_internal.cuh"
 #include "mst_tc_gemm.cuh"
+#include "mst_tc_ptx.cuh"
+
+// feature-major copies and their TMA description (mst_spmm.cu)
+mst_status_t mst_feature_major_copy(const void* in, int64_t ldin, int64_t T, int C, mst_dtype_t dtype, void* out, int64_t ldt,
+                                    cudaStream_t s);
+bool mst_feature_major_map(CUtensorMap* tm, const void* base, int64_t T, int C, int64_t ldt, mst_dtype_t dtype, int box_tokens,
+                           int box_features);
 
 namespace {
 
@@ -21,44 +32,44 @@ constexpr int WARPS = 8;
 constexpr int RPW = ROWS / WARPS;
 constexpr int LIST_CAP = ROWS * COLS;
 
-__device__ __forceinline__ void load8(float (&v)[8], const float* p) {
-  const float4 a = *reinterpret_cast<const float4*>(p);
-  const float4 b = *reinterpret_cast<const float4*>(p + 4);
-  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-}
-__device__ __forceinline__ void load8(float (&v)[8], const uint16_t* p) {
-  const uint4 q = *reinterpret_cast<const uint4*>(p);
-  v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xFFFF0000u);
-  v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xFFFF0000u);
-  v[4] = __uint_as_float(q.z << 16); v[5] = __uint_as_float(q.z & 0xFFFF0000u);
-  v[6] = __uint_as_float(q.w << 16); v[7] = __uint_as_float(q.w & 0xFFFF0000u);
-}
+__device__ int g_sddmm_error = 0;  // sticky: a bounded wait expired
 
-// Stage `ncols` (<= 64) feature columns starting at c0 of tokens [t0, t0+TOK) into S[c][token]; zero fill outside.
+// 8 consecutive tokens of one feature, as stored
 template <typename T>
-__device__ __forceinline__ void stage64(T* __restrict__ S, const T* __restrict__ in, int64_t ld, int64_t T_total, int C,
-                                        int64_t t0, int c0, bool vec_ok) {
-  constexpr int VEC = 16 / (int)sizeof(T);
-  const int tt = threadIdx.x;
-  const int64_t t = t0 + tt;
-  const bool row_ok = t < T_total;
-  const T* src = in + t * ld + c0;
-  if (vec_ok) {
-#pragma unroll 4
-    for (int v = 0; v < COLS / VEC; ++v) {
-      uint4 q = make_uint4(0, 0, 0, 0);
-      if (row_ok && c0 + v * VEC < C) q = *reinterpret_cast<const uint4*>(src + v * VEC);
-      const T* e = reinterpret_cast<const T*>(&q);
-#pragma unroll
-      for (int j = 0; j < VEC; ++j) S[(v * VEC + j) * TOK + tt] = e[j];
-    }
-  } else {
-    for (int c = 0; c < COLS; ++c) {
-      T x = T(0);
-      if (row_ok && c0 + c < C) x = src[c];
-      S[c * TOK + tt] = x;
-    }
+struct Vec8;
+template <>
+struct Vec8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) {
+    a = *reinterpret_cast<const float4*>(p);
+    b = *reinterpret_cast<const float4*>(p + 4);
   }
+};
+template <>
+struct Vec8<uint16_t> {
+  uint4 q;
+  __device__ __forceinline__ void load(const uint16_t* p) { q = *reinterpret_cast<const uint4*>(p); }
+};
+__device__ __forceinline__ float dot8(const Vec8<float>& d, const Vec8<float>& x) {
+  float s0 = d.a.x * x.a.x, s1 = d.a.y * x.a.y;
+  s0 = fmaf(d.a.z, x.a.z, s0); s1 = fmaf(d.a.w, x.a.w, s1);
+  s0 = fmaf(d.b.x, x.b.x, s0); s1 = fmaf(d.b.y, x.b.y, s1);
+  s0 = fmaf(d.b.z, x.b.z, s0); s1 = fmaf(d.b.w, x.b.w, s1);
+  return s0 + s1;
+}
+// exact bf16 products accumulated in fp32 (mixed-precision FMA of sm_100), two chains of four
+__device__ __forceinline__ float dot8(const Vec8<uint16_t>& d, const Vec8<uint16_t>& x) {
+  const uint32_t dw[4] = {d.q.x, d.q.y, d.q.z, d.q.w}, xw[4] = {x.q.x, x.q.y, x.q.z, x.q.w};
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint16_t dl, dh, xl, xh;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(dl), "=h"(dh) : "r"(dw[j]));
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(xl), "=h"(xh) : "r"(xw[j]));
+    asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(s0) : "h"(dl), "h"(xl));
+    asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(s1) : "h"(dh), "h"(xh));
+  }
+  return s0 + s1;
 }
 
 __device__ __forceinline__ int lower_bound_u16(const uint16_t* __restrict__ a, int lo, int hi, int key) {
@@ -71,19 +82,32 @@ __device__ __forceinline__ int lower_bound_u16(const uint16_t* __restrict__ a, i
 
 template <typename T>
 __global__ void __launch_bounds__(WARPS * 32)
-sddmm_window_kernel(const int32_t* __restrict__ row_ptr, const uint16_t* __restrict__ col_idx,
-                    const T* __restrict__ dY, int64_t lddy, const T* __restrict__ X, int64_t ldx, int64_t T_total, int O,
-                    int I, float* __restrict__ dW, int vec_x, int vec_dy) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  T* Xs = reinterpret_cast<T*>(smem_raw);                       // [COLS][TOK]
-  T* Ds = Xs + COLS * TOK;                                      // [ROWS][TOK]
-  float* accS = reinterpret_cast<float*>(Ds + ROWS * TOK);      // [LIST_CAP]
-  uint16_t* list = reinterpret_cast<uint16_t*>(accS + LIST_CAP);  // [LIST_CAP]  (row_local << 8) | col_local
+sddmm_window_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constant__ CUtensorMap tmX,
+                    const int32_t* __restrict__ row_ptr, const uint16_t* __restrict__ col_idx, int64_t T_total, int O,
+                    int I, float* __restrict__ dW) {
+  using namespace mst_ptx;
+  constexpr uint32_t TILE_BYTES = (uint32_t)(COLS * TOK * sizeof(T));
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 127u) & ~127u;
+  unsigned char* tiles = smem_raw + (tiles_base - raw);
+  T* Xs = reinterpret_cast<T*>(tiles);                             // [COLS][TOK]
+  T* Ds = reinterpret_cast<T*>(tiles + TILE_BYTES);                // [ROWS][TOK]
+  float* accS = reinterpret_cast<float*>(tiles + 2 * TILE_BYTES);  // [LIST_CAP]
+  uint16_t* list = reinterpret_cast<uint16_t*>(accS + LIST_CAP);   // [LIST_CAP]  (row_local << 8) | col_local
   __shared__ int ks[ROWS];          // CSR position of the row's first entry inside the window
   __shared__ int lstart[ROWS + 1];  // list offset of each row
+  __shared__ uint64_t bar;
+  __shared__ int abort_sh;
+  volatile int* abort_flag = &abort_sh;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int o0 = blockIdx.x * ROWS, c0 = blockIdx.y * COLS;
+  if (threadIdx.x == 0) {
+    abort_sh = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
 
   // ---- list the stored entries of the window
   if (threadIdx.x < ROWS) {
@@ -118,14 +142,19 @@ sddmm_window_kernel(const int32_t* __restrict__ row_ptr, const uint16_t* __restr
   for (int e = threadIdx.x; e < L; e += WARPS * 32) accS[e] = 0.f;
 
   const int groups = (L + 31) >> 5;
+  uint32_t ph = 0;
   for (int64_t t0 = 0; t0 < T_total; t0 += TOK) {
-    __syncthreads();
-    stage64<T>(Xs, X, ldx, T_total, I, t0, c0, vec_x != 0);
-    stage64<T>(Ds, dY, lddy, T_total, O, t0, o0, vec_dy != 0);
-    __syncthreads();
+    __syncthreads();  // the previous tiles have been read by every warp; list and accumulators are initialised
+    if (threadIdx.x == 0) {
+      mbar_expect_tx(smem_u32(&bar), 2 * TILE_BYTES);
+      tma_load_2d(tiles_base, &tmX, (int)t0, c0, smem_u32(&bar));
+      tma_load_2d(tiles_base + TILE_BYTES, &tmDY, (int)t0, o0, smem_u32(&bar));
+    }
+    if (!mst_ptx::mbar_wait(smem_u32(&bar), ph, abort_flag, &g_sddmm_error)) break;
+    ph ^= 1u;
     for (int g = warp; g < groups; g += WARPS) {
       float p[32];
-      float dy[8];
+      Vec8<T> dy;
       int cur_row = -1;
 #pragma unroll
       for (int j = 0; j < 32; ++j) {
@@ -135,15 +164,12 @@ sddmm_window_kernel(const int32_t* __restrict__ row_ptr, const uint16_t* __restr
           const int ent = list[e];
           const int rl = ent >> 8, cl = ent & 0xFF;
           if (rl != cur_row) {
-            load8(dy, Ds + rl * TOK + lane * 8);
+            dy.load(Ds + rl * TOK + lane * 8);
             cur_row = rl;
           }
-          float x[8];
-          load8(x, Xs + (cl & (COLS - 1)) * TOK + lane * 8);
-          float s = dy[0] * x[0];
-#pragma unroll
-          for (int i = 1; i < 8; ++i) s = fmaf(dy[i], x[i], s);
-          p[j] = s;
+          Vec8<T> x;
+          x.load(Xs + (cl & (COLS - 1)) * TOK + lane * 8);
+          p[j] = dot8(dy, x);
         }
       }
       // transposing reduction: afterwards p[0] in lane j is the sum over all lanes of entry j
@@ -184,20 +210,35 @@ __global__ void sample_dense_kernel(const uint32_t* __restrict__ bits, const int
 template <typename T>
 mst_status_t launch(const mst_layer* L, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T_total,
                     float* dW, cudaStream_t s) {
-  constexpr int VEC = 16 / (int)sizeof(T);
-  const size_t smem = (size_t)(COLS + ROWS) * TOK * sizeof(T) + (size_t)LIST_CAP * (4 + 2);
+  // feature-major copies of both operands in the per-device column scratch: [I x ldt] then [O x ldt]
+  const int64_t ldt = (T_total + 63) / 64 * 64;
+  void* ws = nullptr;
+  MST_TRY(mst_workspace_kind(MST_WS_COLUMNS, (size_t)(L->I + L->O) * ldt * sizeof(T), &ws));
+  T* XT = (T*)ws;
+  T* dYT = XT + (size_t)L->I * ldt;
+  MST_TRY(mst_feature_major_copy(X, ldx, T_total, L->I, L->dtype, XT, ldt, s));
+  MST_TRY(mst_feature_major_copy(dY, lddy, T_total, L->O, L->dtype, dYT, ldt, s));
+  CUtensorMap tmX, tmDY;
+  if (!mst_feature_major_map(&tmX, XT, T_total, L->I, ldt, L->dtype, TOK, COLS) ||
+      !mst_feature_major_map(&tmDY, dYT, T_total, L->O, ldt, L->dtype, TOK, ROWS))
+    return MST_ERR_SHAPE;
+  const size_t smem = (size_t)(COLS + ROWS) * TOK * sizeof(T) + (size_t)LIST_CAP * (4 + 2) + 128;
   MST_CUDA_TRY(cudaFuncSetAttribute(sddmm_window_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  const int vec_x = (ldx % VEC == 0) && (L->I % VEC == 0) && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0);
-  const int vec_dy = (lddy % VEC == 0) && (L->O % VEC == 0) && ((reinterpret_cast<uintptr_t>(dY) & 15u) == 0);
   dim3 grid((unsigned)((L->O + ROWS - 1) / ROWS), (unsigned)((L->I + COLS - 1) / COLS));
   const int c = L->cur;
-  sddmm_window_kernel<T><<<grid, WARPS * 32, smem, s>>>(L->row_ptr[c], L->col_idx[c], (const T*)dY, lddy, (const T*)X,
-                                                      ldx, T_total, L->O, L->I, dW, vec_x, vec_dy);
+  sddmm_window_kernel<T><<<grid, WARPS * 32, smem, s>>>(tmDY, tmX, L->row_ptr[c], L->col_idx[c], T_total, L->O, L->I, dW); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
 
 }  // namespace
+
+mst_status_t mst_sddmm_error_flags(int32_t* flags) {
+  int v = 0;
+  MST_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_sddmm_error, sizeof(int)));
+  *flags = v;
+  return MST_OK;
+}
 
 mst_status_t mst_launch_sddmm(const mst_layer* L, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,
                               float* dW, cudaStream_t s) {
@@ -240,7 +281,7 @@ extern "C" mst_status_t mst_sddmm_from_dense(const mst_layer_t* L, const float* 
   const int c = L->cur;
   const int64_t threads = L->nwords * 32;
   sample_dense_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
-      L->bits[c], L->wscan[c], L->O, L->I, L->wpr, G_dense, dW_vals);
+      L->bits[c], L->wscan[c], L->O, L->I, L->wpr, G_dense, dW_vals); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

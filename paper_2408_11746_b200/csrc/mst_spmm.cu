@@ -4,35 +4,48 @@
 // (r = input feature, idx = output feature, values fetched through the CSC->CSR permutation), so both are gathers
 // with a fixed summation order: no floating-point atomics, run-to-run identical results.
 //
-// A block owns TOK tokens x PANEL rows.  The activation tile is staged feature-major in shared memory, one column
-// chunk at a time (Xs[c][token]), so that a lane that owns 8 consecutive tokens fetches its 8 operands of one
-// nonzero with a single 128-bit (bf16) or two 128-bit (fp32) shared loads.  A warp owns PANEL/8 rows and walks each
-// row's nonzeros with a cursor that advances chunk by chunk (columns ascend inside a row); indices and values are
-// loaded 32 at a time, coalesced, and broadcast with shuffles.  Accumulation is fp32 in registers; the output tile
-// goes through shared memory so that global stores are contiguous along the feature dimension.
+// The activations are first copied feature-major once per call (inT[c][t], one coalesced transpose); after that a
+// nonzero costs one contiguous read of its column.  A block owns 256 tokens x 120 rows of the output.  A producer
+// warp streams [column chunk x 256 tokens] tiles of inT into a ring of shared-memory stages with the TMA unit
+// (cp.async.bulk.tensor, this GPU's memory only, no multicast); 15 compute warps each own 8 rows and hold their
+// 8 x 256 partial sums in registers (lane = 8 consecutive tokens) across all chunks.  Per nonzero: one warp shuffle
+// broadcasts (column, value), one 128-bit shared load fetches the lane's 8 activations, and 8 FMAs accumulate in
+// fp32 -- for bf16 layers with the mixed-precision instruction (bf16 x bf16 + fp32), so no unpacking is issued.
+// Work is proportional to nnz: a (row, chunk) visit costs a ballot over a 32-entry window of the row kept in
+// registers, and global index/value loads happen only when a window is used up (coalesced, 32 entries).
+// Rows of unequal nnz: inside a panel the rows are dealt to the warps in order of decreasing nnz, back and forth,
+// so every warp gets a similar count; panels are many more than SMs and are scheduled dynamically.
+// The output tile leaves through shared memory so that global stores are contiguous along the feature dimension.
+#include <cuda.h>
+
 #include "mst_internal.cuh"
 #include "mst_tc_gemm.cuh"
+#include "mst_tc_ptx.cuh"
 
 namespace {
 
 constexpr int TOK = 256;    // tokens per block (8 per lane)
-constexpr int PANEL = 64;   // rows per block
-constexpr int WARPS = 8;
+constexpr int PANEL = 120;  // rows per block
+constexpr int WARPS = 15;   // compute warps; one more warp produces (512 threads: 128 registers each)
 constexpr int RPW = PANEL / WARPS;
 constexpr int OS_LD = PANEL + 1;
+constexpr int STAGES = 3;
+constexpr int THREADS = (WARPS + 1) * 32;
 
 template <typename T>
 struct Cfg;
 template <>
 struct Cfg<float> {
-  static constexpr int KC = 64;
+  static constexpr int KC = 64;   // columns per stage: 64 KiB
   static constexpr int VEC = 4;
 };
 template <>
 struct Cfg<uint16_t> {
-  static constexpr int KC = 128;
+  static constexpr int KC = 128;  // 64 KiB
   static constexpr int VEC = 8;
 };
+
+__device__ int g_spmm_error = 0;  // sticky: a bounded wait expired
 
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(uint16_t v) { return __uint_as_float(((uint32_t)v) << 16); }
@@ -45,7 +58,9 @@ __device__ __forceinline__ void store_out(uint16_t* p, float v) {
   *p = (uint16_t)(u >> 16);
 }
 
-__device__ __forceinline__ void fma8(float (&acc)[8], float w, const float* xs) {
+// acc[0..7] += w * xs[0..7]
+__device__ __forceinline__ void fma8(float (&acc)[8], uint32_t wbits, const float* xs) {
+  const float w = __uint_as_float(wbits);
   const float4 a = *reinterpret_cast<const float4*>(xs);
   const float4 b = *reinterpret_cast<const float4*>(xs + 4);
   acc[0] = fmaf(w, a.x, acc[0]);
@@ -57,133 +72,280 @@ __device__ __forceinline__ void fma8(float (&acc)[8], float w, const float* xs) 
   acc[6] = fmaf(w, b.z, acc[6]);
   acc[7] = fmaf(w, b.w, acc[7]);
 }
-__device__ __forceinline__ void fma8(float (&acc)[8], float w, const uint16_t* xs) {
-  const uint4 v = *reinterpret_cast<const uint4*>(xs);
-  acc[0] = fmaf(w, __uint_as_float(v.x << 16), acc[0]);
-  acc[1] = fmaf(w, __uint_as_float(v.x & 0xFFFF0000u), acc[1]);
-  acc[2] = fmaf(w, __uint_as_float(v.y << 16), acc[2]);
-  acc[3] = fmaf(w, __uint_as_float(v.y & 0xFFFF0000u), acc[3]);
-  acc[4] = fmaf(w, __uint_as_float(v.z << 16), acc[4]);
-  acc[5] = fmaf(w, __uint_as_float(v.z & 0xFFFF0000u), acc[5]);
-  acc[6] = fmaf(w, __uint_as_float(v.w << 16), acc[6]);
-  acc[7] = fmaf(w, __uint_as_float(v.w & 0xFFFF0000u), acc[7]);
+// bf16 operands, fp32 accumulator: d = a * b + c with the exact product (the mixed-precision FMA of sm_100)
+__device__ __forceinline__ void fma_bf16(float& acc, uint16_t a, uint16_t b) {
+  asm("fma.rn.f32.bf16 %0, %1, %2, %0;" : "+f"(acc) : "h"(a), "h"(b));
 }
-
-// Stage columns [c0, c0+KC) of tokens [t0, t0+TOK) into Xs[c][token]; out-of-range elements become 0.
-template <typename T>
-__device__ __forceinline__ void stage_tile(T* __restrict__ Xs, const T* __restrict__ in, int64_t ld, int64_t T_total,
-                                           int C, int64_t t0, int c0, bool vec_ok) {
-  constexpr int KC = Cfg<T>::KC, VEC = Cfg<T>::VEC;
-  const int tt = threadIdx.x;
-  const int64_t t = t0 + tt;
-  const bool row_ok = t < T_total;
-  const T* src = in + t * ld + c0;
-  if (vec_ok) {
-#pragma unroll 4
-    for (int v = 0; v < KC / VEC; ++v) {
-      uint4 q = make_uint4(0, 0, 0, 0);
-      if (row_ok && c0 + v * VEC < C) q = *reinterpret_cast<const uint4*>(src + v * VEC);
-      const T* e = reinterpret_cast<const T*>(&q);
+__device__ __forceinline__ void fma8(float (&acc)[8], uint32_t wbits, const uint16_t* xs) {
+  const uint4 v = *reinterpret_cast<const uint4*>(xs);
+  const uint16_t w = (uint16_t)wbits;
+  const uint32_t xw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-      for (int j = 0; j < VEC; ++j) Xs[(v * VEC + j) * TOK + tt] = e[j];
-    }
-  } else {
-    for (int c = 0; c < KC; ++c) {
-      T x = T(0);
-      if (row_ok && c0 + c < C) x = src[c];
-      Xs[c * TOK + tt] = x;
-    }
+  for (int j = 0; j < 4; ++j) {
+    uint16_t lo, hi;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(xw[j]));
+    fma_bf16(acc[2 * j], w, lo);
+    fma_bf16(acc[2 * j + 1], w, hi);
+  }
+}
+// two entries of one row: both operand fetches are issued before the first FMA
+__device__ __forceinline__ void fma8x2(float (&acc)[8], uint32_t wa, const float* xa, uint32_t wb, const float* xb) {
+  const float4 a0 = *reinterpret_cast<const float4*>(xa), a1 = *reinterpret_cast<const float4*>(xa + 4);
+  const float4 b0 = *reinterpret_cast<const float4*>(xb), b1 = *reinterpret_cast<const float4*>(xb + 4);
+  const float fa = __uint_as_float(wa), fb = __uint_as_float(wb);
+  acc[0] = fmaf(fa, a0.x, acc[0]); acc[1] = fmaf(fa, a0.y, acc[1]); acc[2] = fmaf(fa, a0.z, acc[2]); acc[3] = fmaf(fa, a0.w, acc[3]);
+  acc[4] = fmaf(fa, a1.x, acc[4]); acc[5] = fmaf(fa, a1.y, acc[5]); acc[6] = fmaf(fa, a1.z, acc[6]); acc[7] = fmaf(fa, a1.w, acc[7]);
+  acc[0] = fmaf(fb, b0.x, acc[0]); acc[1] = fmaf(fb, b0.y, acc[1]); acc[2] = fmaf(fb, b0.z, acc[2]); acc[3] = fmaf(fb, b0.w, acc[3]);
+  acc[4] = fmaf(fb, b1.x, acc[4]); acc[5] = fmaf(fb, b1.y, acc[5]); acc[6] = fmaf(fb, b1.z, acc[6]); acc[7] = fmaf(fb, b1.w, acc[7]);
+}
+__device__ __forceinline__ void fma8x2(float (&acc)[8], uint32_t wa, const uint16_t* xa, uint32_t wb, const uint16_t* xb) {
+  const uint4 va = *reinterpret_cast<const uint4*>(xa);
+  const uint4 vb = *reinterpret_cast<const uint4*>(xb);
+  const uint32_t aw[4] = {va.x, va.y, va.z, va.w}, bw[4] = {vb.x, vb.y, vb.z, vb.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint16_t lo, hi;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(aw[j]));
+    fma_bf16(acc[2 * j], (uint16_t)wa, lo);
+    fma_bf16(acc[2 * j + 1], (uint16_t)wa, hi);
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint16_t lo, hi;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(bw[j]));
+    fma_bf16(acc[2 * j], (uint16_t)wb, lo);
+    fma_bf16(acc[2 * j + 1], (uint16_t)wb, hi);
+  }
+}
+__device__ __forceinline__ uint32_t weight_bits(float v) { return __float_as_uint(v); }
+__device__ __forceinline__ uint32_t weight_bits(uint16_t v) { return (uint32_t)v; }
+
+// inT[c][t] = in[t][c]: 64 x 64 tiles through shared memory, coalesced on both sides.  ldt >= T, multiple of 16 bytes.
+template <typename T>
+__global__ void __launch_bounds__(256) transpose_in_kernel(const T* __restrict__ in, int64_t ldin, int64_t T_total, int C,
+                                                          T* __restrict__ inT, int64_t ldt) {
+  __shared__ T tile[64][64 + (sizeof(T) == 2 ? 2 : 1)];
+  const int64_t t0 = (int64_t)blockIdx.x * 64;
+  const int c0 = blockIdx.y * 64;
+  const int x = threadIdx.x & 63, y = threadIdx.x >> 6;   // 4 rows of 64 per pass
+#pragma unroll 4
+  for (int j = 0; j < 16; ++j) {
+    const int tl = y + 4 * j;
+    const int64_t t = t0 + tl;
+    tile[tl][x] = (t < T_total && c0 + x < C) ? in[t * ldin + c0 + x] : T(0);
+  }
+  __syncthreads();
+#pragma unroll 4
+  for (int j = 0; j < 16; ++j) {
+    const int cl = y + 4 * j;
+    if (c0 + cl < C && t0 + x < ldt) inT[(int64_t)(c0 + cl) * ldt + t0 + x] = tile[x][cl];
   }
 }
 
 template <typename T, bool PERM>
-__global__ void __launch_bounds__(WARPS * 32, 2)
-spmm_panel_kernel(const int32_t* __restrict__ ptr, const uint16_t* __restrict__ idx, const T* __restrict__ vals,
-                  const int32_t* __restrict__ perm, const T* __restrict__ in, int64_t ldin, T* __restrict__ out,
-                  int64_t ldout, int64_t T_total, int R_total, int C, int vec_ok) {
+__global__ void __launch_bounds__(THREADS, 1)
+spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __restrict__ ptr,
+                   const uint16_t* __restrict__ idx, const T* __restrict__ vals, const int32_t* __restrict__ perm,
+                   T* __restrict__ out, int64_t ldout, int64_t T_total, int R_total, int C) {
+  using namespace mst_ptx;
   constexpr int KC = Cfg<T>::KC;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  T* Xs = reinterpret_cast<T*>(smem_raw);
-  float* Os = reinterpret_cast<float*>(smem_raw);
+  constexpr uint32_t STAGE_BYTES = (uint32_t)(KC * TOK * sizeof(T));
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 127u) & ~127u;
+  unsigned char* tiles = smem_raw + (tiles_base - raw);
+  __shared__ uint64_t bars[2 * STAGES];
+  __shared__ int nnz_sh[PANEL];
+  __shared__ unsigned char order_sh[PANEL];   // order_sh[w * RPW + j] = local row of warp w's j-th row
+  __shared__ int abort_sh;
+  volatile int* abort_flag = &abort_sh;
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int r_base = blockIdx.x * PANEL + warp * RPW;
+  const int r0 = blockIdx.x * PANEL;
   const int64_t t0 = (int64_t)blockIdx.y * TOK;
-
-  int32_t kcur[RPW], kend[RPW];
-  float acc[RPW][8];
-#pragma unroll
-  for (int rr = 0; rr < RPW; ++rr) {
-    const int r = r_base + rr;
-    kcur[rr] = r < R_total ? ptr[r] : 0;
-    kend[rr] = r < R_total ? ptr[r + 1] : 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[rr][j] = 0.f;
+  if (threadIdx.x == 0) {
+    abort_sh = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, WARPS);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // rows of the panel in order of decreasing nnz, dealt to the warps back and forth
+  if (threadIdx.x < PANEL) {
+    const int r = r0 + threadIdx.x;
+    nnz_sh[threadIdx.x] = r < R_total ? ptr[r + 1] - ptr[r] : -1;
+  }
+  __syncthreads();
+  if (threadIdx.x < PANEL) {
+    const int mine = nnz_sh[threadIdx.x];
+    int rank = 0;
+    for (int j = 0; j < PANEL; ++j) {
+      const int other = nnz_sh[j];
+      rank += (other > mine || (other == mine && j < (int)threadIdx.x)) ? 1 : 0;
+    }
+    const int round = rank / WARPS, pos = rank % WARPS;
+    const int w = (round & 1) ? WARPS - 1 - pos : pos;
+    order_sh[w * RPW + round] = (unsigned char)threadIdx.x;
+  }
+  __syncthreads();
+  const int nchunks = (C + KC - 1) / KC;
 
-  for (int c0 = 0; c0 < C; c0 += KC) {
-    __syncthreads();  // previous chunk fully consumed
-    stage_tile<T>(Xs, in, ldin, T_total, C, t0, c0, vec_ok != 0);
-    __syncthreads();
-    const uint32_t c_end = (uint32_t)(c0 + KC);
+  if (warp == WARPS) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      for (int c = 0; c < nchunks && !*abort_flag; ++c) {
+        if (!mst_ptx::mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag, &g_spmm_error)) break;
+        mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+        tma_load_2d(tiles_base + (uint32_t)s * STAGE_BYTES, &tmIn, (int)t0, c * KC, full0 + 8 * s);
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ compute warps
+    int rloc[RPW];
+    int32_t kwin[RPW], kend[RPW];
+    uint32_t wci[RPW], wval[RPW];   // this lane's entry of the row's current 32-entry window: column, value bits
+    float acc[RPW][8];
+    auto load_window = [&](int rr) {
+      const int32_t kk = kwin[rr] + lane;
+      wci[rr] = 0xFFFFFFFFu;
+      wval[rr] = 0u;
+      if (kk < kend[rr]) {
+        wci[rr] = (uint32_t)idx[kk];
+        wval[rr] = weight_bits(PERM ? vals[perm[kk]] : vals[kk]);
+      }
+    };
 #pragma unroll
     for (int rr = 0; rr < RPW; ++rr) {
-      int32_t k = kcur[rr];
-      const int32_t e = kend[rr];
-      while (k < e) {
-        const int32_t kk = k + lane;
-        const uint32_t ci = kk < e ? (uint32_t)idx[kk] : 0xFFFFFFFFu;
-        const bool inb = ci < c_end;
-        const unsigned m = __ballot_sync(0xffffffffu, inb);
-        const int n = __popc(m);  // columns ascend, so the in-chunk entries are the first n
-        if (n == 0) break;
-        float w = 0.f;
-        if (inb) w = to_float(PERM ? vals[perm[kk]] : vals[kk]);
-        const int cl = (int)ci - c0;
-        for (int j = 0; j < n; ++j) {
-          const int cj = __shfl_sync(0xffffffffu, cl, j);
-          const float wj = __shfl_sync(0xffffffffu, w, j);
-          fma8(acc[rr], wj, Xs + cj * TOK + lane * 8);
-        }
-        k += n;
-        if (n < 32) break;
-      }
-      kcur[rr] = k;
+      rloc[rr] = order_sh[warp * RPW + rr];
+      const int r = r0 + rloc[rr];
+      kwin[rr] = r < R_total ? ptr[r] : 0;
+      kend[rr] = r < R_total ? ptr[r + 1] : 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[rr][j] = 0.f;
     }
-  }
+#pragma unroll
+    for (int rr = 0; rr < RPW; ++rr) load_window(rr);
 
-  // epilogue: registers -> shared (token-permuted rows, conflict-free) -> global, contiguous along the rows
-  __syncthreads();
+    int s = 0;
+    uint32_t ph = 0;
+    for (int c = 0; c < nchunks; ++c) {
+      if (!mst_ptx::mbar_wait(full0 + 8 * s, ph, abort_flag, &g_spmm_error)) break;
+      const T* Xs = reinterpret_cast<const T*>(tiles + (size_t)s * STAGE_BYTES);
+      const uint32_t c0 = (uint32_t)(c * KC), c_end = c0 + KC;
 #pragma unroll
-  for (int rr = 0; rr < RPW; ++rr)
+      for (int rr = 0; rr < RPW; ++rr) {
+        while (true) {
+          // columns ascend and everything below c0 was consumed in earlier chunks: the entries of this chunk are the
+          // lanes whose column lies below c_end and has not been used yet
+          const unsigned m = __ballot_sync(0xffffffffu, wci[rr] >= c0 && wci[rr] < c_end);
+          if (m == 0) break;
+          const int first = __ffs(m) - 1, n = __popc(m);
+          // bf16: column and value travel in one shuffle (16 bits each); two entries per trip so that the shared
+          // loads of the second overlap the FMAs of the first
+          const uint32_t mine = sizeof(T) == 2 ? (((wci[rr] - c0) << 16) | wval[rr]) : 0u;
+          int j = first;
+          for (; j + 1 < first + n; j += 2) {
+            uint32_t ca, wa, cb, wb;
+            if (sizeof(T) == 2) {
+              const uint32_t pa = __shfl_sync(0xffffffffu, mine, j), pb = __shfl_sync(0xffffffffu, mine, j + 1);
+              ca = pa >> 16; wa = pa & 0xFFFFu; cb = pb >> 16; wb = pb & 0xFFFFu;
+            } else {
+              ca = __shfl_sync(0xffffffffu, wci[rr], j) - c0;
+              wa = __shfl_sync(0xffffffffu, wval[rr], j);
+              cb = __shfl_sync(0xffffffffu, wci[rr], j + 1) - c0;
+              wb = __shfl_sync(0xffffffffu, wval[rr], j + 1);
+            }
+            fma8x2(acc[rr], wa, Xs + ca * TOK + lane * 8, wb, Xs + cb * TOK + lane * 8);
+          }
+          if (j < first + n) {
+            uint32_t ca, wa;
+            if (sizeof(T) == 2) {
+              const uint32_t pa = __shfl_sync(0xffffffffu, mine, j);
+              ca = pa >> 16; wa = pa & 0xFFFFu;
+            } else {
+              ca = __shfl_sync(0xffffffffu, wci[rr], j) - c0;
+              wa = __shfl_sync(0xffffffffu, wval[rr], j);
+            }
+            fma8(acc[rr], wa, Xs + ca * TOK + lane * 8);
+          }
+          if (first + n < 32) break;        // the window still holds entries of later chunks (or the row has ended)
+          kwin[rr] += 32;                   // window used up: next 32 entries of the row
+          load_window(rr);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(empty0 + 8 * s);
+      if (++s == STAGES) { s = 0; ph ^= 1u; }
+    }
+
+    // epilogue: registers -> shared (token-permuted rows, conflict-free) -> global, contiguous along the rows.
+    // Named barrier over the compute warps only: every stage has been consumed, the tiles can be overwritten.
+    asm volatile("bar.sync 1, %0;" ::"n"(WARPS * 32) : "memory");
+    float* Os = reinterpret_cast<float*>(tiles);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) Os[(j * 32 + lane) * OS_LD + warp * RPW + rr] = acc[rr][j];
-  __syncthreads();
-  for (int i = threadIdx.x; i < TOK * PANEL; i += WARPS * 32) {
-    const int tt = i / PANEL, rl = i % PANEL;
-    const int64_t t = t0 + tt;
-    const int r = blockIdx.x * PANEL + rl;
-    if (t < T_total && r < R_total) store_out(out + t * ldout + r, Os[((tt & 7) * 32 + (tt >> 3)) * OS_LD + rl]);
+    for (int rr = 0; rr < RPW; ++rr)
+#pragma unroll
+      for (int j = 0; j < 8; ++j) Os[(j * 32 + lane) * OS_LD + rloc[rr]] = acc[rr][j];
+    asm volatile("bar.sync 1, %0;" ::"n"(WARPS * 32) : "memory");
+    for (int i = threadIdx.x; i < TOK * PANEL; i += WARPS * 32) {
+      const int tt = i / PANEL, rl = i % PANEL;
+      const int64_t t = t0 + tt;
+      const int r = r0 + rl;
+      if (t < T_total && r < R_total) store_out(out + t * ldout + r, Os[((tt & 7) * 32 + (tt >> 3)) * OS_LD + rl]);
+    }
   }
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn spmm_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  }
+  return fn;
+}
+
+}  // namespace
+mst_status_t mst_feature_major_copy(const void* in, int64_t ldin, int64_t T, int C, mst_dtype_t dtype, void* out, int64_t ldt,
+                                    cudaStream_t s);
+bool mst_feature_major_map(CUtensorMap* tm, const void* base, int64_t T, int C, int64_t ldt, mst_dtype_t dtype, int box_tokens,
+                           int box_features);
+namespace {
+
 template <typename T>
 constexpr size_t spmm_smem() {
-  return (size_t)Cfg<T>::KC * TOK * sizeof(T) > (size_t)TOK * OS_LD * 4 ? (size_t)Cfg<T>::KC * TOK * sizeof(T)
-                                                                      : (size_t)TOK * OS_LD * 4;
+  return (size_t)STAGES * Cfg<T>::KC * TOK * sizeof(T) + 128 > (size_t)TOK * OS_LD * 4 + 128
+             ? (size_t)STAGES * Cfg<T>::KC * TOK * sizeof(T) + 128
+             : (size_t)TOK * OS_LD * 4 + 128;
 }
 
 template <typename T, bool PERM>
 mst_status_t launch(const int32_t* ptr, const uint16_t* idx, const void* vals, const int32_t* perm, const void* in,
                     int64_t ldin, void* out, int64_t ldout, int64_t T_total, int R_total, int C, cudaStream_t s) {
+  // feature-major copy of the activations: [C x ldt], ldt a multiple of 64 tokens
+  const int64_t ldt = (T_total + 63) / 64 * 64;
+  const mst_dtype_t dt = sizeof(T) == 2 ? MST_BF16 : MST_F32;
+  void* inT = nullptr;
+  MST_TRY(mst_workspace_kind(MST_WS_COLUMNS, (size_t)C * ldt * sizeof(T), &inT));
+  MST_TRY(mst_feature_major_copy(in, ldin, T_total, C, dt, inT, ldt, s));
+  CUtensorMap tm;
+  if (!mst_feature_major_map(&tm, inT, T_total, C, ldt, dt, TOK, Cfg<T>::KC)) return MST_ERR_SHAPE;
   const size_t smem = spmm_smem<T>();
   // per call: the attribute belongs to the current device's copy of the kernel
-  MST_CUDA_TRY(cudaFuncSetAttribute(spmm_panel_kernel<T, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  constexpr int VEC = Cfg<T>::VEC;
-  const int vec_ok = (ldin % VEC == 0) && (C % VEC == 0) && ((reinterpret_cast<uintptr_t>(in) & 15u) == 0);
+  MST_CUDA_TRY(cudaFuncSetAttribute(spmm_stream_kernel<T, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((unsigned)((R_total + PANEL - 1) / PANEL), (unsigned)((T_total + TOK - 1) / TOK));
-  spmm_panel_kernel<T, PERM><<<grid, WARPS * 32, smem, s>>>(ptr, idx, (const T*)vals, perm, (const T*)in, ldin, (T*)out,
-                                                          ldout, T_total, R_total, C, vec_ok);
+  spmm_stream_kernel<T, PERM><<<grid, THREADS, smem, s>>>(tm, ptr, idx, (const T*)vals, perm, (T*)out, ldout, T_total, R_total, C); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
@@ -212,12 +374,45 @@ mst_status_t launch_act(void* out, int64_t ldout, const void* pre, int64_t ldpre
                         cudaStream_t s) {
   const int64_t n = rows * cols;
   const int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 16);
-  act_rows_kernel<T><<<blocks, 256, 0, s>>>((T*)out, ldout, (const T*)pre, ldpre, rows, cols, act);
+  act_rows_kernel<T><<<blocks, 256, 0, s>>>((T*)out, ldout, (const T*)pre, ldpre, rows, cols, act); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
 
 }  // namespace
+
+// feature-major copy out[c][t] = in[t][c] (zero for T <= t < ldt) and its TMA description with a box of
+// box_tokens x box_features; shared with the weight-gradient kernel
+mst_status_t mst_feature_major_copy(const void* in, int64_t ldin, int64_t T, int C, mst_dtype_t dtype, void* out, int64_t ldt,
+                                    cudaStream_t s) {
+  dim3 grid((unsigned)(ldt / 64), (unsigned)((C + 63) / 64));
+  if (dtype == MST_F32)
+    { transpose_in_kernel<float><<<grid, 256, 0, s>>>((const float*)in, ldin, T, C, (float*)out, ldt); MST_COUNT_LAUNCH(); }
+  else
+    { transpose_in_kernel<uint16_t><<<grid, 256, 0, s>>>((const uint16_t*)in, ldin, T, C, (uint16_t*)out, ldt); MST_COUNT_LAUNCH(); }
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
+}
+bool mst_feature_major_map(CUtensorMap* tm, const void* base, int64_t T, int C, int64_t ldt, mst_dtype_t dtype, int box_tokens,
+                           int box_features) {
+  EncodeTiledFn enc = spmm_encode_fn();
+  if (!enc) return false;
+  const size_t es = dtype == MST_F32 ? 4 : 2;
+  cuuint64_t dims[2] = {(cuuint64_t)T, (cuuint64_t)C};
+  cuuint64_t strides[1] = {(cuuint64_t)ldt * es};
+  cuuint32_t box[2] = {(cuuint32_t)box_tokens, (cuuint32_t)box_features};
+  cuuint32_t estr[2] = {1u, 1u};
+  return enc(tm, dtype == MST_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+             dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+mst_status_t mst_spmm_error_flags(int32_t* flags) {
+  int v = 0;
+  MST_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_spmm_error, sizeof(int)));
+  *flags = v;
+  return MST_OK;
+}
 
 mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in, int64_t ldin, int64_t T, void* out,
                              int64_t ldout, cudaStream_t s, int act, void* pre, int64_t ldpre) {

@@ -282,14 +282,14 @@ int64_t mst_scan_block_sums_len(int64_t n) { return (n + SCAN_TILE - 1) / SCAN_T
 mst_status_t mst_scan_i32_if(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, const int* enabled,
                              cudaStream_t s) {
   if (n <= 0) {
-    scan_empty<<<1, 1, 0, s>>>(out);
+    scan_empty<<<1, 1, 0, s>>>(out); MST_COUNT_LAUNCH();
     MST_CUDA_TRY(cudaGetLastError());
     return MST_OK;
   }
   const int64_t tiles = (n + SCAN_TILE - 1) / SCAN_TILE;
-  scan_tile_sums<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, enabled);
-  scan_sums_inplace<<<1, 1024, 0, s>>>(block_sums, tiles, enabled);
-  scan_tiles<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, out, enabled);
+  scan_tile_sums<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, enabled); MST_COUNT_LAUNCH();
+  scan_sums_inplace<<<1, 1024, 0, s>>>(block_sums, tiles, enabled); MST_COUNT_LAUNCH();
+  scan_tiles<<<(unsigned)tiles, SCAN_THREADS, 0, s>>>(in, n, block_sums, out, enabled); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
@@ -301,17 +301,17 @@ mst_status_t mst_scan_i32(const int32_t* in, int32_t* out, int64_t n, int32_t* b
 // bits[set] must be final.  Computes wscan[set], row_ptr[set], col_idx[set], vals[set].
 mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set,
                                    cudaStream_t s) {
-  popc_words<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[set], L->nwords, L->word_cnt);
+  popc_words<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[set], L->nwords, L->word_cnt); MST_COUNT_LAUNCH();
   MST_TRY(mst_scan_i32(L->word_cnt, L->wscan[set], L->nwords, L->block_sums, s));
   const unsigned grid = blocks_for(L->nwords * 32, 256);
   if (L->dtype == MST_F32) {
     fill_csr<float><<<grid, 256, 0, s>>>(L->bits[set], L->wscan[set], L->O, L->I, L->wpr, L->col_idx[set],
                                          (float*)L->vals[set], L->row_ptr[set], (const float*)dense_W, ldw,
-                                         L->bits[old_set], L->wscan[old_set], (const float*)L->vals[old_set]);
+                                         L->bits[old_set], L->wscan[old_set], (const float*)L->vals[old_set]); MST_COUNT_LAUNCH();
   } else {
     fill_csr<uint16_t><<<grid, 256, 0, s>>>(L->bits[set], L->wscan[set], L->O, L->I, L->wpr, L->col_idx[set],
                                             (uint16_t*)L->vals[set], L->row_ptr[set], (const uint16_t*)dense_W, ldw,
-                                            L->bits[old_set], L->wscan[old_set], (const uint16_t*)L->vals[old_set]);
+                                            L->bits[old_set], L->wscan[old_set], (const uint16_t*)L->vals[old_set]); MST_COUNT_LAUNCH();
   }
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
@@ -321,11 +321,11 @@ mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, i
 mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s) {
   const int c = L->cur;
   transpose_bits<<<blocks_for((int64_t)L->wpc * L->wpr * 32, 256), 256, 0, s>>>(L->bits[c], L->O, L->I, L->wpr, L->wpc,
-                                                                                L->bitsT);
-  popc_words<<<blocks_for(L->nwordsT, 256), 256, 0, s>>>(L->bitsT, L->nwordsT, L->word_cnt);
+                                                                                L->bitsT); MST_COUNT_LAUNCH();
+  popc_words<<<blocks_for(L->nwordsT, 256), 256, 0, s>>>(L->bitsT, L->nwordsT, L->word_cnt); MST_COUNT_LAUNCH();
   MST_TRY(mst_scan_i32(L->word_cnt, L->wscanT, L->nwordsT, L->block_sums, s));
   fill_csc<<<blocks_for(L->nwordsT * 32, 256), 256, 0, s>>>(L->bitsT, L->wscanT, L->O, L->I, L->wpr, L->wpc, L->bits[c],
-                                                            L->wscan[c], L->row_idx, L->perm, L->col_ptr);
+                                                            L->wscan[c], L->row_idx, L->perm, L->col_ptr); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   L->csc_valid = 1;
   return MST_OK;
@@ -338,6 +338,10 @@ mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s) {
 
 mst_status_t mst_densify(const mst_layer* L, cudaStream_t s) {
   const int c = L->cur;
+  // with value tracking the image is reused until the mask or the values change
+  if (L->track_values && L->dense_version == L->version && L->dense_epoch == L->values_epoch) return MST_OK;
+  L->dense_version = L->version;
+  L->dense_epoch = L->values_epoch;
   const int64_t groups = L->N / 8;  // callers guarantee I % 8 == 0
   {
     MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
@@ -351,7 +355,7 @@ mst_status_t mst_densify(const mst_layer* L, cudaStream_t s) {
 // new mask of an update from the three selection results; leaves popcounts in word_cnt
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s) {
   combine_bits<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[L->cur], L->pruned_bits, L->grad_bits, L->rand_bits,
-                                                          L->nwords, L->bits[new_set], L->word_cnt);
+                                                          L->nwords, L->bits[new_set], L->word_cnt); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
@@ -363,8 +367,8 @@ extern "C" mst_status_t mst_pack(mst_layer_t* L, const void* W_dense, int64_t ld
   cudaStream_t s = (cudaStream_t)stream;
   const int set = L->cur;
   L->nnz = -1;
-  mask_bytes_to_bits<<<blocks_for(L->nwords * 32, 256), 256, 0, s>>>(mask, L->O, L->I, L->wpr, L->bits[set]);
-  popc_words<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[set], L->nwords, L->word_cnt);
+  mask_bytes_to_bits<<<blocks_for(L->nwords * 32, 256), 256, 0, s>>>(mask, L->O, L->I, L->wpr, L->bits[set]); MST_COUNT_LAUNCH();
+  popc_words<<<blocks_for(L->nwords, 256), 256, 0, s>>>(L->bits[set], L->nwords, L->word_cnt); MST_COUNT_LAUNCH();
   MST_TRY(mst_scan_i32(L->word_cnt, L->wscan[set], L->nwords, L->block_sums, s));
   int32_t total = 0;
   MST_CUDA_TRY(cudaMemcpyAsync(&total, L->wscan[set] + L->nwords, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
@@ -386,7 +390,7 @@ extern "C" mst_status_t mst_export_csr(const mst_layer_t* L, int32_t* row_ptr, i
   const int c = L->cur;
   if (row_ptr)
     MST_CUDA_TRY(cudaMemcpyAsync(row_ptr, L->row_ptr[c], sizeof(int32_t) * (L->O + 1), cudaMemcpyDeviceToDevice, s));
-  if (col_idx && L->nnz > 0) widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->col_idx[c], L->nnz, col_idx);
+  if (col_idx && L->nnz > 0) { widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->col_idx[c], L->nnz, col_idx); MST_COUNT_LAUNCH(); }
   if (vals && L->nnz > 0)
     MST_CUDA_TRY(cudaMemcpyAsync(vals, L->vals[c], mst_elem_size(L->dtype) * L->nnz, cudaMemcpyDeviceToDevice, s));
   MST_CUDA_TRY(cudaGetLastError());
@@ -401,7 +405,7 @@ extern "C" mst_status_t mst_export_csc(const mst_layer_t* L, int32_t* col_ptr, i
   MST_TRY(mst_ensure_csc(L, s));
   if (col_ptr)
     MST_CUDA_TRY(cudaMemcpyAsync(col_ptr, L->col_ptr, sizeof(int32_t) * (L->I + 1), cudaMemcpyDeviceToDevice, s));
-  if (row_idx && L->nnz > 0) widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->row_idx, L->nnz, row_idx);
+  if (row_idx && L->nnz > 0) { widen_u16<<<blocks_for(L->nnz, 256), 256, 0, s>>>(L->row_idx, L->nnz, row_idx); MST_COUNT_LAUNCH(); }
   if (perm && L->nnz > 0)
     MST_CUDA_TRY(cudaMemcpyAsync(perm, L->perm, sizeof(int32_t) * L->nnz, cudaMemcpyDeviceToDevice, s));
   MST_CUDA_TRY(cudaGetLastError());
@@ -415,9 +419,9 @@ extern "C" mst_status_t mst_validate(const mst_layer_t* L, mst_stream_t stream) 
   const int c = L->cur;
   MST_TRY(mst_ensure_csc(L, s));
   validate_rows<<<blocks_for(L->O, 128), 128, 0, s>>>(L->row_ptr[c], L->col_idx[c], L->bits[c], L->O, L->I, L->wpr,
-                                                     L->nnz, L->flags);
+                                                     L->nnz, L->flags); MST_COUNT_LAUNCH();
   validate_cols<<<blocks_for(L->I, 128), 128, 0, s>>>(L->col_ptr, L->row_idx, L->perm, L->row_ptr[c], L->col_idx[c],
-                                                     L->O, L->I, L->nnz, L->flags);
+                                                     L->O, L->I, L->nnz, L->flags); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   int32_t f = 0;
   MST_CUDA_TRY(cudaMemcpyAsync(&f, L->flags, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
@@ -509,16 +513,16 @@ extern "C" mst_status_t mst_mask_to_csr_noalloc(int32_t O, int32_t I, mst_dtype_
   int32_t* sums = (int32_t*)(base + NOALLOC_OFF_SUMS);
   cudaStream_t s = (cudaStream_t)stream;
   // every word of the scratch that the later kernels read is written first by this call: nothing needs clearing
-  mask_bytes_to_bits<<<blocks_for(nwords * 32, 256), 256, 0, s>>>(mask, O, I, wpr, bits);
-  popc_words<<<blocks_for(nwords, 256), 256, 0, s>>>(bits, nwords, cnt);
+  mask_bytes_to_bits<<<blocks_for(nwords * 32, 256), 256, 0, s>>>(mask, O, I, wpr, bits); MST_COUNT_LAUNCH();
+  popc_words<<<blocks_for(nwords, 256), 256, 0, s>>>(bits, nwords, cnt); MST_COUNT_LAUNCH();
   MST_TRY(mst_scan_i32(cnt, scan, nwords, sums, s));
   const unsigned grid = blocks_for(nwords * 32, 256);
   if (dtype == MST_F32)
-    fill_csr_external<float><<<grid, 256, 0, s>>>(bits, scan, O, I, wpr, (const float*)W_dense, ldw, nnz_capacity,
-                                                  row_ptr, col_idx, (float*)vals);
+    { fill_csr_external<float><<<grid, 256, 0, s>>>(bits, scan, O, I, wpr, (const float*)W_dense, ldw, nnz_capacity,
+                                                  row_ptr, col_idx, (float*)vals); MST_COUNT_LAUNCH(); }
   else
-    fill_csr_external<uint16_t><<<grid, 256, 0, s>>>(bits, scan, O, I, wpr, (const uint16_t*)W_dense, ldw, nnz_capacity,
-                                                     row_ptr, col_idx, (uint16_t*)vals);
+    { fill_csr_external<uint16_t><<<grid, 256, 0, s>>>(bits, scan, O, I, wpr, (const uint16_t*)W_dense, ldw, nnz_capacity,
+                                                     row_ptr, col_idx, (uint16_t*)vals); MST_COUNT_LAUNCH(); }
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

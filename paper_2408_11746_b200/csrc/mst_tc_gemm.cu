@@ -892,8 +892,12 @@ extern "C" mst_status_t mst_device_error_flags(int32_t* flags) {
   MST_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_tc_error, sizeof(int)));
   int32_t att = 0;
   MST_TRY(mst_attention_error_flags(&att));
-  int32_t sp = 0;
+  int32_t sp = 0, cc = 0;
   MST_TRY(mst_sp24_error_flags(&sp));
-  *flags = v | (att << 1) | (sp << 2);
+  MST_TRY(mst_spmm_error_flags(&cc));
+  int32_t sd = 0;
+  MST_TRY(mst_sddmm_error_flags(&sd));
+  cc |= sd;
+  *flags = v | (att << 1) | (sp << 2) | (cc << 3);
   return MST_OK;
 }

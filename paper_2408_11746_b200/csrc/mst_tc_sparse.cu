@@ -10,8 +10,9 @@
 // ([rows x K/2] bf16, K-major) with its 2-bit position metadata in tensor memory; the activations are the B operand,
 // read as stored.  The accumulator therefore holds the TRANSPOSE of the output tile (lanes = rows of S = output
 // features, columns = tokens); the epilogue adds the spill entries of its row from a feature-major copy of the
-// activation columns they touch, and writes token-major rows through a transposing shared-memory box.  Every product
-// is an exact bf16 x bf16 product accumulated in fp32, as on the dense path.
+// activation columns they touch, and writes 64-byte runs of the token-major output rows (32 consecutive features of
+// one token per store instruction).  Every product is an exact bf16 x bf16 product accumulated in fp32, as on the
+// dense path.
 //
 // Kernel: clusters of two blocks (an SM pair) share a 256 (rows of S) x 240 (tokens) tile with
 // tcgen05.mma.sp.cta_group::2.  Per 128-deep K block a block loads its 128 compressed rows (16 KB), its 120 tokens of
@@ -39,23 +40,42 @@ constexpr int SKB = 128;               // logical K per stage (64 compressed ele
 constexpr int S_STAGES = 4;
 constexpr int SA_BYTES = SM_ROWS * (SKB / 2) * 2;       // 16 KiB
 constexpr int SB_BOX_BYTES = (SN / 2) * 64 * 2;         // 15 KiB: 120 tokens x 64 k
-constexpr int SB_BOX_STRIDE = 16384;                    // boxes start on 1024-byte boundaries
+constexpr int SB_BOX_STRIDE = SB_BOX_BYTES;             // 15 KiB: still a multiple of 1024 bytes (swizzle atoms)
 constexpr int SE_BYTES = 128 * 16;                      // metadata of 128 rows x 128 k
-constexpr int S_STAGE_BYTES = SA_BYTES + 2 * SB_BOX_STRIDE + SE_BYTES;   // 50 KiB
+constexpr int S_STAGE_BYTES = SA_BYTES + 2 * SB_BOX_STRIDE + SE_BYTES;   // 48 KiB
 constexpr int S_TX_BYTES = SA_BYTES + 2 * SB_BOX_BYTES + SE_BYTES;
 constexpr int S_EPI_WARPS = 8;
 constexpr int S_THREADS = 64 + 32 * S_EPI_WARPS;
 constexpr int S_CHUNK = 16;                             // tokens per epilogue step
-constexpr int S_OUT_BOX_BYTES = S_CHUNK * 32 * 2;       // 16 tokens x 32 features, bf16
+constexpr int S_FAST_SPILLS = 4;                        // spills per row whose activations are fetched one step ahead
 constexpr int S_TMEM_COLS = 512;
 constexpr int S_META_COL = 2 * SN;                      // metadata slots behind the two accumulators
-constexpr size_t S_SMEM_BYTES = (size_t)S_STAGES * S_STAGE_BYTES + S_EPI_WARPS * S_OUT_BOX_BYTES + 1024 + 256;
+constexpr size_t S_SMEM_BYTES = (size_t)S_STAGES * S_STAGE_BYTES + 1024 + 256;
 constexpr int XR_TOK = 64;                              // token tile of the feature-major column copy
 
 __device__ int g_sp_error = 0;  // sticky: 1 = a bounded wait expired
 
+// Cycle accounting of the roles (compiled in with -DMST_SP_PROFILE, off by default; no effect on results): per block
+//   [0] producer waiting for a free stage   [1] MMA thread waiting for a full stage   [2] MMA thread waiting for a free
+//   accumulator   [3] epilogue warp 2 waiting for a complete accumulator   [4] epilogue warp 2 working
+//   [5] whole kernel
+#ifdef MST_SP_PROFILE
+__device__ long long g_sp_prof[160][8];
+#define SP_PROF_DECL long long prof_t0 = 0, prof_acc0 = 0, prof_acc1 = 0
+#define SP_PROF_BEGIN() prof_t0 = clock64()
+#define SP_PROF_END(acc) acc += clock64() - prof_t0
+#define SP_PROF_STORE(slot, acc) g_sp_prof[blockIdx.x][slot] = acc
+#else
+#define SP_PROF_DECL
+#define SP_PROF_BEGIN()
+#define SP_PROF_END(acc)
+#define SP_PROF_STORE(slot, acc)
+#endif
+
 struct SpParams {
   int64_t R, T;           // rows of S (output features of the product), tokens
+  uint16_t* out;          // [T x ldout] bf16
+  int64_t ldout;
   int kblocks;            // kd_pad / 128
   int m_tiles, n_tiles;   // 256-row tiles of S, 240-token tiles
   int chunks;             // 16-k chunks per row of S
@@ -110,12 +130,11 @@ __device__ __forceinline__ void sp_tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) 
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(S_THREADS, 1)
 tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const __grid_constant__ CUtensorMap tmE, const __grid_constant__ CUtensorMap tmC, const SpParams P) {
+                    const __grid_constant__ CUtensorMap tmE, const SpParams P) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
-  const uint32_t out_base = tiles_base + S_STAGES * S_STAGE_BYTES;
-  const uint32_t bar_base = out_base + S_EPI_WARPS * S_OUT_BOX_BYTES;
+  const uint32_t bar_base = tiles_base + S_STAGES * S_STAGE_BYTES;
   const uint32_t full0 = bar_base, empty0 = bar_base + 8 * S_STAGES, tfull0 = bar_base + 16 * S_STAGES, tempty0 = tfull0 + 16;
   __shared__ uint32_t tmem_base_holder;
   __shared__ int abort_sh;
@@ -148,6 +167,9 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t tmem_base = tmem_base_holder;
   mst_grid_launch_dependents();
   mst_grid_dependency_wait();
+#ifdef MST_SP_PROFILE
+  const long long prof_kernel_t0 = clock64();
+#endif
 
   // work item w: token tile w / m_tiles, row tile w % m_tiles.  Pairs that run at the same time share their token
   // tile (the activations stream through L2 once) and sweep the compressed operand, which stays L2-resident.
@@ -159,23 +181,27 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
+      SP_PROF_DECL;
       for (int64_t w = pair; w < works && !*abort_flag; w += npairs) {
         const int mt = (int)(w % P.m_tiles), nt = (int)(w / P.m_tiles);
         const int row0 = mt * (2 * SM_ROWS) + (int)rank * SM_ROWS;      // this block's rows of S
         const int tok0 = nt * SN + (int)rank * (SN / 2);                // this block's half of the tokens
         const int mt128 = mt * 2 + (int)rank;                           // 128-row tile index for the metadata
         for (int kb = 0; kb < P.kblocks; ++kb) {
+          SP_PROF_BEGIN();
           if (!sp_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
+          SP_PROF_END(prof_acc0);
           const uint32_t fb = sp_in_even_block(full0 + 8 * s);
           const uint32_t sa = tiles_base + s * S_STAGE_BYTES, sb = sa + SA_BYTES, se = sb + 2 * SB_BOX_STRIDE;
           asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(fb), "r"(S_TX_BYTES) : "memory");
           sp_tma_load_2d_pair(sa, &tmA, kb * (SKB / 2), row0, fb);
           sp_tma_load_2d_pair(sb, &tmB, kb * SKB, tok0, fb);
           sp_tma_load_2d_pair(sb + SB_BOX_STRIDE, &tmB, kb * SKB + 64, tok0, fb);
-          sp_tma_load_2d_pair(se, &tmE, 0, (mt128 * P.kblocks + kb) * 128, fb);
+          sp_tma_load_2d_pair(se, &tmE, 0, (mt128 * P.kblocks + kb) * 2, fb);   // two 1 KiB rows = the block's 2 KiB
           if (++s == S_STAGES) { s = 0; ph ^= 1u; }
         }
       }
+      SP_PROF_STORE(0, prof_acc0);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (even block only)
@@ -188,13 +214,18 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint64_t edesc0 = sp_desc_plain(tiles_base + SA_BYTES + 2 * SB_BOX_STRIDE, 128, 128);
       int s = 0, acc = 0, eslot = 0;
       uint32_t ph = 0, acc_ph = 0;
+      SP_PROF_DECL;
       for (int64_t w = pair; w < works && !*abort_flag; w += npairs) {
+        SP_PROF_BEGIN();
         if (!sp_wait(tempty0 + 8 * acc, acc_ph ^ 1u, abort_flag)) break;
+        SP_PROF_END(prof_acc1);
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * SN);
         bool ok = true;
         for (int kb = 0; kb < P.kblocks; ++kb) {
+          SP_PROF_BEGIN();
           if (!sp_wait(full0 + 8 * s, ph, abort_flag)) { ok = false; break; }
+          SP_PROF_END(prof_acc0);
           tc_fence_after();
           const uint64_t soff = (uint64_t)(uint32_t)(s * (S_STAGE_BYTES >> 4));
           const uint32_t e_tmem = tmem_base + (uint32_t)(S_META_COL + 4 * eslot);
@@ -228,14 +259,20 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                      : "memory");
         if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
       }
+      SP_PROF_STORE(1, prof_acc0);
+      SP_PROF_STORE(2, prof_acc1);
     }
   } else {
     // ------------------------------------------------------------------ epilogue (both blocks, own 128 rows of S)
+    // A thread owns one output feature (tensor-memory lane) and reads 16 tokens of it at a time.  For a fixed token the
+    // 32 lanes of a warp hold 32 consecutive features, so each store instruction writes one 64-byte run of an output
+    // row: no staging through shared memory.  The activations of the row's first spills are fetched one step ahead
+    // (they come from L2: the latency would otherwise be paid once per step).
     const int q = warp & 3;                 // tensor-memory lane quarter
     const int c0 = (warp - 2) >> 2;         // the two warps of a quarter take alternate 16-token chunks
-    const uint32_t stage = out_base + (uint32_t)(warp - 2) * S_OUT_BOX_BYTES;
     int acc = 0;
     uint32_t acc_ph = 0;
+    SP_PROF_DECL;
     for (int64_t w = pair; w < works; w += npairs) {
       const int mt = (int)(w % P.m_tiles), nt = (int)(w / P.m_tiles);
       const int64_t row0 = (int64_t)mt * (2 * SM_ROWS) + (int)rank * SM_ROWS + q * 32;
@@ -243,49 +280,82 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int64_t tok0 = (int64_t)nt * SN;
       // third and fourth entries of this row's groups (rows beyond R have none: their counts are zero)
       const int32_t sp0 = P.scan[r * P.chunks], sp1 = P.scan[(r + 1) * P.chunks];
+      const int n_fast = min(sp1 - sp0, S_FAST_SPILLS);
+      const int n_fast_warp = __reduce_max_sync(0xffffffffu, n_fast);
+      float wv[S_FAST_SPILLS];
+      const uint16_t* xrow[S_FAST_SPILLS];
+#pragma unroll
+      for (int j = 0; j < S_FAST_SPILLS; ++j) {
+        const uint32_t ent = j < n_fast ? __ldg(P.spill + sp0 + j) : 0u;
+        wv[j] = __uint_as_float(ent << 16);
+        xrow[j] = P.xr + (int64_t)(ent >> 16) * P.ldxr;
+      }
+      uint4 xn[S_FAST_SPILLS][2];           // activations of the fast spills for the next chunk
+      auto fetch = [&](int c) {
+        const int64_t t0 = tok0 + c * S_CHUNK;
+#pragma unroll
+        for (int j = 0; j < S_FAST_SPILLS; ++j) {
+          xn[j][0] = xn[j][1] = make_uint4(0, 0, 0, 0);
+          if (j < n_fast && c < SN / S_CHUNK && t0 < P.T) {
+            const uint4* src = reinterpret_cast<const uint4*>(xrow[j] + t0);
+            xn[j][0] = __ldg(src);
+            xn[j][1] = __ldg(src + 1);
+          }
+        }
+      };
+      if (n_fast_warp > 0) fetch(c0);
+      SP_PROF_BEGIN();
       if (!sp_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
+      SP_PROF_END(prof_acc0);
       tc_fence_after();
+      SP_PROF_BEGIN();
 #pragma unroll 1
       for (int c = c0; c < SN / S_CHUNK; c += 2) {
         const int64_t t0 = tok0 + c * S_CHUNK;
         if (t0 >= P.T) break;  // uniform
         uint32_t v[16];
+        uint4 xc[S_FAST_SPILLS][2];
+#pragma unroll
+        for (int j = 0; j < S_FAST_SPILLS; ++j) { xc[j][0] = xn[j][0]; xc[j][1] = xn[j][1]; }
+        if (n_fast_warp > 0) fetch(c + 2);
         sp_tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * SN + c * S_CHUNK), v);
-        // each spill multiplies 16 consecutive tokens of one activation column
-        for (int32_t e = sp0; e < sp1; ++e) {
-          const uint32_t ent = __ldg(P.spill + e);
-          const float wv = __uint_as_float(ent << 16);
-          const uint4* src = reinterpret_cast<const uint4*>(P.xr + (int64_t)(ent >> 16) * P.ldxr + t0);
-          const uint4 x0 = __ldg(src), x1 = __ldg(src + 1);
+        auto add_spill = [&](float wj, const uint4& x0, const uint4& x1) {
           const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            v[2 * j] = __float_as_uint(fmaf(wv, __uint_as_float(xw[j] << 16), __uint_as_float(v[2 * j])));
-            v[2 * j + 1] = __float_as_uint(fmaf(wv, __uint_as_float(xw[j] & 0xFFFF0000u), __uint_as_float(v[2 * j + 1])));
+          for (int i = 0; i < 8; ++i) {
+            v[2 * i] = __float_as_uint(fmaf(wj, __uint_as_float(xw[i] << 16), __uint_as_float(v[2 * i])));
+            v[2 * i + 1] = __float_as_uint(fmaf(wj, __uint_as_float(xw[i] & 0xFFFF0000u), __uint_as_float(v[2 * i + 1])));
           }
-        }
-        if (lane == 0) bulk_wait_read();  // the box's previous contents have left shared memory
-        __syncwarp();
-        // transposing box: row j = token t0 + j, 32 features (64 bytes) per row, this thread's feature at column `lane`
+        };
 #pragma unroll
-        for (int j = 0; j < 16; j += 2) {
-          const uint32_t pk = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-          asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage + (uint32_t)(j * 64 + lane * 2)), "h"((uint16_t)(pk & 0xFFFFu)) : "memory");
-          asm volatile("st.shared.u16 [%0], %1;" ::"r"(stage + (uint32_t)((j + 1) * 64 + lane * 2)), "h"((uint16_t)(pk >> 16)) : "memory");
+        for (int j = 0; j < S_FAST_SPILLS; ++j)
+          if (j < n_fast) add_spill(wv[j], xc[j][0], xc[j][1]);
+        // rows with more spills than the prefetch holds: one at a time
+        for (int32_t e = sp0 + S_FAST_SPILLS; e < sp1; ++e) {
+          const uint32_t ent = __ldg(P.spill + e);
+          const uint4* src = reinterpret_cast<const uint4*>(P.xr + (int64_t)(ent >> 16) * P.ldxr + t0);
+          add_spill(__uint_as_float(ent << 16), __ldg(src), __ldg(src + 1));
         }
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0 && row0 < P.R) {
-          tma_store_2d(&tmC, stage, (int)row0, (int)t0);
-          bulk_commit();
+        if (r < P.R) {
+          uint16_t* dst = P.out + t0 * P.ldout + r;
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const uint32_t pk = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+            if (t0 + j < P.T) dst[(int64_t)j * P.ldout] = (uint16_t)(pk & 0xFFFFu);
+            if (t0 + j + 1 < P.T) dst[(int64_t)(j + 1) * P.ldout] = (uint16_t)(pk >> 16);
+          }
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(sp_in_even_block(tempty0 + 8 * acc)) : "memory");
+      SP_PROF_END(prof_acc1);
       if (++acc == 2) { acc = 0; acc_ph ^= 1u; }
     }
-    if (lane == 0) bulk_wait_all();
+    if (warp == 2 && lane == 0) {
+      SP_PROF_STORE(3, prof_acc0);
+      SP_PROF_STORE(4, prof_acc1);
+    }
   }
 
   // ------------------------------------------------------------------ teardown
@@ -294,6 +364,9 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
   tc_fence_before();
   __syncthreads();
+#ifdef MST_SP_PROFILE
+  if (threadIdx.x == 0) g_sp_prof[blockIdx.x][5] = clock64() - prof_kernel_t0;
+#endif
   sp_cluster_sync();
   if (warp == 1) {
     tc_fence_after();
@@ -465,7 +538,7 @@ __global__ void sp24_slot_cols_kernel(const int32_t* __restrict__ col_flag, cons
 // Feature-major copy of the activation columns that spills multiply: xr[slot][t] = in[t][slot_col[slot]], zero for
 // t >= T.  A block moves 32 columns x 64 tokens through shared memory: reads walk along the token rows (consecutive
 // slots are ascending, mostly adjacent columns), writes are 128-byte rows.  Blocks beyond the number of such columns
-// leave at once.
+// do nothing.
 __global__ void __launch_bounds__(256) sp24_gather_cols_kernel(const uint16_t* __restrict__ in, int64_t ldin, int64_t T,
                                                               const int32_t* __restrict__ slot_col,
                                                               const int32_t* __restrict__ n_cols_ptr,
@@ -474,26 +547,30 @@ __global__ void __launch_bounds__(256) sp24_gather_cols_kernel(const uint16_t* _
   mst_grid_dependency_wait();
   __shared__ uint16_t tile[32][XR_TOK + 2];
   const int n_cols = *n_cols_ptr;
-  const int slot0 = blockIdx.x * 32;
-  if (slot0 >= n_cols) return;
-  const int64_t t0 = (int64_t)blockIdx.y * XR_TOK;
+  const int64_t tok_tiles = ldxr / XR_TOK;
+  const int64_t items = (int64_t)((n_cols + 31) / 32) * tok_tiles;   // the grid is sized for the layer, not for n_cols
   const int x = threadIdx.x & 31, y = threadIdx.x >> 5;
-  const int slot = slot0 + x;
-  const int k = slot < n_cols ? slot_col[slot] : -1;
+  for (int64_t it = blockIdx.x; it < items; it += gridDim.x) {
+    const int slot0 = (int)(it / tok_tiles) * 32;
+    const int64_t t0 = (it % tok_tiles) * XR_TOK;
+    const int slot = slot0 + x;
+    const int k = slot < n_cols ? slot_col[slot] : -1;
 #pragma unroll
-  for (int j = 0; j < XR_TOK / 8; ++j) {
-    const int tl = y * (XR_TOK / 8) + j;
-    const int64_t t = t0 + tl;
-    tile[x][tl] = (k >= 0 && t < T) ? in[t * ldin + k] : (uint16_t)0;
-  }
-  __syncthreads();
-  // warp y writes slots 4y .. 4y+3; eight lanes per slot, eight tokens (16 bytes) per lane
-  const int sl = y * 4 + (x >> 3), piece = x & 7;
-  if (slot0 + sl < n_cols) {
-    uint32_t w[4];
+    for (int j = 0; j < XR_TOK / 8; ++j) {
+      const int tl = y * (XR_TOK / 8) + j;
+      const int64_t t = t0 + tl;
+      tile[x][tl] = (k >= 0 && t < T) ? in[t * ldin + k] : (uint16_t)0;
+    }
+    __syncthreads();
+    // warp y writes slots 4y .. 4y+3; eight lanes per slot, eight tokens (16 bytes) per lane
+    const int sl = y * 4 + (x >> 3), piece = x & 7;
+    if (slot0 + sl < n_cols) {
+      uint32_t w[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) w[j] = (uint32_t)tile[sl][piece * 8 + 2 * j] | ((uint32_t)tile[sl][piece * 8 + 2 * j + 1] << 16);
-    *reinterpret_cast<uint4*>(xr + (int64_t)(slot0 + sl) * ldxr + t0 + piece * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int j = 0; j < 4; ++j) w[j] = (uint32_t)tile[sl][piece * 8 + 2 * j] | ((uint32_t)tile[sl][piece * 8 + 2 * j + 1] << 16);
+      *reinterpret_cast<uint4*>(xr + (int64_t)(slot0 + sl) * ldxr + t0 + piece * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __syncthreads();
   }
 }
 
@@ -601,10 +678,14 @@ mst_status_t sp24_refresh(mst_layer* L, int dir, cudaStream_t s) {
     MST_TRY(dir == 0 ? sp24_launch_compress<0>(L, 0, s) : sp24_launch_compress<1>(L, 0, s));
     MST_TRY(mst_scan_i32(S.cnt, S.scan, S.r_pad * S.chunks, S.bsums, s));
     MST_TRY(mst_scan_i32(S.col_flag, S.col_slot, S.kd_pad, S.bsums, s));
-    sp24_slot_cols_kernel<<<(unsigned)((S.kd_pad + 255) / 256), 256, 0, s>>>(S.col_flag, S.col_slot, S.kd_pad, S.slot_col);
+    sp24_slot_cols_kernel<<<(unsigned)((S.kd_pad + 255) / 256), 256, 0, s>>>(S.col_flag, S.col_slot, S.kd_pad, S.slot_col); MST_COUNT_LAUNCH();
     MST_CUDA_TRY(cudaGetLastError());
     S.struct_version = L->version;
+    S.values_epoch = -1;
   }
+  // with value tracking the compressed operand is reused until the values change
+  if (L->track_values && S.values_epoch == L->values_epoch) return MST_OK;
+  S.values_epoch = L->values_epoch;
   return dir == 0 ? sp24_launch_compress<0>(L, 1, s) : sp24_launch_compress<1>(L, 1, s);
 }
 
@@ -634,22 +715,26 @@ mst_status_t mst_sp24_product(mst_layer* L, int dir, const void* in, int64_t ldi
   const int64_t ldxr = (T + XR_TOK - 1) / XR_TOK * XR_TOK;
   void* xr = nullptr;
   MST_TRY(mst_workspace_kind(MST_WS_COLUMNS, (size_t)S.kd_pad * ldxr * 2, &xr));
-  MST_CUDA_TRY(mst_launch_overlapped(sp24_gather_cols_kernel, dim3((unsigned)(S.kd_pad / 32), (unsigned)(ldxr / XR_TOK)),
-                                     dim3(256), 0, s, (const uint16_t*)in, ldin, T, (const int32_t*)S.slot_col,
+  const int64_t gather_items = (int64_t)(S.kd_pad / 32) * (ldxr / XR_TOK);
+  const int64_t gather_grid = gather_items < (int64_t)sp_sm_count() * 8 ? gather_items : (int64_t)sp_sm_count() * 8;
+  MST_CUDA_TRY(mst_launch_overlapped(sp24_gather_cols_kernel, dim3((unsigned)gather_grid), dim3(256), 0, s, (const uint16_t*)in, ldin, T, (const int32_t*)S.slot_col,
                                      (const int32_t*)(S.col_slot + S.kd_pad), (uint16_t*)xr, ldxr));
   MST_CUDA_TRY(cudaGetLastError());
 
-  CUtensorMap tmA, tmB, tmE, tmC;
+  CUtensorMap tmA, tmB, tmE;
   const bool ok = sp_map_2d(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, S.ac, S.r_pad, S.kd_pad / 2, S.kd_pad / 2, 64, SM_ROWS,
                             CU_TENSOR_MAP_SWIZZLE_128B) &&
                   sp_map_2d(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, in, T, S.Kd, ldin, 64, SN / 2, CU_TENSOR_MAP_SWIZZLE_128B) &&
-                  sp_map_2d(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, S.meta, (int64_t)(S.r_pad / 128) * S.kblocks * 128, 4, 4, 4,
-                            128, CU_TENSOR_MAP_SWIZZLE_NONE) &&
-                  sp_map_2d(&tmC, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, out, T, S.R, ldout, 32, S_CHUNK, CU_TENSOR_MAP_SWIZZLE_NONE);
+                  // metadata blocks are contiguous 2 KiB pieces: described as rows of 256 words so that a block is
+                  // fetched as sixteen full lines (a box of 128 rows x 16 bytes would be 128 separate requests)
+                  sp_map_2d(&tmE, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, S.meta, (int64_t)(S.r_pad / 128) * S.kblocks * 2, 256, 256, 256,
+                            2, CU_TENSOR_MAP_SWIZZLE_NONE);
   if (!ok) return MST_ERR_SHAPE;
   SpParams P = {};
   P.R = S.R;
   P.T = T;
+  P.out = (uint16_t*)out;
+  P.ldout = ldout;
   P.kblocks = S.kblocks;
   P.m_tiles = (int)(S.r_pad / (2 * SM_ROWS));
   P.n_tiles = (int)((T + SN - 1) / SN);
@@ -662,10 +747,20 @@ mst_status_t mst_sp24_product(mst_layer* L, int dir, const void* in, int64_t ldi
   const int64_t works = (int64_t)P.m_tiles * P.n_tiles;
   const int64_t max_pairs = sp_sm_count() / 2;
   const int grid = 2 * (int)(works < max_pairs ? works : max_pairs);
-  MST_CUDA_TRY(mst_launch_overlapped(tc_sp24_pair_kernel, dim3(grid), dim3(S_THREADS), S_SMEM_BYTES, s, tmA, tmB, tmE, tmC, P));
+  MST_CUDA_TRY(mst_launch_overlapped(tc_sp24_pair_kernel, dim3(grid), dim3(S_THREADS), S_SMEM_BYTES, s, tmA, tmB, tmE, P));
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
+
+#ifdef MST_SP_PROFILE
+// cycle counters of the last launch: out[block][8], `blocks` rows (profiling builds only)
+extern "C" mst_status_t mst_sp24_profile(long long* out, int blocks) {
+  if (!out || blocks < 0 || blocks > 160) return MST_ERR_INVALID_ARG;
+  MST_CUDA_TRY(cudaDeviceSynchronize());
+  MST_CUDA_TRY(cudaMemcpyFromSymbol(out, g_sp_prof, sizeof(long long) * 8 * (size_t)blocks));
+  return MST_OK;
+}
+#endif
 
 mst_status_t mst_sp24_error_flags(int32_t* flags) {
   int v = 0;

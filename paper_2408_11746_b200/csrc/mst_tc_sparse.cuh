@@ -30,6 +30,7 @@ struct mst_sp24 {
   int kd_pad = 0, kblocks = 0, chunks = 0;
   int64_t spill_cap = 0;
   int64_t struct_version = -1;    // layer structure version the spill positions belong to
+  int64_t values_epoch = -1;      // values epoch the compressed operand was built from (value tracking only)
 };
 
 // true when the operands can be described to the TMA unit and the layer's nnz fits the spill capacity

@@ -301,15 +301,15 @@ mst_status_t run_select(mst_layer* L, const SelParams& P, int64_t k, uint32_t* o
     return MST_OK;
   }
   constexpr int passes = num_passes(KeyBits<MODE>::value);
-  select_init<<<1, 256, 0, s>>>(L->sel, (long long)k, L->hist, L->counter);
+  select_init<<<1, 256, 0, s>>>(L->sel, (long long)k, L->hist, L->counter); MST_COUNT_LAUNCH();
   int64_t blocks = (L->nwords * 32 + HIST_THREADS - 1) / HIST_THREADS;
   if (blocks > 2 * 148) blocks = 2 * 148;  // all SMs fully occupied; each block ends with one global add per non-empty bin
   for (int p = 0; p < passes; ++p)
-    select_hist<MODE><<<(unsigned)blocks, HIST_THREADS, 0, s>>>(P, p, L->sel, L->hist, L->counter, L->flags);
+    { select_hist<MODE><<<(unsigned)blocks, HIST_THREADS, 0, s>>>(P, p, L->sel, L->hist, L->counter, L->flags); MST_COUNT_LAUNCH(); }
   const unsigned wgrid = (unsigned)((L->nwords * 32 + 255) / 256);
-  select_count_equal<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_cnt);
+  select_count_equal<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_cnt); MST_COUNT_LAUNCH();
   MST_TRY(mst_scan_i32_if(L->word_cnt, L->word_scan, L->nwords, L->block_sums, &L->sel->need_rank, s));
-  select_mark<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_scan, out_bits);
+  select_mark<MODE><<<wgrid, 256, 0, s>>>(P, L->sel, L->word_scan, out_bits); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
@@ -881,6 +881,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     cfg.attrs = attr;
     cfg.numAttrs = mst_pdl_enabled() ? 2 : 1;
     MST_CUDA_TRY(cudaLaunchKernelExC(&cfg, fn, args));
+    MST_COUNT_LAUNCH();
   } else {
     MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
     MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
@@ -891,7 +892,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   const int64_t nnz_before = L->nnz;
   if (stats) {
     // the fused kernel records the longest row itself only when it also builds the CSC view
-    if (!fused || !L->csc_valid) max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags);
+    if (!fused || !L->csc_valid) { max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags); MST_COUNT_LAUNCH(); }
     int32_t f[4] = {0, 0, 0, 0};
     int32_t total = 0;
     MST_CUDA_TRY(cudaMemcpyAsync(f, L->flags, sizeof(f), cudaMemcpyDeviceToHost, s));

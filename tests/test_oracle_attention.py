@@ -88,3 +88,85 @@ def test_matches_position_by_position_loop(n, stride):
     if n > stride > 1:
         band = np.tril(np.ones((n, n), bool)) & ~np.tril(np.ones((n, n), bool), -stride)
         assert (att.strided_mask(n, stride) != band).any()
+
+
+# ------------------------------------------------------------------ backward pass
+def _rand_qkv(B, H, n, d, seed):
+    rng = np.random.default_rng(seed)
+    return tuple(rng.normal(size=(B, H, n, d)) for _ in range(4))      # Q, K, V, dO
+
+
+@pytest.mark.parametrize("n,stride", [(7, 3), (12, 4), (9, 16)])
+def test_backward_matches_central_differences(n, stride):
+    Q, K, V, dO = _rand_qkv(1, 2, n, 5, 100 + n)
+    dQ, dK, dV = att.strided_attention_bwd(Q, K, V, dO, stride)
+
+    def loss(q, k, v):
+        return float((att.strided_attention(q, k, v, stride)[0] * dO).sum())
+    h = 1e-6
+    rng = np.random.default_rng(5)
+    for name, X, dX in (("q", Q, dQ), ("k", K, dK), ("v", V, dV)):
+        for _ in range(25):
+            idx = tuple(rng.integers(0, s) for s in X.shape)
+            Xp, Xm = X.copy(), X.copy()
+            Xp[idx] += h
+            Xm[idx] -= h
+            args_p = [Q, K, V]; args_m = [Q, K, V]
+            j = "qkv".index(name)
+            args_p[j], args_m[j] = Xp, Xm
+            num = (loss(*args_p) - loss(*args_m)) / (2 * h)
+            assert abs(num - dX[idx]) <= 1e-6 * max(1.0, abs(num)), (name, idx)
+
+
+def test_backward_directional_identity():
+    # first-order change of <dO, Out> along a random direction equals the inner products with the gradients
+    Q, K, V, dO = _rand_qkv(2, 3, 20, 8, 7)
+    dq, dk, dv, _ = _rand_qkv(2, 3, 20, 8, 8)
+    dQ, dK, dV = att.strided_attention_bwd(Q, K, V, dO, 6)
+    eps = 1e-6
+    f = lambda t: float((att.strided_attention(Q + t * dq, K + t * dk, V + t * dv, 6)[0] * dO).sum())
+    num = (f(eps) - f(-eps)) / (2 * eps)
+    ana = float((dQ * dq).sum() + (dK * dk).sum() + (dV * dv).sum())
+    assert abs(num - ana) <= 1e-6 * max(1.0, abs(ana))
+
+
+def test_backward_position_by_position_loop():
+    # the same derivative written without matrices: one query position at a time, explicit key sets
+    Q, K, V, dO = _rand_qkv(1, 1, 11, 4, 3)
+    stride = 4
+    n, d = 11, 4
+    dQ = np.zeros((n, d)); dK = np.zeros((n, d)); dV = np.zeros((n, d))
+    for i in range(n):
+        js = [j for j in range(i + 1) if i - j < stride or (i - j) % stride == 0]
+        s = np.array([Q[0, 0, i] @ K[0, 0, j] for j in js]) / np.sqrt(d)
+        p = np.exp(s - s.max()); p /= p.sum()
+        dp = np.array([dO[0, 0, i] @ V[0, 0, j] for j in js])
+        ds = p * (dp - (p * dp).sum())
+        for a, j in enumerate(js):
+            dV[j] += p[a] * dO[0, 0, i]
+            dQ[i] += ds[a] * K[0, 0, j] / np.sqrt(d)
+            dK[j] += ds[a] * Q[0, 0, i] / np.sqrt(d)
+    g = att.strided_attention_bwd(Q, K, V, dO, stride)
+    np.testing.assert_allclose(g[0][0, 0], dQ, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(g[1][0, 0], dK, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(g[2][0, 0], dV, rtol=1e-12, atol=1e-12)
+
+
+def test_backward_invariants():
+    Q, K, V, dO = _rand_qkv(1, 2, 16, 4, 11)
+    dQ, dK, dV = att.strided_attention_bwd(Q, K, V, dO, 5)
+    # every row of P sums to one: the gradients of all values add up to the sum of the upstream gradients
+    np.testing.assert_allclose(dV.sum(axis=-2), dO.sum(axis=-2), rtol=1e-12, atol=1e-12)
+    # the first position attends only to itself: its softmax is constant, so its query gets no gradient
+    np.testing.assert_allclose(dQ[..., 0, :], 0.0, atol=1e-15)
+    # the last key is seen by the last query only
+    np.testing.assert_allclose(dV[..., -1, :], dO[..., -1, :] * _p_last(Q, K, 5), rtol=1e-12)
+
+
+def _p_last(Q, K, stride):
+    n, d = Q.shape[-2], Q.shape[-1]
+    i = n - 1
+    js = [j for j in range(n) if i - j < stride or (i - j) % stride == 0]
+    s = np.einsum("bhd,bhjd->bhj", Q[..., i, :], K[..., js, :]) / np.sqrt(d)
+    p = np.exp(s - s.max(-1, keepdims=True)); p /= p.sum(-1, keepdims=True)
+    return p[..., -1:]          # weight of key n-1 in row n-1
