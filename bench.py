@@ -194,6 +194,11 @@ def run_attention(args) -> None:
     for stride in (256, 128):
         t = timed(lambda: mst.mst_strided_attention_fwd(base, base + 2 * C, base + 4 * C, 3 * C, B, n, H, d, stride, out,
                                                         C, lse))
+        dO = torch.randn((B * n, C), device=dev, dtype=torch.float32).to(torch.bfloat16)
+        dqkv = torch.empty_like(qkv)
+        gb = dqkv.data_ptr()
+        t_bwd = timed(lambda: mst.mst_strided_attention_bwd(base, base + 2 * C, base + 4 * C, 3 * C, out, C, dO, C, lse, B, n,
+                                                            H, d, stride, gb, gb + 2 * C, gb + 4 * C, 3 * C))
         kept = sum(min(i, stride - 1) + 1 + i // stride for i in range(n))        # |S_i| summed over positions
         useful = 4.0 * d * kept * B * H                                            # scores + weighted sum, kept pairs
         executed = 4.0 * d * n * (stride + 128) * B * H                            # the two tile products as issued
@@ -204,6 +209,7 @@ def run_attention(args) -> None:
             "kept_fraction": kept / float(n * n),
             "roofline": {"bound": "hbm", "achieved": bytes_alg / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": bytes_alg / t / 1e9 / peaks["hbm_gbs"]},
+            "backward_us": t_bwd * 1e6, "backward_useful_tflops": 2.5 * useful / t_bwd / 1e12,
             "torch_dense_causal_us": t_dense * 1e6}))
     assert mst.mst_device_error_flags() == 0
 

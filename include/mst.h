@@ -184,6 +184,21 @@ mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, const void*
                                        int32_t seq_len, int32_t heads, int32_t head_dim, int32_t stride, void* Out,
                                        int64_t ldo, float* lse, mst_stream_t stream);
 
+/* Backward of mst_strided_attention_fwd (same passage; the derivative of the definition above):
+ *   delta_i = dOut_i . Out_i,  P_ij = exp(q_i . k_j / sqrt(d) - lse_i),  dS_ij = P_ij (dOut_i . v_j - delta_i),
+ *   dV_j = sum_i P_ij dOut_i,  dK_j = sum_i dS_ij q_i / sqrt(d),  dQ_i = sum_j dS_ij k_j / sqrt(d)   (sums over the pairs
+ *   with j in S_i).
+ * Q, K, V, ld as in the forward call; Out [batch*seq_len x ldo] the forward output, dOut [batch*seq_len x lddo] the
+ * upstream gradient, lse [batch, heads, seq_len] the forward's log-sum-exp (all device, bf16 except lse).
+ * dQ, dK, dV: device bf16, ldg elements between tokens, head h in columns h*head_dim .. (three column slices of one
+ * fused gradient buffer may be passed).  Supported: head_dim = 64, seq_len and stride multiples of 64, leading
+ * dimensions multiples of 8, 16-byte aligned pointers; anything else MST_ERR_SHAPE.  Deterministic (no atomics).
+ * Keeps one float per (token, head) in a per-device scratch buffer: calls must not overlap on the GPU. */
+mst_status_t mst_strided_attention_bwd(const void* Q, const void* K, const void* V, int64_t ld, const void* Out,
+                                       int64_t ldo, const void* dOut, int64_t lddo, const float* lse, int32_t batch,
+                                       int32_t seq_len, int32_t heads, int32_t head_dim, int32_t stride, void* dQ,
+                                       void* dK, void* dV, int64_t ldg, mst_stream_t stream);
+
 /* Weight gradient on the mask only, dW[k] = sum_t dY[t,o_k] X[t,i_k] for the k-th active entry in CSR order
  * (same passage).  dW_vals device float [nnz].  May use the per-device split scratch (see the conventions above). */
 mst_status_t mst_sddmm_dw(const mst_layer_t* layer, const void* dY, int64_t lddy, const void* X, int64_t ldx, int64_t T,

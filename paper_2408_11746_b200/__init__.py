@@ -24,7 +24,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 5: "MST_ERR_INFEASIBLE", 6: "MST_ERR_NONFINITE", 7: "MST_ERR_CORRUPT", 8: "MST_ERR_CUDA",
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_path_in_use", "mst_launch_count", "mst_track_values", "mst_values_changed", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
-           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_strided_attention_fwd", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
+           "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_strided_attention_fwd", "mst_strided_attention_bwd", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
            "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
            "mst_status_string"]
@@ -81,6 +81,8 @@ _sig = {
     "mst_spmm_fwd_gelu": [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp],
     "mst_spmm_bwd_x_gelu": [_vp, _vp, _i64, _i64, _vp, _i64, _vp, _i64, _vp],
     "mst_strided_attention_fwd": [_vp, _vp, _vp, _i64, _i32, _i32, _i32, _i32, _i32, _vp, _i64, _vp, _vp],
+    "mst_strided_attention_bwd": [_vp, _vp, _vp, _i64, _vp, _i64, _vp, _i64, _vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp,
+                                  _i64, _vp],
     "mst_sddmm_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp],
     "mst_dense_grad": [_vp, _i64, _vp, _i64, _i64, _i32, _i32, ctypes.c_int, _vp, _vp],
     "mst_sddmm_from_dense": [_vp, _vp, _vp, _vp],
@@ -228,6 +230,13 @@ def mst_strided_attention_fwd(Q, K, V, ld: int, batch: int, seq_len: int, heads:
                               ldo: int, lse=None, stream=None) -> None:
     _check(_lib.mst_strided_attention_fwd(_ptr(Q), _ptr(K), _ptr(V), ld, batch, seq_len, heads, head_dim, stride,
                                           _ptr(Out), ldo, _ptr(lse), _stream(stream)), "mst_strided_attention_fwd")
+
+
+def mst_strided_attention_bwd(Q, K, V, ld: int, Out, ldo: int, dOut, lddo: int, lse, batch: int, seq_len: int, heads: int,
+                              head_dim: int, stride: int, dQ, dK, dV, ldg: int, stream=None) -> None:
+    _check(_lib.mst_strided_attention_bwd(_ptr(Q), _ptr(K), _ptr(V), ld, _ptr(Out), ldo, _ptr(dOut), lddo, _ptr(lse), batch,
+                                          seq_len, heads, head_dim, stride, _ptr(dQ), _ptr(dK), _ptr(dV), ldg,
+                                          _stream(stream)), "mst_strided_attention_bwd")
 
 
 def mst_sddmm_dw(layer: int, dY, lddy: int, X, ldx: int, T: int, dW_vals, stream=None) -> None:

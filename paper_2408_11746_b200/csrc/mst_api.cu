@@ -83,11 +83,6 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
     o_col[s] = cv.take(2 * (size_t)cap);
     o_vals[s] = cv.take(es * (size_t)cap);
   }
-  const size_t o_bitsT = cv.take(4 * (size_t)L->nwordsT);
-  const size_t o_wscanT = cv.take(4 * (size_t)(L->nwordsT + 1));
-  const size_t o_colptr = cv.take(4 * (size_t)(I + 1));
-  const size_t o_rowidx = cv.take(2 * (size_t)cap);
-  const size_t o_perm = cv.take(4 * (size_t)cap);
   const size_t o_pruned = cv.take(4 * (size_t)L->nwords);
   const size_t o_grad = cv.take(4 * (size_t)L->nwords);
   const size_t o_rand = cv.take(4 * (size_t)L->nwords);
@@ -98,7 +93,6 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   const size_t o_sel = cv.take(sizeof(mst_select_state));
   const size_t o_flags = cv.take(4 * 4);
   const size_t o_counter = cv.take(4);
-  const size_t o_dense = dtype == MST_BF16 ? cv.take(2 * (size_t)N) : 0;
 
   unsigned char* base = nullptr;
   if (cudaMalloc((void**)&base, cv.off) != cudaSuccess) {
@@ -117,11 +111,12 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
     L->col_idx[s] = (uint16_t*)(base + o_col[s]);
     L->vals[s] = (void*)(base + o_vals[s]);
   }
-  L->bitsT = (uint32_t*)(base + o_bitsT);
-  L->wscanT = (int32_t*)(base + o_wscanT);
-  L->col_ptr = (int32_t*)(base + o_colptr);
-  L->row_idx = (uint16_t*)(base + o_rowidx);
-  L->perm = (int32_t*)(base + o_perm);
+  L->csc_base = nullptr;
+  L->bitsT = nullptr;
+  L->wscanT = nullptr;
+  L->col_ptr = nullptr;
+  L->row_idx = nullptr;
+  L->perm = nullptr;
   L->pruned_bits = (uint32_t*)(base + o_pruned);
   L->grad_bits = (uint32_t*)(base + o_grad);
   L->rand_bits = (uint32_t*)(base + o_rand);
@@ -132,7 +127,7 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->sel = (mst_select_state*)(base + o_sel);
   L->flags = (int32_t*)(base + o_flags);
   L->counter = (unsigned int*)(base + o_counter);
-  L->dense_w = dtype == MST_BF16 ? (uint16_t*)(base + o_dense) : nullptr;
+  L->dense_w = nullptr;
   L->csc_valid = 0;
   L->path = MST_PATH_AUTO;
   L->stg_x = L->stg_dy = L->stg_y = L->stg_dx = nullptr;
@@ -140,6 +135,36 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->stg_tokens = 0;
   L->async_ready = 0;
   *out = L;
+  return MST_OK;
+}
+
+// The CSC view (column pointers, row indices, CSC->CSR permutation, transposed bit mask and its scan) and the dense
+// bf16 image live in allocations of their own, made when a call first needs them: a layer that stays on the tensor
+// path never allocates the view, a layer on the CUDA-core or structured-sparse path never allocates the image.
+mst_status_t mst_alloc_csc(mst_layer* L) {
+  if (L->csc_base) return MST_OK;
+  Carver cv;
+  const size_t o_bitsT = cv.take(4 * (size_t)L->nwordsT);
+  const size_t o_wscanT = cv.take(4 * (size_t)(L->nwordsT + 1));
+  const size_t o_colptr = cv.take(4 * (size_t)(L->I + 1));
+  const size_t o_rowidx = cv.take(2 * (size_t)L->cap);
+  const size_t o_perm = cv.take(4 * (size_t)L->cap);
+  unsigned char* base = nullptr;
+  MST_CUDA_TRY(cudaMalloc((void**)&base, cv.off));
+  L->csc_base = base;
+  L->bitsT = (uint32_t*)(base + o_bitsT);
+  L->wscanT = (int32_t*)(base + o_wscanT);
+  L->col_ptr = (int32_t*)(base + o_colptr);
+  L->row_idx = (uint16_t*)(base + o_rowidx);
+  L->perm = (int32_t*)(base + o_perm);
+  L->csc_valid = 0;
+  return MST_OK;
+}
+
+mst_status_t mst_alloc_dense(mst_layer* L) {
+  if (L->dense_w || L->dtype != MST_BF16) return MST_OK;
+  MST_CUDA_TRY(cudaMalloc((void**)&L->dense_w, 2 * (size_t)L->N));
+  L->dense_version = L->dense_epoch = -1;
   return MST_OK;
 }
 
@@ -156,7 +181,9 @@ extern "C" mst_status_t mst_layer_destroy(mst_layer_t* L) {
   }
   free_staging(L);
   mst_sp24_free(L);
-  cudaFree(L->bits[0]);  // base of the single allocation
+  cudaFree(L->csc_base);
+  cudaFree(L->dense_w);
+  cudaFree(L->bits[0]);  // base of the main allocation
   delete L;
   return MST_OK;
 }

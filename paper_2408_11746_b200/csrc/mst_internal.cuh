@@ -109,7 +109,9 @@ struct mst_layer {
 
   // CSC view of the live structure.  Built at pack; the fused update skips it for layers whose input gradient runs
   // on the tensor path (which reads the dense image, not the CSC view) and it is then rebuilt on first use.
+  // Allocated on first use (mst_alloc_csc): layers that never leave the tensor path never pay for it.
   mutable int csc_valid;
+  unsigned char* csc_base;  // the view's own allocation, nullptr until it is needed
   uint32_t* bitsT;       // [nwordsT]
   int32_t* wscanT;       // [nwordsT+1]
   int32_t* col_ptr;      // [I+1]
@@ -129,7 +131,7 @@ struct mst_layer {
   unsigned int* counter;  // [1] block-completion counter
 
   // dense bf16 image of W.M for the tensor-core path (bf16 layers only): [O x I]; the input gradient reads it as an
-  // MN-major operand, so no transposed copy is kept
+  // MN-major operand, so no transposed copy is kept.  Allocated on first use (mst_alloc_dense).
   uint16_t* dense_w;
   int path;  // mst_compute_path_t
   // 2:4 split of W.M (forward) and of its transpose (input gradient) for the structured-sparse tensor-core path;
@@ -155,10 +157,12 @@ int64_t mst_scan_block_sums_len(int64_t n);
 mst_status_t mst_scan_i32_if(const int32_t* in, int32_t* out, int64_t n, int32_t* block_sums, const int* enabled,
                              cudaStream_t s);
 mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, int64_t ldw, int old_set, cudaStream_t s);
+mst_status_t mst_alloc_csc(mst_layer* L);     // no-op when the view's arrays exist
+mst_status_t mst_alloc_dense(mst_layer* L);   // no-op when the dense image exists
 mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s);
 mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s);  // builds the CSC view if it is stale
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
-mst_status_t mst_densify(const mst_layer* L, cudaStream_t s);
+mst_status_t mst_densify(const mst_layer* L, cudaStream_t s, const uint16_t** image);
 bool mst_use_tensor_path(const mst_layer* L);
 bool mst_use_sparse_tc_path(const mst_layer* L);
 

@@ -5,7 +5,7 @@
 // with a fixed summation order: no floating-point atomics, run-to-run identical results.
 //
 // The activations are first copied feature-major once per call (inT[c][t], one coalesced transpose); after that a
-// nonzero costs one contiguous read of its column.  A block owns 256 tokens x 120 rows of the output.  A producer
+// nonzero costs one contiguous read of its column.  A block owns 256 tokens x 120 rows of the output (fewer rows per warp when the grid would not fill the GPU).  A producer
 // warp streams [column chunk x 256 tokens] tiles of inT into a ring of shared-memory stages with the TMA unit
 // (cp.async.bulk.tensor, this GPU's memory only, no multicast); 15 compute warps each own 8 rows and hold their
 // 8 x 256 partial sums in registers (lane = 8 consecutive tokens) across all chunks.  Per nonzero: one warp shuffle
@@ -25,10 +25,9 @@
 namespace {
 
 constexpr int TOK = 256;    // tokens per block (8 per lane)
-constexpr int PANEL = 120;  // rows per block
 constexpr int WARPS = 15;   // compute warps; one more warp produces (512 threads: 128 registers each)
-constexpr int RPW = PANEL / WARPS;
-constexpr int OS_LD = PANEL + 1;
+constexpr int MAX_RPW = 8;  // rows per warp: 8 (120-row panels) for large outputs, fewer when the grid would not fill the GPU
+constexpr int MAX_PANEL = WARPS * MAX_RPW;
 constexpr int STAGES = 3;
 constexpr int THREADS = (WARPS + 1) * 32;
 
@@ -142,13 +141,15 @@ __global__ void __launch_bounds__(256) transpose_in_kernel(const T* __restrict__
   }
 }
 
-template <typename T, bool PERM>
+template <typename T, bool PERM, int RPW>
 __global__ void __launch_bounds__(THREADS, 1)
 spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __restrict__ ptr,
                    const uint16_t* __restrict__ idx, const T* __restrict__ vals, const int32_t* __restrict__ perm,
                    T* __restrict__ out, int64_t ldout, int64_t T_total, int R_total, int C) {
   using namespace mst_ptx;
   constexpr int KC = Cfg<T>::KC;
+  constexpr int PANEL = WARPS * RPW;
+  constexpr int OS_LD = PANEL + 1;
   constexpr uint32_t STAGE_BYTES = (uint32_t)(KC * TOK * sizeof(T));
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -325,9 +326,22 @@ namespace {
 
 template <typename T>
 constexpr size_t spmm_smem() {
-  return (size_t)STAGES * Cfg<T>::KC * TOK * sizeof(T) + 128 > (size_t)TOK * OS_LD * 4 + 128
+  return (size_t)STAGES * Cfg<T>::KC * TOK * sizeof(T) + 128 > (size_t)TOK * (MAX_PANEL + 1) * 4 + 128
              ? (size_t)STAGES * Cfg<T>::KC * TOK * sizeof(T) + 128
-             : (size_t)TOK * OS_LD * 4 + 128;
+             : (size_t)TOK * (MAX_PANEL + 1) * 4 + 128;
+}
+
+template <typename T, bool PERM, int RPW>
+mst_status_t launch_rpw(const CUtensorMap& tm, const int32_t* ptr, const uint16_t* idx, const void* vals, const int32_t* perm,
+                        void* out, int64_t ldout, int64_t T_total, int R_total, int C, cudaStream_t s) {
+  constexpr int PANEL = WARPS * RPW;
+  const size_t smem = spmm_smem<T>();
+  // per call: the attribute belongs to the current device's copy of the kernel
+  MST_CUDA_TRY(cudaFuncSetAttribute(spmm_stream_kernel<T, PERM, RPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid((unsigned)((R_total + PANEL - 1) / PANEL), (unsigned)((T_total + TOK - 1) / TOK));
+  spmm_stream_kernel<T, PERM, RPW><<<grid, THREADS, smem, s>>>(tm, ptr, idx, (const T*)vals, perm, (T*)out, ldout, T_total, R_total, C); MST_COUNT_LAUNCH();
+  MST_CUDA_TRY(cudaGetLastError());
+  return MST_OK;
 }
 
 template <typename T, bool PERM>
@@ -341,13 +355,19 @@ mst_status_t launch(const int32_t* ptr, const uint16_t* idx, const void* vals, c
   MST_TRY(mst_feature_major_copy(in, ldin, T_total, C, dt, inT, ldt, s));
   CUtensorMap tm;
   if (!mst_feature_major_map(&tm, inT, T_total, C, ldt, dt, TOK, Cfg<T>::KC)) return MST_ERR_SHAPE;
-  const size_t smem = spmm_smem<T>();
-  // per call: the attribute belongs to the current device's copy of the kernel
-  MST_CUDA_TRY(cudaFuncSetAttribute(spmm_stream_kernel<T, PERM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  dim3 grid((unsigned)((R_total + PANEL - 1) / PANEL), (unsigned)((T_total + TOK - 1) / TOK));
-  spmm_stream_kernel<T, PERM><<<grid, THREADS, smem, s>>>(tm, ptr, idx, (const T*)vals, perm, (T*)out, ldout, T_total, R_total, C); MST_COUNT_LAUNCH();
-  MST_CUDA_TRY(cudaGetLastError());
-  return MST_OK;
+  // rows per warp: the largest panel that still gives every SM a block (small token counts, narrow outputs)
+  const int64_t ttiles = (T_total + TOK - 1) / TOK;
+  int sms = 148;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+  }
+  auto blocks = [&](int rpw) { return ((int64_t)R_total + WARPS * rpw - 1) / (WARPS * rpw) * ttiles; };
+  if (blocks(8) >= 2 * sms) return launch_rpw<T, PERM, 8>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
+  if (blocks(4) >= 2 * sms) return launch_rpw<T, PERM, 4>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
+  if (blocks(2) >= sms) return launch_rpw<T, PERM, 2>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
+  return launch_rpw<T, PERM, 1>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
 }
 
 // Element-wise pass behind the CUDA-core product (the tensor path fuses it into its epilogue instead).
@@ -425,9 +445,10 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
   if (act == MST_ACT_NONE && mst_use_sparse_tc_path(L) && mst_sp24_usable(L, transpose ? 1 : 0, in, ldin, out, ldout))
     return mst_sp24_product(const_cast<mst_layer*>(L), transpose ? 1 : 0, in, ldin, T, out, ldout, s);
   if (mst_use_tensor_path(L) && (ldout % 8 == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0)) {
-    const uint16_t* image = L->dense_w;
-    if (mst_tc_gemm_usable(in, ldin, image, L->I)) {
-      MST_TRY(mst_densify(L, s));
+    // the image is 256-byte aligned by construction: only the activations and the row length decide
+    if (mst_tc_gemm_usable(in, ldin, in, L->I)) {
+      const uint16_t* image = nullptr;
+      MST_TRY(mst_densify(L, s, &image));
       mst_tc_gemm_args a = {};
       a.A = in; a.lda = ldin; a.a_mn_major = 0;
       a.B = image; a.ldb = L->I; a.b_mn_major = transpose ? 1 : 0;

@@ -6,6 +6,7 @@
 // The same holds for the CSC view on the transposed bit mask.  Everything below is integer work,
 // stream-ordered, with no inter-block waiting (the scan is three plain kernels).
 #include "mst_internal.cuh"
+#include "mst_tc_gemm.cuh"
 #include "mst_bits.cuh"
 
 #include <cuda_bf16.h>
@@ -319,6 +320,7 @@ mst_status_t mst_rebuild_from_bits(mst_layer* L, int set, const void* dense_W, i
 
 // CSC view of the live set.
 mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s) {
+  MST_TRY(mst_alloc_csc(L));
   const int c = L->cur;
   transpose_bits<<<blocks_for((int64_t)L->wpc * L->wpr * 32, 256), 256, 0, s>>>(L->bits[c], L->O, L->I, L->wpr, L->wpc,
                                                                                 L->bitsT); MST_COUNT_LAUNCH();
@@ -336,18 +338,30 @@ mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s) {
   return mst_build_csc(const_cast<mst_layer*>(L), s);
 }
 
-mst_status_t mst_densify(const mst_layer* L, cudaStream_t s) {
+// Dense bf16 image of W.M for the dense-tile kernels.  Without value tracking the image is rebuilt at every call
+// anyway, so it lives in a per-device scratch buffer shared by all layers (no per-layer memory; like the other
+// scratch kinds, calls that use it must not overlap on the GPU).  With value tracking the layer keeps its own image
+// and reuses it until the mask or the values change.
+mst_status_t mst_densify(const mst_layer* L, cudaStream_t s, const uint16_t** image) {
   const int c = L->cur;
-  // with value tracking the image is reused until the mask or the values change
-  if (L->track_values && L->dense_version == L->version && L->dense_epoch == L->values_epoch) return MST_OK;
-  L->dense_version = L->version;
-  L->dense_epoch = L->values_epoch;
-  const int64_t groups = L->N / 8;  // callers guarantee I % 8 == 0
-  {
-    MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
-                                       (const uint32_t*)L->bits[c], (const int32_t*)L->wscan[c], L->O, L->I, L->wpr,
-                                       (const uint16_t*)L->vals[c], (const int32_t*)nullptr, L->dense_w));
+  uint16_t* dst = nullptr;
+  if (L->track_values) {
+    MST_TRY(mst_alloc_dense(const_cast<mst_layer*>(L)));
+    dst = L->dense_w;
+    *image = dst;
+    if (L->dense_version == L->version && L->dense_epoch == L->values_epoch) return MST_OK;
+    L->dense_version = L->version;
+    L->dense_epoch = L->values_epoch;
+  } else {
+    void* ws = nullptr;
+    MST_TRY(mst_workspace_kind(MST_WS_IMAGE, 2 * (size_t)L->N, &ws));
+    dst = (uint16_t*)ws;
+    *image = dst;
   }
+  const int64_t groups = L->N / 8;  // callers guarantee I % 8 == 0
+  MST_CUDA_TRY(mst_launch_overlapped(densify_from_bits, dim3(blocks_for(groups, 256)), dim3(256), 0, s,
+                                     (const uint32_t*)L->bits[c], (const int32_t*)L->wscan[c], L->O, L->I, L->wpr,
+                                     (const uint16_t*)L->vals[c], (const int32_t*)nullptr, dst));
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
@@ -377,7 +391,10 @@ extern "C" mst_status_t mst_pack(mst_layer_t* L, const void* W_dense, int64_t ld
   MST_TRY(mst_rebuild_from_bits(L, set, W_dense, ldw, set, s));
   L->nnz = total;
   ++L->version;
-  MST_TRY(mst_build_csc(L, s));
+  // the CSC view serves the CUDA-core input gradient, the CSC export and the structure check: layers on the tensor
+  // path get it on demand
+  if (mst_use_tensor_path(L)) L->csc_valid = 0;
+  else MST_TRY(mst_build_csc(L, s));
   MST_CUDA_TRY(cudaStreamSynchronize(s));
   return MST_OK;
 }

@@ -205,12 +205,18 @@ __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_bas
       const int64_t wi = m * P.wpr + (n >> 5);
       const uint32_t word = P.bits[wi];
       float* dst = (P.splits > 1 ? P.partial + (int64_t)split * P.nnz : reinterpret_cast<float*>(P.out)) + P.wscan[wi];
-      int rank = 0;
+      if (word == 0xFFFFFFFFu) {
+        // dense stretch (a restored layer, a saturated row): the 32 values are contiguous in CSR order
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        if ((word >> j) & 1u) {
-          dst[rank] = __uint_as_float(r[j]);
-          ++rank;
+        for (int j = 0; j < 32; ++j) dst[j] = __uint_as_float(r[j]);
+      } else {
+        int rank = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if ((word >> j) & 1u) {
+            dst[rank] = __uint_as_float(r[j]);
+            ++rank;
+          }
         }
       }
     }
@@ -765,7 +771,11 @@ int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double ou
 //                   buffer, so two such calls must not overlap on the GPU (mst_dense_grad, mst_dense_grad_dw,
 //                   mst_sddmm_dw and the host-step calls on the tensor path): keep them on one stream or order them
 //                   with events.
-//   MST_WS_COLUMNS  feature-major copy of activation columns for the structured-sparse path (same rule).
+//   MST_WS_COLUMNS  feature-major copies of activations for the structured-sparse path and the CUDA-core kernels
+//                   (same rule).
+//   MST_WS_ATTENTION  per-row dot products of the attention backward pass (same rule).
+//   MST_WS_IMAGE    dense bf16 image of W.M of the layer being multiplied, for layers without value tracking
+//                   (same rule).
 mst_status_t mst_workspace_kind(int kind, size_t bytes, void** ptr) {
   constexpr int MAX_DEVICES = 64;
   static void* buf[MST_WS_KINDS][MAX_DEVICES] = {};

@@ -62,5 +62,5 @@ int mst_tc_pick_splits(int64_t works1, int64_t slots, int64_t kblocks, double ou
 // Calls that use it must not overlap on the GPU.
 mst_status_t mst_workspace(size_t bytes, void** ptr);
 // The same per purpose: split partial sums, feature-major activation columns of the structured-sparse path.
-enum { MST_WS_SPLIT = 0, MST_WS_COLUMNS = 1, MST_WS_KINDS = 2 };
+enum { MST_WS_SPLIT = 0, MST_WS_COLUMNS = 1, MST_WS_ATTENTION = 2, MST_WS_IMAGE = 3, MST_WS_KINDS = 4 };
 mst_status_t mst_workspace_kind(int kind, size_t bytes, void** ptr);

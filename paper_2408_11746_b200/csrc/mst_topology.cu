@@ -854,6 +854,7 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
   }
   if (fused) {
     MST_CUDA_TRY(cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * BINS, s));
+    if (!mst_use_tensor_path(L)) MST_TRY(mst_alloc_csc(L));   // the kernel fills the view's arrays for such layers
     FusedParams F;
     F.sel = P;
     F.n_prune = n_prune; F.n_grad = n_grad; F.n_rand = n_rand;

@@ -492,3 +492,65 @@ def test_csc_view_is_rebuilt_on_demand_after_an_update():
     np.testing.assert_array_equal(pm, order)
     np.testing.assert_array_equal(cp, np.concatenate([[0], np.cumsum(np.bincount(ci, minlength=320))]))
     L.close()
+
+
+# ------------------------------------------------------------ value tracking, path query, launch counter
+def test_value_tracking_reuses_and_refreshes_derived_operands():
+    from cuda.bindings import runtime as cudart
+    p = _problem(192, 256, 300, "bf16", 0.2, 4321)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    for path in (mst.MST_PATH_TENSOR_CORE, mst.MST_PATH_SPARSE_TC):
+        L = make_layer(p)
+        L.set_path(path)
+        L.track_values(True)
+        T, O, I = p.tokens, p.out_features, p.in_features
+        X, dY = to_dev(p, "X"), to_dev(p, "dY")
+        Y = torch.empty((T, O), dtype=torch.bfloat16, device=dev())
+        dX = torch.empty((T, I), dtype=torch.bfloat16, device=dev())
+
+        def run():
+            L.fwd(X, Y, T); L.bwd_x(dY, dX, T)
+            torch.cuda.synchronize()
+            return host(Y), host(dX)
+        n0 = mst.mst_launch_count()
+        Y1, dX1 = run()
+        n1 = mst.mst_launch_count()
+        Y2, dX2 = run()                      # nothing changed: the derived operands are reused, fewer launches
+        n2 = mst.mst_launch_count()
+        assert n2 - n1 < n1 - n0
+        np.testing.assert_array_equal(Y1.view(np.uint32), Y2.view(np.uint32))
+        assert rel_err(Y1, oracle.fwd(p.X, W, p.mask)) <= TOL["bf16"]
+        # an optimizer step in place (every value doubled: exact in bf16), announced to the library
+        ptr, nnz = mst.mst_values(L.handle)
+        v2 = (2.0 * oracle.to_csr(W, p.mask)[2]).astype(np.float32)
+        bits = torch.from_numpy(mst_inputs.f32_to_bf16_bits(v2).view(np.int16)).to(dev())
+        (err,) = cudart.cudaMemcpy(ptr, bits.data_ptr(), 2 * nnz, cudart.cudaMemcpyKind.cudaMemcpyDeviceToDevice)
+        assert int(err) == 0
+        L.values_changed()
+        Y3, dX3 = run()
+        assert rel_err(Y3, oracle.fwd(p.X, 2.0 * W, p.mask)) <= TOL["bf16"]
+        assert rel_err(dX3, oracle.bwd_x(p.dY, 2.0 * W, p.mask)) <= TOL["bf16"]
+        # a topology update announces itself
+        G = oracle.dense_grad(p.dY, p.X).astype(np.float32)
+        st = mst.mst_topology_update(L.handle, 0.3, -1, 0.25, 3, 0, False, torch.from_numpy(G).to(dev()))
+        Wn, Mn, *_ = oracle.mg_update((2.0 * W).astype(np.float32), p.mask.copy(), G, st.n_prune, st.n_grad, st.n_rand, 3, 0,
+                                      p.layer_id)
+        Y4, dX4 = run()
+        assert rel_err(Y4, oracle.fwd(p.X, Wn, Mn)) <= TOL["bf16"]
+        assert rel_err(dX4, oracle.bwd_x(p.dY, Wn, Mn)) <= TOL["bf16"]
+        L.close()
+
+
+def test_path_in_use_reports_the_resolved_path():
+    p = _problem(64, 64, 8, "bf16", 0.1, 1)
+    L = make_layer(p)
+    assert L.path_in_use() == mst.MST_PATH_TENSOR_CORE           # AUTO on an aligned bf16 layer
+    L.set_path(mst.MST_PATH_CUDA_CORE)
+    assert L.path_in_use() == mst.MST_PATH_CUDA_CORE
+    L.set_path(mst.MST_PATH_SPARSE_TC)
+    assert L.path_in_use() == mst.MST_PATH_SPARSE_TC
+    L.close()
+    q = _problem(64, 64, 8, "f32", 0.1, 1)
+    L = make_layer(q)
+    assert L.path_in_use() == mst.MST_PATH_CUDA_CORE             # fp32 layers never leave the CUDA cores
+    L.close()
