@@ -381,6 +381,68 @@ def run_sweep(args) -> None:
                                   measured_peaks(), dev)))
 
 
+# ------------------------------------------------------------------------------------------ small cases for a profiler
+def run_profile_case(args) -> None:
+    """A few launches of one kernel family on a case small enough for a counter capture (inputs still larger than L2,
+    a few hundred MB on the device): the command line the summaries in profiles/ were captured with."""
+    import torch
+    import paper_2408_11746_b200 as mst
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    case = args.profile_case
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(1)
+    if case == "attention_bwd":
+        B, n, H, d = 4, 1024, 12, 64
+        C = H * d
+        qkv = torch.randn(B * n, 3 * C, device=dev, dtype=torch.bfloat16, generator=gen)
+        dO = torch.randn(B * n, C, device=dev, dtype=torch.bfloat16, generator=gen)
+        out = torch.empty(B * n, C, device=dev, dtype=torch.bfloat16)
+        lse = torch.empty(B, H, n, device=dev, dtype=torch.float32)
+        dqkv = torch.empty_like(qkv)
+        b0, g0 = qkv.data_ptr(), dqkv.data_ptr()
+        for _ in range(3):
+            mst.mst_strided_attention_fwd(b0, b0 + 2 * C, b0 + 4 * C, 3 * C, B, n, H, d, 256, out, C, lse)
+            mst.mst_strided_attention_bwd(b0, b0 + 2 * C, b0 + 4 * C, 3 * C, out, C, dO, C, lse, B, n, H, d, 256,
+                                          g0, g0 + 2 * C, g0 + 4 * C, 3 * C)
+        torch.cuda.synchronize()
+        return
+    O, I, T = 5120, 1280, 8192                       # fc1 of GPT-2 large, half the sweep's tokens
+    density = {"dense_tiles": 0.1, "sparse_tc": 0.02, "cuda_core": 0.1, "update": 0.1}[case]
+    nnz = mst_inputs.exact_nnz(O, I, density)
+    Wd = (torch.randn(O, I, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+    mask = torch.from_numpy(mst_inputs.uniform_mask(O, I, nnz, mst_inputs.BASE_SEED + 5, 2)).to(dev)
+    X = torch.randn(T, I, device=dev, dtype=torch.bfloat16, generator=gen)
+    dY = (torch.randn(T, O, device=dev, dtype=torch.float32, generator=gen) * 1e-2).to(torch.bfloat16)
+    Y = torch.empty(T, O, device=dev, dtype=torch.bfloat16)
+    dX = torch.empty(T, I, device=dev, dtype=torch.bfloat16)
+    dW = torch.empty(nnz, device=dev, dtype=torch.float32)
+    G = torch.empty(O, I, device=dev, dtype=torch.float32)
+    if case == "update":
+        layers = []
+        for li in range(4):
+            L = mst.Layer(li, O, I, mst.MST_BF16)
+            L.pack(Wd, mask)
+            layers.append(L)
+        G.normal_(generator=gen)
+        for k in range(3):
+            rules = [mst.RegrowRule(-1, 0.25, 5, k, 0, 0.0) for _ in layers]
+            mst.mst_topology_update_many([L.handle for L in layers], [0.3] * 4, rules, [G] * 4, want_stats=False)
+            layers[0].update(0.3, target_nnz=-1, random_ratio=0.25, seed=6, step=k, G_dense=G, want_stats=False)
+        torch.cuda.synchronize()
+        return
+    L = mst.Layer(2, O, I, mst.MST_BF16)
+    L.pack(Wd, mask)
+    L.set_path({"dense_tiles": mst.MST_PATH_TENSOR_CORE, "sparse_tc": mst.MST_PATH_SPARSE_TC,
+                "cuda_core": mst.MST_PATH_CUDA_CORE}[case])
+    for _ in range(3):
+        L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW)
+        if case == "dense_tiles":
+            L.dense_grad(dY, X, T, G)
+    torch.cuda.synchronize()
+    assert mst.mst_device_error_flags() == 0
+
+
 # ------------------------------------------------------------------------------------------ other workloads
 def other_legs(reps: int, dev):
     """Timed legs of the workloads the headline does not cover: the single fp32 layer (CUDA-core kernels), the
@@ -416,7 +478,9 @@ def other_legs(reps: int, dev):
             for L, p, X, dY, Y, dX, dW, G in slots:
                 L.fwd(X, Y, p.tokens); L.bwd_x(dY, dX, p.tokens); L.sddmm(dY, X, p.tokens, dW)
                 L.dense_grad(dY, X, p.tokens, G)
-                L.update(zeta, target_nnz=-1, random_ratio=0.25, seed=9, step=k[0], G_dense=G, want_stats=False)
+            rules = [mst.RegrowRule(-1, 0.25, 9, k[0], 0, 0.0) for _ in slots]
+            mst.mst_topology_update_many([s[0].handle for s in slots], [zeta] * len(slots), rules, [s[7] for s in slots],
+                                         want_stats=False)
         t_prod, _ = median_ms(products, reps)
         useful = sum(6.0 * p.tokens * p.nnz for _, p, *_ in slots)
         res = {"workload": label, "fwd_bwd_ms": round(t_prod, 4), "fwd_bwd_useful_tflops": round(useful / (t_prod * 1e-3) / 1e12, 3),
@@ -450,6 +514,8 @@ def main() -> None:
     ap.add_argument("--sweep-reps", type=int, default=50)
     ap.add_argument("--sweep", default=None, choices=["medium", "large", "small"],
                     help="density sweep report alone (not the bench line)")
+    ap.add_argument("--profile-case", default=None, choices=["dense_tiles", "sparse_tc", "cuda_core", "update", "attention_bwd"],
+                    help="run a few launches of one kernel family on a small case (for ncu; prints nothing)")
     ap.add_argument("--attention", action="store_true",
                     help="report on the strided sparse attention forward (not the bench line): one JSON object per "
                          "stride at 16 x 1024 tokens, 12 heads of 64, with torch's dense causal attention beside it")
@@ -458,6 +524,9 @@ def main() -> None:
                          "fc2 input gradient with GELU', against the plain products, GPT-2 small, 16384 tokens")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.profile_case:
+        run_profile_case(args)
+        return
     if args.attention:
         run_attention(args)
         return
@@ -523,6 +592,14 @@ def main() -> None:
         e.record(stream)
         return e
 
+    handles = [s.L.handle for s in slots]
+    Gs = [s.G for s in slots]
+
+    def update_all(k: int, seed: int):
+        # all layers of the block in one call: same results as one call per layer, shared grid barriers
+        rules = [mst.RegrowRule(-1, 0.25, seed, k, 0, 0.0) for _ in slots]
+        mst.mst_topology_update_many(handles, [0.3] * len(slots), rules, Gs, want_stats=False)
+
     def step(k: int, timed: bool):
         for s in slots:
             marks = [ev()] if timed else None
@@ -533,12 +610,14 @@ def main() -> None:
             s.L.sddmm(s.dY, s.X, T, s.dW)
             if timed: marks.append(ev())
             s.L.dense_grad(s.dY, s.X, T, s.G)
-            if timed: marks.append(ev())
-            s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=1, step=k, G_dense=s.G, want_stats=False)
             if timed:
                 marks.append(ev())
-                for j, name in enumerate(KERNELS):
-                    timers[name].append((s, marks[j], marks[j + 1]))
+                for j, name in enumerate(KERNELS[:4]):
+                    timers[name].append(([s], marks[j], marks[j + 1]))
+        a = ev() if timed else None
+        update_all(k, 1)
+        if timed:
+            timers["topology_update"].append((slots, a, ev()))
 
     def barrier():
         if dist is not None:
@@ -586,9 +665,9 @@ def main() -> None:
 
     def roofline_of(name):
         ms_tot = sum(a.elapsed_time(b) for _, a, b in timers[name])
-        fl = sum(algorithmic(name, s)[0] for s, _, _ in timers[name])
-        by = sum(algorithmic(name, s)[1] for s, _, _ in timers[name])
-        pipe = algorithmic(name, timers[name][0][0])[2]
+        fl = sum(algorithmic(name, s)[0] for ss, _, _ in timers[name] for s in ss)
+        by = sum(algorithmic(name, s)[1] for ss, _, _ in timers[name] for s in ss)
+        pipe = algorithmic(name, timers[name][0][0][0])[2]
         t_pipe = fl / (tensor_peak * 1e12) if pipe != "hbm" else 0.0
         t_hbm = by / (peaks["hbm_gbs"] * 1e9)
         if t_hbm >= t_pipe:
@@ -625,7 +704,7 @@ def main() -> None:
                             "not repeated here because the capture is not regenerated with every kernel change")
     if dom_family == "contraction":
         # what the tensor pipe itself sustains: executed dense flops of this call kind over its time
-        dense_fl = sum(2.0 * T * s.O * s.I for s, _, _ in timers[dom])
+        dense_fl = sum(2.0 * T * s.O * s.I for ss, _, _ in timers[dom] for s in ss)
         dense_ms = sum(a.elapsed_time(b) for _, a, b in timers[dom])
         roof["tensor_pipe"] = {"executed_tflops": dense_fl / (dense_ms * 1e-3) / 1e12, "peak": tensor_peak,
                                "frac": dense_fl / (dense_ms * 1e-3) / 1e12 / tensor_peak,
@@ -642,7 +721,7 @@ def main() -> None:
         for s in slots:
             mst.mst_layer_step_host_async(s.L.handle, s.Xh, s.dYh, T, s.Yh, s.dXh, s.dWh)
             s.L.dense_grad(s.dY, s.X, T, s.G)
-            s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=2, step=k, G_dense=s.G, want_stats=False)
+        update_all(k, 2)
 
     def e2e_wait():
         for s in slots:
@@ -671,7 +750,7 @@ def main() -> None:
             s.L.fwd(s.X, s.Y, T)
             s.L.bwd_x(s.dY, s.dX, T)
             s.L.dense_grad_dw(s.dY, s.X, T, s.G, s.dW)
-            s.L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=3, step=k, G_dense=s.G, want_stats=False)
+        update_all(k, 3)
     for k in range(3):
         shared_step(k)
     barrier()
@@ -694,7 +773,7 @@ def main() -> None:
         "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: four layers' distinct buffers, %.0f MB touched "
                    "per step" % (sum(2 * T * (p.in_features + p.out_features) * es for p in probs) / 1e6),
                    "update": "every step, zeta=0.3, R=0.25 (gradient growth by |G| over the inactive entries), "
-                   "target = current nnz", "paths": paths, "replicas": world},
+                   "target = current nnz; the four layers in one mst_topology_update_many call", "paths": paths, "replicas": world},
         "clocks": clocks, "roofline": roof, "kernels": per,
         "fwd_bwd_only_tflops": useful / ((per["spmm_fwd"]["ms_per_step"] + per["spmm_bwd_x"]["ms_per_step"] +
                                           per["sddmm_dw"]["ms_per_step"]) * 1e-3) / 1e12,

@@ -239,6 +239,18 @@ mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_t target_nn
 mst_status_t mst_topology_update(mst_layer_t* layer, double prune_frac, const mst_regrow_rule_t* regrow_rule,
                                  const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream);
 
+/* The same update for several layers in one call (in training all layers are updated on the same step): identical
+ * results, bit for bit, to calling mst_topology_update on each layer in turn, but the layers' selection passes share
+ * their grid-wide barriers inside one cooperative launch (up to 8 layers per launch), which is where a single update
+ * spends most of its time.  prune_frac[i], rules[i], G_dense[i] belong to layers[i]; stats is NULL or an array of
+ * n_layers entries (same meaning as above, the call then synchronises once per layer).  A layer may appear once.
+ * All arguments are validated before anything is launched.  Layers that cannot join a batch (fp32 or CUDA-core
+ * layers, which also rebuild their CSC view; very large layers) are updated by the single-layer kernels.
+ * Returns the first error met; layers before and after it are still completed. */
+mst_status_t mst_topology_update_many(int32_t n_layers, mst_layer_t* const* layers, const double* prune_frac,
+                                      const mst_regrow_rule_t* rules, const float* const* G_dense,
+                                      mst_update_stats_t* stats, mst_stream_t stream);
+
 /* One training step of the layer from HOST buffers (pinned memory recommended): copies X [T x I] and dY [T x O]
  * (contiguous, layer dtype) to the device, runs forward, input gradient and weight gradient, and copies
  * Y [T x O], dX [T x I] (layer dtype) and dW_vals float [nnz] back.  Any output may be NULL to skip its copy.

@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_path_in_use", "mst_launch_count", "mst_track_values", "mst_values_changed", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_strided_attention_fwd", "mst_strided_attention_bwd", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
-           "mst_update_counts", "mst_topology_update", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
+           "mst_update_counts", "mst_topology_update", "mst_topology_update_many", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
            "mst_status_string"]
 
@@ -89,6 +89,8 @@ _sig = {
     "mst_dense_grad_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp, _vp],
     "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
+    "mst_topology_update_many": [_i32, ctypes.POINTER(_vp), ctypes.POINTER(_f64), ctypes.POINTER(RegrowRule), ctypes.POINTER(_vp),
+                                 ctypes.POINTER(UpdateStats), _vp],
     "mst_layer_step_host": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
     "mst_layer_step_host_async": [_vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp],
     "mst_layer_step_host_wait": [_vp],
@@ -276,6 +278,18 @@ def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, ran
                                     ctypes.byref(stats) if want_stats else None, _stream(stream)),
            "mst_topology_update")
     return stats
+
+
+def mst_topology_update_many(layers, prune_frac, rules, G_dense, want_stats: bool = True, stream=None):
+    """layers: handles; prune_frac: floats; rules: RegrowRule objects; G_dense: device arrays or None, one per layer."""
+    n = len(layers)
+    hs = (_vp * n)(*[int(h) for h in layers])
+    zs = (_f64 * n)(*[float(z) for z in prune_frac])
+    rs = (RegrowRule * n)(*rules)
+    gs = (_vp * n)(*[_ptr(g) for g in G_dense])
+    stats = (UpdateStats * n)() if want_stats else None
+    _check(_lib.mst_topology_update_many(n, hs, zs, rs, gs, stats, _stream(stream)), "mst_topology_update_many")
+    return list(stats) if want_stats else None
 
 
 def mst_layer_step_host(layer: int, X_host, dY_host, T: int, Y_host, dX_host, dW_vals_host, stream=None) -> None:

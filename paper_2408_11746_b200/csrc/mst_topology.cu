@@ -14,6 +14,7 @@
 #include <cooperative_groups.h>
 
 #include <cstdlib>
+#include <new>
 
 #include "mst_bits.cuh"
 #include "mst_internal.cuh"
@@ -760,6 +761,452 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
                           F.row_idx, F.perm, F.col_ptr, totT);
 }
 
+// ------------------------------------------------------------------------------------------------ batched update
+// The updates of several layers in ONE cooperative launch.  The single-layer kernel above is a chain of about ten
+// grid-wide barriers with little work between them; here every round does, for each layer in turn, the work of that
+// layer's current phase, and then ALL layers share one barrier.  A layer's phases and their order are those of the
+// single-layer kernel (histogram pass -> digit pick, tie count -> scan -> mark, mask rewrite -> scan -> CSR fill), its
+// selection state lives in shared memory per layer, and every block takes every decision from the same global
+// histograms, so all blocks walk through the same sequence.  Results are bit-identical to updating the layers one
+// after the other.  Keys are recomputed from global memory in every pass (no register cache: a block holds slices of
+// all layers), and the CSC view is not built (layers that need it take the single-layer path).
+constexpr int BATCH_MAX = 8;
+enum { PH_NEW = 0, PH_HIST = 1, PH_TIE = 2, PH_REWRITE = 3, PH_DONE = 4 };
+
+struct BatchParams {
+  FusedParams L[BATCH_MAX];
+  int smem_off[BATCH_MAX];  // word offset of the layer's three slices (old mask, its scan, gradient marks) in dynamic smem
+  int n;
+};
+
+struct BatchLayerState {
+  unsigned long long prefix, tau;
+  long long k, rem;
+  int need_rank, done, found;
+  int sel;    // 0 prune, 1 gradient, 2 random, 3 rewrite
+  int phase;  // which barrier the layer waits for next
+  int pass, gpass, gscan;
+};
+
+struct BatchShared {
+  unsigned int hist[BINS];
+  unsigned int warp_tot[FUSED_WARPS];
+  int red[FUSED_WARPS];
+  BatchLayerState st[BATCH_MAX];
+};
+
+struct BatchSlice {
+  int64_t lo, hi;
+  uint32_t* s_old;
+  int32_t* s_base;
+  uint32_t* s_grad;
+};
+
+__device__ __forceinline__ int batch_block_sum(int v, int* red) {
+  for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  int r = 0;
+#pragma unroll
+  for (int w = 0; w < FUSED_WARPS; ++w) r += red[w];
+  return r;
+}
+__device__ __forceinline__ int batch_block_excl_scan(int v, int& total, int* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int x = v;
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();
+  if (lane == 31) red[warp] = x;
+  __syncthreads();
+  int before = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < FUSED_WARPS; ++w) {
+    const int t = red[w];
+    if (w < warp) before += t;
+    tot += t;
+  }
+  total = tot;
+  return before + x - v;
+}
+
+// first half of a grid-wide scan: this block's sum of cnt[lo, hi) into the layer's current partial-sum area
+__device__ void batch_scan_begin(const int32_t* cnt, int64_t lo, int64_t hi, int32_t* bsums, int gscan, int* red) {
+  int v = 0;
+  for (int64_t i = lo + threadIdx.x; i < hi; i += FUSED_THREADS) v += cnt[i];
+  const int bs = batch_block_sum(v, red);
+  if (threadIdx.x == 0) bsums[(gscan & 1) * (int)gridDim.x + blockIdx.x] = bs;
+}
+// second half, behind the barrier: out[lo, hi) = exclusive scan, out[n] = total
+__device__ int batch_scan_end(const int32_t* cnt, int32_t* out, int64_t n, int64_t lo, int64_t hi, const int32_t* bsums,
+                               int gscan, int* red) {
+  const int32_t* area = bsums + (gscan & 1) * (int)gridDim.x;
+  int off = 0, tot = 0;
+  for (int j = threadIdx.x; j < (int)gridDim.x; j += FUSED_THREADS) {
+    const int x = __ldcg(area + j);
+    tot += x;
+    if (j < (int)blockIdx.x) off += x;
+  }
+  off = batch_block_sum(off, red);
+  tot = batch_block_sum(tot, red);
+  int carry = off;
+  for (int64_t base = lo; base < hi; base += FUSED_THREADS) {
+    const int64_t i = base + threadIdx.x;
+    const int x = i < hi ? cnt[i] : 0;
+    int tile_total;
+    const int ex = batch_block_excl_scan(x, tile_total, red);
+    if (i < hi) out[i] = carry + ex;
+    carry += tile_total;
+  }
+  if (threadIdx.x == 0) out[n] = tot;
+  __syncthreads();
+  return tot;
+}
+
+template <int MODE>
+__device__ void batch_hist_sweep(const FusedParams& F, BatchLayerState& st, const BatchSlice& sl, BatchShared& sh) {
+  constexpr int KB = KeyBits<MODE>::value;
+  typedef typename KeyWord<MODE>::type K;
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int pass = st.pass;
+  const int shift = pass_shift(KB, pass), width = pass_width(KB, pass);
+  const unsigned dmask = (1u << width) - 1u;
+  const int hi_shift = shift + width;
+  const K prefix = (K)st.prefix;
+  unsigned int* gh = F.hist + (st.gpass % 3) * BINS;
+  __syncthreads();  // the state was written by the previous step
+  for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
+  __syncthreads();
+  bool saw_nonfinite = false;
+  constexpr int BATCH = 8;
+  for (int64_t w0 = sl.lo + warp; w0 < sl.hi; w0 += FUSED_WARPS * BATCH) {
+    unsigned digit[BATCH];
+    bool live[BATCH];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
+      unsigned long long key64 = 0;
+      bool nf = false;
+      const int64_t li = w < sl.hi ? w - sl.lo : 0;
+      const bool c = w < sl.hi && cand_key_w<MODE>(P, w, lane, sl.s_old[li], sl.s_base[li], sl.s_grad[li], key64, nf);
+      const K key = (K)key64;
+      saw_nonfinite |= (c && nf);
+      live[j] = c && (pass == 0 || (K)(key >> hi_shift) == prefix);
+      digit[j] = live[j] ? (unsigned)((key >> shift) & (K)dmask) : (unsigned)BINS;
+    }
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      if (live[j]) atomicAdd(&sh.hist[digit[j]], 1u);
+    }
+  }
+  if (pass == 0 && saw_nonfinite) atomicOr(&F.flags[0], MST_FLAG_NONFINITE);
+  __syncthreads();
+  for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS)
+    if (sh.hist[b]) atomicAdd(&gh[b], sh.hist[b]);
+}
+
+// behind the barrier: every block picks the digit from the complete histogram (same arithmetic as the single-layer
+// kernel) and advances the layer's selection state
+template <int MODE>
+__device__ void batch_hist_pick(const FusedParams& F, BatchLayerState& st, BatchShared& sh) {
+  constexpr int KB = KeyBits<MODE>::value;
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int pass = st.pass;
+  const int shift = pass_shift(KB, pass), width = pass_width(KB, pass);
+  const unsigned long long prefix = st.prefix;
+  const long long k = st.k;
+  const int gpass = st.gpass;
+  unsigned int* gh = F.hist + (gpass % 3) * BINS;
+  unsigned int mine[FUSED_BPT];
+  unsigned int tsum = 0;
+#pragma unroll
+  for (int j = 0; j < FUSED_BPT; ++j) {
+    mine[j] = __ldcg(gh + threadIdx.x * FUSED_BPT + j);
+    tsum += mine[j];
+  }
+  if (blockIdx.x == 0) {  // clear the buffer of pass gpass + 2 (last read before this barrier)
+    unsigned int* gz = F.hist + ((gpass + 2) % 3) * BINS;
+    for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) gz[b] = 0;
+  }
+  unsigned int incl = tsum;
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  __syncthreads();  // everyone has read the state; warp_tot is free
+  if (threadIdx.x == 0) st.found = 0;
+  if (lane == 31) sh.warp_tot[warp] = incl;
+  __syncthreads();
+  unsigned int before = incl - tsum;
+  for (int wv = 0; wv < warp; ++wv) before += sh.warp_tot[wv];
+  const bool owner = (long long)before < k && k <= (long long)before + (long long)tsum;
+  if (owner) {
+    long long cum = before;
+    int bin = 0;
+    unsigned int bcount = 0;
+    for (int j = 0; j < FUSED_BPT; ++j) {
+      if (cum + (long long)mine[j] >= k) { bin = j; bcount = mine[j]; break; }
+      cum += mine[j];
+    }
+    const unsigned long long np = (prefix << width) | (unsigned long long)(threadIdx.x * FUSED_BPT + bin);
+    st.prefix = np;
+    st.k = k - cum;
+    st.found = 1;
+    if (shift == 0) {
+      st.tau = np;
+      st.rem = k - cum;
+      st.need_rank = ((long long)bcount > k - cum) ? 1 : 0;
+      st.done = 1;
+    } else if ((long long)bcount == k - cum) {
+      st.tau = (np << shift) | ((1ULL << shift) - 1ULL);
+      st.rem = k - cum;
+      st.need_rank = 0;
+      st.done = 1;
+    } else if (MODE == MODE_PRUNE && shift <= P.low_zero) {
+      st.tau = np << shift;
+      st.rem = k - cum;
+      st.need_rank = 1;
+      st.done = 1;
+    }
+  }
+  __syncthreads();
+  if (!st.found) {  // fewer candidates than requested (ruled out by the host counts): take everything
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      st.tau = ~0ULL;
+      st.rem = 0x7FFFFFFFFFFFFFFFLL;
+      st.need_rank = 0;
+      st.done = 1;
+      if (blockIdx.x == 0) atomicOr(&F.flags[0], MST_FLAG_CORRUPT);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    st.gpass = gpass + 1;
+    st.pass = pass + 1;
+  }
+  __syncthreads();
+}
+
+template <int MODE>
+__device__ void batch_tie_count(const FusedParams& F, const BatchLayerState& st, const BatchSlice& sl, BatchShared& sh) {
+  typedef typename KeyWord<MODE>::type K;
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const K tau = (K)st.tau;
+  for (int64_t w = sl.lo + warp; w < sl.hi; w += FUSED_WARPS) {
+    unsigned long long key64;
+    bool nf;
+    const bool c = cand_key_w<MODE>(P, w, lane, sl.s_old[w - sl.lo], sl.s_base[w - sl.lo], sl.s_grad[w - sl.lo], key64, nf);
+    const unsigned eq = __ballot_sync(0xffffffffu, c && (K)key64 == tau);
+    if (lane == 0) F.cnt[w] = __popc(eq);
+  }
+  __syncthreads();
+  batch_scan_begin(F.cnt, sl.lo, sl.hi, F.bsums, st.gscan, sh.red);
+}
+
+template <int MODE>
+__device__ void batch_mark(const FusedParams& F, const BatchLayerState& st, const BatchSlice& sl, uint32_t* out_bits) {
+  typedef typename KeyWord<MODE>::type K;
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const K tau = (K)st.tau;
+  const long long rem = st.rem;
+  const bool need_rank = st.need_rank != 0;
+  constexpr int MB = 4;
+  for (int64_t w0 = sl.lo + warp; w0 < sl.hi; w0 += FUSED_WARPS * MB) {
+    bool c[MB], iseq[MB];
+    K key[MB];
+#pragma unroll
+    for (int j = 0; j < MB; ++j) {
+      const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
+      bool nf = false;
+      unsigned long long key64 = 0;
+      const int64_t li = w < sl.hi ? w - sl.lo : 0;
+      c[j] = w < sl.hi && cand_key_w<MODE>(P, w, lane, sl.s_old[li], sl.s_base[li], sl.s_grad[li], key64, nf);
+      key[j] = (K)key64;
+      iseq[j] = c[j] && key[j] == tau;
+    }
+#pragma unroll
+    for (int j = 0; j < MB; ++j) {
+      const int64_t w = w0 + (int64_t)j * FUSED_WARPS;
+      if (w >= sl.hi) continue;  // uniform over the warp
+      const unsigned eq = __ballot_sync(0xffffffffu, iseq[j]);
+      const long long rank = need_rank ? (long long)F.scan[w] + __popc(eq & lanemask_lt()) : -1;
+      const bool take = c[j] && (key[j] < tau || (iseq[j] && rank < rem));
+      const unsigned bits = __ballot_sync(0xffffffffu, take);
+      if (lane == 0) {
+        out_bits[w] = bits;
+        if (MODE == MODE_GRAD) sl.s_grad[w - sl.lo] = bits;  // the random selection of this block reads it from here
+      }
+    }
+  }
+  __syncthreads();
+}
+
+__device__ __forceinline__ long long batch_sel_count(const FusedParams& F, int sel) {
+  return sel == 0 ? F.n_prune : (sel == 1 ? F.n_grad : F.n_rand);
+}
+__device__ __forceinline__ uint32_t* batch_sel_bits(const FusedParams& F, int sel) {
+  return sel == 0 ? F.pruned_bits : (sel == 1 ? F.grad_bits : F.rand_bits);
+}
+
+// Non-barrier work until the layer reaches its next barrier phase: selections that take nothing write empty masks,
+// the next selection with work gets its state, after the last one the mask rewrite is due.
+__device__ void batch_advance(const FusedParams& F, BatchLayerState& st, const BatchSlice& sl) {
+  __syncthreads();
+  int sel = st.sel;
+  while (sel <= 2 && batch_sel_count(F, sel) <= 0) {
+    uint32_t* out = batch_sel_bits(F, sel);
+    for (int64_t w = sl.lo + threadIdx.x; w < sl.hi; w += FUSED_THREADS) {
+      out[w] = 0;
+      if (sel == 1) sl.s_grad[w - sl.lo] = 0;
+    }
+    ++sel;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    st.sel = sel;
+    if (sel <= 2) {
+      st.prefix = 0;
+      st.k = batch_sel_count(F, sel);
+      st.tau = 0;
+      st.rem = 0;
+      st.need_rank = 0;
+      st.done = 0;
+      st.pass = 0;
+      st.phase = PH_HIST;
+    } else {
+      st.phase = PH_REWRITE;
+    }
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_batch_kernel(const BatchParams B) {
+  cg::grid_group grid = cg::this_grid();
+  __shared__ BatchShared sh;
+  extern __shared__ uint32_t s_dyn[];
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  BatchSlice sl[BATCH_MAX];
+#pragma unroll
+  for (int l = 0; l < BATCH_MAX; ++l) {
+    if (l >= B.n) break;
+    const SelParams& P = B.L[l].sel;
+    const int64_t per = (P.nwords + gridDim.x - 1) / gridDim.x;
+    sl[l].lo = per * blockIdx.x < P.nwords ? per * blockIdx.x : P.nwords;
+    sl[l].hi = sl[l].lo + per < P.nwords ? sl[l].lo + per : P.nwords;
+    sl[l].s_old = s_dyn + B.smem_off[l];
+    sl[l].s_base = reinterpret_cast<int32_t*>(s_dyn + B.smem_off[l] + per);
+    sl[l].s_grad = s_dyn + B.smem_off[l] + 2 * per;
+    for (int64_t w = sl[l].lo + threadIdx.x; w < sl[l].hi; w += FUSED_THREADS) {
+      sl[l].s_old[w - sl[l].lo] = P.old_bits[w];
+      sl[l].s_base[w - sl[l].lo] = P.old_wscan[w];
+      sl[l].s_grad[w - sl[l].lo] = 0;
+    }
+    if (threadIdx.x == 0) {
+      sh.st[l].sel = 0;
+      sh.st[l].phase = PH_NEW;
+      sh.st[l].gpass = 0;
+      sh.st[l].gscan = 0;
+    }
+  }
+  __syncthreads();
+  for (int l = 0; l < B.n; ++l) batch_advance(B.L[l], sh.st[l], sl[l]);
+
+  for (;;) {
+    // ---- work in front of the shared barrier
+    bool pending = false;
+    for (int l = 0; l < B.n; ++l) {
+      const FusedParams& F = B.L[l];
+      BatchLayerState& st = sh.st[l];
+      const int phase = st.phase, sel = st.sel;   // uniform: written behind block barriers
+      if (phase == PH_DONE) continue;
+      pending = true;
+      if (phase == PH_HIST) {
+        if (sel == 0) batch_hist_sweep<MODE_PRUNE>(F, st, sl[l], sh);
+        else if (sel == 1) batch_hist_sweep<MODE_GRAD>(F, st, sl[l], sh);
+        else batch_hist_sweep<MODE_RAND>(F, st, sl[l], sh);
+      } else if (phase == PH_TIE) {
+        if (sel == 0) batch_tie_count<MODE_PRUNE>(F, st, sl[l], sh);
+        else if (sel == 1) batch_tie_count<MODE_GRAD>(F, st, sl[l], sh);
+        else batch_tie_count<MODE_RAND>(F, st, sl[l], sh);
+      } else {  // PH_REWRITE: new = (old & ~pruned) | grad | rand, and its popcounts
+        const SelParams& P = F.sel;
+        for (int64_t w = sl[l].lo + threadIdx.x; w < sl[l].hi; w += FUSED_THREADS) {
+          const uint32_t b = (P.old_bits[w] & ~F.pruned_bits[w]) | F.grad_bits[w] | F.rand_bits[w];
+          F.new_bits[w] = b;
+          F.cnt[w] = __popc(b);
+        }
+        __syncthreads();
+        batch_scan_begin(F.cnt, sl[l].lo, sl[l].hi, F.bsums, st.gscan, sh.red);
+      }
+    }
+    if (!pending) break;   // same decision in every block
+    grid.sync();
+    // ---- work behind it
+    for (int l = 0; l < B.n; ++l) {
+      const FusedParams& F = B.L[l];
+      BatchLayerState& st = sh.st[l];
+      const int phase = st.phase, sel = st.sel;
+      if (phase == PH_DONE) continue;
+      if (phase == PH_HIST) {
+        constexpr int passes_mag = num_passes(32), passes_hash = num_passes(64);
+        if (sel == 0) batch_hist_pick<MODE_PRUNE>(F, st, sh);
+        else if (sel == 1) batch_hist_pick<MODE_GRAD>(F, st, sh);
+        else batch_hist_pick<MODE_RAND>(F, st, sh);
+        const bool finished = st.done || st.pass >= (sel == 2 ? passes_hash : passes_mag);
+        if (!finished) continue;
+        if (st.need_rank) {
+          __syncthreads();
+          if (threadIdx.x == 0) st.phase = PH_TIE;
+          __syncthreads();
+          continue;
+        }
+      } else if (phase == PH_TIE) {
+        batch_scan_end(F.cnt, F.scan, F.sel.nwords, sl[l].lo, sl[l].hi, F.bsums, st.gscan, sh.red);
+        __syncthreads();
+        if (threadIdx.x == 0) st.gscan = st.gscan + 1;
+        __syncthreads();
+      } else {  // PH_REWRITE
+        batch_scan_end(F.cnt, F.new_wscan, F.sel.nwords, sl[l].lo, sl[l].hi, F.bsums, st.gscan, sh.red);
+        const SelParams& P = F.sel;
+        for (int64_t w0 = sl[l].lo + warp; w0 < sl[l].hi; w0 += FUSED_WARPS * 4) {
+          if (P.bf16)
+            mst_fill_csr_words<uint16_t, 4>(w0, FUSED_WARPS, sl[l].hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col,
+                                            (uint16_t*)F.new_vals, F.new_row_ptr, P.old_bits, P.old_wscan,
+                                            (const uint16_t*)P.vals, nullptr);
+          else
+            mst_fill_csr_words<float, 4>(w0, FUSED_WARPS, sl[l].hi, lane, F.new_bits, F.new_wscan, P.O, P.wpr, F.new_col,
+                                         (float*)F.new_vals, F.new_row_ptr, P.old_bits, P.old_wscan, (const float*)P.vals,
+                                         nullptr);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) st.phase = PH_DONE;
+        __syncthreads();
+        continue;
+      }
+      // the selection is settled (threshold known, ties ranked if needed): mark it and move on
+      if (sel == 0) batch_mark<MODE_PRUNE>(F, st, sl[l], F.pruned_bits);
+      else if (sel == 1) batch_mark<MODE_GRAD>(F, st, sl[l], F.grad_bits);
+      else batch_mark<MODE_RAND>(F, st, sl[l], F.rand_bits);
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        st.sel = sel + 1;
+        st.phase = PH_NEW;
+      }
+      batch_advance(F, st, sl[l]);
+    }
+  }
+}
+
 inline unsigned long long host_mix(unsigned long long z) {
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
   z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
@@ -791,27 +1238,35 @@ extern "C" mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_
   return MST_OK;
 }
 
-extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, const mst_regrow_rule_t* rule,
-                                            const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream) {
+namespace {
+
+// One layer's update, planned on the host: counts, selection parameters, which buffer set is built.
+struct UpdatePlan {
+  mst_layer* L;
+  int64_t n_prune, n_rand, n_grad, target;
+  int c, n;  // live set, set being built
+  SelParams P;
+};
+
+mst_status_t plan_update(mst_layer* L, double prune_frac, const mst_regrow_rule_t* rule, const float* G_dense, UpdatePlan* pl) {
   if (!L || !rule) return MST_ERR_INVALID_ARG;
   if (L->nnz < 0) return MST_ERR_NOT_PACKED;
-  cudaStream_t s = (cudaStream_t)stream;
   int64_t cnt[4];
   MST_TRY(mst_update_counts(prune_frac, L->nnz, rule->target_nnz, L->N, rule->random_ratio, cnt));
-  const int64_t n_prune = cnt[0], n_rand = cnt[2], n_grad = cnt[3];
-  const int64_t target = rule->target_nnz < 0 ? L->nnz : rule->target_nnz;
-  if (target > L->cap) return MST_ERR_CAPACITY;
+  pl->L = L;
+  pl->n_prune = cnt[0];
+  pl->n_rand = cnt[2];
+  pl->n_grad = cnt[3];
+  pl->target = rule->target_nnz < 0 ? L->nnz : rule->target_nnz;
+  if (pl->target > L->cap) return MST_ERR_CAPACITY;
   if (!(rule->prune_grad_weight >= 0.f)) return MST_ERR_INVALID_ARG;
-  if ((n_grad > 0 || (rule->prune_grad_weight != 0.f && n_prune > 0)) && !G_dense) return MST_ERR_INVALID_ARG;
-
-  const int c = L->cur, n = c ^ 1;
-  // flags[0] (error bits) stays set until a reporting call has returned it; only the per-update statistic is cleared
-  MST_CUDA_TRY(cudaMemsetAsync(L->flags + 1, 0, sizeof(int32_t) * 3, s));
-
-  SelParams P;
-  P.old_bits = L->bits[c];
-  P.old_wscan = L->wscan[c];
-  P.vals = L->vals[c];
+  if ((pl->n_grad > 0 || (rule->prune_grad_weight != 0.f && pl->n_prune > 0)) && !G_dense) return MST_ERR_INVALID_ARG;
+  pl->c = L->cur;
+  pl->n = L->cur ^ 1;
+  SelParams& P = pl->P;
+  P.old_bits = L->bits[pl->c];
+  P.old_wscan = L->wscan[pl->c];
+  P.vals = L->vals[pl->c];
   P.bf16 = L->dtype == MST_BF16;
   P.G = G_dense;
   P.pruned_bits = L->pruned_bits;
@@ -829,21 +1284,105 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     const unsigned long long b = host_mix((a ^ rule->step) + SM64_GAMMA);
     P.stream = host_mix((b ^ (unsigned long long)(int64_t)L->layer_id) + SM64_GAMMA);
   }
+  return MST_OK;
+}
 
+void fill_fused_params(const UpdatePlan& pl, FusedParams& F) {
+  mst_layer* L = pl.L;
+  const int n = pl.n;
+  F.sel = pl.P;
+  F.n_prune = pl.n_prune; F.n_grad = pl.n_grad; F.n_rand = pl.n_rand;
+  F.pruned_bits = L->pruned_bits; F.grad_bits = L->grad_bits; F.rand_bits = L->rand_bits; F.new_bits = L->bits[n];
+  F.cnt = L->word_cnt; F.scan = L->word_scan; F.bsums = L->block_sums;
+  F.hist = L->hist; F.flags = L->flags;
+  F.new_wscan = L->wscan[n]; F.new_row_ptr = L->row_ptr[n]; F.new_col = L->col_idx[n]; F.new_vals = L->vals[n];
+  F.bitsT = L->bitsT; F.wscanT = L->wscanT; F.col_ptr = L->col_ptr; F.row_idx = L->row_idx; F.perm = L->perm;
+  F.wpc = L->wpc; F.nwordsT = L->nwordsT;
+  F.build_csc = mst_use_tensor_path(L) ? 0 : 1;
+}
+
+// Host epilogue of an update whose kernels have been enqueued: statistics and error report when asked for, then the
+// flip to the new buffer set.  `fused`: the structure was built by a fused kernel (single-layer or batched).
+mst_status_t finish_update(const UpdatePlan& pl, bool fused, mst_update_stats_t* stats, cudaStream_t s) {
+  mst_layer* L = pl.L;
+  const int n = pl.n;
+  const int64_t nnz_before = L->nnz;
+  if (stats) {
+    // the fused kernel records the longest row itself only when it also builds the CSC view
+    if (!fused || !L->csc_valid) { max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags); MST_COUNT_LAUNCH(); }
+    int32_t f[4] = {0, 0, 0, 0};
+    int32_t total = 0;
+    MST_CUDA_TRY(cudaMemcpyAsync(f, L->flags, sizeof(f), cudaMemcpyDeviceToHost, s));
+    MST_CUDA_TRY(cudaMemcpyAsync(&total, L->wscan[n] + L->nwords, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+    MST_CUDA_TRY(cudaStreamSynchronize(s));
+    stats->nnz_before = nnz_before;
+    stats->nnz_after = total;
+    stats->n_prune = pl.n_prune;
+    stats->n_grad = pl.n_grad;
+    stats->n_rand = pl.n_rand;
+    stats->max_row_nnz = f[1];
+    const bool bad = (f[0] & (MST_FLAG_NONFINITE | MST_FLAG_CORRUPT)) || total != pl.target;
+    if (bad) {
+      // A rejected update is not applied: the structure built in the other buffer set is dropped and the layer keeps
+      // its mask, values and nnz.  The CSC arrays may hold the rejected structure, so the view is rebuilt on next use.
+      L->csc_valid = 0;
+      MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t), s));  // reported: cleared
+      stats->nnz_after = nnz_before;
+      return (f[0] & MST_FLAG_NONFINITE) ? MST_ERR_NONFINITE : MST_ERR_CORRUPT;
+    }
+  }
+  L->cur = n;
+  L->nnz = pl.target;
+  ++L->version;
+  if (!fused) MST_TRY(mst_build_csc(L, s));
+  return MST_OK;
+}
+
+// grid of the fused kernels on the current device (0: cooperative launch unavailable)
+int fused_grid_limit(const void* fn) {
+  int dev = 0, coop = 0, sms = 0, occ = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, FUSED_THREADS, 0) != cudaSuccess || !coop || occ < 1)
+    return 0;
+  if (occ > 2) occ = 2;
+  return sms * occ;
+}
+
+mst_status_t launch_cooperative(const void* fn, void** args, int grid_blocks, size_t smem, cudaStream_t s) {
+  // cooperative launch that may also start while its predecessor drains (the kernel waits before its first access)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid_blocks);
+  cfg.blockDim = dim3(FUSED_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = mst_pdl_enabled() ? 2 : 1;
+  MST_CUDA_TRY(cudaLaunchKernelExC(&cfg, fn, args));
+  MST_COUNT_LAUNCH();
+  return MST_OK;
+}
+
+// kernels of one layer's update (everything except the host epilogue); *fused_out tells which form ran
+mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fused_out) {
+  mst_layer* L = pl.L;
+  const SelParams& P = pl.P;
+  // flags[0] (error bits) stays set until a reporting call has returned it; only the per-update statistic is cleared
+  MST_CUDA_TRY(cudaMemsetAsync(L->flags + 1, 0, sizeof(int32_t) * 3, s));
   bool fused = true;
   if (const char* e = getenv("MST_UPDATE_FUSED")) fused = (e[0] != '0');
   int grid_blocks = 0;
   size_t fused_smem = 0;
+  const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
   if (fused) {
-    int dev = 0, coop = 0, sms = 0, occ = 0;
-    const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, FUSED_THREADS, 0) != cudaSuccess || !coop || occ < 1)
-      fused = false;
+    grid_blocks = fused_grid_limit(fn);
+    if (grid_blocks == 0) fused = false;
     else {
-      if (occ > 2) occ = 2;
-      grid_blocks = sms * occ;
       const int64_t useful = (L->nwords + FUSED_WARPS - 1) / FUSED_WARPS;  // at least one word per warp
       if (grid_blocks > useful) grid_blocks = (int)(useful < 1 ? 1 : useful);
       // two alternating partial-sum areas of grid_blocks entries each (the buffer carries 1024 spare entries)
@@ -856,68 +1395,104 @@ extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, c
     MST_CUDA_TRY(cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * BINS, s));
     if (!mst_use_tensor_path(L)) MST_TRY(mst_alloc_csc(L));   // the kernel fills the view's arrays for such layers
     FusedParams F;
-    F.sel = P;
-    F.n_prune = n_prune; F.n_grad = n_grad; F.n_rand = n_rand;
-    F.pruned_bits = L->pruned_bits; F.grad_bits = L->grad_bits; F.rand_bits = L->rand_bits; F.new_bits = L->bits[n];
-    F.cnt = L->word_cnt; F.scan = L->word_scan; F.bsums = L->block_sums;
-    F.hist = L->hist; F.flags = L->flags;
-    F.new_wscan = L->wscan[n]; F.new_row_ptr = L->row_ptr[n]; F.new_col = L->col_idx[n]; F.new_vals = L->vals[n];
-    F.bitsT = L->bitsT; F.wscanT = L->wscanT; F.col_ptr = L->col_ptr; F.row_idx = L->row_idx; F.perm = L->perm;
-    F.wpc = L->wpc; F.nwordsT = L->nwordsT;
-    F.build_csc = mst_use_tensor_path(L) ? 0 : 1;
+    fill_fused_params(pl, F);
     L->csc_valid = F.build_csc;
     void* args[] = {&F};
-    const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
-    // cooperative launch that may also start while its predecessor drains (the kernel waits before its first access)
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid_blocks);
-    cfg.blockDim = dim3(FUSED_THREADS);
-    cfg.dynamicSmemBytes = fused_smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeCooperative;
-    attr[0].val.cooperative = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = mst_pdl_enabled() ? 2 : 1;
-    MST_CUDA_TRY(cudaLaunchKernelExC(&cfg, fn, args));
-    MST_COUNT_LAUNCH();
+    MST_TRY(launch_cooperative(fn, args, grid_blocks, fused_smem, s));
   } else {
-    MST_TRY(run_select<MODE_PRUNE>(L, P, n_prune, L->pruned_bits, s));
-    MST_TRY(run_select<MODE_GRAD>(L, P, n_grad, L->grad_bits, s));
-    MST_TRY(run_select<MODE_RAND>(L, P, n_rand, L->rand_bits, s));
-    MST_TRY(mst_combine_update_bits(L, n, s));
-    MST_TRY(mst_rebuild_from_bits(L, n, nullptr, 0, c, s));
+    MST_TRY(run_select<MODE_PRUNE>(L, P, pl.n_prune, L->pruned_bits, s));
+    MST_TRY(run_select<MODE_GRAD>(L, P, pl.n_grad, L->grad_bits, s));
+    MST_TRY(run_select<MODE_RAND>(L, P, pl.n_rand, L->rand_bits, s));
+    MST_TRY(mst_combine_update_bits(L, pl.n, s));
+    MST_TRY(mst_rebuild_from_bits(L, pl.n, nullptr, 0, pl.c, s));
   }
-  const int64_t nnz_before = L->nnz;
-  if (stats) {
-    // the fused kernel records the longest row itself only when it also builds the CSC view
-    if (!fused || !L->csc_valid) { max_row_nnz<<<(L->O + 255) / 256, 256, 0, s>>>(L->row_ptr[n], L->O, L->flags); MST_COUNT_LAUNCH(); }
-    int32_t f[4] = {0, 0, 0, 0};
-    int32_t total = 0;
-    MST_CUDA_TRY(cudaMemcpyAsync(f, L->flags, sizeof(f), cudaMemcpyDeviceToHost, s));
-    MST_CUDA_TRY(cudaMemcpyAsync(&total, L->wscan[n] + L->nwords, sizeof(int32_t), cudaMemcpyDeviceToHost, s));
-    MST_CUDA_TRY(cudaStreamSynchronize(s));
-    stats->nnz_before = nnz_before;
-    stats->nnz_after = total;
-    stats->n_prune = n_prune;
-    stats->n_grad = n_grad;
-    stats->n_rand = n_rand;
-    stats->max_row_nnz = f[1];
-    const bool bad = (f[0] & (MST_FLAG_NONFINITE | MST_FLAG_CORRUPT)) || total != target;
-    if (bad) {
-      // A rejected update is not applied: the structure built in the other buffer set is dropped and the layer keeps
-      // its mask, values and nnz.  The CSC arrays may hold the rejected structure, so the view is rebuilt on next use.
-      L->csc_valid = 0;
-      MST_CUDA_TRY(cudaMemsetAsync(L->flags, 0, sizeof(int32_t), s));  // reported: cleared
-      stats->nnz_after = nnz_before;
-      return (f[0] & MST_FLAG_NONFINITE) ? MST_ERR_NONFINITE : MST_ERR_CORRUPT;
+  *fused_out = fused;
+  return MST_OK;
+}
+
+}  // namespace
+
+extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, const mst_regrow_rule_t* rule,
+                                            const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  UpdatePlan pl;
+  MST_TRY(plan_update(L, prune_frac, rule, G_dense, &pl));
+  bool fused = false;
+  MST_TRY(launch_single_update(pl, s, &fused));
+  return finish_update(pl, fused, stats, s);
+}
+
+extern "C" mst_status_t mst_topology_update_many(int32_t n_layers, mst_layer_t* const* layers, const double* prune_frac,
+                                                 const mst_regrow_rule_t* rules, const float* const* G_dense,
+                                                 mst_update_stats_t* stats, mst_stream_t stream) {
+  if (n_layers < 0 || (n_layers > 0 && (!layers || !prune_frac || !rules || !G_dense))) return MST_ERR_INVALID_ARG;
+  if (n_layers == 0) return MST_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  // every layer is validated before anything is launched: an argument error leaves all layers untouched
+  UpdatePlan* plans = new (std::nothrow) UpdatePlan[n_layers];
+  char* mode = new (std::nothrow) char[n_layers];   // 0: not launched yet, 1: batched, 2: single fused, 3: kernel per phase
+  if (!plans || !mode) { delete[] plans; delete[] mode; return MST_ERR_INVALID_ARG; }
+  mst_status_t st = MST_OK;
+  for (int i = 0; i < n_layers && st == MST_OK; ++i) {
+    st = plan_update(layers[i], prune_frac[i], &rules[i], G_dense[i], &plans[i]);
+    mode[i] = 0;
+    for (int j = 0; j < i && st == MST_OK; ++j)
+      if (layers[j] == layers[i]) st = MST_ERR_INVALID_ARG;   // a layer may appear once
+  }
+  const int grid_limit = st == MST_OK ? fused_grid_limit((const void*)mg_update_batch_kernel) : 0;
+  bool batching = grid_limit > 0;
+  if (const char* e = getenv("MST_UPDATE_BATCH")) batching = batching && (e[0] != '0');
+  int i = 0;
+  while (st == MST_OK && i < n_layers) {
+    // collect the next run of layers that can share a launch: tensor-path layers (no CSC view to build) whose slices
+    // fit shared memory together and whose scan scratch holds two partial-sum areas of the grid
+    BatchParams B;
+    B.n = 0;
+    size_t words = 0;
+    int first = i;
+    while (batching && i < n_layers && B.n < BATCH_MAX) {
+      mst_layer* L = plans[i].L;
+      const size_t per = (size_t)((L->nwords + grid_limit - 1) / grid_limit);
+      const bool ok = mst_use_tensor_path(L) && 2 * (int64_t)grid_limit <= mst_scan_block_sums_len(L->nwords) + 1024 &&
+                      (words + 3 * per) * 4 <= 40 * 1024;
+      if (!ok) break;
+      B.smem_off[B.n] = (int)words;
+      words += 3 * per;
+      fill_fused_params(plans[i], B.L[B.n]);
+      B.L[B.n].build_csc = 0;
+      ++B.n;
+      ++i;
+    }
+    if (B.n >= 2) {
+      for (int j = first; j < i && st == MST_OK; ++j) {
+        mst_layer* L = plans[j].L;
+        if (cudaMemsetAsync(L->flags + 1, 0, sizeof(int32_t) * 3, s) != cudaSuccess ||
+            cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * BINS, s) != cudaSuccess)
+          st = MST_ERR_CUDA;
+        L->csc_valid = 0;
+        mode[j] = 1;
+      }
+      if (st == MST_OK) {
+        void* args[] = {&B};
+        st = launch_cooperative((const void*)mg_update_batch_kernel, args, grid_limit, words * 4, s);
+      }
+    } else {
+      // a run of one (or a layer that cannot be batched): the single-layer path
+      i = first;
+      bool fused = false;
+      st = launch_single_update(plans[i], s, &fused);
+      mode[i] = fused ? 2 : 3;
+      ++i;
     }
   }
-  L->cur = n;
-  L->nnz = target;
-  ++L->version;
-  if (!fused) MST_TRY(mst_build_csc(L, s));
-  return MST_OK;
+  // host epilogues in order; the first failure is reported, later layers are still finished so that no layer is left
+  // with kernels enqueued but its buffer sets not flipped
+  for (int j = 0; j < n_layers; ++j) {
+    if (mode[j] == 0) continue;
+    const mst_status_t fj = finish_update(plans[j], mode[j] != 3, stats ? &stats[j] : nullptr, s);
+    if (st == MST_OK) st = fj;
+  }
+  delete[] plans;
+  delete[] mode;
+  return st;
 }

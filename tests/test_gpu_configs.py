@@ -204,3 +204,30 @@ def test_lm_head_shape_large_out_features():
     _update_and_compare(L, p, W, p.mask.copy(), host(G), 0.3, 0.25, 11, 0)
     L.close()
     assert mst.mst_device_error_flags() == 0
+
+
+def test_config3_block_updated_in_one_call():
+    # the four layers of an ultra-sparse block (Zipf rows) updated together, every step, against the oracle
+    probs = mst_inputs.config3(blocks=1, first_block=3)
+    layers = [make_layer(p) for p in probs]
+    rng = np.random.default_rng(33)
+    Ws = [np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32) for p in probs]
+    Ms = [p.mask.copy() for p in probs]
+    Gh = [rng.normal(size=p.mask.shape).astype(np.float32) for p in probs]
+    Gd = [torch.from_numpy(g).to(dev()) for g in Gh]
+    for step in range(3):
+        rules = [mst.RegrowRule(-1, 0.25, 77, step, 0, 0.0) for _ in probs]
+        stats = mst.mst_topology_update_many([L.handle for L in layers], [0.1] * 4, rules, Gd)
+        for j, (p, L, st) in enumerate(zip(probs, layers, stats)):
+            n_prune, _, n_rand, n_grad = oracle.mg_counts(0.1, int(Ms[j].sum()), -1, Ms[j].size, 0.25)
+            assert (st.n_prune, st.n_rand, st.n_grad) == (n_prune, n_rand, n_grad)
+            Ws[j], Ms[j], *_ = oracle.mg_update(Ws[j], Ms[j], Gh[j], n_prune, n_grad, n_rand, 77, step, p.layer_id)
+            rp, ci, vb = export_csr(L, p.dtype)
+            rp_r, ci_r, v_r = oracle.to_csr(Ws[j], Ms[j])
+            np.testing.assert_array_equal(rp, rp_r)
+            np.testing.assert_array_equal(ci, ci_r)
+            np.testing.assert_array_equal(vb, value_bits(v_r, p.dtype))
+    for L in layers:
+        L.validate()
+        L.close()
+    assert mst.mst_device_error_flags() == 0

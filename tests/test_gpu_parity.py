@@ -554,3 +554,49 @@ def test_path_in_use_reports_the_resolved_path():
     L = make_layer(q)
     assert L.path_in_use() == mst.MST_PATH_CUDA_CORE             # fp32 layers never leave the CUDA cores
     L.close()
+
+
+# ------------------------------------------------------------ several layers updated in one call
+def test_update_many_is_bit_identical_to_single_updates():
+    shapes = [(96, 160, "bf16", 0.2), (130, 257, "bf16", 0.1), (64, 64, "f32", 0.3), (200, 96, "bf16", 0.05),
+              (300, 200, "bf16", 0.5)]
+    probs = [_problem(O, I, 4, dt, d, 700 + k) for k, (O, I, dt, d) in enumerate(shapes)]
+    rng = np.random.default_rng(12)
+    Gs = [np.round(rng.normal(size=(p.out_features, p.in_features)) * 4).astype(np.float32) / 4 for p in probs]   # many equal |g|
+    Gd = [torch.from_numpy(g).to(dev()) for g in Gs]
+    A = [make_layer(p) for p in probs]      # updated one by one
+    Bm = [make_layer(p) for p in probs]     # updated together
+    # growth, shrinkage, pure pruning (ties among the zeros grown before), R = 0 and R = 1
+    plan = [(0.3, None, 0.25), (0.2, 0.9, 0.0), (0.1, 1.2, 1.0), (0.5, None, 0.5), (0.0, 0.5, 0.25), (0.3, None, 0.25)]
+    for step, (zeta, scale, R) in enumerate(plan):
+        targets = [-1 if scale is None else min(p.mask.size, max(0, int(L.nnz * scale))) for p, L in zip(probs, A)]
+        for L, t, g in zip(A, targets, Gd):
+            mst.mst_topology_update(L.handle, zeta, t, R, 21, step, False, g)
+        rules = [mst.RegrowRule(int(t), float(R), 21, step, 0, 0.0) for t in targets]
+        stats = mst.mst_topology_update_many([L.handle for L in Bm], [zeta] * len(Bm), rules, Gd)
+        for p, La, Lb, st in zip(probs, A, Bm, stats):
+            assert La.nnz == Lb.nnz == st.nnz_after
+            for x, y in zip(export_csr(La, p.dtype), export_csr(Lb, p.dtype)):
+                np.testing.assert_array_equal(x, y)
+            Lb.validate()
+    assert mst.mst_device_error_flags() == 0
+    for L in A + Bm:
+        L.close()
+
+
+def test_update_many_checks_every_layer_first():
+    p = _problem(64, 96, 4, "bf16", 0.2, 31)
+    L1, L2 = make_layer(p), make_layer(p)
+    n1, n2 = L1.nnz, L2.nnz
+    G = torch.zeros((64, 96), dtype=torch.float32, device=dev())
+    rules = [mst.RegrowRule(-1, 0.25, 1, 0, 0, 0.0), mst.RegrowRule(64 * 96 + 1, 0.25, 1, 0, 0, 0.0)]   # second: infeasible target
+    with pytest.raises(mst.MstError) as e:
+        mst.mst_topology_update_many([L1.handle, L2.handle], [0.3, 0.3], rules, [G, G])
+    assert e.value.status == 5
+    before = export_csr(L1, "bf16")
+    assert (L1.nnz, L2.nnz) == (n1, n2)
+    with pytest.raises(mst.MstError):            # the same layer twice
+        mst.mst_topology_update_many([L1.handle, L1.handle], [0.3, 0.3], [rules[0], rules[0]], [G, G])
+    for x, y in zip(before, export_csr(L1, "bf16")):
+        np.testing.assert_array_equal(x, y)
+    L1.close(); L2.close()
