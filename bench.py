@@ -408,7 +408,7 @@ def run_profile_case(args) -> None:
         torch.cuda.synchronize()
         return
     O, I, T = 5120, 1280, 8192                       # fc1 of GPT-2 large, half the sweep's tokens
-    density = {"dense_tiles": 0.1, "sparse_tc": 0.02, "cuda_core": 0.1, "update": 0.1}[case]
+    density = {"dense_tiles": 0.1, "sparse_tc": 0.02, "sparse_tc_cycles": 0.02, "cuda_core": 0.1, "update": 0.1}[case]
     nnz = mst_inputs.exact_nnz(O, I, density)
     Wd = (torch.randn(O, I, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
     mask = torch.from_numpy(mst_inputs.uniform_mask(O, I, nnz, mst_inputs.BASE_SEED + 5, 2)).to(dev)
@@ -433,6 +433,26 @@ def run_profile_case(args) -> None:
         return
     L = mst.Layer(2, O, I, mst.MST_BF16)
     L.pack(Wd, mask)
+    if case == "sparse_tc_cycles":
+        # needs a library built with MST_NVCC_EXTRA=-DMST_SP_PROFILE (python paper_2408_11746_b200/csrc/build.py --force):
+        # per-role cycle counters of the structured-sparse kernel's last launch, mean over the blocks of each parity
+        import ctypes
+        lib = ctypes.CDLL(os.path.join(ROOT, "paper_2408_11746_b200", "libmst.so"))
+        if not hasattr(lib, "mst_sp24_profile"):
+            raise SystemExit("libmst.so was built without -DMST_SP_PROFILE")
+        L.set_path(mst.MST_PATH_SPARSE_TC)
+        names = ["producer waits for a free stage", "MMA thread waits for a full stage", "MMA thread waits for a free accumulator",
+                 "epilogue warp waits for a complete accumulator", "epilogue warp busy", "whole kernel"]
+        for label, fn in (("forward (K = 1280)", lambda: L.fwd(X, Y, T)), ("input gradient (K = 5120)", lambda: L.bwd_x(dY, dX, T))):
+            for _ in range(3):
+                fn()
+            buf = (ctypes.c_longlong * (148 * 8))()
+            assert lib.mst_sp24_profile(buf, 148) == 0
+            a = np.array(buf[:]).reshape(148, 8)
+            print(json.dumps({"call": label, "tokens": T, "density": density, "cycles_even_block_mean":
+                              {n: float(a[0::2, j].mean()) for j, n in enumerate(names)},
+                              "cycles_odd_block_mean": {n: float(a[1::2, j].mean()) for j, n in enumerate(names)}}))
+        return
     L.set_path({"dense_tiles": mst.MST_PATH_TENSOR_CORE, "sparse_tc": mst.MST_PATH_SPARSE_TC,
                 "cuda_core": mst.MST_PATH_CUDA_CORE}[case])
     for _ in range(3):
@@ -514,7 +534,7 @@ def main() -> None:
     ap.add_argument("--sweep-reps", type=int, default=50)
     ap.add_argument("--sweep", default=None, choices=["medium", "large", "small"],
                     help="density sweep report alone (not the bench line)")
-    ap.add_argument("--profile-case", default=None, choices=["dense_tiles", "sparse_tc", "cuda_core", "update", "attention_bwd"],
+    ap.add_argument("--profile-case", default=None, choices=["dense_tiles", "sparse_tc", "sparse_tc_cycles", "cuda_core", "update", "attention_bwd"],
                     help="run a few launches of one kernel family on a small case (for ncu; prints nothing)")
     ap.add_argument("--attention", action="store_true",
                     help="report on the strided sparse attention forward (not the bench line): one JSON object per "

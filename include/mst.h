@@ -240,12 +240,12 @@ mst_status_t mst_topology_update(mst_layer_t* layer, double prune_frac, const ms
                                  const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream);
 
 /* The same update for several layers in one call (in training all layers are updated on the same step): identical
- * results, bit for bit, to calling mst_topology_update on each layer in turn, but the layers' selection passes share
- * their grid-wide barriers inside one cooperative launch (up to 8 layers per launch), which is where a single update
- * spends most of its time.  prune_frac[i], rules[i], G_dense[i] belong to layers[i]; stats is NULL or an array of
- * n_layers entries (same meaning as above, the call then synchronises once per layer).  A layer may appear once.
- * All arguments are validated before anything is launched.  Layers that cannot join a batch (fp32 or CUDA-core
- * layers, which also rebuild their CSC view; very large layers) are updated by the single-layer kernels.
+ * results, bit for bit, to calling mst_topology_update on each layer in turn.  prune_frac[i], rules[i], G_dense[i]
+ * belong to layers[i]; stats is NULL or an array of n_layers entries (same meaning as above, the call then
+ * synchronises once per layer).  A layer may appear once.  All arguments are validated before anything is launched.
+ * With MST_UPDATE_BATCH=1 in the environment up to 8 tensor-path layers share one cooperative launch and its grid-wide
+ * barriers; measured slower than one launch per layer on GPT-2 shapes (the shared launch cannot keep the layers'
+ * keys on chip between passes), so it is off by default.
  * Returns the first error met; layers before and after it are still completed. */
 mst_status_t mst_topology_update_many(int32_t n_layers, mst_layer_t* const* layers, const double* prune_frac,
                                       const mst_regrow_rule_t* rules, const float* const* G_dense,

@@ -60,6 +60,23 @@ __device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat1
   }
 }
 
+// the same copy issued asynchronously (cp.async, 16 bytes per request); complete after async_wait_all + a barrier
+__device__ __forceinline__ void load_tile_async(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int64_t r0) {
+  for (int e = threadIdx.x; e < TS * D / 8; e += BW_THREADS) {
+    const int r = e >> 3, c = (e & 7) * 8;
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + r * LDB + c);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + (r0 + r) * ld + c) : "memory");
+  }
+}
+__device__ __forceinline__ void load_floats_async(float* dst, const float* src, int n) {
+  for (int e = threadIdx.x; e < n; e += BW_THREADS) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + e);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(src + e) : "memory");
+  }
+}
+__device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 __global__ void attn_delta_kernel(BwdParams P) {
   const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;   // (token, head)
   const int lane = threadIdx.x & 31;
@@ -119,9 +136,8 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dq_kernel(BwdParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem);   // [64][LDB]
   __nv_bfloat16* Gs = Qs + TS * LDB;                             // dOut tile
-  __nv_bfloat16* Ks = Gs + TS * LDB;
-  __nv_bfloat16* Vs = Ks + TS * LDB;
-  __nv_bfloat16* Sb = Vs + TS * LDB;                             // dS, bf16
+  __nv_bfloat16* KV = Gs + TS * LDB;                             // two (K tile, V tile) buffers: the next pair is fetched
+  __nv_bfloat16* Sb = KV + 4 * TS * LDB;                         //   while the current one is used
   float* Sf = reinterpret_cast<float*>(Sb + TS * LDB);           // scores, later dQ   [64][LDF]
   float* Pf = Sf + TS * LDF;                                     // dP
   __shared__ float lse_s[TS], del_s[TS];
@@ -142,11 +158,20 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dq_kernel(BwdParams P) {
   for (int nb = 0; nb < 4; ++nb) wmma::fill_fragment(acc[nb], 0.f);
   const int r_base = warp * 16;
   const int k_first = q0 - l > 0 ? q0 - l : 0;
-  for (int k0 = k_first; k0 <= q0; k0 += TS) {
-    __syncthreads();   // the previous key tile has been consumed (first trip: the query tiles are in place)
-    load_tile(Ks, P.K + h * D, P.ld, row0 + k0);
-    load_tile(Vs, P.V + h * D, P.ld, row0 + k0);
-    __syncthreads();
+  load_tile_async(KV, P.K + h * D, P.ld, row0 + k_first);
+  load_tile_async(KV + TS * LDB, P.V + h * D, P.ld, row0 + k_first);
+  async_commit();
+  int buf = 0;
+  for (int k0 = k_first; k0 <= q0; k0 += TS, buf ^= 1) {
+    async_wait_all();
+    __syncthreads();   // this tile has landed for everyone; the other buffer's tile has been consumed
+    const __nv_bfloat16* Ks = KV + buf * 2 * TS * LDB;
+    const __nv_bfloat16* Vs = Ks + TS * LDB;
+    if (k0 + TS <= q0) {
+      load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB, P.K + h * D, P.ld, row0 + k0 + TS);
+      load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB + TS * LDB, P.V + h * D, P.ld, row0 + k0 + TS);
+      async_commit();
+    }
     strip_abt(Sf + r_base * LDF, Qs + r_base * LDB, Ks);
     strip_abt(Pf + r_base * LDF, Gs + r_base * LDB, Vs);
     __syncwarp();
@@ -194,13 +219,12 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dkv_kernel(BwdParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem);
   __nv_bfloat16* Vs = Ks + TS * LDB;
-  __nv_bfloat16* Qs = Vs + TS * LDB;
-  __nv_bfloat16* Gs = Qs + TS * LDB;
-  __nv_bfloat16* Pb = Gs + TS * LDB;                             // P^T, bf16   [key][query]
+  __nv_bfloat16* QG = Vs + TS * LDB;                             // two (Q tile, dOut tile) buffers
+  __nv_bfloat16* Pb = QG + 4 * TS * LDB;                         // P^T, bf16   [key][query]
   __nv_bfloat16* Sb = Pb + TS * LDB;                             // dS^T, bf16
   float* Sf = reinterpret_cast<float*>(Sb + TS * LDB);           // S^T, later dK
   float* Pf = Sf + TS * LDF;                                     // dP^T, later dV
-  __shared__ float lse_s[TS], del_s[TS];
+  __shared__ float stat_s[2][2 * TS];   // per buffer: log-sum-exp and delta of the tile's queries
 
   const int kt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int k0 = kt * TS, l = P.stride;
@@ -217,15 +241,23 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dkv_kernel(BwdParams P) {
   }
   const int r_base = warp * 16;   // this warp's keys
   const int q_last = k0 + l < P.seq - TS ? k0 + l : P.seq - TS;
-  for (int q0 = k0; q0 <= q_last; q0 += TS) {
-    __syncthreads();
-    load_tile(Qs, P.Q + h * D, P.ld, row0 + q0);
-    load_tile(Gs, P.dOut + h * D, P.lddo, row0 + q0);
-    if (threadIdx.x < TS) {
-      lse_s[threadIdx.x] = P.lse[stat0 + q0 + threadIdx.x];
-      del_s[threadIdx.x] = P.delta[stat0 + q0 + threadIdx.x];
-    }
-    __syncthreads();
+  auto fetch = [&](int q0, int bf) {
+    load_tile_async(QG + bf * 2 * TS * LDB, P.Q + h * D, P.ld, row0 + q0);
+    load_tile_async(QG + bf * 2 * TS * LDB + TS * LDB, P.dOut + h * D, P.lddo, row0 + q0);
+    load_floats_async(stat_s[bf], P.lse + stat0 + q0, TS);
+    load_floats_async(stat_s[bf] + TS, P.delta + stat0 + q0, TS);
+    async_commit();
+  };
+  fetch(k0, 0);
+  int buf = 0;
+  for (int q0 = k0; q0 <= q_last; q0 += TS, buf ^= 1) {
+    async_wait_all();
+    __syncthreads();   // this query tile has landed for everyone (first trip: also K and V); the other buffer is free
+    const __nv_bfloat16* Qs = QG + buf * 2 * TS * LDB;
+    const __nv_bfloat16* Gs = Qs + TS * LDB;
+    const float* lse_s = stat_s[buf];
+    const float* del_s = stat_s[buf] + TS;
+    if (q0 + TS <= q_last) fetch(q0 + TS, buf ^ 1);
     strip_abt(Sf + r_base * LDF, Ks + r_base * LDB, Qs);   // S^T[key][query]
     strip_abt(Pf + r_base * LDF, Vs + r_base * LDB, Gs);   // dP^T[key][query]
     __syncwarp();
@@ -309,8 +341,8 @@ extern "C" mst_status_t mst_strided_attention_bwd(const void* Q, const void* K, 
   P.batch = batch; P.seq = seq_len; P.heads = heads; P.stride = stride;
   const int64_t warps = (int64_t)batch * seq_len * heads;
   attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, s>>>(P); MST_COUNT_LAUNCH();
-  const size_t smem_q = (size_t)(5 * TS * LDB) * 2 + (size_t)2 * TS * LDF * 4 + 128;
-  const size_t smem_kv = (size_t)(6 * TS * LDB) * 2 + (size_t)2 * TS * LDF * 4 + 128;
+  const size_t smem_q = (size_t)(7 * TS * LDB) * 2 + (size_t)2 * TS * LDF * 4 + 128;
+  const size_t smem_kv = (size_t)(8 * TS * LDB) * 2 + (size_t)2 * TS * LDF * 4 + 128;
   MST_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_q));
   MST_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv));
   dim3 grid((unsigned)(seq_len / TS), (unsigned)heads, (unsigned)batch);

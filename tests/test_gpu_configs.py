@@ -206,7 +206,9 @@ def test_lm_head_shape_large_out_features():
     assert mst.mst_device_error_flags() == 0
 
 
-def test_config3_block_updated_in_one_call():
+@pytest.mark.parametrize("shared_launch", ["0", "1"])
+def test_config3_block_updated_in_one_call(shared_launch, monkeypatch):
+    monkeypatch.setenv("MST_UPDATE_BATCH", shared_launch)
     # the four layers of an ultra-sparse block (Zipf rows) updated together, every step, against the oracle
     probs = mst_inputs.config3(blocks=1, first_block=3)
     layers = [make_layer(p) for p in probs]

@@ -557,7 +557,9 @@ def test_path_in_use_reports_the_resolved_path():
 
 
 # ------------------------------------------------------------ several layers updated in one call
-def test_update_many_is_bit_identical_to_single_updates():
+@pytest.mark.parametrize("shared_launch", ["0", "1"])
+def test_update_many_is_bit_identical_to_single_updates(shared_launch, monkeypatch):
+    monkeypatch.setenv("MST_UPDATE_BATCH", shared_launch)      # read by the library at every call
     shapes = [(96, 160, "bf16", 0.2), (130, 257, "bf16", 0.1), (64, 64, "f32", 0.3), (200, 96, "bf16", 0.05),
               (300, 200, "bf16", 0.5)]
     probs = [_problem(O, I, 4, dt, d, 700 + k) for k, (O, I, dt, d) in enumerate(shapes)]
