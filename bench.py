@@ -415,7 +415,7 @@ def run_profile_case(args) -> None:
         torch.cuda.synchronize()
         return
     O, I, T = 5120, 1280, 8192                       # fc1 of GPT-2 large, half the sweep's tokens
-    density = {"dense_tiles": 0.1, "sparse_tc": 0.02, "sparse_tc_cycles": 0.02, "cuda_core": 0.1, "update": 0.1}[case]
+    density = {"dense_tiles": 0.1, "sparse_tc": 0.02, "sparse_tc_cycles": 0.02, "cuda_core": 0.1, "update": 0.1, "update_phases": 0.1}[case]
     nnz = mst_inputs.exact_nnz(O, I, density)
     Wd = (torch.randn(O, I, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
     mask = torch.from_numpy(mst_inputs.uniform_mask(O, I, nnz, mst_inputs.BASE_SEED + 5, 2)).to(dev)
@@ -425,6 +425,37 @@ def run_profile_case(args) -> None:
     dX = torch.empty(T, I, device=dev, dtype=torch.bfloat16)
     dW = torch.empty(nnz, device=dev, dtype=torch.float32)
     G = torch.empty(O, I, device=dev, dtype=torch.float32)
+    if case == "update_phases":
+        # needs a library built with MST_NVCC_EXTRA=-DMST_UPD_PROFILE (python paper_2408_11746_b200/csrc/build.py --force):
+        # SM-clock stamps of block 0 at the phase boundaries of the last fused update kernel
+        import ctypes
+        lib = ctypes.CDLL(os.path.join(ROOT, "paper_2408_11746_b200", "libmst.so"))
+        if not hasattr(lib, "mst_update_profile"):
+            raise SystemExit("libmst.so was built without -DMST_UPD_PROFILE")
+        names = {2: "slice loaded", 4: "hash test of the inactive entries", 3: "keys and first histogram", 40: "tie ranking",
+                 41: "marking sweep", 42: "bracket list + barrier", 43: "threshold among the listed", 44: "random marks + new mask",
+                 49: "-", 51: "-", 52: "scan of the new mask (barrier inside)", 53: "CSR fill", 54: "scratch cleared",
+                 60: "prune selection (sequential form)", 61: "gradient selection (sequential form)", 62: "random selection (general form)"}
+        for p in range(3):
+            names[10 + p] = "histogram sweep %d" % p
+            names[20 + p] = "flush + barrier %d" % p
+            names[30 + p] = "digit picks %d" % p
+        O, I = 4096, 1024                                # fc1 of GPT-2 medium
+        nnz = mst_inputs.exact_nnz(O, I, 0.1)
+        Wd = (torch.randn(O, I, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+        mask = torch.from_numpy(mst_inputs.uniform_mask(O, I, nnz, mst_inputs.BASE_SEED + 5, 2)).to(dev)
+        L = mst.Layer(2, O, I, mst.MST_BF16)
+        L.pack(Wd, mask)
+        G = torch.randn(O, I, device=dev, generator=gen)
+        for k in range(4):
+            L.update(0.3, target_nnz=-1, random_ratio=0.25, seed=6, step=k, G_dense=G, want_stats=False)
+        buf = (ctypes.c_longlong * 64)()
+        n = lib.mst_update_profile(buf, 32)
+        a = np.array(buf[:2 * n]).reshape(n, 2)
+        print(json.dumps({"layer": "fc1 of GPT-2 medium (4096 x 1024), d = 0.1, zeta = 0.3, R = 0.25", "unit": "SM cycles, block 0",
+                          "phases": [[names.get(int(a[i, 0]), str(int(a[i, 0]))), int(a[i, 1] - a[i - 1, 1])] for i in range(1, n)],
+                          "total": int(a[-1, 1] - a[0, 1])}))
+        return
     if case == "update":
         layers = []
         for li in range(4):
@@ -543,7 +574,7 @@ def main() -> None:
                     help="density sweep report alone (not the bench line)")
     ap.add_argument("--sweep-path", default="auto", choices=["auto", "cuda_core", "dense_tiles", "sparse_tc"],
                     help="with --sweep: force one kernel family instead of the automatic choice")
-    ap.add_argument("--profile-case", default=None, choices=["dense_tiles", "sparse_tc", "sparse_tc_cycles", "cuda_core", "update", "attention_bwd"],
+    ap.add_argument("--profile-case", default=None, choices=["dense_tiles", "sparse_tc", "sparse_tc_cycles", "cuda_core", "update", "update_phases", "attention_bwd"],
                     help="run a few launches of one kernel family on a small case (for ncu; prints nothing)")
     ap.add_argument("--attention", action="store_true",
                     help="report on the strided sparse attention forward (not the bench line): one JSON object per "

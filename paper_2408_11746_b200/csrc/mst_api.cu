@@ -89,7 +89,12 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   const size_t o_cnt = cv.take(4 * (size_t)(wmax + 1));
   const size_t o_scan = cv.take(4 * (size_t)(wmax + 1));
   const size_t o_bsum = cv.take(4 * (size_t)(mst_scan_block_sums_len(wmax) + 1024));
-  const size_t o_hist = cv.take(4 * (size_t)MST_SELECT_BINS * 3);
+  const size_t o_hist = cv.take(4 * (size_t)MST_SELECT_BINS * 2 * 3);
+  int64_t rand_cap = N / 64;
+  if (rand_cap < 1024) rand_cap = 1024;
+  if (rand_cap > 32768) rand_cap = 32768;
+  const size_t o_rlist = cv.take(16 * (size_t)rand_cap);
+  const size_t o_rctr = cv.take(16);
   const size_t o_sel = cv.take(sizeof(mst_select_state));
   const size_t o_flags = cv.take(4 * 4);
   const size_t o_counter = cv.take(4);
@@ -124,6 +129,10 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->word_scan = (int32_t*)(base + o_scan);
   L->block_sums = (int32_t*)(base + o_bsum);
   L->hist = (unsigned int*)(base + o_hist);
+  L->rand_list = (unsigned long long*)(base + o_rlist);
+  L->rand_ctr = (unsigned long long*)(base + o_rctr);
+  L->rand_cap = (int)rand_cap;
+  L->scratch_clean = 1;   // the allocation was cleared above
   L->sel = (mst_select_state*)(base + o_sel);
   L->flags = (int32_t*)(base + o_flags);
   L->counter = (unsigned int*)(base + o_counter);

@@ -32,7 +32,8 @@ using namespace nvcuda;
 
 constexpr int D = 64;        // head dimension
 constexpr int TS = 64;       // tile side (queries and keys)
-constexpr int BW_THREADS = 128;
+constexpr int BW_THREADS = 256;
+constexpr int BW_WARPS = BW_THREADS / 32;
 constexpr int LDB = 72;      // row pitch of the bf16 tiles in shared memory (64 + 8: rows 144 bytes apart, no bank aliasing)
 constexpr int LDF = 68;      // row pitch of the fp32 tiles
 constexpr float SCALE = 0.125f;   // 1 / sqrt(64)
@@ -98,34 +99,40 @@ typedef wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::col_majo
 typedef wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::row_major> FragB;    // B given as [k][n] rows
 typedef wmma::fragment<wmma::accumulator, 16, 16, 16, float> FragC;
 
-// out strip [16 x 64] (fp32, ld 64) = A strip [16 x 64] * B^T, B stored as 64 rows of 64 (row n holds B^T's column n)
-__device__ __forceinline__ void strip_abt(float* out, const __nv_bfloat16* a_strip, const __nv_bfloat16* b_rows) {
+// Eight warps per block: warp = (strip of 16 rows, half of the 64 columns).  A warp forms its 16 x 32 part of the two
+// score-shaped products, applies the softmax algebra to it, and after a block barrier accumulates its 16 x 32 part of
+// the gradient tiles from the complete 16 x 64 strip of weights.
+
+// out [16 x 32] (fp32, pitch LDF) = A strip [16 x 64] * B^T for 32 of B's rows (row n of b_rows holds B^T's column n)
+__device__ __forceinline__ void half_abt(float* out, const __nv_bfloat16* a_strip, const __nv_bfloat16* b_rows) {
+  FragA a[4];
 #pragma unroll
-  for (int nb = 0; nb < 4; ++nb) {
+  for (int kb = 0; kb < 4; ++kb) wmma::load_matrix_sync(a[kb], a_strip + kb * 16, LDB);
+#pragma unroll
+  for (int nb = 0; nb < 2; ++nb) {
     FragC c;
     wmma::fill_fragment(c, 0.f);
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) {
-      FragA a;
       FragBt b;
-      wmma::load_matrix_sync(a, a_strip + kb * 16, LDB);
       wmma::load_matrix_sync(b, b_rows + nb * 16 * LDB + kb * 16, LDB);
-      wmma::mma_sync(c, a, b, c);
+      wmma::mma_sync(c, a[kb], b, c);
     }
     wmma::store_matrix_sync(out + nb * 16, c, LDF, wmma::mem_row_major);
   }
 }
 
-// acc[4] (a 16 x 64 strip of fp32 fragments) += A strip [16 x 64] (bf16, ld 64) * B [64 x 64] (bf16 rows)
-__device__ __forceinline__ void strip_ab_acc(FragC (&acc)[4], const __nv_bfloat16* a_strip, const __nv_bfloat16* b_rows) {
+// acc[2] (16 x 32, fp32 fragments) += A strip [16 x 64] (bf16) * 32 columns of B [64 x 64] (bf16 rows; b_cols points
+// at the first of the 32 columns)
+__device__ __forceinline__ void half_ab_acc(FragC (&acc)[2], const __nv_bfloat16* a_strip, const __nv_bfloat16* b_cols) {
 #pragma unroll
   for (int kb = 0; kb < 4; ++kb) {
     FragA a;
     wmma::load_matrix_sync(a, a_strip + kb * 16, LDB);
 #pragma unroll
-    for (int nb = 0; nb < 4; ++nb) {
+    for (int nb = 0; nb < 2; ++nb) {
       FragB b;
-      wmma::load_matrix_sync(b, b_rows + kb * 16 * LDB + nb * 16, LDB);
+      wmma::load_matrix_sync(b, b_cols + kb * 16 * LDB + nb * 16, LDB);
       wmma::mma_sync(acc[nb], a, b, acc[nb]);
     }
   }
@@ -153,10 +160,10 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dq_kernel(BwdParams P) {
     lse_s[threadIdx.x] = P.lse[stat0 + q0 + threadIdx.x];
     del_s[threadIdx.x] = P.delta[stat0 + q0 + threadIdx.x];
   }
-  FragC acc[4];
+  FragC acc[2];
 #pragma unroll
-  for (int nb = 0; nb < 4; ++nb) wmma::fill_fragment(acc[nb], 0.f);
-  const int r_base = warp * 16;
+  for (int nb = 0; nb < 2; ++nb) wmma::fill_fragment(acc[nb], 0.f);
+  const int r_base = (warp & 3) * 16, c_base = (warp >> 2) * 32;
   const int k_first = q0 - l > 0 ? q0 - l : 0;
   load_tile_async(KV, P.K + h * D, P.ld, row0 + k_first);
   load_tile_async(KV + TS * LDB, P.V + h * D, P.ld, row0 + k_first);
@@ -164,7 +171,7 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dq_kernel(BwdParams P) {
   int buf = 0;
   for (int k0 = k_first; k0 <= q0; k0 += TS, buf ^= 1) {
     async_wait_all();
-    __syncthreads();   // this tile has landed for everyone; the other buffer's tile has been consumed
+    __syncthreads();   // this tile has landed for everyone; the other buffer's tile and the weights have been consumed
     const __nv_bfloat16* Ks = KV + buf * 2 * TS * LDB;
     const __nv_bfloat16* Vs = Ks + TS * LDB;
     if (k0 + TS <= q0) {
@@ -172,27 +179,32 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dq_kernel(BwdParams P) {
       load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB + TS * LDB, P.V + h * D, P.ld, row0 + k0 + TS);
       async_commit();
     }
-    strip_abt(Sf + r_base * LDF, Qs + r_base * LDB, Ks);
-    strip_abt(Pf + r_base * LDF, Gs + r_base * LDB, Vs);
+    half_abt(Sf + r_base * LDF + c_base, Qs + r_base * LDB, Ks + c_base * LDB);
+    half_abt(Pf + r_base * LDF + c_base, Gs + r_base * LDB, Vs + c_base * LDB);
     __syncwarp();
-    for (int e = lane; e < 16 * TS; e += 32) {
-      const int r = r_base + (e >> 6), c = e & 63;
+    // the visited key tiles lie within l + 64 positions behind the queries: a pair is kept iff 0 <= i - j <= l
+    // (the window, and the first strided position i - l)
+    const int d0 = q0 - k0;
+    for (int e = lane; e < 16 * 32; e += 32) {
+      const int r = r_base + (e >> 5), c = c_base + (e & 31);
+      const int back = d0 + r - c;
       float ds = 0.f;
-      if (attends(q0 + r, k0 + c, l)) {
+      if (back >= 0 && back <= l) {
         const float p = __expf(Sf[r * LDF + c] * SCALE - lse_s[r]);
         ds = p * (Pf[r * LDF + c] - del_s[r]);
       }
       Sb[r * LDB + c] = __float2bfloat16(ds);
     }
-    __syncwarp();
-    strip_ab_acc(acc, Sb + r_base * LDB, Ks);
+    __syncthreads();   // the strip of weights is complete (both column halves)
+    half_ab_acc(acc, Sb + r_base * LDB, Ks + c_base);
   }
-  __syncwarp();
+  __syncthreads();     // every warp has read its scores: the array takes dQ now
 #pragma unroll
-  for (int nb = 0; nb < 4; ++nb) wmma::store_matrix_sync(Sf + r_base * LDF + nb * 16, acc[nb], LDF, wmma::mem_row_major);
-  __syncwarp();
+  for (int nb = 0; nb < 2; ++nb)
+    wmma::store_matrix_sync(Sf + r_base * LDF + c_base + nb * 16, acc[nb], LDF, wmma::mem_row_major);
+  __syncthreads();
   // strided keys beyond the tiles: i - 2l, i - 3l, ...   (lane = two head dimensions)
-  for (int r = r_base; r < r_base + 16; ++r) {
+  for (int r = warp * (TS / BW_WARPS); r < (warp + 1) * (TS / BW_WARPS); ++r) {
     const int i = q0 + r;
     const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Qs + r * LDB + 2 * lane));
     const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Gs + r * LDB + 2 * lane));
@@ -233,13 +245,13 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dkv_kernel(BwdParams P) {
   const int64_t stat0 = ((int64_t)b * P.heads + h) * P.seq;
   load_tile(Ks, P.K + h * D, P.ld, row0 + k0);
   load_tile(Vs, P.V + h * D, P.ld, row0 + k0);
-  FragC acc_k[4], acc_v[4];
+  FragC acc_k[2], acc_v[2];
 #pragma unroll
-  for (int nb = 0; nb < 4; ++nb) {
+  for (int nb = 0; nb < 2; ++nb) {
     wmma::fill_fragment(acc_k[nb], 0.f);
     wmma::fill_fragment(acc_v[nb], 0.f);
   }
-  const int r_base = warp * 16;   // this warp's keys
+  const int r_base = (warp & 3) * 16, c_base = (warp >> 2) * 32;   // this warp's keys, and its half of the columns
   const int q_last = k0 + l < P.seq - TS ? k0 + l : P.seq - TS;
   auto fetch = [&](int q0, int bf) {
     load_tile_async(QG + bf * 2 * TS * LDB, P.Q + h * D, P.ld, row0 + q0);
@@ -252,38 +264,41 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dkv_kernel(BwdParams P) {
   int buf = 0;
   for (int q0 = k0; q0 <= q_last; q0 += TS, buf ^= 1) {
     async_wait_all();
-    __syncthreads();   // this query tile has landed for everyone (first trip: also K and V); the other buffer is free
+    __syncthreads();   // this query tile has landed for everyone (first trip: also K and V); the other buffer and the
+                       // weights of the previous tile have been consumed
     const __nv_bfloat16* Qs = QG + buf * 2 * TS * LDB;
     const __nv_bfloat16* Gs = Qs + TS * LDB;
     const float* lse_s = stat_s[buf];
     const float* del_s = stat_s[buf] + TS;
     if (q0 + TS <= q_last) fetch(q0 + TS, buf ^ 1);
-    strip_abt(Sf + r_base * LDF, Ks + r_base * LDB, Qs);   // S^T[key][query]
-    strip_abt(Pf + r_base * LDF, Vs + r_base * LDB, Gs);   // dP^T[key][query]
+    half_abt(Sf + r_base * LDF + c_base, Ks + r_base * LDB, Qs + c_base * LDB);   // S^T[key][query]
+    half_abt(Pf + r_base * LDF + c_base, Vs + r_base * LDB, Gs + c_base * LDB);   // dP^T[key][query]
     __syncwarp();
-    for (int e = lane; e < 16 * TS; e += 32) {
-      const int r = r_base + (e >> 6), c = e & 63;      // key r, query c
+    const int d0 = q0 - k0;   // the visited query tiles lie within l + 64 positions ahead: kept iff 0 <= i - j <= l
+    for (int e = lane; e < 16 * 32; e += 32) {
+      const int r = r_base + (e >> 5), c = c_base + (e & 31);      // key r, query c
+      const int back = d0 + c - r;
       float p = 0.f, ds = 0.f;
-      if (attends(q0 + c, k0 + r, l)) {
+      if (back >= 0 && back <= l) {
         p = __expf(Sf[r * LDF + c] * SCALE - lse_s[c]);
         ds = p * (Pf[r * LDF + c] - del_s[c]);
       }
       Pb[r * LDB + c] = __float2bfloat16(p);
       Sb[r * LDB + c] = __float2bfloat16(ds);
     }
-    __syncwarp();
-    strip_ab_acc(acc_v, Pb + r_base * LDB, Gs);
-    strip_ab_acc(acc_k, Sb + r_base * LDB, Qs);
+    __syncthreads();   // the strips of weights are complete (both query halves)
+    half_ab_acc(acc_v, Pb + r_base * LDB, Gs + c_base);
+    half_ab_acc(acc_k, Sb + r_base * LDB, Qs + c_base);
   }
-  __syncwarp();
+  __syncthreads();     // every warp has read its scores: the arrays take dK and dV now
 #pragma unroll
-  for (int nb = 0; nb < 4; ++nb) {
-    wmma::store_matrix_sync(Sf + r_base * LDF + nb * 16, acc_k[nb], LDF, wmma::mem_row_major);
-    wmma::store_matrix_sync(Pf + r_base * LDF + nb * 16, acc_v[nb], LDF, wmma::mem_row_major);
+  for (int nb = 0; nb < 2; ++nb) {
+    wmma::store_matrix_sync(Sf + r_base * LDF + c_base + nb * 16, acc_k[nb], LDF, wmma::mem_row_major);
+    wmma::store_matrix_sync(Pf + r_base * LDF + c_base + nb * 16, acc_v[nb], LDF, wmma::mem_row_major);
   }
-  __syncwarp();
+  __syncthreads();
   // queries further on that see this key through the stride: j + 2l, j + 3l, ...
-  for (int r = r_base; r < r_base + 16; ++r) {
+  for (int r = warp * (TS / BW_WARPS); r < (warp + 1) * (TS / BW_WARPS); ++r) {
     const int j = k0 + r;
     const float2 k = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Ks + r * LDB + 2 * lane));
     const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Vs + r * LDB + 2 * lane));

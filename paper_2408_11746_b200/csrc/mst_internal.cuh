@@ -125,7 +125,11 @@ struct mst_layer {
   int32_t* word_cnt;      // [max(nwords, nwordsT)+1]
   int32_t* word_scan;     // [max(nwords, nwordsT)+1]
   int32_t* block_sums;    // scan partials
-  unsigned int* hist;     // [3][MST_SELECT_BINS]: rotating global histograms of the radix select
+  unsigned int* hist;     // [3][2 * MST_SELECT_BINS]: rotating global histograms of the radix select (two selections side by side)
+  unsigned long long* rand_list;  // [rand_cap][2]: hash key and flat index of the random-growth candidates inside the bracket
+  unsigned long long* rand_ctr;   // [2]: candidates below the bracket, list length
+  int rand_cap;
+  int scratch_clean;      // hist and rand_ctr are known to be zero (the fused update kernel leaves them so)
   mst_select_state* sel;  // [1]
   int32_t* flags;         // [4]: error bits, max row nnz, spare
   unsigned int* counter;  // [1] block-completion counter

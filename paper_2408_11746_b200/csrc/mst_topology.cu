@@ -9,10 +9,17 @@
 // mst_structure.cu.  Integer keys, integer atomics only: the outcome is deterministic and bit-exact.
 //
 // Work layout: one warp per 32-bit mask word, lane = column inside the word, so reads of G and of the value array are
-// coalesced.  The last block to finish a histogram pass picks the digit (completion counter, no waiting).  The tie
-// ranking (count, scan) is skipped on the device when the threshold key has no surplus ties.
+// coalesced.  Three forms, all with the same results:
+//  - kernel per phase (run_select): the last block to finish a histogram pass picks the digit;
+//  - one cooperative kernel, one selection after the other (fused_select);
+//  - one cooperative kernel with the prune and the gradient selection side by side and the random growth by bracket
+//    (fused_dual_update), the default whenever just-pruned links may not be regrown: keys of a block's slice in
+//    shared memory, gradients copied there asynchronously, work on the few active entries of a word done by one
+//    thread per word, the random threshold found among the few candidates whose hash falls into a precomputed bracket.
+// The tie ranking (count, scan) is skipped on the device when the threshold key has no surplus ties.
 #include <cooperative_groups.h>
 
+#include <cmath>
 #include <cstdlib>
 #include <new>
 
@@ -323,6 +330,25 @@ mst_status_t run_select(mst_layer* L, const SelParams& P, int64_t k, uint32_t* o
 // (three rotating histogram buffers: the one for pass p+2 is cleared after the barrier of pass p).
 namespace cg = cooperative_groups;
 
+#ifdef MST_UPD_PROFILE
+// phase stamps of block 0 of the last fused update (SM clock), read back through mst_update_profile
+__device__ long long g_upd_stamps[64];
+__device__ int g_upd_nstamps;
+#define UPD_STAMP(id)                                                      \
+  do {                                                                     \
+    if (blockIdx.x == 0 && threadIdx.x == 0) {                             \
+      const int at_ = g_upd_nstamps;                                       \
+      if (at_ < 31) {                                                      \
+        g_upd_stamps[2 * at_] = (id);                                      \
+        g_upd_stamps[2 * at_ + 1] = clock64();                             \
+        g_upd_nstamps = at_ + 1;                                           \
+      }                                                                    \
+    }                                                                      \
+  } while (0)
+#else
+#define UPD_STAMP(id) do { } while (0)
+#endif
+
 constexpr int FUSED_THREADS = 512;
 constexpr int FUSED_WARPS = FUSED_THREADS / 32;
 constexpr int FUSED_BPT = BINS / FUSED_THREADS;  // histogram bins per thread in the pick
@@ -332,7 +358,7 @@ struct FusedParams {
   long long n_prune, n_grad, n_rand;
   uint32_t *pruned_bits, *grad_bits, *rand_bits, *new_bits;
   int32_t *cnt, *scan, *bsums;
-  unsigned int* hist;  // [3][BINS], all zero at launch
+  unsigned int* hist;  // [3][HSTRIDE], all zero at launch and again at exit
   int32_t* flags;
   int32_t *new_wscan, *new_row_ptr;
   uint16_t* new_col;
@@ -345,15 +371,33 @@ struct FusedParams {
   int64_t nwordsT;
   int build_csc;  // 0: leave the CSC view stale (the layer's input gradient reads the dense image instead)
   int smem_keys;  // 1: the launch carries shared memory for the key cache (slices too large for the registers)
+  int dual;       // 1: prune and gradient selections run side by side (their candidate sets are disjoint)
+  int g_bulk;     // 1: a slice's gradients are one contiguous, 16-byte aligned run (mask words tile the flat index space)
+  // random growth by bracket: hash keys are uniform, so the n_rand-th smallest lies in [rand_lo, rand_hi) with
+  // overwhelming probability; the candidates inside are listed and the threshold is found among them
+  int rand_bracket;
+  int rand_cap;                    // entries the list holds
+  unsigned long long rand_lo, rand_hi;
+  unsigned long long* rand_list;   // [rand_cap][2]: key, flat index
+  unsigned long long* rand_ctr;    // [2]: candidates below rand_lo, list length; zero at launch and again at exit
 };
 
+constexpr int HSTRIDE = 2 * BINS;   // one rotating histogram buffer: two selections side by side
 struct FusedShared {
-  unsigned int hist[BINS];
+  unsigned int hist[BINS];   // side-by-side selections count in the two 16-bit halves of a bin (a slice has < 65536 entries)
   unsigned int warp_tot[FUSED_WARPS];
   int red[FUSED_WARPS];
   unsigned long long prefix, tau;
   long long k, rem;
   int need_rank, done, found;
+  // two selections side by side (0: prune, 1: gradient growth)
+  uint32_t d_prefix[2], d_tau[2];
+  long long d_k[2], d_rem[2];
+  int d_need_rank[2], d_done[2], d_found[2];
+  // random growth by bracket
+  unsigned long long r_tau, r_tau_f;
+  long long r_rank;
+  int r_ok, r_bin, r_n;
 };
 
 __device__ __forceinline__ int fused_block_sum(int v, FusedShared& sh) {
@@ -517,7 +561,7 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     const int hi_shift = shift + width;
     const K prefix = (K)sh.prefix;
     const long long k = sh.k;
-    unsigned int* gh = F.hist + (gpass % 3) * BINS;
+    unsigned int* gh = F.hist + (gpass % 3) * HSTRIDE;
     for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
     __syncthreads();
     bool saw_nonfinite = cache_nonfinite;
@@ -589,8 +633,8 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
       tsum += mine[j];
     }
     if (blockIdx.x == 0) {  // clear the buffer of pass gpass + 2 (last read before this barrier)
-      unsigned int* gz = F.hist + ((gpass + 2) % 3) * BINS;
-      for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) gz[b] = 0;
+      unsigned int* gz = F.hist + ((gpass + 2) % 3) * HSTRIDE;
+      for (int b = threadIdx.x; b < HSTRIDE; b += FUSED_THREADS) gz[b] = 0;
     }
     unsigned int incl = tsum;
     for (int o = 1; o < 32; o <<= 1) {
@@ -775,6 +819,594 @@ __device__ void fused_select(const FusedParams& F, long long k_total, uint32_t* 
     }
   }
   __syncthreads();
+  UPD_STAMP(60 + MODE);
+}
+
+// ---------------------------------------------------------------------------------- two selections side by side
+// Under the default reading of the candidate sets the prune selection looks only at active entries and the gradient
+// selection only at inactive ones, so every entry carries exactly one 32-bit key and the two radix selects can share
+// their sweeps and their barriers: pass p of both runs in one sweep into two histograms, both digits are picked behind
+// one barrier, and one marking sweep writes both bit masks.
+
+// columns of mask word w that exist (the last word of a row is ragged when I is not a multiple of 32)
+__device__ __forceinline__ uint32_t word_valid_mask(const SelParams& P, int64_t w) {
+  if (P.aligned) return 0xFFFFFFFFu;
+  const unsigned wu = (unsigned)w, wpr = (unsigned)P.wpr;
+  const int c0 = (int)(wu % wpr) * 32;
+  const int nv = P.I - c0;
+  return nv >= 32 ? 0xFFFFFFFFu : ((1u << nv) - 1u);
+}
+
+__device__ __forceinline__ long long word_flat_index(const SelParams& P, int64_t w, int lane) {
+  if (P.aligned) return (long long)w * 32 + lane;
+  const unsigned wu = (unsigned)w, wpr = (unsigned)P.wpr;
+  const int o = (int)(wu / wpr), c = (int)(wu - (unsigned)o * wpr) * 32 + lane;
+  return (long long)o * P.I + c;
+}
+
+// digit picks of the two selections from their complete histograms gh[0..BINS) and gh[BINS..2 BINS) (every block, same
+// result); `todo` bit s: selection s still runs
+__device__ void dual_pick(FusedShared& sh, unsigned todo, const unsigned int* gh, int shift, int width, int low_zero_a,
+                          int32_t* flags) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned int mine[2][FUSED_BPT];
+  unsigned int tsum[2] = {0u, 0u}, incl[2];
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+#pragma unroll
+    for (int j = 0; j < FUSED_BPT; ++j) {
+      mine[s][j] = ((todo >> s) & 1u) ? __ldcg(gh + s * BINS + threadIdx.x * FUSED_BPT + j) : 0u;
+      tsum[s] += mine[s][j];
+    }
+  }
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+    incl[s] = tsum[s];
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int y = __shfl_up_sync(0xffffffffu, incl[s], o);
+      if (lane >= o) incl[s] += y;
+    }
+  }
+  const uint32_t prefix[2] = {sh.d_prefix[0], sh.d_prefix[1]};
+  const long long k[2] = {sh.d_k[0], sh.d_k[1]};
+  __syncthreads();  // the totals' arrays are free, every thread has read the selection state
+  if (threadIdx.x < 2) sh.d_found[threadIdx.x] = 0;
+  if (lane == 31) {
+    sh.warp_tot[warp] = incl[0];
+    sh.red[warp] = (int)incl[1];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int s = 0; s < 2; ++s) {
+    if (!((todo >> s) & 1u)) continue;  // uniform
+    unsigned int before = incl[s] - tsum[s];
+    for (int wv = 0; wv < warp; ++wv) before += s ? (unsigned int)sh.red[wv] : sh.warp_tot[wv];
+    const bool owner = (long long)before < k[s] && k[s] <= (long long)before + (long long)tsum[s];
+    if (owner) {
+      long long cum = before;
+      int bin = 0;
+      unsigned int bcount = 0;
+      for (int j = 0; j < FUSED_BPT; ++j) {
+        if (cum + (long long)mine[s][j] >= k[s]) { bin = j; bcount = mine[s][j]; break; }
+        cum += mine[s][j];
+      }
+      const uint32_t np = (width < 32 ? (prefix[s] << width) : 0u) | (uint32_t)(threadIdx.x * FUSED_BPT + bin);
+      sh.d_prefix[s] = np;
+      sh.d_k[s] = k[s] - cum;
+      sh.d_found[s] = 1;
+      if (shift == 0) {
+        sh.d_tau[s] = np;
+        sh.d_rem[s] = k[s] - cum;
+        sh.d_need_rank[s] = ((long long)bcount > k[s] - cum) ? 1 : 0;
+        sh.d_done[s] = 1;
+      } else if ((long long)bcount == k[s] - cum) {
+        sh.d_tau[s] = (np << shift) | ((1u << shift) - 1u);
+        sh.d_rem[s] = k[s] - cum;
+        sh.d_need_rank[s] = 0;
+        sh.d_done[s] = 1;
+      } else if (s == 0 && shift <= low_zero_a) {
+        // the undecided low bits are zero in every prune key: the bucket is one run of equal keys
+        sh.d_tau[s] = np << shift;
+        sh.d_rem[s] = k[s] - cum;
+        sh.d_need_rank[s] = 1;
+        sh.d_done[s] = 1;
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < 2 && ((todo >> threadIdx.x) & 1u) && !sh.d_found[threadIdx.x]) {
+    // fewer candidates than requested (ruled out by the host counts): take everything
+    const int s = threadIdx.x;
+    sh.d_tau[s] = 0xFFFFFFFFu;
+    sh.d_rem[s] = 0x7FFFFFFFFFFFFFFFLL;
+    sh.d_need_rank[s] = 0;
+    sh.d_done[s] = 1;
+    if (blockIdx.x == 0) atomicOr(&flags[0], MST_FLAG_CORRUPT);
+  }
+  __syncthreads();
+}
+
+// Shared-memory arrays of a block's slice in the side-by-side form of the update (one entry per mask word, keys one
+// per entry).
+struct DualSlice {
+  uint32_t* old;   // mask words before the update
+  int32_t* base;   // their exclusive popcount scan (position of a word's first entry in the value array)
+  uint32_t* grad;  // entries grown by gradient
+  uint32_t* prn;   // entries pruned
+  uint32_t* hc;    // random growth: inactive entries whose hash can still be below the bracket's upper end
+  uint32_t* key;   // [words][32] the 32-bit key of every entry
+};
+
+__device__ __forceinline__ unsigned long long entry_hash(const SelParams& P, long long f) {
+  return sm64_mix(P.stream + SM64_GAMMA * ((unsigned long long)f + 1ULL));
+}
+
+// Prune and gradient selections side by side over keys kept in shared memory, random growth by bracket, mask rewrite.
+// Sweeps over the slice: (0) keys, first histogram pass and the hash test of every inactive entry; (1, 2) the later
+// histogram passes; (3) marking of pruned and gradient-grown entries, then one thread per word lists the random
+// candidates inside the bracket; (4) behind the bracket's barrier, one thread per word marks the randomly grown
+// entries and writes the new mask word.  Returns false (uniform over the grid) when the random growth still has to
+// be done by the general radix select (no bracket, or the bracket missed); the new mask is not written then.
+__device__ bool fused_dual_update(const FusedParams& F, int64_t lo, int nloc, int& gpass, int& gscan, cg::grid_group& grid,
+                                  FusedShared& sh, const DualSlice& S) {
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool wantA = F.n_prune > 0, wantB = F.n_grad > 0;
+  const bool wantR = F.rand_bracket && F.n_rand > 0;
+  const bool aligned = P.aligned != 0;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) {
+      sh.d_prefix[s] = 0;
+      sh.d_k[s] = s ? F.n_grad : F.n_prune;
+      sh.d_tau[s] = 0;
+      sh.d_rem[s] = 0;
+      sh.d_need_rank[s] = 0;
+      sh.d_done[s] = (s ? wantB : wantA) ? 0 : 1;
+    }
+  }
+  for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
+  __syncthreads();
+  // ---- sweep 0
+  {
+    const uint32_t rhi_hi = (uint32_t)(F.rand_hi >> 32);
+    const bool lam = P.lambda != 0.f;
+    bool saw_nonfinite = false;
+    const bool bulk = F.g_bulk && wantB;   // uniform over the grid
+    if (bulk) {
+      // mask words tile the flat index space: the slice's gradients are one contiguous run, copied asynchronously
+      // into the key array while the hashes below are computed
+      const float* src = P.G + lo * 32;
+      const uint32_t dst = (uint32_t)__cvta_generic_to_shared(S.key);
+      for (int i = threadIdx.x; i < nloc * 8; i += FUSED_THREADS)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i), "l"(src + 4 * (size_t)i) : "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    // random growth: which inactive entries have a hash whose high word does not exceed the bracket's upper end
+    if (wantR && aligned) {
+      // flat index (lo + li) * 32 + lane: the generator's argument advances by a constant from one of this warp's
+      // words to the next
+      unsigned long long z = P.stream + SM64_GAMMA * ((unsigned long long)(lo + warp) * 32ULL + (unsigned long long)lane + 1ULL);
+      constexpr unsigned long long ZSTEP = SM64_GAMMA * 32ULL * (unsigned long long)FUSED_WARPS;
+#pragma unroll 4
+      for (int li = warp; li < nloc; li += FUSED_WARPS) {
+        const bool act = (S.old[li] >> lane) & 1u;
+        const bool h_ok = !act && (uint32_t)(sm64_mix(z) >> 32) <= rhi_hi;
+        z += ZSTEP;
+        const unsigned hm = __ballot_sync(0xffffffffu, h_ok);
+        if (lane == 0) S.hc[li] = hm;
+      }
+    } else if (wantR) {
+#pragma unroll 4
+      for (int li = warp; li < nloc; li += FUSED_WARPS) {
+        const bool act = (S.old[li] >> lane) & 1u;
+        const bool valid = (word_valid_mask(P, lo + li) >> lane) & 1u;
+        bool h_ok = false;
+        if (!act && valid) h_ok = (uint32_t)(entry_hash(P, word_flat_index(P, lo + li, lane)) >> 32) <= rhi_hi;
+        const unsigned hm = __ballot_sync(0xffffffffu, h_ok);
+        if (lane == 0) S.hc[li] = hm;
+      }
+    } else {
+      for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) S.hc[li] = 0u;
+    }
+    UPD_STAMP(4);
+    if (bulk) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncthreads();
+    }
+    // gradient keys of the inactive entries, lane per entry (the active entries' slots are written below)
+    if (wantB) {
+      constexpr int GB = 4;  // words per trip, loads first
+      for (int l0 = warp; l0 < nloc; l0 += FUSED_WARPS * GB) {
+        uint32_t kk[GB], ow[GB];
+#pragma unroll
+        for (int j = 0; j < GB; ++j) {
+          const int li = l0 + j * FUSED_WARPS;
+          kk[j] = 0u;
+          ow[j] = 0xFFFFFFFFu;
+          if (li < nloc) {  // uniform over the warp
+            ow[j] = S.old[li];
+            const bool c = !((ow[j] >> lane) & 1u) && (aligned || ((word_valid_mask(P, lo + li) >> lane) & 1u));
+            if (bulk) kk[j] = S.key[li * 32 + lane] & 0x7FFFFFFFu;
+            else if (c) kk[j] = __float_as_uint(P.G[word_flat_index(P, lo + li, lane)]) & 0x7FFFFFFFu;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < GB; ++j) {
+          const int li = l0 + j * FUSED_WARPS;
+          if (li >= nloc) break;  // uniform over the warp
+          const bool c = !((ow[j] >> lane) & 1u) && (aligned || ((word_valid_mask(P, lo + li) >> lane) & 1u));
+          const uint32_t key = 0xFFFFFFFFu - kk[j];  // largest magnitude first
+          if (c) {
+            saw_nonfinite |= kk[j] >= 0x7F800000u;
+            atomicAdd(&sh.hist[key >> pass_shift(32, 0)], 0x10000u);
+          }
+          S.key[li * 32 + lane] = key;
+        }
+      }
+      __syncthreads();  // the active entries' slots are rewritten by other threads below
+    }
+    // prune keys of the active entries, one thread per word
+    if (wantA) {
+      for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) {
+        uint32_t m = S.old[li];
+        int32_t pos = S.base[li];
+        while (m) {
+          const int b = __ffs(m) - 1;
+          m &= m - 1;
+          uint32_t k = (P.bf16 ? (uint32_t)((const uint16_t*)P.vals)[pos] << 16 : ((const uint32_t*)P.vals)[pos]) & 0x7FFFFFFFu;
+          ++pos;
+          if (lam) {  // MEST criterion, fp32 with one rounding per operation (never contracted to an FMA)
+            const float g = fabsf(P.G[word_flat_index(P, lo + li, b)]);
+            k = __float_as_uint(__fadd_rn(__uint_as_float(k), __fmul_rn(P.lambda, g))) & 0x7FFFFFFFu;
+          }
+          saw_nonfinite |= k >= 0x7F800000u;
+          S.key[li * 32 + b] = k;
+          atomicAdd(&sh.hist[k >> pass_shift(32, 0)], 1u);
+        }
+      }
+    }
+    if (saw_nonfinite) atomicOr(&F.flags[0], MST_FLAG_NONFINITE);
+  }
+  UPD_STAMP(3);
+  // ---- histogram passes (the first one was filled by sweep 0)
+  constexpr int passes = num_passes(32);
+  for (int pass = 0; pass < passes; ++pass) {
+    const bool doneA = sh.d_done[0] != 0, doneB = sh.d_done[1] != 0;
+    if (doneA && doneB) break;  // same decision in every block
+    const int shift = pass_shift(32, pass), width = pass_width(32, pass);
+    unsigned int* gh = F.hist + (gpass % 3) * HSTRIDE;
+    if (pass > 0) {
+      const unsigned dmask = (1u << width) - 1u;
+      const int hi_shift = shift + width;
+      const uint32_t prefA = sh.d_prefix[0], prefB = sh.d_prefix[1];
+      const bool liveA = wantA && !doneA, liveB = wantB && !doneB;
+      __syncthreads();  // every thread has read the selection state
+      for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
+      __syncthreads();
+      constexpr int PB = 4;  // words per trip: the shared-memory atomics would otherwise keep the next loads behind them
+      for (int l0 = warp; l0 < nloc; l0 += FUSED_WARPS * PB) {
+        uint32_t key[PB], ow[PB];
+#pragma unroll
+        for (int j = 0; j < PB; ++j) {
+          const int li = l0 + j * FUSED_WARPS;
+          const bool ok = li < nloc;  // uniform over the warp
+          key[j] = ok ? S.key[li * 32 + lane] : 0u;
+          ow[j] = ok ? S.old[li] : 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < PB; ++j) {
+          const int li = l0 + j * FUSED_WARPS;
+          if (li >= nloc) break;  // uniform over the warp
+          const bool act = (ow[j] >> lane) & 1u;
+          const bool valid = aligned || ((word_valid_mask(P, lo + li) >> lane) & 1u);
+          const bool lv = (act ? liveA : (liveB && valid)) && (key[j] >> hi_shift) == (act ? prefA : prefB);
+          if (lv) atomicAdd(&sh.hist[(key[j] >> shift) & dmask], act ? 1u : 0x10000u);
+        }
+      }
+    }
+    __syncthreads();
+    UPD_STAMP(10 + pass);
+    for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) {
+      const unsigned int v = sh.hist[b];
+      if (v & 0xFFFFu) atomicAdd(&gh[b], v & 0xFFFFu);
+      if (v >> 16) atomicAdd(&gh[BINS + b], v >> 16);
+    }
+    grid.sync();
+    UPD_STAMP(20 + pass);
+    dual_pick(sh, (doneA ? 0u : 1u) | (doneB ? 0u : 2u), gh, shift, width, P.low_zero, F.flags);
+    if (blockIdx.x == 0) {  // clear the buffer of pass gpass + 2 (last read before this barrier)
+      unsigned int* gz = F.hist + ((gpass + 2) % 3) * HSTRIDE;
+      for (int b = threadIdx.x; b < HSTRIDE; b += FUSED_THREADS) gz[b] = 0;
+    }
+    __syncthreads();
+    UPD_STAMP(30 + pass);
+    ++gpass;
+  }
+  const uint32_t tauA = sh.d_tau[0], tauB = sh.d_tau[1];
+  const long long remA = sh.d_rem[0], remB = sh.d_rem[1];
+  const bool rankA = sh.d_need_rank[0] != 0, rankB = sh.d_need_rank[1] != 0;
+  // tie ranking in index order, one scan per selection that needs it (the second into the array of the new mask's
+  // scan, which is not written before the mask rewrite)
+  for (int s = 0; s < 2; ++s) {
+    if (!(s ? rankB : rankA)) continue;  // uniform over the grid
+    const uint32_t tau = s ? tauB : tauA;
+    for (int li = warp; li < nloc; li += FUSED_WARPS) {
+      const bool act = (S.old[li] >> lane) & 1u;
+      const bool valid = aligned || ((word_valid_mask(P, lo + li) >> lane) & 1u);
+      const bool c = s ? (!act && valid) : act;
+      const unsigned eq = __ballot_sync(0xffffffffu, c && S.key[li * 32 + lane] == tau);
+      if (lane == 0) F.cnt[lo + li] = __popc(eq);
+    }
+    __syncthreads();
+    fused_grid_scan(F.cnt, s ? F.new_wscan : F.scan, P.nwords, lo, lo + nloc, F.bsums, gscan, grid, sh);
+  }
+  UPD_STAMP(40);
+  // ---- sweep 3: marking
+  if (!rankA && !rankB) {
+    // no tie has to be ranked: an entry is taken when its key does not exceed its selection's threshold
+    const uint32_t enA = wantA ? 0xFFFFFFFFu : 0u, enB = wantB ? 0xFFFFFFFFu : 0u;
+    constexpr int MB = 4;  // words per trip, loads first
+    for (int l0 = warp; l0 < nloc; l0 += FUSED_WARPS * MB) {
+      uint32_t key[MB], ow[MB];
+#pragma unroll
+      for (int j = 0; j < MB; ++j) {
+        const int li = l0 + j * FUSED_WARPS;
+        const bool ok = li < nloc;  // uniform over the warp
+        key[j] = ok ? S.key[li * 32 + lane] : 0u;
+        ow[j] = ok ? S.old[li] : 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < MB; ++j) {
+        const int li = l0 + j * FUSED_WARPS;
+        if (li >= nloc) break;  // uniform over the warp
+        const bool act = (ow[j] >> lane) & 1u;
+        const unsigned all = __ballot_sync(0xffffffffu, key[j] <= (act ? tauA : tauB));
+        if (lane == 0) {
+          S.prn[li] = all & ow[j] & enA;
+          S.grad[li] = all & ~ow[j] & enB & (aligned ? 0xFFFFFFFFu : word_valid_mask(P, lo + li));
+        }
+      }
+    }
+  } else
+  for (int li = warp; li < nloc; li += FUSED_WARPS) {
+    const uint32_t key = S.key[li * 32 + lane];
+    const bool act = (S.old[li] >> lane) & 1u;
+    const bool valid = aligned || ((word_valid_mask(P, lo + li) >> lane) & 1u);
+    bool takeA = wantA && act && key < tauA, takeB = wantB && !act && valid && key < tauB;
+    const bool eqA = wantA && act && key == tauA, eqB = wantB && !act && valid && key == tauB;
+    if (rankA) {  // uniform
+      const unsigned m = __ballot_sync(0xffffffffu, eqA);
+      takeA |= eqA && (long long)F.scan[lo + li] + __popc(m & lanemask_lt()) < remA;
+    } else {
+      takeA |= eqA;
+    }
+    if (rankB) {
+      const unsigned m = __ballot_sync(0xffffffffu, eqB);
+      takeB |= eqB && (long long)F.new_wscan[lo + li] + __popc(m & lanemask_lt()) < remB;
+    } else {
+      takeB |= eqB;
+    }
+    const unsigned bA = __ballot_sync(0xffffffffu, takeA), bB = __ballot_sync(0xffffffffu, takeB);
+    if (lane == 0) {
+      S.prn[li] = bA;
+      S.grad[li] = bB;
+    }
+  }
+  __syncthreads();
+  UPD_STAMP(41);
+  if (!wantR && F.n_rand > 0) return false;  // uniform over the grid: no bracket was planned
+  if (wantR) {
+    // one thread per word: the remaining candidates whose hash lies below the bracket are counted, those inside
+    // listed (counted first, so that a block reserves its part of the list with one atomic)
+    unsigned long long below_lo = 0;
+    int n_in = 0;
+    for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) {
+      uint32_t m = S.hc[li] & ~S.grad[li], keep = 0;
+      while (m) {
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        const unsigned long long h = entry_hash(P, word_flat_index(P, lo + li, b));
+        if (h < F.rand_lo) {
+          ++below_lo;
+          keep |= 1u << b;
+        } else if (h < F.rand_hi) {
+          ++n_in;
+          keep |= 1u << b;
+        }
+      }
+      S.hc[li] = keep;  // what can still be taken
+    }
+    int blk_in = 0;
+    const int my_at = fused_block_excl_scan(n_in, blk_in, sh);
+    __syncthreads();
+    if (threadIdx.x == 0) sh.r_tau = blk_in ? atomicAdd(&F.rand_ctr[1], (unsigned long long)blk_in) : 0ULL;
+    __syncthreads();
+    if (n_in) {
+      unsigned long long at = sh.r_tau + (unsigned long long)my_at;
+      for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) {
+        uint32_t m = S.hc[li];
+        while (m) {
+          const int b = __ffs(m) - 1;
+          m &= m - 1;
+          const long long f = word_flat_index(P, lo + li, b);
+          const unsigned long long h = entry_hash(P, f);
+          if (h >= F.rand_lo) {
+            if (at < (unsigned long long)F.rand_cap) {
+              F.rand_list[2 * at] = h;
+              F.rand_list[2 * at + 1] = (unsigned long long)f;
+            }
+            ++at;
+          }
+        }
+      }
+    }
+    for (int o = 16; o; o >>= 1) below_lo += __shfl_xor_sync(0xffffffffu, below_lo, o);
+    if (lane == 0 && below_lo) atomicAdd(&F.rand_ctr[0], below_lo);
+    grid.sync();
+    UPD_STAMP(42);
+    const unsigned long long c_lo = __ldcg(&F.rand_ctr[0]), n_list = __ldcg(&F.rand_ctr[1]);
+    const unsigned long long k = (unsigned long long)F.n_rand;
+    if (!(c_lo < k && k <= c_lo + n_list && n_list <= (unsigned long long)F.rand_cap)) return false;  // uniform over the grid
+    const int n = (int)n_list;
+    const long long r = (long long)(k - c_lo);  // 1-based rank inside the list
+    const unsigned long long range = F.rand_hi - F.rand_lo;
+    // bin of a key: (key - lo) >> bshift, below BINS because range >> bshift < BINS
+    const int bshift = (range >> RADIX_BITS) ? 64 - RADIX_BITS - __clzll((long long)range) : 0;
+    __syncthreads();
+    for (int b = threadIdx.x; b < BINS; b += FUSED_THREADS) sh.hist[b] = 0;
+    if (threadIdx.x == 0) { sh.r_ok = 0; sh.r_n = 0; }
+    __syncthreads();
+    // the keys of the selections are not needed any more: their array stages the listed hash keys
+    unsigned long long* staged = reinterpret_cast<unsigned long long*>(S.key);
+    const bool stage = n <= nloc * 16;  // uniform over the block
+    for (int i = threadIdx.x; i < n; i += FUSED_THREADS) {
+      const unsigned long long key = __ldcg(&F.rand_list[2 * (size_t)i]);
+      if (stage) staged[i] = key;
+      atomicAdd(&sh.hist[(unsigned)((key - F.rand_lo) >> bshift)], 1u);
+    }
+    __syncthreads();
+    {
+      unsigned int mine[FUSED_BPT];
+      unsigned int tsum = 0;
+#pragma unroll
+      for (int j = 0; j < FUSED_BPT; ++j) {
+        mine[j] = sh.hist[threadIdx.x * FUSED_BPT + j];
+        tsum += mine[j];
+      }
+      unsigned int incl = tsum;
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      if (lane == 31) sh.warp_tot[warp] = incl;
+      __syncthreads();
+      unsigned int before = incl - tsum;
+      for (int wv = 0; wv < warp; ++wv) before += sh.warp_tot[wv];
+      if ((long long)before < r && r <= (long long)before + (long long)tsum) {
+        long long cum = before;
+        for (int j = 0; j < FUSED_BPT; ++j) {
+          if (cum + (long long)mine[j] >= r) {
+            sh.r_bin = threadIdx.x * FUSED_BPT + j;
+            sh.r_rank = r - cum;                                  // 1-based rank inside the bin
+            sh.r_ok = mine[j] <= (unsigned)(BINS / 4) ? 1 : 0;   // the bin's entries must fit the shared array below
+            break;
+          }
+          cum += mine[j];
+        }
+      }
+      __syncthreads();
+    }
+    if (!sh.r_ok) return false;  // same data in every block: same decision
+    const unsigned rbin = (unsigned)sh.r_bin;
+    const long long rr = sh.r_rank;
+    __syncthreads();
+    // the entries of that bin, gathered over the histogram's storage (BINS words = BINS / 4 pairs of 64-bit words)
+    unsigned long long* small = reinterpret_cast<unsigned long long*>(sh.hist);
+    for (int i = threadIdx.x; i < n; i += FUSED_THREADS) {
+      const unsigned long long key = stage ? staged[i] : __ldcg(&F.rand_list[2 * (size_t)i]);
+      if ((unsigned)((key - F.rand_lo) >> bshift) == rbin) {
+        const int at = atomicAdd(&sh.r_n, 1);
+        small[2 * at] = key;
+        small[2 * at + 1] = __ldcg(&F.rand_list[2 * (size_t)i + 1]);
+      }
+    }
+    __syncthreads();
+    const int m = sh.r_n;
+    for (int i = threadIdx.x; i < m; i += FUSED_THREADS) {
+      const unsigned long long key = small[2 * i], f = small[2 * i + 1];
+      int rank = 0;
+      for (int q = 0; q < m; ++q) {
+        const unsigned long long kq = small[2 * q], fq = small[2 * q + 1];
+        rank += (kq < key || (kq == key && fq < f)) ? 1 : 0;
+      }
+      if (rank == (int)(rr - 1)) { sh.r_tau = key; sh.r_tau_f = f; }
+    }
+    __syncthreads();
+    UPD_STAMP(43);
+  }
+  // ---- sweep 4, one thread per word: randomly grown entries and the new mask word
+  const unsigned long long tau = wantR ? sh.r_tau : 0ULL, tau_f = wantR ? sh.r_tau_f : 0ULL;
+  for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) {
+    uint32_t m = wantR ? S.hc[li] : 0u, bR = 0;
+    while (m) {
+      const int b = __ffs(m) - 1;
+      m &= m - 1;
+      const unsigned long long f = (unsigned long long)word_flat_index(P, lo + li, b);
+      const unsigned long long h = entry_hash(P, (long long)f);
+      if (h < tau || (h == tau && f <= tau_f)) bR |= 1u << b;
+    }
+    const uint32_t nb = (S.old[li] & ~S.prn[li]) | S.grad[li] | bR;
+    F.new_bits[lo + li] = nb;
+    F.cnt[lo + li] = __popc(nb);
+    S.hc[li] = nb;  // for the rebuild below
+  }
+  __syncthreads();
+  UPD_STAMP(44);
+  return true;
+}
+
+// Scan of the new mask and CSR fill from the slice kept in shared memory (new mask words in S.hc): the same result
+// as fused_grid_scan + mst_fill_csr_words, without fetching masks and scans again.  One grid barrier inside.
+template <typename V>
+__device__ void fused_dual_rebuild(const FusedParams& F, int64_t lo, int nloc, int& gscan, cg::grid_group& grid,
+                                   FusedShared& sh, const DualSlice& S) {
+  const SelParams& P = F.sel;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int32_t* bsums = F.bsums + (gscan & 1) * (int)gridDim.x;
+  ++gscan;
+  int v = 0;
+  for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) v += __popc(S.hc[li]);
+  const int bs = fused_block_sum(v, sh);
+  if (threadIdx.x == 0) bsums[blockIdx.x] = bs;
+  grid.sync();
+  int off = 0, tot = 0;
+  for (int j = threadIdx.x; j < (int)gridDim.x; j += FUSED_THREADS) {
+    const int x = __ldcg(bsums + j);
+    tot += x;
+    if (j < (int)blockIdx.x) off += x;
+  }
+  off = fused_block_sum(off, sh);
+  tot = fused_block_sum(tot, sh);
+  int carry = off;
+  int32_t* nbase = reinterpret_cast<int32_t*>(S.prn);  // the pruned bits are not needed any more
+  for (int b0 = 0; b0 < nloc; b0 += FUSED_THREADS) {
+    const int li = b0 + threadIdx.x;
+    const int x = li < nloc ? __popc(S.hc[li]) : 0;
+    int tile_total;
+    const int ex = fused_block_excl_scan(x, tile_total, sh);
+    if (li < nloc) {
+      nbase[li] = carry + ex;
+      F.new_wscan[lo + li] = carry + ex;
+    }
+    carry += tile_total;
+  }
+  if (threadIdx.x == 0) F.new_wscan[P.nwords] = tot;
+  __syncthreads();
+  UPD_STAMP(52);
+  // fill, one thread per word: a word holds few entries, and the lanes of a warp-per-word loop would mostly idle
+  const V* old_vals = (const V*)P.vals;
+  V* new_vals = (V*)F.new_vals;
+  for (int li = threadIdx.x; li < nloc; li += FUSED_THREADS) {
+    const uint32_t nb = S.hc[li], ob = S.old[li];
+    const unsigned wu = (unsigned)(lo + li);
+    const int o = (int)(wu / (unsigned)P.wpr), wc = (int)(wu - (unsigned)o * (unsigned)P.wpr);
+    int32_t pos = nbase[li];
+    if (wc == 0) {
+      F.new_row_ptr[o] = pos;
+      if (o == P.O - 1) F.new_row_ptr[P.O] = tot;
+    }
+    const int32_t obase = S.base[li];
+    uint32_t m = nb;
+    while (m) {
+      const int b = __ffs(m) - 1;
+      m &= m - 1;
+      V v = V(0);
+      if ((ob >> b) & 1u) v = old_vals[obase + __popc(ob & ((1u << b) - 1u))];
+      F.new_col[pos] = (uint16_t)(wc * 32 + b);
+      new_vals[pos] = v;
+      ++pos;
+    }
+  }
 }
 
 template <typename V>
@@ -793,42 +1425,75 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
   const int64_t hiT = loT + perT < F.nwordsT ? loT + perT : F.nwordsT;
 
   // this block's slice of the old mask and of its scan stays in shared memory for every selection pass
-  extern __shared__ uint32_t s_dyn[];
-  uint32_t* s_old = s_dyn;
-  int32_t* s_base = reinterpret_cast<int32_t*>(s_dyn + per);
-  uint32_t* s_grad = s_dyn + 2 * per;
-  uint32_t* scand = s_dyn + 3 * per;          // only present (and used) when the launch asked for the key cache
-  uint32_t* skey = s_dyn + 4 * per;
+  extern __shared__ __align__(16) uint32_t s_dyn[];
+  uint32_t* skey = s_dyn;                     // only present (and used) when the launch asked for the key cache
+  uint32_t* s_small = s_dyn + (F.smem_keys ? 32 * per : 0);
+  uint32_t* s_old = s_small;
+  int32_t* s_base = reinterpret_cast<int32_t*>(s_small + per);
+  uint32_t* s_grad = s_small + 2 * per;
+  uint32_t* scand = s_small + 3 * per;        // candidate words of the running selection
+  uint32_t* s_prn = s_small + 4 * per;        // side-by-side form: pruned bits
   for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
     s_old[w - lo] = P.old_bits[w];
     s_base[w - lo] = P.old_wscan[w];
     s_grad[w - lo] = 0;
   }
+  if (blockIdx.x == 0 && threadIdx.x < 3) F.flags[1 + threadIdx.x] = 0;  // per-update statistics (first used behind a barrier)
+#ifdef MST_UPD_PROFILE
+  if (blockIdx.x == 0 && threadIdx.x == 0) g_upd_nstamps = 0;
+#endif
   __syncthreads();
+  UPD_STAMP(2);
 
   int gpass = 0, gscan = 0;
-  if (per <= (int64_t)FUSED_WARPS * KEYS_PER_LANE) {  // uniform over the grid: every warp's words fit its key registers
+  const int cache = F.smem_keys ? CACHE_SMEM : (per <= (int64_t)FUSED_WARPS * KEYS_PER_LANE ? CACHE_REGS : CACHE_NONE);  // uniform over the grid
+  bool rewritten = false;
+  if (F.dual) {  // the launch carries the key cache
+    DualSlice S;
+    S.old = s_old; S.base = s_base; S.grad = s_grad; S.prn = s_prn; S.hc = scand; S.key = skey;
+    rewritten = fused_dual_update(F, lo, (int)(hi - lo), gpass, gscan, grid, sh, S);
+  } else if (cache == CACHE_REGS) {
     fused_select<MODE_PRUNE, CACHE_REGS>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
     fused_select<MODE_GRAD, CACHE_REGS>(F, F.n_grad, F.grad_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
-    fused_select<MODE_RAND, CACHE_REGS>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
-  } else if (F.smem_keys) {  // uniform over the grid
+  } else if (cache == CACHE_SMEM) {
     fused_select<MODE_PRUNE, CACHE_SMEM>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
     fused_select<MODE_GRAD, CACHE_SMEM>(F, F.n_grad, F.grad_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
-    fused_select<MODE_RAND, CACHE_SMEM>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
   } else {
     fused_select<MODE_PRUNE, CACHE_NONE>(F, F.n_prune, F.pruned_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
     fused_select<MODE_GRAD, CACHE_NONE>(F, F.n_grad, F.grad_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
-    fused_select<MODE_RAND, CACHE_NONE>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
   }
-
-  // mask rewrite: new = (old & ~pruned) | grad | rand, and its popcounts
-  for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
-    const uint32_t b = (P.old_bits[w] & ~F.pruned_bits[w]) | F.grad_bits[w] | F.rand_bits[w];
-    F.new_bits[w] = b;
-    F.cnt[w] = __popc(b);
+  UPD_STAMP(49);
+  if (!rewritten) {  // uniform over the grid: random growth by the general radix select, then the mask rewrite
+    if (cache == CACHE_REGS)
+      fused_select<MODE_RAND, CACHE_REGS>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
+    else if (cache == CACHE_SMEM)
+      fused_select<MODE_RAND, CACHE_SMEM>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
+    else
+      fused_select<MODE_RAND, CACHE_NONE>(F, F.n_rand, F.rand_bits, lo, hi, gpass, gscan, grid, sh, s_old, s_base, s_grad, skey, scand);
+    // mask rewrite: new = (old & ~pruned) | grad | rand, and its popcounts
+    for (int64_t w = lo + threadIdx.x; w < hi; w += FUSED_THREADS) {
+      const uint32_t pw = F.dual ? s_prn[w - lo] : F.pruned_bits[w], gw = F.dual ? s_grad[w - lo] : F.grad_bits[w];
+      const uint32_t b = (s_old[w - lo] & ~pw) | gw | F.rand_bits[w];
+      F.new_bits[w] = b;
+      F.cnt[w] = __popc(b);
+    }
+    __syncthreads();
   }
-  __syncthreads();
+  UPD_STAMP(51);
+  if (rewritten && !F.build_csc) {  // uniform over the grid: the slice's new mask is still in shared memory
+    DualSlice S;
+    S.old = s_old; S.base = s_base; S.grad = s_grad; S.prn = s_prn; S.hc = scand; S.key = skey;
+    fused_dual_rebuild<V>(F, lo, (int)(hi - lo), gscan, grid, sh, S);
+    UPD_STAMP(53);
+    if (blockIdx.x == 0) {  // every pick and every list read lies before the last barrier: leave the scratch zero
+      for (int b = threadIdx.x; b < 3 * HSTRIDE; b += FUSED_THREADS) F.hist[b] = 0;
+      if (threadIdx.x < 2) F.rand_ctr[threadIdx.x] = 0;
+    }
+    UPD_STAMP(54);
+    return;
+  }
   fused_grid_scan(F.cnt, F.new_wscan, P.nwords, lo, hi, F.bsums, gscan, grid, sh);
+  UPD_STAMP(52);
   // the barrier inside the scan came after every block wrote its part of the new mask: transpose it now
   if (F.build_csc) {
     const int64_t tiles = (int64_t)F.wpc * P.wpr;
@@ -841,6 +1506,12 @@ __global__ void __launch_bounds__(FUSED_THREADS, 2) mg_update_fused_kernel(const
                              F.new_row_ptr, P.old_bits, P.old_wscan, (const V*)P.vals,
                              F.build_csc ? &F.flags[1] : nullptr);  // without the barrier above the next row's scan entry
                                                                     // may belong to a block that has not written it yet
+  UPD_STAMP(53);
+  if (blockIdx.x == 0) {  // every pick and every list read lies before the last barrier: leave the scratch zero
+    for (int b = threadIdx.x; b < 3 * HSTRIDE; b += FUSED_THREADS) F.hist[b] = 0;
+    if (threadIdx.x < 2) F.rand_ctr[threadIdx.x] = 0;
+  }
+  UPD_STAMP(54);
   if (!F.build_csc) return;  // uniform over the grid
   for (int64_t w = loT + threadIdx.x; w < hiT; w += FUSED_THREADS) F.cnt[w] = __popc(F.bitsT[w]);
   __syncthreads();
@@ -1389,6 +2060,35 @@ void fill_fused_params(const UpdatePlan& pl, FusedParams& F) {
   F.wpc = L->wpc; F.nwordsT = L->nwordsT;
   F.build_csc = mst_use_tensor_path(L) ? 0 : 1;
   F.smem_keys = 0;
+  F.dual = 0;
+  F.g_bulk = 0;
+  F.rand_bracket = 0;
+  F.rand_cap = L->rand_cap;
+  F.rand_lo = F.rand_hi = 0;
+  F.rand_list = L->rand_list;
+  F.rand_ctr = L->rand_ctr;
+}
+
+// Bracket for the random growth: the n_rand-th smallest of C independent uniform 64-bit keys lies, with probability
+// 1 - 1e-8 or better, between the quantiles (k - m) / C and (k + m) / C with m = sigmas * sqrt(k) + 16 (the count of
+// keys below a quantile is binomial with a standard deviation below sqrt(k)).  The kernel checks the bracket against
+// the exact counts and falls back to the general radix select when it missed, so the choice only affects speed.
+void plan_rand_bracket(const UpdatePlan& pl, FusedParams& F) {
+  const mst_layer* L = pl.L;
+  const long long k = pl.n_rand;
+  const long long C = (L->N - L->nnz) - pl.n_grad;   // candidates: inactive entries the gradient growth left
+  if (k <= 0 || C <= 0 || k > C) return;
+  double sigmas = 6.0;
+  if (const char* e = getenv("MST_UPDATE_RAND_SIGMAS")) sigmas = atof(e);
+  if (!(sigmas > 0.0)) return;                        // 0 switches the bracket off
+  const long long m = (long long)(sigmas * sqrt((double)k)) + 16;
+  if (3 * m > L->rand_cap) return;                    // expected list length 2m: leave room for its own spread
+  const long long lo_cnt = k - m > 0 ? k - m : 0, hi_cnt = k + m;
+  const unsigned __int128 one = (unsigned __int128)1 << 64;
+  F.rand_lo = (unsigned long long)(one * (unsigned __int128)lo_cnt / (unsigned __int128)C);
+  F.rand_hi = hi_cnt >= C ? ~0ULL : (unsigned long long)(one * (unsigned __int128)hi_cnt / (unsigned __int128)C);
+  if (F.rand_hi <= F.rand_lo) return;
+  F.rand_bracket = 1;
 }
 
 // Host epilogue of an update whose kernels have been enqueued: statistics and error report when asked for, then the
@@ -1462,14 +2162,16 @@ mst_status_t launch_cooperative(const void* fn, void** args, int grid_blocks, si
 mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fused_out) {
   mst_layer* L = pl.L;
   const SelParams& P = pl.P;
-  // flags[0] (error bits) stays set until a reporting call has returned it; only the per-update statistic is cleared
-  MST_CUDA_TRY(cudaMemsetAsync(L->flags + 1, 0, sizeof(int32_t) * 3, s));
   bool fused = true;
   if (const char* e = getenv("MST_UPDATE_FUSED")) fused = (e[0] != '0');
   int grid_blocks = 0;
   size_t fused_smem = 0;
   const void* fn = L->dtype == MST_F32 ? (const void*)mg_update_fused_kernel<float> : (const void*)mg_update_fused_kernel<uint16_t>;
   int smem_keys = 0;
+  // Side-by-side selections: not with regrowth of just-pruned links (the gradient candidates then depend on the prune
+  // result)
+  bool want_dual = !P.allow;
+  if (const char* e = getenv("MST_UPDATE_DUAL")) want_dual = want_dual && (e[0] != '0');
   if (fused) {
     grid_blocks = fused_grid_limit(fn);
     if (grid_blocks == 0) fused = false;
@@ -1477,10 +2179,11 @@ mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fu
       const int64_t useful = (L->nwords + FUSED_WARPS - 1) / FUSED_WARPS;  // at least one word per warp
       if (grid_blocks > useful) grid_blocks = (int)(useful < 1 ? 1 : useful);
       int64_t per = (L->nwords + grid_blocks - 1) / grid_blocks;
-      fused_smem = (size_t)per * 12;  // slice of mask, scan and grad words
-      if (per > (int64_t)FUSED_WARPS * KEYS_PER_LANE && !getenv("MST_UPDATE_NO_SMEM_KEYS")) {
-        // the slice's keys do not fit the registers: keep them in shared memory (128 bytes per mask word plus a
-        // candidate word) if a block can have that much, with two blocks per SM or, for the largest layers, one
+      fused_smem = (size_t)per * 20;  // slice of mask, scan, grown, candidate and pruned words
+      if ((per > (int64_t)FUSED_WARPS * KEYS_PER_LANE || want_dual) && !getenv("MST_UPDATE_NO_SMEM_KEYS")) {
+        // keys in shared memory (128 bytes per mask word): always for the side-by-side form, otherwise when the
+        // slice's keys do not fit the registers; if a block can have that much, with two blocks per SM or, for the
+        // largest layers, one
         int dev = 0, sms = 0, optin = 0;
         if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
             cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) == cudaSuccess) {
@@ -1488,7 +2191,7 @@ mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fu
             int g = sms * occ_want;
             if (g > grid_blocks) g = grid_blocks;
             const int64_t per_k = (L->nwords + g - 1) / g;
-            const size_t need = (size_t)per_k * (12 + 4 + 128);
+            const size_t need = (size_t)per_k * (20 + 128);
             if (need + 10 * 1024 > (size_t)optin) continue;
             if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess) continue;
             int occ = 0;
@@ -1507,15 +2210,29 @@ mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fu
     }
   }
   if (fused) {
-    MST_CUDA_TRY(cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * BINS, s));
+    // flags[0] (error bits) stays set until a reporting call has returned it; the kernel clears the per-update
+    // statistics itself and leaves the histograms and the bracket counters zero for the next launch
+    if (!L->scratch_clean) {
+      MST_CUDA_TRY(cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * HSTRIDE, s));
+      MST_CUDA_TRY(cudaMemsetAsync(L->rand_ctr, 0, 2 * sizeof(unsigned long long), s));
+    }
     if (!mst_use_tensor_path(L)) MST_TRY(mst_alloc_csc(L));   // the kernel fills the view's arrays for such layers
     FusedParams F;
     fill_fused_params(pl, F);
     F.smem_keys = smem_keys;
+    // the packed histogram of the side-by-side form needs fewer than 65536 entries per block
+    const bool dual = want_dual && smem_keys && ((L->nwords + grid_blocks - 1) / grid_blocks) * 32 < 65536;
+    F.dual = dual ? 1 : 0;
+    F.g_bulk = (dual && P.aligned && P.G && ((uintptr_t)P.G % 16 == 0)) ? 1 : 0;
+    if (dual) plan_rand_bracket(pl, F);
     L->csc_valid = F.build_csc;
     void* args[] = {&F};
+    L->scratch_clean = 0;
     MST_TRY(launch_cooperative(fn, args, grid_blocks, fused_smem, s));
+    L->scratch_clean = 1;
   } else {
+    MST_CUDA_TRY(cudaMemsetAsync(L->flags + 1, 0, sizeof(int32_t) * 3, s));
+    L->scratch_clean = 0;
     MST_TRY(run_select<MODE_PRUNE>(L, P, pl.n_prune, L->pruned_bits, s));
     MST_TRY(run_select<MODE_GRAD>(L, P, pl.n_grad, L->grad_bits, s));
     MST_TRY(run_select<MODE_RAND>(L, P, pl.n_rand, L->rand_bits, s));
@@ -1527,6 +2244,20 @@ mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fu
 }
 
 }  // namespace
+
+#ifdef MST_UPD_PROFILE
+// (id, SM clock) pairs stamped by block 0 of the last fused update kernel; returns the number of pairs
+extern "C" int mst_update_profile(long long* out, int max_pairs) {
+  long long h[64];
+  int n = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpyFromSymbol(h, g_upd_stamps, sizeof(h)) != cudaSuccess ||
+      cudaMemcpyFromSymbol(&n, g_upd_nstamps, sizeof(int)) != cudaSuccess)
+    return -1;
+  if (n > max_pairs) n = max_pairs;
+  for (int i = 0; i < 2 * n; ++i) out[i] = h[i];
+  return n;
+}
+#endif
 
 extern "C" mst_status_t mst_topology_update(mst_layer_t* L, double prune_frac, const mst_regrow_rule_t* rule,
                                             const float* G_dense, mst_update_stats_t* stats, mst_stream_t stream) {
@@ -1590,6 +2321,7 @@ extern "C" mst_status_t mst_topology_update_many(int32_t n_layers, mst_layer_t* 
             cudaMemsetAsync(L->hist, 0, sizeof(unsigned int) * 3 * BINS, s) != cudaSuccess)
           st = MST_ERR_CUDA;
         L->csc_valid = 0;
+        L->scratch_clean = 0;
         mode[j] = 1;
       }
       if (st == MST_OK) {

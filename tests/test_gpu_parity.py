@@ -157,15 +157,44 @@ def _update_both(L, p, W, M, G, zeta, target, R, seed, step, allow=False):
     return Wn, Mn
 
 
+def _set_update_variant(monkeypatch, variant):
+    env = {"fused": {}, "phases": {"MST_UPDATE_FUSED": "0"}, "fused_sequential": {"MST_UPDATE_DUAL": "0"},
+           "fused_bracket_miss": {"MST_UPDATE_RAND_SIGMAS": "0.001"}, "fused_no_bracket": {"MST_UPDATE_RAND_SIGMAS": "0"},
+           "fused_no_key_cache": {"MST_UPDATE_NO_SMEM_KEYS": "1"}}[variant]
+    for k in ("MST_UPDATE_FUSED", "MST_UPDATE_DUAL", "MST_UPDATE_RAND_SIGMAS", "MST_UPDATE_NO_SMEM_KEYS"):
+        monkeypatch.delenv(k, raising=False)
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)             # read by the library at every call
+
+
+@pytest.mark.parametrize("variant", ["fused", "fused_no_key_cache", "fused_bracket_miss", "fused_sequential"])
+def test_update_of_a_layer_beyond_the_register_key_cache(variant, monkeypatch):
+    # 2.6 M entries: a block's slice no longer fits the key registers; keys live in shared memory or are recomputed
+    _set_update_variant(monkeypatch, variant)
+    O, I = 1024, 2560
+    p = _problem(O, I, 4, "bf16", 0.05, 4100, "uniform")
+    L = make_layer(p)
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    M = p.mask.copy()
+    rng = np.random.default_rng(9)
+    for step in range(3):
+        G = rng.standard_normal((O, I)).astype(np.float32)
+        G.reshape(-1)[::7] = np.float32(0.125)
+        W, M = _update_both(L, p, W, M, G, 0.3, -1, 0.25, 11, step)
+    L.close()
+
+
 @pytest.mark.parametrize("O,I,dtype,density,kind,zeta,R,allow", [
     (96, 160, "f32", 0.25, "uniform", 0.3, 0.25, False), (130, 257, "bf16", 0.1, "uniform", 0.3, 0.25, False),
     (256, 512, "bf16", 0.05, "zipf", 0.1, 0.25, False), (64, 96, "f32", 0.3, "uniform", 0.3, 0.0, False),
     (64, 96, "bf16", 0.3, "uniform", 0.3, 1.0, False), (96, 160, "bf16", 0.25, "uniform", 0.5, 0.25, True),
     (33, 31, "f32", 0.5, "uniform", 1.0, 0.5, False)])
-@pytest.mark.parametrize("fused", ["1", "0"])
-def test_update_is_bit_exact_over_consecutive_steps(O, I, dtype, density, kind, zeta, R, allow, fused, monkeypatch):
-    # both implementations of the update: the single cooperative kernel and the kernel-per-phase sequence
-    monkeypatch.setenv("MST_UPDATE_FUSED", fused)
+@pytest.mark.parametrize("variant", ["fused", "phases", "fused_sequential", "fused_bracket_miss", "fused_no_bracket"])
+def test_update_is_bit_exact_over_consecutive_steps(O, I, dtype, density, kind, zeta, R, allow, variant, monkeypatch):
+    # every implementation of the update: the single cooperative kernel (prune and gradient selections side by side,
+    # random growth by bracket), the kernel-per-phase sequence, the cooperative kernel with one selection after the
+    # other, with a bracket so narrow that it usually misses (general radix select takes over), and without bracket
+    _set_update_variant(monkeypatch, variant)
     p = _problem(O, I, 4, dtype, density, 300 + O + I, kind)
     L = make_layer(p)
     W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
