@@ -547,6 +547,14 @@ def other_legs(reps: int, dev):
             t_all, _ = median_ms(whole, reps)
             res["step_with_dense_grad_and_update_ms"] = round(t_all, 4)
             res["step_useful_tflops"] = round(useful / (t_all * 1e-3) / 1e12, 3)
+
+            def update_only():
+                k[0] += 1
+                rules = [mst.RegrowRule(-1, 0.25, 9, k[0], 0, 0.0) for _ in slots]
+                mst.mst_topology_update_many([s[0].handle for s in slots], [zeta] * len(slots), rules, [s[7] for s in slots],
+                                             want_stats=False)
+            t_upd, _ = median_ms(update_only, reps)
+            res["topology_update_ms"] = round(t_upd, 4)
         for s in slots:
             s[0].close()
         return res
@@ -660,8 +668,12 @@ def main() -> None:
         rules = [mst.RegrowRule(-1, 0.25, seed, k, 0, 0.0) for _ in slots]
         mst.mst_topology_update_many(handles, [0.3] * len(slots), rules, Gs, want_stats=False)
 
+    for s in slots:
+        s.L.track_values(True)      # the dense image of W.M is rebuilt when values or structure changed, not per call
+
     def step(k: int, timed: bool):
         for s in slots:
+            s.L.values_changed()    # what an optimizer step does once per training step
             marks = [ev()] if timed else None
             s.L.fwd(s.X, s.Y, T)
             if timed: marks.append(ev())
@@ -693,13 +705,19 @@ def main() -> None:
     w0 = time.time()
     e0 = ev()
     for k in range(args.steps):
-        step(args.warmup + k, True)
+        step(args.warmup + k, False)
     e1 = ev()
     barrier()
     w1 = time.time()
     clocks = sampler.stop(w0, w1)
     gpu_launches = mst.mst_launch_count() - launches0
     ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    # the same K steps once more with an event pair around every call: the per-kernel times and the roofline's launch
+    # durations.  (Events between the calls keep a launch from starting under its predecessor's tail, so these times
+    # add up to more than the step time above.)
+    for k in range(args.steps):
+        step(args.warmup + args.steps + k, True)
+    barrier()
     useful = 6.0 * T * sum(s.nnz for s in slots)          # per step, per replica
     value = aggregate_value(useful, args.steps, world, ms)
 
@@ -812,6 +830,7 @@ def main() -> None:
     # which keeps every call of the path as its own launch.
     def shared_step(k):
         for s in slots:
+            s.L.values_changed()
             s.L.fwd(s.X, s.Y, T)
             s.L.bwd_x(s.dY, s.dX, T)
             s.L.dense_grad_dw(s.dY, s.X, T, s.G, s.dW)
@@ -838,8 +857,12 @@ def main() -> None:
         "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: four layers' distinct buffers, %.0f MB touched "
                    "per step" % (sum(2 * T * (p.in_features + p.out_features) * es for p in probs) / 1e6),
                    "update": "every step, zeta=0.3, R=0.25 (gradient growth by |G| over the inactive entries), "
-                   "target = current nnz; the four layers in one mst_topology_update_many call", "paths": paths, "replicas": world},
+                   "target = current nnz; the four layers in one mst_topology_update_many call",
+                   "values": "mst_values_changed once per layer and step (an optimizer step): the dense image of W.M is "
+                   "rebuilt once per step, not per product", "paths": paths, "replicas": world},
         "clocks": clocks, "roofline": roof, "kernels": per,
+        "kernels_note": "per-call times from a second pass of the same steps with a CUDA-event pair around every call; "
+                        "ms_per_step and value come from the first pass, which has no events inside",
         "fwd_bwd_only_tflops": useful / ((per["spmm_fwd"]["ms_per_step"] + per["spmm_bwd_x"]["ms_per_step"] +
                                           per["sddmm_dw"]["ms_per_step"]) * 1e-3) / 1e12,
         "shared_gradient_step": {"ms_per_step": shared_ms, "value": aggregate_value(useful, 1, world, shared_ms),
