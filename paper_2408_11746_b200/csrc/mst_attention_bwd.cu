@@ -10,30 +10,28 @@
 //   1. delta: one warp per (token, head).
 //   2. dQ, query-centric: a block owns 64 queries of one (sequence, head) and walks the key tiles of their window
 //      (stride / 64 + 1 tiles of 64 keys; the tile that starts `stride` positions back also holds the first strided
-//      key of every query).  Per tile: S = Q K^T and dP = dOut V^T on the tensor cores (warp-level 16x16x16 bf16
-//      fragments, fp32 accumulators), the softmax algebra element-wise on the fp32 tiles in shared memory, then
-//      dQ += dS K with dS rounded to bf16.  The strided keys further back (i - 2l, i - 3l, ...: single keys, not
-//      tiles) are handled on the CUDA cores.
+//      key of every query).  Per tile: S = Q K^T and dP = dOut V^T on the tensor cores (warp-level mma.sync
+//      m16n8k16, bf16 operands fetched with ldmatrix, fp32 accumulators), the softmax algebra on the accumulator
+//      registers, then dQ += dS K with dS rounded to bf16 and used as the next A operand straight from the registers
+//      (the accumulator layout of two neighbouring 16 x 8 tiles is the A layout).  The strided keys further back (i - 2l, i - 3l, ...) are
+//      visited as further tiles of which only the diagonal is kept.
 //   3. dK and dV, key-centric: a block owns 64 keys and walks the query tiles that can see them, with the
 //      transposed products (S^T = K Q^T, dP^T = V dOut^T), dV += P^T dOut and dK += dS^T Q; far queries
-//      (j + 2l, j + 3l, ...) on the CUDA cores.
+//      (j + 2l, j + 3l, ...) as further tiles, diagonal only.
 // Every warp owns a 16-row strip of each tile, so the element-wise steps need no block-wide barrier; the barriers
 // are around the cooperative tile loads only.  Scores, sums and deltas are fp32; P and dS are rounded to bf16 where
 // they enter a tensor-core product (as the forward kernel does with P).
 #include <cuda_bf16.h>
-#include <mma.h>
 
 #include "mst_internal.cuh"
 #include "mst_tc_gemm.cuh"
 
 namespace {
 
-using namespace nvcuda;
 
 constexpr int D = 64;        // head dimension
 constexpr int TS = 64;       // tile side (queries and keys)
-constexpr int BW_THREADS = 256;
-constexpr int BW_WARPS = BW_THREADS / 32;
+constexpr int BW_THREADS = 128;
 constexpr int LDB = 72;      // row pitch of the bf16 tiles in shared memory (64 + 8: rows 144 bytes apart, no bank aliasing)
 constexpr int LDF = 68;      // row pitch of the fp32 tiles
 constexpr float SCALE = 0.125f;   // 1 / sqrt(64)
@@ -48,20 +46,8 @@ struct BwdParams {
   int batch, seq, heads, stride;
 };
 
-__device__ __forceinline__ bool attends(int i, int j, int l) {
-  const int back = i - j;
-  return back >= 0 && (back < l || back % l == 0);
-}
-
-// rows [r0, r0 + 64) of one head's 64 columns -> dst[64][LDB] (row-major, bf16), 16 bytes per thread and step
-__device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int64_t r0) {
-  for (int e = threadIdx.x; e < TS * D / 8; e += BW_THREADS) {
-    const int r = e >> 3, c = (e & 7) * 8;
-    *reinterpret_cast<uint4*>(dst + r * LDB + c) = *reinterpret_cast<const uint4*>(src + (r0 + r) * ld + c);
-  }
-}
-
-// the same copy issued asynchronously (cp.async, 16 bytes per request); complete after async_wait_all + a barrier
+// rows [r0, r0 + 64) of one head's 64 columns -> dst[64][LDB] (row-major, bf16), issued asynchronously (cp.async, 16 bytes per
+// request); complete after async_wait_all + a barrier
 __device__ __forceinline__ void load_tile_async(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int64_t r0) {
   for (int e = threadIdx.x; e < TS * D / 8; e += BW_THREADS) {
     const int r = e >> 3, c = (e & 7) * 8;
@@ -94,165 +80,193 @@ __global__ void attn_delta_kernel(BwdParams P) {
   if (lane == 0) P.delta[(b * P.heads + h) * P.seq + i] = s;
 }
 
-typedef wmma::fragment<wmma::matrix_a, 16, 16, 16, __nv_bfloat16, wmma::row_major> FragA;
-typedef wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::col_major> FragBt;   // B given as [n][k] rows
-typedef wmma::fragment<wmma::matrix_b, 16, 16, 16, __nv_bfloat16, wmma::row_major> FragB;    // B given as [k][n] rows
-typedef wmma::fragment<wmma::accumulator, 16, 16, 16, float> FragC;
-
-// Eight warps per block: warp = (strip of 16 rows, half of the 64 columns).  A warp forms its 16 x 32 part of the two
-// score-shaped products, applies the softmax algebra to it, and after a block barrier accumulates its 16 x 32 part of
-// the gradient tiles from the complete 16 x 64 strip of weights.
-
-// out [16 x 32] (fp32, pitch LDF) = A strip [16 x 64] * B^T for 32 of B's rows (row n of b_rows holds B^T's column n)
-__device__ __forceinline__ void half_abt(float* out, const __nv_bfloat16* a_strip, const __nv_bfloat16* b_rows) {
-  FragA a[4];
+// Warp-level tensor-core pieces (mma.sync m16n8k16, bf16 in, fp32 accumulate) with the published fragment layouts:
+// with g = lane / 4 and t = lane % 4, an accumulator tile (16 x 8) holds rows g, g + 8 and columns 2t, 2t + 1 in its
+// four registers, and an A operand (16 x 16, row-major) holds the same rows and columns 2t, 2t + 1, 2t + 8, 2t + 9 —
+// so two neighbouring accumulator tiles, rounded to bf16, ARE the A operand of the next product and the scores never
+// leave the registers.
+__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const __nv_bfloat16* p) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const __nv_bfloat16* p) {
+  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+// A operand: rows r0 .. r0 + 16, columns 16 kb .. 16 kb + 16 of a bf16 tile with row pitch LDB
+__device__ __forceinline__ void load_a(uint32_t (&a)[4], const __nv_bfloat16* tile, int r0, int kb, int lane) {
+  ldsm_x4(a, tile + (r0 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDB + kb * 16 + (lane >> 4) * 8);
+}
+// c[16 x 8] += A strip (four k-steps over the 64 head dimensions, in registers) * rows n0 .. n0 + 8 of `tile`, transposed
+__device__ __forceinline__ void mma_rows(float (&c)[4], const uint32_t (&a)[4][4], const __nv_bfloat16* tile, int n0, int lane) {
 #pragma unroll
-  for (int kb = 0; kb < 4; ++kb) wmma::load_matrix_sync(a[kb], a_strip + kb * 16, LDB);
-#pragma unroll
-  for (int nb = 0; nb < 2; ++nb) {
-    FragC c;
-    wmma::fill_fragment(c, 0.f);
-#pragma unroll
-    for (int kb = 0; kb < 4; ++kb) {
-      FragBt b;
-      wmma::load_matrix_sync(b, b_rows + nb * 16 * LDB + kb * 16, LDB);
-      wmma::mma_sync(c, a[kb], b, c);
-    }
-    wmma::store_matrix_sync(out + nb * 16, c, LDF, wmma::mem_row_major);
+  for (int k2 = 0; k2 < 2; ++k2) {
+    uint32_t b[4];
+    ldsm_x4(b, tile + (n0 + (lane & 7)) * LDB + k2 * 32 + (lane >> 3) * 8);
+    mma_bf16(c, a[2 * k2], b[0], b[1]);
+    mma_bf16(c, a[2 * k2 + 1], b[2], b[3]);
   }
 }
-
-// acc[2] (16 x 32, fp32 fragments) += A strip [16 x 64] (bf16) * 32 columns of B [64 x 64] (bf16 rows; b_cols points
-// at the first of the 32 columns)
-__device__ __forceinline__ void half_ab_acc(FragC (&acc)[2], const __nv_bfloat16* a_strip, const __nv_bfloat16* b_cols) {
+// acc[16 x 64] += A (16 x 16, in registers) * rows k0 .. k0 + 16 of `tile` (64 columns)
+__device__ __forceinline__ void mma_cols(float (&acc)[8][4], const uint32_t (&a)[4], const __nv_bfloat16* tile, int k0, int lane) {
 #pragma unroll
-  for (int kb = 0; kb < 4; ++kb) {
-    FragA a;
-    wmma::load_matrix_sync(a, a_strip + kb * 16, LDB);
+  for (int n2 = 0; n2 < 4; ++n2) {
+    uint32_t b[4];
+    ldsm_x4_t(b, tile + (k0 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDB + n2 * 16 + (lane >> 4) * 8);
+    mma_bf16(acc[2 * n2], a, b[0], b[1]);
+    mma_bf16(acc[2 * n2 + 1], a, b[2], b[3]);
+  }
+}
+// accumulators (16 x 64) -> fp32 tile in shared memory, rows r0 .. r0 + 16
+__device__ __forceinline__ void store_acc(float* out, const float (&acc)[8][4], int r0, int lane) {
+  const int g = lane >> 2, t = lane & 3;
 #pragma unroll
-    for (int nb = 0; nb < 2; ++nb) {
-      FragB b;
-      wmma::load_matrix_sync(b, b_cols + kb * 16 * LDB + nb * 16, LDB);
-      wmma::mma_sync(acc[nb], a, b, acc[nb]);
-    }
+  for (int nb = 0; nb < 8; ++nb) {
+    *reinterpret_cast<float2*>(out + (r0 + g) * LDF + nb * 8 + 2 * t) = make_float2(acc[nb][0], acc[nb][1]);
+    *reinterpret_cast<float2*>(out + (r0 + g + 8) * LDF + nb * 8 + 2 * t) = make_float2(acc[nb][2], acc[nb][3]);
   }
 }
 
 // ------------------------------------------------------------------------------------------- dQ
-__global__ void __launch_bounds__(BW_THREADS) attn_bwd_dq_kernel(BwdParams P) {
+__global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dq_kernel(BwdParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem);   // [64][LDB]
   __nv_bfloat16* Gs = Qs + TS * LDB;                             // dOut tile
   __nv_bfloat16* KV = Gs + TS * LDB;                             // two (K tile, V tile) buffers: the next pair is fetched
-  __nv_bfloat16* Sb = KV + 4 * TS * LDB;                         //   while the current one is used
-  float* Sf = reinterpret_cast<float*>(Sb + TS * LDB);           // scores, later dQ   [64][LDF]
-  float* Pf = Sf + TS * LDF;                                     // dP
+  float* Sf = reinterpret_cast<float*>(KV);                      //   while the current one is used; dQ [64][LDF] is staged
+                                                                 //   over them when the last tile has been consumed
   __shared__ float lse_s[TS], del_s[TS];
 
   const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int q0 = qt * TS, l = P.stride;
   const int64_t row0 = (int64_t)b * P.seq;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
   const int64_t stat0 = ((int64_t)b * P.heads + h) * P.seq;
-  load_tile(Qs, P.Q + h * D, P.ld, row0 + q0);
-  load_tile(Gs, P.dOut + h * D, P.lddo, row0 + q0);
+  load_tile_async(Qs, P.Q + h * D, P.ld, row0 + q0);       // all first loads in flight together
+  load_tile_async(Gs, P.dOut + h * D, P.lddo, row0 + q0);
   if (threadIdx.x < TS) {
     lse_s[threadIdx.x] = P.lse[stat0 + q0 + threadIdx.x];
     del_s[threadIdx.x] = P.delta[stat0 + q0 + threadIdx.x];
   }
-  FragC acc[2];
-#pragma unroll
-  for (int nb = 0; nb < 2; ++nb) wmma::fill_fragment(acc[nb], 0.f);
-  const int r_base = (warp & 3) * 16, c_base = (warp >> 2) * 32;
+  const int r_base = warp * 16;
+  // key tiles: the window's tiles, then one tile per strided position further back (i - 2l, i - 3l, ...), of which
+  // only the diagonal (query r, key r) is attended
   const int k_first = q0 - l > 0 ? q0 - l : 0;
+  const int n_near = (q0 - k_first) / TS + 1;
+  const int n_tiles = n_near + (q0 / l > 1 ? q0 / l - 1 : 0);
+  auto tile_start = [&](int ti) { return ti < n_near ? k_first + ti * TS : q0 - (ti - n_near + 2) * l; };
   load_tile_async(KV, P.K + h * D, P.ld, row0 + k_first);
   load_tile_async(KV + TS * LDB, P.V + h * D, P.ld, row0 + k_first);
   async_commit();
+  async_wait_all();
+  __syncthreads();   // Q, dOut, the statistics and the first key tile are in place
+  uint32_t qa[4][4], ga[4][4];
+#pragma unroll
+  for (int kb = 0; kb < 4; ++kb) {
+    load_a(qa[kb], Qs, r_base, kb, lane);
+    load_a(ga[kb], Gs, r_base, kb, lane);
+  }
+  const float lse0 = lse_s[r_base + g], lse1 = lse_s[r_base + g + 8];
+  const float del0 = del_s[r_base + g], del1 = del_s[r_base + g + 8];
+  float acc[8][4];
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb) acc[nb][0] = acc[nb][1] = acc[nb][2] = acc[nb][3] = 0.f;
   int buf = 0;
-  for (int k0 = k_first; k0 <= q0; k0 += TS, buf ^= 1) {
+  for (int ti = 0; ti < n_tiles; ++ti, buf ^= 1) {
+    const int k0 = tile_start(ti);
     async_wait_all();
-    __syncthreads();   // this tile has landed for everyone; the other buffer's tile and the weights have been consumed
+    __syncthreads();   // this tile has landed for everyone; the other buffer's tile has been consumed
     const __nv_bfloat16* Ks = KV + buf * 2 * TS * LDB;
     const __nv_bfloat16* Vs = Ks + TS * LDB;
-    if (k0 + TS <= q0) {
-      load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB, P.K + h * D, P.ld, row0 + k0 + TS);
-      load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB + TS * LDB, P.V + h * D, P.ld, row0 + k0 + TS);
+    if (ti + 1 < n_tiles) {
+      const int kn = tile_start(ti + 1);
+      load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB, P.K + h * D, P.ld, row0 + kn);
+      load_tile_async(KV + (buf ^ 1) * 2 * TS * LDB + TS * LDB, P.V + h * D, P.ld, row0 + kn);
       async_commit();
     }
-    half_abt(Sf + r_base * LDF + c_base, Qs + r_base * LDB, Ks + c_base * LDB);
-    half_abt(Pf + r_base * LDF + c_base, Gs + r_base * LDB, Vs + c_base * LDB);
-    __syncwarp();
-    // the visited key tiles lie within l + 64 positions behind the queries: a pair is kept iff 0 <= i - j <= l
-    // (the window, and the first strided position i - l)
-    const int d0 = q0 - k0;
-    for (int e = lane; e < 16 * 32; e += 32) {
-      const int r = r_base + (e >> 5), c = c_base + (e & 31);
-      const int back = d0 + r - c;
-      float ds = 0.f;
-      if (back >= 0 && back <= l) {
-        const float p = __expf(Sf[r * LDF + c] * SCALE - lse_s[r]);
-        ds = p * (Pf[r * LDF + c] - del_s[r]);
-      }
-      Sb[r * LDB + c] = __float2bfloat16(ds);
-    }
-    __syncthreads();   // the strip of weights is complete (both column halves)
-    half_ab_acc(acc, Sb + r_base * LDB, Ks + c_base);
-  }
-  __syncthreads();     // every warp has read its scores: the array takes dQ now
+    // a window tile lies within l + 64 positions behind the queries: a pair is kept iff 0 <= i - j <= l (the window,
+    // and the first strided position i - l); in a tile further back iff i - j is the tile's own distance
+    const int back_lo = ti < n_near ? 0 : q0 - k0, back_hi = ti < n_near ? l : q0 - k0;
+    const int back0 = q0 - k0 + r_base + g - 2 * t;   // i - j of this lane's first element of key column 0
 #pragma unroll
-  for (int nb = 0; nb < 2; ++nb)
-    wmma::store_matrix_sync(Sf + r_base * LDF + c_base + nb * 16, acc[nb], LDF, wmma::mem_row_major);
-  __syncthreads();
-  // strided keys beyond the tiles: i - 2l, i - 3l, ...   (lane = two head dimensions)
-  for (int r = warp * (TS / BW_WARPS); r < (warp + 1) * (TS / BW_WARPS); ++r) {
-    const int i = q0 + r;
-    const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Qs + r * LDB + 2 * lane));
-    const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Gs + r * LDB + 2 * lane));
-    float ax = 0.f, ay = 0.f;
-    for (int j = i - 2 * l; j >= 0; j -= l) {
-      const float2 k = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(P.K + (row0 + j) * P.ld + h * D + 2 * lane));
-      const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(P.V + (row0 + j) * P.ld + h * D + 2 * lane));
-      float s = q.x * k.x + q.y * k.y, dp = g.x * v.x + g.y * v.y;
-      for (int off = 16; off; off >>= 1) {
-        s += __shfl_xor_sync(0xffffffffu, s, off);
-        dp += __shfl_xor_sync(0xffffffffu, dp, off);
+    for (int half = 0; half < 2; ++half) {            // 32 keys at a time
+      float sc[4][4], dp[4][4];
+#pragma unroll
+      for (int nb = 0; nb < 4; ++nb) {
+        sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
+        dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
+        mma_rows(sc[nb], qa, Ks, half * 32 + nb * 8, lane);
+        mma_rows(dp[nb], ga, Vs, half * 32 + nb * 8, lane);
       }
-      const float ds = __expf(s * SCALE - lse_s[r]) * (dp - del_s[r]);
-      ax = fmaf(ds, k.x, ax);
-      ay = fmaf(ds, k.y, ay);
+#pragma unroll
+      for (int nb = 0; nb < 4; ++nb) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int back = back0 + (i >> 1) * 8 - (half * 32 + nb * 8 + (i & 1));
+          float ds = 0.f;
+          if (back >= back_lo && back <= back_hi) {
+            const float p = __expf(sc[nb][i] * SCALE - ((i >> 1) ? lse1 : lse0));
+            ds = p * (dp[nb][i] - ((i >> 1) ? del1 : del0));
+          }
+          sc[nb][i] = ds;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {                   // 16 keys per step
+        uint32_t a[4];
+        a[0] = pack_bf16(sc[2 * j][0], sc[2 * j][1]);
+        a[1] = pack_bf16(sc[2 * j][2], sc[2 * j][3]);
+        a[2] = pack_bf16(sc[2 * j + 1][0], sc[2 * j + 1][1]);
+        a[3] = pack_bf16(sc[2 * j + 1][2], sc[2 * j + 1][3]);
+        mma_cols(acc, a, Ks, half * 32 + j * 16, lane);
+      }
     }
-    const float ox = (Sf[r * LDF + 2 * lane] + ax) * SCALE, oy = (Sf[r * LDF + 2 * lane + 1] + ay) * SCALE;
-    *reinterpret_cast<__nv_bfloat162*>(P.dQ + (row0 + i) * P.ldg + h * D + 2 * lane) = __floats2bfloat162_rn(ox, oy);
+  }
+  __syncthreads();   // every warp is done with the key tiles: their storage takes dQ
+  store_acc(Sf, acc, r_base, lane);
+  __syncwarp();
+  for (int r = r_base; r < r_base + 16; ++r) {   // lane = two head dimensions
+    const float ox = Sf[r * LDF + 2 * lane] * SCALE, oy = Sf[r * LDF + 2 * lane + 1] * SCALE;
+    *reinterpret_cast<__nv_bfloat162*>(P.dQ + (row0 + q0 + r) * P.ldg + h * D + 2 * lane) = __floats2bfloat162_rn(ox, oy);
   }
 }
 
 // ------------------------------------------------------------------------------------------- dK, dV
-__global__ void __launch_bounds__(BW_THREADS) attn_bwd_dkv_kernel(BwdParams P) {
+__global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dkv_kernel(BwdParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem);
   __nv_bfloat16* Vs = Ks + TS * LDB;
   __nv_bfloat16* QG = Vs + TS * LDB;                             // two (Q tile, dOut tile) buffers
-  __nv_bfloat16* Pb = QG + 4 * TS * LDB;                         // P^T, bf16   [key][query]
-  __nv_bfloat16* Sb = Pb + TS * LDB;                             // dS^T, bf16
-  float* Sf = reinterpret_cast<float*>(Sb + TS * LDB);           // S^T, later dK
-  float* Pf = Sf + TS * LDF;                                     // dP^T, later dV
+  float* Sf = reinterpret_cast<float*>(QG);                      // dK [64][LDF] and dV are staged over the query buffers
+  float* Pf = Sf + TS * LDF;                                     //   when the last tile has been consumed
   __shared__ float stat_s[2][2 * TS];   // per buffer: log-sum-exp and delta of the tile's queries
 
   const int kt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int k0 = kt * TS, l = P.stride;
   const int64_t row0 = (int64_t)b * P.seq;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
   const int64_t stat0 = ((int64_t)b * P.heads + h) * P.seq;
-  load_tile(Ks, P.K + h * D, P.ld, row0 + k0);
-  load_tile(Vs, P.V + h * D, P.ld, row0 + k0);
-  FragC acc_k[2], acc_v[2];
-#pragma unroll
-  for (int nb = 0; nb < 2; ++nb) {
-    wmma::fill_fragment(acc_k[nb], 0.f);
-    wmma::fill_fragment(acc_v[nb], 0.f);
-  }
-  const int r_base = (warp & 3) * 16, c_base = (warp >> 2) * 32;   // this warp's keys, and its half of the columns
+  load_tile_async(Ks, P.K + h * D, P.ld, row0 + k0);         // all first loads in flight together
+  load_tile_async(Vs, P.V + h * D, P.ld, row0 + k0);
+  const int r_base = warp * 16;   // this warp's keys
+  // query tiles: those whose window reaches these keys, then one tile per strided position further on
+  // (j + 2l, j + 3l, ...), of which only the diagonal is attended
   const int q_last = k0 + l < P.seq - TS ? k0 + l : P.seq - TS;
+  const int n_near = (q_last - k0) / TS + 1;
+  const int m_max = (P.seq - TS - k0) / l;
+  const int n_tiles = n_near + (m_max > 1 ? m_max - 1 : 0);
+  auto tile_start = [&](int ti) { return ti < n_near ? k0 + ti * TS : k0 + (ti - n_near + 2) * l; };
   auto fetch = [&](int q0, int bf) {
     load_tile_async(QG + bf * 2 * TS * LDB, P.Q + h * D, P.ld, row0 + q0);
     load_tile_async(QG + bf * 2 * TS * LDB + TS * LDB, P.dOut + h * D, P.lddo, row0 + q0);
@@ -261,67 +275,84 @@ __global__ void __launch_bounds__(BW_THREADS) attn_bwd_dkv_kernel(BwdParams P) {
     async_commit();
   };
   fetch(k0, 0);
+  async_wait_all();
+  __syncthreads();   // K, V and the first query tile are in place
+  uint32_t ka[4][4], va[4][4];
+#pragma unroll
+  for (int kb = 0; kb < 4; ++kb) {
+    load_a(ka[kb], Ks, r_base, kb, lane);
+    load_a(va[kb], Vs, r_base, kb, lane);
+  }
+  float acc_k[8][4], acc_v[8][4];
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb) {
+    acc_k[nb][0] = acc_k[nb][1] = acc_k[nb][2] = acc_k[nb][3] = 0.f;
+    acc_v[nb][0] = acc_v[nb][1] = acc_v[nb][2] = acc_v[nb][3] = 0.f;
+  }
   int buf = 0;
-  for (int q0 = k0; q0 <= q_last; q0 += TS, buf ^= 1) {
+  for (int ti = 0; ti < n_tiles; ++ti, buf ^= 1) {
+    const int q0 = tile_start(ti);
     async_wait_all();
-    __syncthreads();   // this query tile has landed for everyone (first trip: also K and V); the other buffer and the
-                       // weights of the previous tile have been consumed
+    __syncthreads();   // this query tile has landed for everyone; the other buffer has been consumed
     const __nv_bfloat16* Qs = QG + buf * 2 * TS * LDB;
     const __nv_bfloat16* Gs = Qs + TS * LDB;
     const float* lse_s = stat_s[buf];
     const float* del_s = stat_s[buf] + TS;
-    if (q0 + TS <= q_last) fetch(q0 + TS, buf ^ 1);
-    half_abt(Sf + r_base * LDF + c_base, Ks + r_base * LDB, Qs + c_base * LDB);   // S^T[key][query]
-    half_abt(Pf + r_base * LDF + c_base, Vs + r_base * LDB, Gs + c_base * LDB);   // dP^T[key][query]
-    __syncwarp();
-    const int d0 = q0 - k0;   // the visited query tiles lie within l + 64 positions ahead: kept iff 0 <= i - j <= l
-    for (int e = lane; e < 16 * 32; e += 32) {
-      const int r = r_base + (e >> 5), c = c_base + (e & 31);      // key r, query c
-      const int back = d0 + c - r;
-      float p = 0.f, ds = 0.f;
-      if (back >= 0 && back <= l) {
-        p = __expf(Sf[r * LDF + c] * SCALE - lse_s[c]);
-        ds = p * (Pf[r * LDF + c] - del_s[c]);
-      }
-      Pb[r * LDB + c] = __float2bfloat16(p);
-      Sb[r * LDB + c] = __float2bfloat16(ds);
-    }
-    __syncthreads();   // the strips of weights are complete (both query halves)
-    half_ab_acc(acc_v, Pb + r_base * LDB, Gs + c_base);
-    half_ab_acc(acc_k, Sb + r_base * LDB, Qs + c_base);
-  }
-  __syncthreads();     // every warp has read its scores: the arrays take dK and dV now
+    if (ti + 1 < n_tiles) fetch(tile_start(ti + 1), buf ^ 1);
+    // a window tile lies within l + 64 positions ahead of the keys: a pair is kept iff 0 <= i - j <= l; in a tile
+    // further on iff i - j is the tile's own distance
+    const int back_lo = ti < n_near ? 0 : q0 - k0, back_hi = ti < n_near ? l : q0 - k0;
+    const int back0 = q0 - k0 - (r_base + g) + 2 * t;   // i - j of this lane's first element of query column 0
 #pragma unroll
-  for (int nb = 0; nb < 2; ++nb) {
-    wmma::store_matrix_sync(Sf + r_base * LDF + c_base + nb * 16, acc_k[nb], LDF, wmma::mem_row_major);
-    wmma::store_matrix_sync(Pf + r_base * LDF + c_base + nb * 16, acc_v[nb], LDF, wmma::mem_row_major);
-  }
-  __syncthreads();
-  // queries further on that see this key through the stride: j + 2l, j + 3l, ...
-  for (int r = warp * (TS / BW_WARPS); r < (warp + 1) * (TS / BW_WARPS); ++r) {
-    const int j = k0 + r;
-    const float2 k = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Ks + r * LDB + 2 * lane));
-    const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Vs + r * LDB + 2 * lane));
-    float kx = 0.f, ky = 0.f, vx = 0.f, vy = 0.f;
-    for (int i = j + 2 * l; i < P.seq; i += l) {
-      const float2 q = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(P.Q + (row0 + i) * P.ld + h * D + 2 * lane));
-      const float2 g = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(P.dOut + (row0 + i) * P.lddo + h * D + 2 * lane));
-      float s = q.x * k.x + q.y * k.y, dp = g.x * v.x + g.y * v.y;
-      for (int off = 16; off; off >>= 1) {
-        s += __shfl_xor_sync(0xffffffffu, s, off);
-        dp += __shfl_xor_sync(0xffffffffu, dp, off);
+    for (int half = 0; half < 2; ++half) {              // 32 queries at a time
+      float st[4][4], dp[4][4];                         // S^T and dP^T: rows = keys, columns = queries
+#pragma unroll
+      for (int nb = 0; nb < 4; ++nb) {
+        st[nb][0] = st[nb][1] = st[nb][2] = st[nb][3] = 0.f;
+        dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
+        mma_rows(st[nb], ka, Qs, half * 32 + nb * 8, lane);
+        mma_rows(dp[nb], va, Gs, half * 32 + nb * 8, lane);
       }
-      const float p = __expf(s * SCALE - P.lse[stat0 + i]);
-      const float ds = p * (dp - P.delta[stat0 + i]);
-      vx = fmaf(p, g.x, vx);
-      vy = fmaf(p, g.y, vy);
-      kx = fmaf(ds, q.x, kx);
-      ky = fmaf(ds, q.y, ky);
+#pragma unroll
+      for (int nb = 0; nb < 4; ++nb) {
+        const int c = half * 32 + nb * 8 + 2 * t;
+        const float2 ls = *reinterpret_cast<const float2*>(lse_s + c), dl = *reinterpret_cast<const float2*>(del_s + c);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int back = back0 + (half * 32 + nb * 8 + (i & 1)) - (i >> 1) * 8;
+          float p = 0.f, ds = 0.f;
+          if (back >= back_lo && back <= back_hi) {
+            p = __expf(st[nb][i] * SCALE - ((i & 1) ? ls.y : ls.x));
+            ds = p * (dp[nb][i] - ((i & 1) ? dl.y : dl.x));
+          }
+          st[nb][i] = p;
+          dp[nb][i] = ds;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {                     // 16 queries per step
+        uint32_t pa[4], da[4];
+        pa[0] = pack_bf16(st[2 * j][0], st[2 * j][1]);
+        pa[1] = pack_bf16(st[2 * j][2], st[2 * j][3]);
+        pa[2] = pack_bf16(st[2 * j + 1][0], st[2 * j + 1][1]);
+        pa[3] = pack_bf16(st[2 * j + 1][2], st[2 * j + 1][3]);
+        da[0] = pack_bf16(dp[2 * j][0], dp[2 * j][1]);
+        da[1] = pack_bf16(dp[2 * j][2], dp[2 * j][3]);
+        da[2] = pack_bf16(dp[2 * j + 1][0], dp[2 * j + 1][1]);
+        da[3] = pack_bf16(dp[2 * j + 1][2], dp[2 * j + 1][3]);
+        mma_cols(acc_v, pa, Gs, half * 32 + j * 16, lane);
+        mma_cols(acc_k, da, Qs, half * 32 + j * 16, lane);
+      }
     }
-    const int64_t o = (row0 + j) * P.ldg + h * D + 2 * lane;
-    *reinterpret_cast<__nv_bfloat162*>(P.dK + o) =
-        __floats2bfloat162_rn((Sf[r * LDF + 2 * lane] + kx) * SCALE, (Sf[r * LDF + 2 * lane + 1] + ky) * SCALE);
-    *reinterpret_cast<__nv_bfloat162*>(P.dV + o) = __floats2bfloat162_rn(Pf[r * LDF + 2 * lane] + vx, Pf[r * LDF + 2 * lane + 1] + vy);
+  }
+  __syncthreads();   // every warp is done with the query tiles: their storage takes dK and dV
+  store_acc(Sf, acc_k, r_base, lane);
+  store_acc(Pf, acc_v, r_base, lane);
+  __syncwarp();
+  for (int r = r_base; r < r_base + 16; ++r) {   // lane = two head dimensions
+    const int64_t o = (row0 + k0 + r) * P.ldg + h * D + 2 * lane;
+    *reinterpret_cast<__nv_bfloat162*>(P.dK + o) = __floats2bfloat162_rn(Sf[r * LDF + 2 * lane] * SCALE, Sf[r * LDF + 2 * lane + 1] * SCALE);
+    *reinterpret_cast<__nv_bfloat162*>(P.dV + o) = __floats2bfloat162_rn(Pf[r * LDF + 2 * lane], Pf[r * LDF + 2 * lane + 1]);
   }
 }
 
@@ -356,8 +387,9 @@ extern "C" mst_status_t mst_strided_attention_bwd(const void* Q, const void* K, 
   P.batch = batch; P.seq = seq_len; P.heads = heads; P.stride = stride;
   const int64_t warps = (int64_t)batch * seq_len * heads;
   attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, s>>>(P); MST_COUNT_LAUNCH();
-  const size_t smem_q = (size_t)(7 * TS * LDB) * 2 + (size_t)2 * TS * LDF * 4 + 128;
-  const size_t smem_kv = (size_t)(8 * TS * LDB) * 2 + (size_t)2 * TS * LDF * 4 + 128;
+  static_assert(2 * TS * LDF * 4 <= 4 * TS * LDB * 2, "the staged gradients must fit the tile buffers");
+  const size_t smem_q = (size_t)(6 * TS * LDB) * 2 + 128;
+  const size_t smem_kv = (size_t)(6 * TS * LDB) * 2 + 128;
   MST_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_q));
   MST_CUDA_TRY(cudaFuncSetAttribute(attn_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_kv));
   dim3 grid((unsigned)(seq_len / TS), (unsigned)heads, (unsigned)batch);
