@@ -137,7 +137,7 @@ __device__ __forceinline__ void store_acc(float* out, const float (&acc)[8][4], 
 }
 
 // ------------------------------------------------------------------------------------------- dQ
-__global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dq_kernel(BwdParams P) {
+__global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P) {
   extern __shared__ __align__(128) unsigned char smem[];
   __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem);   // [64][LDB]
   __nv_bfloat16* Gs = Qs + TS * LDB;                             // dOut tile

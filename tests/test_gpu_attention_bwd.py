@@ -45,7 +45,9 @@ def _run(B, n, H, stride, seed, pad=0, std=1.0):
     (2, 512, 3, 128, 0, 1.0),       # far keys i - 2l, i - 3l; two sequences
     (1, 1024, 2, 256, 8, 1.0),      # the paper's stride at n = 1024, padded leading dimension
     (1, 512, 2, 512, 0, 1.0),       # stride = n: plain causal attention
-    (1, 384, 2, 64, 0, 2.0)])       # smallest stride, peaked scores
+    (1, 384, 2, 64, 0, 2.0),        # smallest stride, peaked scores
+    (1, 1024, 1, 64, 0, 1.0),       # up to fourteen strided positions beyond the window: many diagonal-only tiles
+    (1, 768, 2, 192, 8, 1.0)])      # a stride that is not a power of two
 def test_attention_bwd_matches_oracle(B, n, H, stride, pad, std):
     got, ref, _ = _run(B, n, H, stride, 900 + n + stride, pad, std)
     for a, b, name in zip(got, ref, ("dQ", "dK", "dV")):
