@@ -480,7 +480,8 @@ def run_profile_case(args) -> None:
             raise SystemExit("libmst.so was built without -DMST_SP_PROFILE")
         L.set_path(mst.MST_PATH_SPARSE_TC)
         names = ["producer waits for a free stage", "MMA thread waits for a full stage", "MMA thread waits for a free accumulator",
-                 "epilogue warp waits for a complete accumulator", "epilogue warp busy", "whole kernel"]
+                 "epilogue warp waits for a complete accumulator", "epilogue warp busy", "whole kernel",
+                 "epilogue warp waits for tensor-memory loads", "epilogue warp fetches its rows' spill lists"]
         for label, fn in (("forward (K = 1280)", lambda: L.fwd(X, Y, T)), ("input gradient (K = 5120)", lambda: L.bwd_x(dY, dX, T))):
             for _ in range(3):
                 fn()

@@ -61,12 +61,16 @@ __device__ int g_sp_error = 0;  // sticky: 1 = a bounded wait expired
 //   [5] whole kernel
 #ifdef MST_SP_PROFILE
 __device__ long long g_sp_prof[160][8];
-#define SP_PROF_DECL long long prof_t0 = 0, prof_acc0 = 0, prof_acc1 = 0
+#define SP_PROF_DECL long long prof_t0 = 0, prof_acc0 = 0, prof_acc1 = 0, prof_t1 = 0, prof_acc2 = 0, prof_acc3 = 0
+#define SP_PROF_BEGIN1() prof_t1 = clock64()
+#define SP_PROF_END1(acc) acc += clock64() - prof_t1
 #define SP_PROF_BEGIN() prof_t0 = clock64()
 #define SP_PROF_END(acc) acc += clock64() - prof_t0
 #define SP_PROF_STORE(slot, acc) g_sp_prof[blockIdx.x][slot] = acc
 #else
 #define SP_PROF_DECL
+#define SP_PROF_BEGIN1()
+#define SP_PROF_END1(acc)
 #define SP_PROF_BEGIN()
 #define SP_PROF_END(acc)
 #define SP_PROF_STORE(slot, acc)
@@ -117,7 +121,8 @@ __device__ __forceinline__ uint64_t sp_desc_plain(uint32_t saddr, uint32_t lbo, 
   d |= (uint64_t)1 << 46;
   return d;
 }
-__device__ __forceinline__ void sp_tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+// sixteen columns of this thread's tensor-memory lane, issued without waiting: the registers are valid after sp_tmem_wait on them
+__device__ __forceinline__ void sp_tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -125,7 +130,14 @@ __device__ __forceinline__ void sp_tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) 
         "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// wait for the outstanding tensor-memory loads; the registers are operands so that no use of them moves above the wait
+__device__ __forceinline__ void sp_tmem_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(S_THREADS, 1)
@@ -266,8 +278,9 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------------ epilogue (both blocks, own 128 rows of S)
     // A thread owns one output feature (tensor-memory lane) and reads 16 tokens of it at a time.  For a fixed token the
     // 32 lanes of a warp hold 32 consecutive features, so each store instruction writes one 64-byte run of an output
-    // row: no staging through shared memory.  The activations of the row's first spills are fetched one step ahead
-    // (they come from L2: the latency would otherwise be paid once per step).
+    // row.  (Staging the chunk in shared memory for a bulk tensor store was measured slower: 94 K against 87 K cycles
+    // for the forward product of a 5120 x 1280 layer over 8192 tokens.)  The activations of the row's first spills are
+    // fetched one step ahead (they come from L2: the latency would otherwise be paid once per step).
     const int q = warp & 3;                 // tensor-memory lane quarter
     const int c0 = (warp - 2) >> 2;         // the two warps of a quarter take alternate 16-token chunks
     int acc = 0;
@@ -279,6 +292,7 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int64_t r = row0 + lane;        // this thread's row of S = output feature
       const int64_t tok0 = (int64_t)nt * SN;
       // third and fourth entries of this row's groups (rows beyond R have none: their counts are zero)
+      SP_PROF_BEGIN1();
       const int32_t sp0 = P.scan[r * P.chunks], sp1 = P.scan[(r + 1) * P.chunks];
       const int n_fast = min(sp1 - sp0, S_FAST_SPILLS);
       const int n_fast_warp = __reduce_max_sync(0xffffffffu, n_fast);
@@ -304,47 +318,75 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       };
       if (n_fast_warp > 0) fetch(c0);
+      SP_PROF_END1(prof_acc3);
       SP_PROF_BEGIN();
       if (!sp_wait(tfull0 + 8 * acc, acc_ph, abort_flag)) break;
       SP_PROF_END(prof_acc0);
       tc_fence_after();
       SP_PROF_BEGIN();
-#pragma unroll 1
-      for (int c = c0; c < SN / S_CHUNK; c += 2) {
+      // one 16-token chunk: spills added, rounded, written.  The tensor-memory load of the warp's next chunk is issued
+      // before the chunk in hand is processed, so its latency hides behind the stores.
+      auto chunk = [&](int c, uint32_t (&v)[16]) {
         const int64_t t0 = tok0 + c * S_CHUNK;
-        if (t0 >= P.T) break;  // uniform
-        uint32_t v[16];
-        uint4 xc[S_FAST_SPILLS][2];
+        if (n_fast_warp > 0) {   // uniform over the warp: some row of this warp has spills in this tile
+          uint4 xc[S_FAST_SPILLS][2];
 #pragma unroll
-        for (int j = 0; j < S_FAST_SPILLS; ++j) { xc[j][0] = xn[j][0]; xc[j][1] = xn[j][1]; }
-        if (n_fast_warp > 0) fetch(c + 2);
-        sp_tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * SN + c * S_CHUNK), v);
-        auto add_spill = [&](float wj, const uint4& x0, const uint4& x1) {
-          const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+          for (int j = 0; j < S_FAST_SPILLS; ++j) { xc[j][0] = xn[j][0]; xc[j][1] = xn[j][1]; }
+          fetch(c + 2);
+          auto add_spill = [&](float wj, const uint4& x0, const uint4& x1) {
+            const uint32_t xw[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            v[2 * i] = __float_as_uint(fmaf(wj, __uint_as_float(xw[i] << 16), __uint_as_float(v[2 * i])));
-            v[2 * i + 1] = __float_as_uint(fmaf(wj, __uint_as_float(xw[i] & 0xFFFF0000u), __uint_as_float(v[2 * i + 1])));
+            for (int i = 0; i < 8; ++i) {
+              v[2 * i] = __float_as_uint(fmaf(wj, __uint_as_float(xw[i] << 16), __uint_as_float(v[2 * i])));
+              v[2 * i + 1] = __float_as_uint(fmaf(wj, __uint_as_float(xw[i] & 0xFFFF0000u), __uint_as_float(v[2 * i + 1])));
+            }
+          };
+#pragma unroll
+          for (int j = 0; j < S_FAST_SPILLS; ++j)
+            if (j < n_fast) add_spill(wv[j], xc[j][0], xc[j][1]);
+          // rows with more spills than the prefetch holds: one at a time
+          for (int32_t e = sp0 + S_FAST_SPILLS; e < sp1; ++e) {
+            const uint32_t ent = __ldg(P.spill + e);
+            const uint4* src = reinterpret_cast<const uint4*>(P.xr + (int64_t)(ent >> 16) * P.ldxr + t0);
+            add_spill(__uint_as_float(ent << 16), __ldg(src), __ldg(src + 1));
           }
-        };
-#pragma unroll
-        for (int j = 0; j < S_FAST_SPILLS; ++j)
-          if (j < n_fast) add_spill(wv[j], xc[j][0], xc[j][1]);
-        // rows with more spills than the prefetch holds: one at a time
-        for (int32_t e = sp0 + S_FAST_SPILLS; e < sp1; ++e) {
-          const uint32_t ent = __ldg(P.spill + e);
-          const uint4* src = reinterpret_cast<const uint4*>(P.xr + (int64_t)(ent >> 16) * P.ldxr + t0);
-          add_spill(__uint_as_float(ent << 16), __ldg(src), __ldg(src + 1));
         }
         if (r < P.R) {
           uint16_t* dst = P.out + t0 * P.ldout + r;
+          if (t0 + S_CHUNK <= P.T) {   // uniform: the whole chunk lies inside
 #pragma unroll
-          for (int j = 0; j < 16; j += 2) {
-            const uint32_t pk = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-            if (t0 + j < P.T) dst[(int64_t)j * P.ldout] = (uint16_t)(pk & 0xFFFFu);
-            if (t0 + j + 1 < P.T) dst[(int64_t)(j + 1) * P.ldout] = (uint16_t)(pk >> 16);
+            for (int j = 0; j < 16; j += 2) {
+              const uint32_t pk = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+              dst[(int64_t)j * P.ldout] = (uint16_t)(pk & 0xFFFFu);
+              dst[(int64_t)(j + 1) * P.ldout] = (uint16_t)(pk >> 16);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+              const uint32_t pk = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+              if (t0 + j < P.T) dst[(int64_t)j * P.ldout] = (uint16_t)(pk & 0xFFFFu);
+              if (t0 + j + 1 < P.T) dst[(int64_t)(j + 1) * P.ldout] = (uint16_t)(pk >> 16);
+            }
           }
         }
+      };
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * SN);
+      auto chunk_valid = [&](int c) { return c < SN / S_CHUNK && tok0 + (int64_t)c * S_CHUNK < P.T; };   // uniform
+      uint32_t va[16], vb[16];
+      if (chunk_valid(c0)) sp_tmem_ld16_issue(tacc + (uint32_t)(c0 * S_CHUNK), va);
+#pragma unroll 1
+      for (int c = c0; chunk_valid(c); c += 4) {
+        SP_PROF_BEGIN1();
+        sp_tmem_wait(va);
+        SP_PROF_END1(prof_acc2);
+        if (chunk_valid(c + 2)) sp_tmem_ld16_issue(tacc + (uint32_t)((c + 2) * S_CHUNK), vb);
+        chunk(c, va);
+        if (!chunk_valid(c + 2)) break;
+        SP_PROF_BEGIN1();
+        sp_tmem_wait(vb);
+        SP_PROF_END1(prof_acc2);
+        if (chunk_valid(c + 4)) sp_tmem_ld16_issue(tacc + (uint32_t)((c + 4) * S_CHUNK), va);
+        chunk(c + 2, vb);
       }
       tc_fence_before();
       __syncwarp();
@@ -355,6 +397,8 @@ tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 2 && lane == 0) {
       SP_PROF_STORE(3, prof_acc0);
       SP_PROF_STORE(4, prof_acc1);
+      SP_PROF_STORE(6, prof_acc2);
+      SP_PROF_STORE(7, prof_acc3);
     }
   }
 
