@@ -469,7 +469,8 @@ __global__ void sp24_compress_kernel(const uint32_t* __restrict__ bits, const in
                                      int kblocks, int chunks, uint16_t* __restrict__ ac, uint16_t* __restrict__ meta16,
                                      int32_t* __restrict__ cnt, const int32_t* __restrict__ scan,
                                      int32_t* __restrict__ col_flag, const int32_t* __restrict__ col_slot,
-                                     uint32_t* __restrict__ spill, int64_t spill_cap, int mode) {
+                                     uint32_t* __restrict__ spill, int64_t spill_cap, int32_t* __restrict__ place,
+                                     int mode) {
   mst_grid_launch_dependents();
   mst_grid_dependency_wait();
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -546,6 +547,11 @@ __global__ void sp24_compress_kernel(const uint32_t* __restrict__ bits, const in
     const uint32_t lo = s0 >= 0 ? (uint32_t)vals[s0] : 0u;
     const uint32_t hi = s1 >= 0 ? (uint32_t)vals[s1] : 0u;
     outw[g] = lo | (hi << 16);
+    if (place && mode == 1) {
+      const int32_t at = (int32_t)(r * (kd_pad >> 1) + (k0 >> 1) + 2 * g);
+      if (s0 >= 0) place[s0] = at;
+      if (s1 >= 0) place[s1] = at + 1;
+    }
     m16 |= G.nib << (4 * g);
     if (n > 2) {
       extra += n - 2;
@@ -560,6 +566,7 @@ __global__ void sp24_compress_kernel(const uint32_t* __restrict__ bits, const in
               col_flag[k] = 1;
             } else if (e_at < spill_cap) {
               spill[e_at] = ((uint32_t)col_slot[k] << 16) | (uint32_t)vals[seen == 2 ? ent[2] : ent[3]];
+              if (place) place[seen == 2 ? ent[2] : ent[3]] = -(e_at + 1);
               ++e_at;
             }
           }
@@ -571,6 +578,20 @@ __global__ void sp24_compress_kernel(const uint32_t* __restrict__ bits, const in
   *reinterpret_cast<uint4*>(ac + r * (kd_pad >> 1) + (k0 >> 1)) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
   meta16[meta_half_index(r, k0, kblocks)] = (uint16_t)m16;
   if (mode == 0) cnt[r * chunks + chunk] = extra;
+}
+
+// The values of the stored entries have changed, the mask has not: every value goes to the place the last compression
+// gave its entry (an element of the compressed operand, or the low half of a spill word).
+__global__ void sp24_scatter_values_kernel(const uint16_t* __restrict__ vals, const int32_t* __restrict__ place, int64_t nnz,
+                                           uint16_t* __restrict__ ac, uint32_t* __restrict__ spill) {
+  mst_grid_launch_dependents();
+  mst_grid_dependency_wait();
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= nnz) return;
+  const int32_t at = place[e];
+  const uint16_t v = vals[e];
+  if (at >= 0) ac[at] = v;
+  else reinterpret_cast<uint16_t*>(spill)[2 * (int64_t)(-(at + 1))] = v;   // little-endian: the value is the low half
 }
 
 __global__ void sp24_slot_cols_kernel(const int32_t* __restrict__ col_flag, const int32_t* __restrict__ col_slot, int kd_pad,
@@ -683,6 +704,9 @@ mst_status_t sp24_ensure(mst_layer* L, int dir) {
   const size_t o_slot = cv.take(4 * (size_t)(S.kd_pad + 1));
   const size_t o_scol = cv.take(4 * (size_t)S.kd_pad);
   const size_t o_bsum = cv.take(4 * (size_t)(mst_scan_block_sums_len(n_cnt) + 1024));
+  // places of the stored entries, when an element index of the compressed operand fits 32 bits
+  const bool keep_place = S.r_pad * (S.kd_pad / 2) < 0x7FFFFFFFLL;
+  const size_t o_place = keep_place ? cv.take(4 * (size_t)(L->cap > 0 ? L->cap : 1)) : 0;
   MST_CUDA_TRY(cudaMalloc((void**)&S.base, cv.off));
   S.ac = (uint16_t*)(S.base + o_ac);
   S.meta = (uint32_t*)(S.base + o_meta);
@@ -693,6 +717,8 @@ mst_status_t sp24_ensure(mst_layer* L, int dir) {
   S.col_slot = (int32_t*)(S.base + o_slot);
   S.slot_col = (int32_t*)(S.base + o_scol);
   S.bsums = (int32_t*)(S.base + o_bsum);
+  S.place = keep_place ? (int32_t*)(S.base + o_place) : nullptr;
+  S.place_version = -1;
   S.struct_version = -1;
   return MST_OK;
 }
@@ -706,14 +732,14 @@ mst_status_t sp24_launch_compress(mst_layer* L, int mode, cudaStream_t s) {
   MST_CUDA_TRY(mst_launch_overlapped(sp24_compress_kernel<DIR>, dim3(blocks), dim3(256), 0, s, (const uint32_t*)L->bits[c],
                                      (const int32_t*)L->wscan[c], (const uint16_t*)L->vals[c], L->O, L->I, L->wpr, S.r_pad,
                                      S.kd_pad, S.kblocks, S.chunks, S.ac, (uint16_t*)S.meta, S.cnt, (const int32_t*)S.scan,
-                                     S.col_flag, (const int32_t*)S.col_slot, S.spill, S.spill_cap, mode));
+                                     S.col_flag, (const int32_t*)S.col_slot, S.spill, S.spill_cap, S.place, mode));
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
 
-// Compressed operand, metadata and spill list of the live structure and the current values.  The values may have been
-// changed in place since the last call, so the compression runs every time; the positions of the spills depend on the
-// mask only and are rebuilt when it has changed.
+// Compressed operand, metadata and spill list of the live structure and the current values.  The positions depend on
+// the mask only and are rebuilt when it has changed; the values may have been changed in place since the last call,
+// so they are written again every time (a scatter over the stored entries to the places the compression recorded).
 mst_status_t sp24_refresh(mst_layer* L, int dir, cudaStream_t s) {
   MST_TRY(sp24_ensure(L, dir));
   mst_sp24& S = L->sp[dir];
@@ -730,7 +756,16 @@ mst_status_t sp24_refresh(mst_layer* L, int dir, cudaStream_t s) {
   // with value tracking the compressed operand is reused until the values change
   if (L->track_values && S.values_epoch == L->values_epoch) return MST_OK;
   S.values_epoch = L->values_epoch;
-  return dir == 0 ? sp24_launch_compress<0>(L, 1, s) : sp24_launch_compress<1>(L, 1, s);
+  if (S.place && S.place_version == L->version) {
+    if (L->nnz == 0) return MST_OK;
+    MST_CUDA_TRY(mst_launch_overlapped(sp24_scatter_values_kernel, dim3((unsigned)((L->nnz + 255) / 256)), dim3(256), 0, s,
+                                       (const uint16_t*)L->vals[L->cur], (const int32_t*)S.place, (int64_t)L->nnz, S.ac, S.spill));
+    MST_CUDA_TRY(cudaGetLastError());
+    return MST_OK;
+  }
+  MST_TRY(dir == 0 ? sp24_launch_compress<0>(L, 1, s) : sp24_launch_compress<1>(L, 1, s));
+  S.place_version = L->version;
+  return MST_OK;
 }
 
 }  // namespace

@@ -25,12 +25,14 @@ struct mst_sp24 {
   int32_t* col_slot = nullptr;    // [kd_pad + 1] exclusive scan of col_flag; col_slot[kd_pad] = number of such columns
   int32_t* slot_col = nullptr;    // [kd_pad]     inverse map
   int32_t* bsums = nullptr;       // scan partials
+  int32_t* place = nullptr;       // [cap] where stored entry e went: >= 0 element of ac, < 0 spill -(index + 1); nullptr: not kept
   int R = 0, Kd = 0;
   int64_t r_pad = 0;
   int kd_pad = 0, kblocks = 0, chunks = 0;
   int64_t spill_cap = 0;
   int64_t struct_version = -1;    // layer structure version the spill positions belong to
   int64_t values_epoch = -1;      // values epoch the compressed operand was built from (value tracking only)
+  int64_t place_version = -1;     // layer structure version `place` belongs to
 };
 
 // true when the operands can be described to the TMA unit and the layer's nnz fits the spill capacity
