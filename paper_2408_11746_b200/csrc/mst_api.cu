@@ -133,6 +133,7 @@ extern "C" mst_status_t mst_layer_create(mst_layer_t** out, int32_t layer_id, in
   L->rand_ctr = (unsigned long long*)(base + o_rctr);
   L->rand_cap = (int)rand_cap;
   L->scratch_clean = 1;   // the allocation was cleared above
+  L->longest_row_version = -1;
   L->sel = (mst_select_state*)(base + o_sel);
   L->flags = (int32_t*)(base + o_flags);
   L->counter = (unsigned int*)(base + o_counter);

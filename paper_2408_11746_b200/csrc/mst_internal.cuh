@@ -131,7 +131,8 @@ struct mst_layer {
   int rand_cap;
   int scratch_clean;      // hist and rand_ctr are known to be zero (the fused update kernel leaves them so)
   mst_select_state* sel;  // [1]
-  int32_t* flags;         // [4]: error bits, max row nnz, spare
+  int32_t* flags;         // [4]: error bits, max row nnz of the last update, longest row (CUDA-core forward), spare
+  mutable int64_t longest_row_version;  // structure version flags[2] belongs to
   unsigned int* counter;  // [1] block-completion counter
 
   // dense bf16 image of W.M for the tensor-core path (bf16 layers only): [O x I]; the input gradient reads it as an

@@ -14,7 +14,12 @@
 // Work is proportional to nnz: a (row, chunk) visit costs a ballot over a 32-entry window of the row kept in
 // registers, and global index/value loads happen only when a window is used up (coalesced, 32 entries).
 // Rows of unequal nnz: inside a panel the rows are dealt to the warps in order of decreasing nnz, back and forth,
-// so every warp gets a similar count; panels are many more than SMs and are scheduled dynamically.
+// so every warp gets a similar count; panels are many more than SMs and are scheduled dynamically.  When the longest
+// row of the matrix has a thousand entries or more and is far above the mean (recorded on the device when the
+// structure changes), a panel keeps a fifth of its row slots free and hands them to its longest rows as extra
+// segments (every cnt-th entry of the row each, so that a segment has its share of every column chunk): a long row
+// is then summed by up to 1 + 3 x (rows per warp) warps, and the epilogue adds the segments' partial sums in a fixed
+// order.
 // The output tile leaves through shared memory so that global stores are contiguous along the feature dimension.
 #include <cuda.h>
 
@@ -141,14 +146,27 @@ __global__ void __launch_bounds__(256) transpose_in_kernel(const T* __restrict__
   }
 }
 
+constexpr int SPLIT_MIN = 64;   // a segment of a split row keeps at least this many entries
+constexpr int SPLIT_LONGEST = 1024;   // rows are split only in matrices whose longest row has at least this many
+
+// longest row of the matrix (rows = the ptr array's rows) into *out, which the caller cleared
+__global__ void longest_row_kernel(const int32_t* __restrict__ ptr, int R, int32_t* out) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  int v = r < R ? ptr[r + 1] - ptr[r] : 0;
+  for (int o = 16; o; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  if ((threadIdx.x & 31) == 0 && v > 0) atomicMax(out, v);
+}
+
 template <typename T, bool PERM, int RPW>
 __global__ void __launch_bounds__(THREADS, 1)
 spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __restrict__ ptr,
                    const uint16_t* __restrict__ idx, const T* __restrict__ vals, const int32_t* __restrict__ perm,
-                   T* __restrict__ out, int64_t ldout, int64_t T_total, int R_total, int C) {
+                   T* __restrict__ out, int64_t ldout, int64_t T_total, int R_total, int C,
+                   const int32_t* __restrict__ longest_row) {
   using namespace mst_ptx;
   constexpr int KC = Cfg<T>::KC;
-  constexpr int PANEL = WARPS * RPW;
+  constexpr int PANEL = WARPS * RPW;          // row slots of a block
+  constexpr int SPARE = 3 * RPW;              // slots kept free for extra segments when rows are split
   constexpr int OS_LD = PANEL + 1;
   constexpr uint32_t STAGE_BYTES = (uint32_t)(KC * TOK * sizeof(T));
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -156,14 +174,26 @@ spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __re
   const uint32_t tiles_base = (raw + 127u) & ~127u;
   unsigned char* tiles = smem_raw + (tiles_base - raw);
   __shared__ uint64_t bars[2 * STAGES];
-  __shared__ int nnz_sh[PANEL];
-  __shared__ unsigned char order_sh[PANEL];   // order_sh[w * RPW + j] = local row of warp w's j-th row
+  __shared__ int nnz_sh[PANEL];               // entries of a slot
+  __shared__ int rown_sh[PANEL];              // entries of a row of the panel
+  __shared__ int slot_beg[PANEL], slot_end[PANEL];
+  __shared__ unsigned char seg_first[PANEL], seg_cnt[PANEL];   // a row's slots: seg_first[row] .. + seg_cnt[row]
+  __shared__ unsigned char slot_step[PANEL];  // a slot takes every slot_step-th entry of its row (1: the whole row)
+  __shared__ unsigned char order_sh[PANEL];   // order_sh[w * RPW + j] = slot of warp w's j-th row
   __shared__ int abort_sh;
   volatile int* abort_flag = &abort_sh;
   const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[STAGES]);
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int r0 = blockIdx.x * PANEL;
+  // rows are split when the longest row of the matrix is far above the mean (uniform over the grid; the grid is
+  // sized for the split form, whose panels hold fewer rows: without splitting the surplus blocks have nothing to do)
+  const int longest = longest_row ? *longest_row : 0;
+  // (measured on GPT-2-small shapes with Zipf rows: a gain for rows of thousands of entries, 0.51 -> 0.36 ms on a
+  // 768 x 3072 layer; a loss for 768-wide layers, where a fifth more panels cost more than the balance gains)
+  const bool split = longest >= SPLIT_LONGEST && (int64_t)longest * R_total > 4 * (int64_t)ptr[R_total] + 64 * (int64_t)R_total;
+  const int rows_here = split ? PANEL - SPARE : PANEL;
+  const int r0 = blockIdx.x * rows_here;
+  if (r0 >= R_total) return;
   const int64_t t0 = (int64_t)blockIdx.y * TOK;
   if (threadIdx.x == 0) {
     abort_sh = 0;
@@ -173,12 +203,89 @@ spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __re
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // rows of the panel in order of decreasing nnz, dealt to the warps back and forth
+  // slots: one per row, or several for the longest rows of the panel when rows are split
   if (threadIdx.x < PANEL) {
     const int r = r0 + threadIdx.x;
-    nnz_sh[threadIdx.x] = r < R_total ? ptr[r + 1] - ptr[r] : -1;
+    const bool have = (int)threadIdx.x < rows_here && r < R_total;
+    rown_sh[threadIdx.x] = have ? ptr[r + 1] - ptr[r] : -1;
+    seg_cnt[threadIdx.x] = 1;
+    slot_step[threadIdx.x] = 1;
+    seg_first[threadIdx.x] = (unsigned char)threadIdx.x;
+    nnz_sh[threadIdx.x] = have ? ptr[r + 1] - ptr[r] : -1;
+    slot_beg[threadIdx.x] = have ? ptr[r] : 0;
+    slot_end[threadIdx.x] = have ? ptr[r + 1] : 0;
   }
   __syncthreads();
+  if (split) {   // uniform over the block
+    if (warp == 0) {
+      // the free slots go, one at a time, to the row whose segments are longest (ties: the lower row)
+      int seg[4] = {1, 1, 1, 1};   // rows lane, lane + 32, lane + 64, lane + 96
+      for (int it = 0; it < SPARE; ++it) {
+        int best = 0, best_row = 0x7FFFFFFF;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int rl = lane + 32 * k;
+          if (rl < rows_here) {
+            const int n = rown_sh[rl];
+            const int per = n > 0 ? (n + seg[k] - 1) / seg[k] : 0;
+            if (per > best || (per == best && rl < best_row)) { best = per; best_row = rl; }
+          }
+        }
+        for (int o = 16; o; o >>= 1) {
+          const int ob = __shfl_xor_sync(0xffffffffu, best, o), orow = __shfl_xor_sync(0xffffffffu, best_row, o);
+          if (ob > best || (ob == best && orow < best_row)) { best = ob; best_row = orow; }
+        }
+        if (best < 2 * SPLIT_MIN) break;   // uniform: splitting further would leave segments below the minimum
+        if ((best_row & 31) == lane) ++seg[best_row >> 5];
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (lane + 32 * k < rows_here) seg_cnt[lane + 32 * k] = (unsigned char)seg[k];
+      __syncwarp();
+      // first slot of every row: exclusive prefix of the segment counts in row order (lane = four consecutive rows)
+      int mine[4], tot = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int rl = lane * 4 + k;
+        mine[k] = rl < rows_here ? seg_cnt[rl] : 0;
+        tot += mine[k];
+      }
+      int incl = tot;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      int at = incl - tot;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int rl = lane * 4 + k;
+        if (rl < rows_here) seg_first[rl] = (unsigned char)at;
+        at += mine[k];
+      }
+      const int used = __shfl_sync(0xffffffffu, incl, 31);
+      for (int sl = used + lane; sl < PANEL; sl += 32) {   // slots left over
+        nnz_sh[sl] = -1;
+        slot_beg[sl] = slot_end[sl] = 0;
+        slot_step[sl] = 1;
+      }
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < rows_here) {
+      const int r = r0 + threadIdx.x;
+      // segment j of a row split in cnt takes the entries j, j + cnt, j + 2 cnt, ... of the row: columns still ascend
+      // inside a segment, and every segment has its share of every column chunk
+      const int n = rown_sh[threadIdx.x], cnt = seg_cnt[threadIdx.x], first = seg_first[threadIdx.x];
+      const int beg = n >= 0 ? ptr[r] : 0, end = n >= 0 ? beg + n : 0;
+      for (int j = 0; j < cnt; ++j) {
+        slot_beg[first + j] = beg + j < end ? beg + j : end;
+        slot_end[first + j] = end;
+        slot_step[first + j] = (unsigned char)cnt;
+        nnz_sh[first + j] = n >= 0 ? (n - j + cnt - 1) / cnt : -1;
+      }
+    }
+    __syncthreads();
+  }
+  // slots in order of decreasing nnz, dealt to the warps back and forth
   if (threadIdx.x < PANEL) {
     const int mine = nnz_sh[threadIdx.x];
     int rank = 0;
@@ -212,7 +319,7 @@ spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __re
     uint32_t wci[RPW], wval[RPW];   // this lane's entry of the row's current 32-entry window: column, value bits
     float acc[RPW][8];
     auto load_window = [&](int rr) {
-      const int32_t kk = kwin[rr] + lane;
+      const int32_t kk = kwin[rr] + lane * (int)slot_step[rloc[rr]];
       wci[rr] = 0xFFFFFFFFu;
       wval[rr] = 0u;
       if (kk < kend[rr]) {
@@ -223,9 +330,8 @@ spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __re
 #pragma unroll
     for (int rr = 0; rr < RPW; ++rr) {
       rloc[rr] = order_sh[warp * RPW + rr];
-      const int r = r0 + rloc[rr];
-      kwin[rr] = r < R_total ? ptr[r] : 0;
-      kend[rr] = r < R_total ? ptr[r + 1] : 0;
+      kwin[rr] = slot_beg[rloc[rr]];
+      kend[rr] = slot_end[rloc[rr]];
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[rr][j] = 0.f;
     }
@@ -275,7 +381,7 @@ spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __re
             fma8(acc[rr], wa, Xs + ca * TOK + lane * 8);
           }
           if (first + n < 32) break;        // the window still holds entries of later chunks (or the row has ended)
-          kwin[rr] += 32;                   // window used up: next 32 entries of the row
+          kwin[rr] += 32 * (int)slot_step[rloc[rr]];   // window used up: next 32 entries of the slot
           load_window(rr);
         }
       }
@@ -293,11 +399,26 @@ spmm_stream_kernel(const __grid_constant__ CUtensorMap tmIn, const int32_t* __re
 #pragma unroll
       for (int j = 0; j < 8; ++j) Os[(j * 32 + lane) * OS_LD + rloc[rr]] = acc[rr][j];
     asm volatile("bar.sync 1, %0;" ::"n"(WARPS * 32) : "memory");
-    for (int i = threadIdx.x; i < TOK * PANEL; i += WARPS * 32) {
-      const int tt = i / PANEL, rl = i % PANEL;
-      const int64_t t = t0 + tt;
-      const int r = r0 + rl;
-      if (t < T_total && r < R_total) store_out(out + t * ldout + r, Os[((tt & 7) * 32 + (tt >> 3)) * OS_LD + rl]);
+    if (!split) {
+      for (int i = threadIdx.x; i < TOK * PANEL; i += WARPS * 32) {
+        const int tt = i / PANEL, rl = i % PANEL;
+        const int64_t t = t0 + tt;
+        const int r = r0 + rl;
+        if (t < T_total && r < R_total) store_out(out + t * ldout + r, Os[((tt & 7) * 32 + (tt >> 3)) * OS_LD + rl]);
+      }
+    } else {
+      constexpr int ROWS = PANEL - SPARE;
+      for (int i = threadIdx.x; i < TOK * ROWS; i += WARPS * 32) {
+        const int tt = i / ROWS, rl = i % ROWS;
+        const int64_t t = t0 + tt;
+        const int r = r0 + rl;
+        if (t < T_total && r < R_total) {
+          const float* o = Os + ((tt & 7) * 32 + (tt >> 3)) * OS_LD + seg_first[rl];
+          float v = o[0];
+          for (int j = 1; j < (int)seg_cnt[rl]; ++j) v += o[j];   // a split row's segments, in order
+          store_out(out + t * ldout + r, v);
+        }
+      }
     }
   }
 }
@@ -333,20 +454,23 @@ constexpr size_t spmm_smem() {
 
 template <typename T, bool PERM, int RPW>
 mst_status_t launch_rpw(const CUtensorMap& tm, const int32_t* ptr, const uint16_t* idx, const void* vals, const int32_t* perm,
-                        void* out, int64_t ldout, int64_t T_total, int R_total, int C, cudaStream_t s) {
-  constexpr int PANEL = WARPS * RPW;
+                        void* out, int64_t ldout, int64_t T_total, int R_total, int C, const int32_t* longest_row, cudaStream_t s) {
+  // with a longest-row record the kernel may split rows: its panels then hold a fifth fewer rows, and the grid is
+  // sized for that form
+  const int PANEL = longest_row ? WARPS * RPW - 3 * RPW : WARPS * RPW;
   const size_t smem = spmm_smem<T>();
   // per call: the attribute belongs to the current device's copy of the kernel
   MST_CUDA_TRY(cudaFuncSetAttribute(spmm_stream_kernel<T, PERM, RPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((unsigned)((R_total + PANEL - 1) / PANEL), (unsigned)((T_total + TOK - 1) / TOK));
-  spmm_stream_kernel<T, PERM, RPW><<<grid, THREADS, smem, s>>>(tm, ptr, idx, (const T*)vals, perm, (T*)out, ldout, T_total, R_total, C); MST_COUNT_LAUNCH();
+  spmm_stream_kernel<T, PERM, RPW><<<grid, THREADS, smem, s>>>(tm, ptr, idx, (const T*)vals, perm, (T*)out, ldout, T_total, R_total, C, longest_row); MST_COUNT_LAUNCH();
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }
 
 template <typename T, bool PERM>
 mst_status_t launch(const int32_t* ptr, const uint16_t* idx, const void* vals, const int32_t* perm, const void* in,
-                    int64_t ldin, void* out, int64_t ldout, int64_t T_total, int R_total, int C, cudaStream_t s) {
+                    int64_t ldin, void* out, int64_t ldout, int64_t T_total, int R_total, int C, const int32_t* longest_row,
+                    cudaStream_t s) {
   // feature-major copy of the activations: [C x ldt], ldt a multiple of 64 tokens
   const int64_t ldt = (T_total + 63) / 64 * 64;
   const mst_dtype_t dt = sizeof(T) == 2 ? MST_BF16 : MST_F32;
@@ -364,10 +488,10 @@ mst_status_t launch(const int32_t* ptr, const uint16_t* idx, const void* vals, c
       sms = 148;
   }
   auto blocks = [&](int rpw) { return ((int64_t)R_total + WARPS * rpw - 1) / (WARPS * rpw) * ttiles; };
-  if (blocks(8) >= 2 * sms) return launch_rpw<T, PERM, 8>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
-  if (blocks(4) >= 2 * sms) return launch_rpw<T, PERM, 4>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
-  if (blocks(2) >= sms) return launch_rpw<T, PERM, 2>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
-  return launch_rpw<T, PERM, 1>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, s);
+  if (blocks(8) >= 2 * sms) return launch_rpw<T, PERM, 8>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, longest_row, s);
+  if (blocks(4) >= 2 * sms) return launch_rpw<T, PERM, 4>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, longest_row, s);
+  if (blocks(2) >= sms) return launch_rpw<T, PERM, 2>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, longest_row, s);
+  return launch_rpw<T, PERM, 1>(tm, ptr, idx, vals, perm, out, ldout, T_total, R_total, C, longest_row, s);
 }
 
 // Element-wise pass behind the CUDA-core product (the tensor path fuses it into its epilogue instead).
@@ -464,14 +588,22 @@ mst_status_t mst_launch_spmm(const mst_layer* L, bool transpose, const void* in,
   const int64_t ldprod = (act == MST_ACT_GELU && pre) ? ldpre : ldout;
   mst_status_t st;
   if (!transpose) {
+    // the longest row of the live structure, kept on the device for the kernel's choice between whole and split rows
+    int32_t* longest = L->flags + 2;
+    if (L->longest_row_version != L->version) {
+      MST_CUDA_TRY(cudaMemsetAsync(longest, 0, sizeof(int32_t), s));
+      longest_row_kernel<<<(unsigned)((L->O + 255) / 256), 256, 0, s>>>(L->row_ptr[c], L->O, longest); MST_COUNT_LAUNCH();
+      MST_CUDA_TRY(cudaGetLastError());
+      L->longest_row_version = L->version;
+    }
     st = L->dtype == MST_F32
-             ? launch<float, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, s)
-             : launch<uint16_t, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, s);
+             ? launch<float, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, longest, s)
+             : launch<uint16_t, false>(L->row_ptr[c], L->col_idx[c], L->vals[c], nullptr, in, ldin, prod, ldprod, T, L->O, L->I, longest, s);
   } else {
     MST_TRY(mst_ensure_csc(L, s));
     st = L->dtype == MST_F32
-             ? launch<float, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, s)
-             : launch<uint16_t, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, s);
+             ? launch<float, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, nullptr, s)
+             : launch<uint16_t, true>(L->col_ptr, L->row_idx, L->vals[c], L->perm, in, ldin, prod, ldprod, T, L->I, L->O, nullptr, s);
   }
   if (st != MST_OK || act == MST_ACT_NONE) return st;
   return L->dtype == MST_F32 ? launch_act<float>(out, ldout, pre, ldpre, T, rows, act, s)

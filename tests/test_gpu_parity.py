@@ -137,6 +137,33 @@ def test_step_host_matches_device_entry_points():
     L.close()
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("O,I,T,n_full", [(400, 1536, 300, 3), (1200, 2048, 520, 5), (97, 1024, 64, 1), (400, 768, 300, 3)])
+def test_cuda_core_forward_splits_long_rows(O, I, T, n_full, dtype):
+    # a few complete rows in an otherwise 3 % dense mask: the longest row is far above the mean, so the CUDA-core
+    # forward hands the long rows (a thousand entries or more; the last case stays below that) to several warps; same
+    # results as the checker, identical bits from run to run
+    p = _problem(O, I, T, dtype, 0.03, 5200 + O, "uniform")
+    rng = np.random.default_rng(O + T)
+    full = rng.choice(O, size=n_full, replace=False)
+    p.mask[full, :] = 1
+    p.mask[full[0], ::3] = 0                       # one long row that is not complete
+    L = make_layer(p)
+    L.set_path(mst.MST_PATH_CUDA_CORE)
+    Wm = np.where(p.mask == 1, p.W, np.float32(0))
+    X = to_dev(p, "X")
+    outs = []
+    for rep in range(2):
+        Y = torch.full((T, O), float("nan"), dtype=tdtype(p), device=dev())
+        mst.mst_spmm_fwd(L.handle, X, I, T, Y, O)
+        torch.cuda.synchronize()
+        outs.append(host(Y))
+    assert rel_err(outs[0], oracle.fwd(p.X, Wm, p.mask)) <= TOL[dtype]
+    np.testing.assert_array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
+    assert mst.mst_device_error_flags() == 0
+    L.close()
+
+
 # ------------------------------------------------------------ topology update
 def _update_both(L, p, W, M, G, zeta, target, R, seed, step, allow=False):
     """Run one update on the GPU and in the oracle from the same state; compare bit-exactly."""
