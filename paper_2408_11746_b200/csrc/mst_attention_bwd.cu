@@ -98,6 +98,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+constexpr float SCALE_LOG2E = SCALE * 1.4426950408889634f;   // exp(s / sqrt(d) - lse) = 2^(s * SCALE_LOG2E - lse * log2(e))
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -176,7 +182,7 @@ __global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P)
     load_a(qa[kb], Qs, r_base, kb, lane);
     load_a(ga[kb], Gs, r_base, kb, lane);
   }
-  const float lse0 = lse_s[r_base + g], lse1 = lse_s[r_base + g + 8];
+  const float nl0 = -lse_s[r_base + g] * 1.4426950408889634f, nl1 = -lse_s[r_base + g + 8] * 1.4426950408889634f;
   const float del0 = del_s[r_base + g], del1 = del_s[r_base + g + 8];
   float acc[8][4];
 #pragma unroll
@@ -198,6 +204,41 @@ __global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P)
     // and the first strided position i - l); in a tile further back iff i - j is the tile's own distance
     const int back_lo = ti < n_near ? 0 : q0 - k0, back_hi = ti < n_near ? l : q0 - k0;
     const int back0 = q0 - k0 + r_base + g - 2 * t;   // i - j of this lane's first element of key column 0
+    if (ti >= n_near) {
+      // a tile further back: query r sees key r of the tile only, so of the 64 keys just the 16 in line with this
+      // warp's rows matter (two score tiles of 16 x 8, one 16-key step of the second product)
+      const int c0 = r_base;                            // first of those keys
+      float sc[2][4], dp[2][4];
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb) {
+        sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
+        dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
+        mma_rows(sc[nb], qa, Ks, c0 + nb * 8, lane);
+        mma_rows(dp[nb], ga, Vs, c0 + nb * 8, lane);
+      }
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          // row r_base + g + 8 (i >> 1) against key c0 + 8 nb + 2 t + (i & 1): kept on the diagonal
+          float ds = 0.f;
+          if (g + (i >> 1) * 8 == nb * 8 + 2 * t + (i & 1)) {
+            const float p = ex2_approx(fmaf(sc[nb][i], SCALE_LOG2E, (i >> 1) ? nl1 : nl0));
+            ds = p * (dp[nb][i] - ((i >> 1) ? del1 : del0));
+          }
+          sc[nb][i] = ds;
+        }
+      }
+      uint32_t a[4];
+      a[0] = pack_bf16(sc[0][0], sc[0][1]);
+      a[1] = pack_bf16(sc[0][2], sc[0][3]);
+      a[2] = pack_bf16(sc[1][0], sc[1][1]);
+      a[3] = pack_bf16(sc[1][2], sc[1][3]);
+      mma_cols(acc, a, Ks, c0, lane);
+      continue;
+    }
+    // every pair of this warp's rows with the tile's keys is kept: no mask arithmetic (uniform over the warp)
+    const bool full = q0 - k0 + r_base - 63 >= back_lo && q0 - k0 + r_base + 15 <= back_hi;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {            // 32 keys at a time
       float sc[4][4], dp[4][4];
@@ -208,17 +249,28 @@ __global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P)
         mma_rows(sc[nb], qa, Ks, half * 32 + nb * 8, lane);
         mma_rows(dp[nb], ga, Vs, half * 32 + nb * 8, lane);
       }
+      if (full) {
 #pragma unroll
-      for (int nb = 0; nb < 4; ++nb) {
+        for (int nb = 0; nb < 4; ++nb) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int back = back0 + (i >> 1) * 8 - (half * 32 + nb * 8 + (i & 1));
-          float ds = 0.f;
-          if (back >= back_lo && back <= back_hi) {
-            const float p = __expf(sc[nb][i] * SCALE - ((i >> 1) ? lse1 : lse0));
-            ds = p * (dp[nb][i] - ((i >> 1) ? del1 : del0));
+          for (int i = 0; i < 4; ++i) {
+            const float p = ex2_approx(fmaf(sc[nb][i], SCALE_LOG2E, (i >> 1) ? nl1 : nl0));
+            sc[nb][i] = p * (dp[nb][i] - ((i >> 1) ? del1 : del0));
           }
-          sc[nb][i] = ds;
+        }
+      } else {
+#pragma unroll
+        for (int nb = 0; nb < 4; ++nb) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int back = back0 + (i >> 1) * 8 - (half * 32 + nb * 8 + (i & 1));
+            float ds = 0.f;
+            if (back >= back_lo && back <= back_hi) {
+              const float p = ex2_approx(fmaf(sc[nb][i], SCALE_LOG2E, (i >> 1) ? nl1 : nl0));
+              ds = p * (dp[nb][i] - ((i >> 1) ? del1 : del0));
+            }
+            sc[nb][i] = ds;
+          }
         }
       }
 #pragma unroll
@@ -303,6 +355,48 @@ __global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dkv_kernel(BwdParams P
     // further on iff i - j is the tile's own distance
     const int back_lo = ti < n_near ? 0 : q0 - k0, back_hi = ti < n_near ? l : q0 - k0;
     const int back0 = q0 - k0 - (r_base + g) + 2 * t;   // i - j of this lane's first element of query column 0
+    if (ti >= n_near) {
+      // a tile further on: key r is seen by query r of the tile only, so just the 16 queries in line with this warp's
+      // keys matter
+      const int c0 = r_base;
+      float st[2][4], dp[2][4];
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb) {
+        st[nb][0] = st[nb][1] = st[nb][2] = st[nb][3] = 0.f;
+        dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
+        mma_rows(st[nb], ka, Qs, c0 + nb * 8, lane);
+        mma_rows(dp[nb], va, Gs, c0 + nb * 8, lane);
+      }
+#pragma unroll
+      for (int nb = 0; nb < 2; ++nb) {
+        const int c = c0 + nb * 8 + 2 * t;
+        const float2 ls = *reinterpret_cast<const float2*>(lse_s + c), dl = *reinterpret_cast<const float2*>(del_s + c);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float p = 0.f, ds = 0.f;
+          if (g + (i >> 1) * 8 == nb * 8 + 2 * t + (i & 1)) {
+            p = ex2_approx(fmaf(st[nb][i], SCALE_LOG2E, -1.4426950408889634f * ((i & 1) ? ls.y : ls.x)));
+            ds = p * (dp[nb][i] - ((i & 1) ? dl.y : dl.x));
+          }
+          st[nb][i] = p;
+          dp[nb][i] = ds;
+        }
+      }
+      uint32_t pa[4], da[4];
+      pa[0] = pack_bf16(st[0][0], st[0][1]);
+      pa[1] = pack_bf16(st[0][2], st[0][3]);
+      pa[2] = pack_bf16(st[1][0], st[1][1]);
+      pa[3] = pack_bf16(st[1][2], st[1][3]);
+      da[0] = pack_bf16(dp[0][0], dp[0][1]);
+      da[1] = pack_bf16(dp[0][2], dp[0][3]);
+      da[2] = pack_bf16(dp[1][0], dp[1][1]);
+      da[3] = pack_bf16(dp[1][2], dp[1][3]);
+      mma_cols(acc_v, pa, Gs, c0, lane);
+      mma_cols(acc_k, da, Qs, c0, lane);
+      continue;
+    }
+    // every pair of the tile's queries with this warp's keys is kept: no mask arithmetic (uniform over the warp)
+    const bool full = q0 - k0 - r_base - 15 >= back_lo && q0 - k0 - r_base + 63 <= back_hi;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {              // 32 queries at a time
       float st[4][4], dp[4][4];                         // S^T and dP^T: rows = keys, columns = queries
@@ -316,17 +410,29 @@ __global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dkv_kernel(BwdParams P
 #pragma unroll
       for (int nb = 0; nb < 4; ++nb) {
         const int c = half * 32 + nb * 8 + 2 * t;
-        const float2 ls = *reinterpret_cast<const float2*>(lse_s + c), dl = *reinterpret_cast<const float2*>(del_s + c);
+        float2 ls = *reinterpret_cast<const float2*>(lse_s + c);
+        const float2 dl = *reinterpret_cast<const float2*>(del_s + c);
+        ls.x *= -1.4426950408889634f;
+        ls.y *= -1.4426950408889634f;
+        if (full) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int back = back0 + (half * 32 + nb * 8 + (i & 1)) - (i >> 1) * 8;
-          float p = 0.f, ds = 0.f;
-          if (back >= back_lo && back <= back_hi) {
-            p = __expf(st[nb][i] * SCALE - ((i & 1) ? ls.y : ls.x));
-            ds = p * (dp[nb][i] - ((i & 1) ? dl.y : dl.x));
+          for (int i = 0; i < 4; ++i) {
+            const float p = ex2_approx(fmaf(st[nb][i], SCALE_LOG2E, (i & 1) ? ls.y : ls.x));
+            st[nb][i] = p;
+            dp[nb][i] = p * (dp[nb][i] - ((i & 1) ? dl.y : dl.x));
           }
-          st[nb][i] = p;
-          dp[nb][i] = ds;
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int back = back0 + (half * 32 + nb * 8 + (i & 1)) - (i >> 1) * 8;
+            float p = 0.f, ds = 0.f;
+            if (back >= back_lo && back <= back_hi) {
+              p = ex2_approx(fmaf(st[nb][i], SCALE_LOG2E, (i & 1) ? ls.y : ls.x));
+              ds = p * (dp[nb][i] - ((i & 1) ? dl.y : dl.x));
+            }
+            st[nb][i] = p;
+            dp[nb][i] = ds;
+          }
         }
       }
 #pragma unroll
