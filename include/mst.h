@@ -226,6 +226,17 @@ mst_status_t mst_dense_grad_dw(const mst_layer_t* layer, const void* dY, int64_t
 mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_t target_nnz, int64_t numel, double random_ratio,
                                int64_t counts[4]);
 
+/* Planning helper of the random growth (host only, no device work).  The hash keys of the `candidates` entries that may
+ * be grown at random are independent and uniform over 64 bits, so the k-th smallest of them lies, with probability
+ * 1 - 1e-8 or better at sigmas = 6, in [lo, hi) = [(k - m) / candidates, (k + m) / candidates) * 2^64 with
+ * m = sigmas * sqrt(k) + 16 (the count of keys below a quantile is binomial with a standard deviation below sqrt(k)).
+ * The update kernel lists the about 2m candidates inside the bracket and finds the threshold among them; it checks the
+ * bracket against the exact counts and falls back to a general selection when it missed, so the bracket affects
+ * speed only.  *planned = 0 (and lo = hi = 0) when there is nothing to bracket (k <= 0, k > candidates), sigmas <= 0,
+ * or 3m exceeds list_capacity, the number of candidates the layer's list can hold. */
+mst_status_t mst_rand_bracket(int64_t k, int64_t candidates, double sigmas, int64_t list_capacity, uint64_t* lo,
+                              uint64_t* hi, int32_t* planned);
+
 /* One Mixed-Growing topology update (Algorithm 1): prune the n_prune active entries of smallest |w|, grow the n_grad
  * empty slots of largest |g| and n_rand more at random, rewrite the mask, drop pruned values, start grown values at
  * +0.0, rebuild CSR/CSC in place.  Ties are broken by the smaller flat index.  Selection is bit-exact and

@@ -25,7 +25,7 @@ STATUS_NAMES = {0: "MST_OK", 1: "MST_ERR_INVALID_ARG", 2: "MST_ERR_SHAPE", 3: "M
                 9: "MST_ERR_NOT_PACKED"}
 EXPORTS = ["mst_layer_create", "mst_layer_destroy", "mst_set_compute_path", "mst_layer_path_in_use", "mst_launch_count", "mst_track_values", "mst_values_changed", "mst_layer_nnz", "mst_pack", "mst_export_csr", "mst_export_csc",
            "mst_values", "mst_validate", "mst_spmm_fwd", "mst_spmm_bwd_x", "mst_spmm_fwd_gelu", "mst_spmm_bwd_x_gelu", "mst_strided_attention_fwd", "mst_strided_attention_bwd", "mst_sddmm_dw", "mst_dense_grad", "mst_sddmm_from_dense", "mst_dense_grad_dw",
-           "mst_update_counts", "mst_topology_update", "mst_topology_update_many", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
+           "mst_update_counts", "mst_rand_bracket", "mst_topology_update", "mst_topology_update_many", "mst_layer_step_host", "mst_layer_step_host_async", "mst_layer_step_host_wait", "mst_mask_to_csr_noalloc",
            "mst_device_error_flags", "mst_sv_sparsity", "mst_sv_update_fraction", "mst_er_densities",
            "mst_status_string"]
 
@@ -88,6 +88,7 @@ _sig = {
     "mst_sddmm_from_dense": [_vp, _vp, _vp, _vp],
     "mst_dense_grad_dw": [_vp, _vp, _i64, _vp, _i64, _i64, _vp, _vp, _vp],
     "mst_update_counts": [_f64, _i64, _i64, _i64, _f64, ctypes.POINTER(_i64)],
+    "mst_rand_bracket": [_i64, _i64, _f64, _i64, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(_i32)],
     "mst_topology_update": [_vp, _f64, ctypes.POINTER(RegrowRule), _vp, ctypes.POINTER(UpdateStats), _vp],
     "mst_topology_update_many": [_i32, ctypes.POINTER(_vp), ctypes.POINTER(_f64), ctypes.POINTER(RegrowRule), ctypes.POINTER(_vp),
                                  ctypes.POINTER(UpdateStats), _vp],
@@ -265,6 +266,14 @@ def mst_update_counts(prune_frac: float, nnz: int, target_nnz: int, numel: int, 
     out = (_i64 * 4)()
     _check(_lib.mst_update_counts(prune_frac, nnz, target_nnz, numel, random_ratio, out), "mst_update_counts")
     return tuple(int(v) for v in out)
+
+
+def mst_rand_bracket(k: int, candidates: int, sigmas: float = 6.0, list_capacity: int = 32768):
+    """(lo, hi) of the hash-key bracket planned for the k-th smallest of `candidates` uniform keys, or None."""
+    lo, hi, planned = ctypes.c_uint64(), ctypes.c_uint64(), _i32()
+    _check(_lib.mst_rand_bracket(k, candidates, sigmas, list_capacity, ctypes.byref(lo), ctypes.byref(hi), ctypes.byref(planned)),
+           "mst_rand_bracket")
+    return (int(lo.value), int(hi.value)) if planned.value else None
 
 
 def mst_topology_update(layer: int, prune_frac: float, target_nnz: int = -1, random_ratio: float = 0.25,

@@ -1998,6 +1998,25 @@ extern "C" mst_status_t mst_update_counts(double prune_frac, int64_t nnz, int64_
   return MST_OK;
 }
 
+extern "C" mst_status_t mst_rand_bracket(int64_t k, int64_t candidates, double sigmas, int64_t list_capacity, uint64_t* lo,
+                                         uint64_t* hi, int32_t* planned) {
+  if (!lo || !hi || !planned || list_capacity < 0) return MST_ERR_INVALID_ARG;
+  *lo = *hi = 0;
+  *planned = 0;
+  if (k <= 0 || candidates <= 0 || k > candidates || !(sigmas > 0.0)) return MST_OK;   // nothing to bracket, or switched off
+  const int64_t m = (int64_t)(sigmas * sqrt((double)k)) + 16;
+  if (3 * m > list_capacity) return MST_OK;               // expected list length 2m: leave room for its own spread
+  const int64_t lo_cnt = k - m > 0 ? k - m : 0, hi_cnt = k + m;
+  const unsigned __int128 one = (unsigned __int128)1 << 64;
+  const uint64_t l = (uint64_t)(one * (unsigned __int128)lo_cnt / (unsigned __int128)candidates);
+  const uint64_t h = hi_cnt >= candidates ? ~(uint64_t)0 : (uint64_t)(one * (unsigned __int128)hi_cnt / (unsigned __int128)candidates);
+  if (h <= l) return MST_OK;
+  *lo = l;
+  *hi = h;
+  *planned = 1;
+  return MST_OK;
+}
+
 namespace {
 
 // One layer's update, planned on the host: counts, selection parameters, which buffer set is built.
@@ -2075,19 +2094,14 @@ void fill_fused_params(const UpdatePlan& pl, FusedParams& F) {
 // the exact counts and falls back to the general radix select when it missed, so the choice only affects speed.
 void plan_rand_bracket(const UpdatePlan& pl, FusedParams& F) {
   const mst_layer* L = pl.L;
-  const long long k = pl.n_rand;
-  const long long C = (L->N - L->nnz) - pl.n_grad;   // candidates: inactive entries the gradient growth left
-  if (k <= 0 || C <= 0 || k > C) return;
   double sigmas = 6.0;
   if (const char* e = getenv("MST_UPDATE_RAND_SIGMAS")) sigmas = atof(e);
-  if (!(sigmas > 0.0)) return;                        // 0 switches the bracket off
-  const long long m = (long long)(sigmas * sqrt((double)k)) + 16;
-  if (3 * m > L->rand_cap) return;                    // expected list length 2m: leave room for its own spread
-  const long long lo_cnt = k - m > 0 ? k - m : 0, hi_cnt = k + m;
-  const unsigned __int128 one = (unsigned __int128)1 << 64;
-  F.rand_lo = (unsigned long long)(one * (unsigned __int128)lo_cnt / (unsigned __int128)C);
-  F.rand_hi = hi_cnt >= C ? ~0ULL : (unsigned long long)(one * (unsigned __int128)hi_cnt / (unsigned __int128)C);
-  if (F.rand_hi <= F.rand_lo) return;
+  uint64_t lo = 0, hi = 0;
+  int32_t planned = 0;
+  // candidates: inactive entries the gradient growth left
+  if (mst_rand_bracket(pl.n_rand, (L->N - L->nnz) - pl.n_grad, sigmas, L->rand_cap, &lo, &hi, &planned) != MST_OK || !planned) return;
+  F.rand_lo = lo;
+  F.rand_hi = hi;
   F.rand_bracket = 1;
 }
 

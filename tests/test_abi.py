@@ -64,3 +64,29 @@ def test_update_counts_agree_with_oracle(mst):
     with pytest.raises(mst.MstError) as e:
         mst.mst_update_counts(-0.1, 10, 10, 40, 0.25)
     assert e.value.status == 1
+
+
+def test_random_growth_bracket_holds_the_kth_smallest_of_uniform_keys(mst):
+    # host logic of the bracket the update kernel lists its random candidates in: on uniform 64-bit keys the k-th
+    # smallest falls inside, the list it implies fits, and the degenerate requests plan nothing
+    rng = np.random.default_rng(5)
+    for C, k in [(1000, 1), (1000, 1000), (5000, 37), (200_000, 1500), (1_000_000, 7500), (1_000_000, 999_000), (3_000_000, 31_457)]:
+        br = mst.mst_rand_bracket(k, C, 6.0, 32768)
+        assert br is not None
+        lo, hi = br
+        assert 0 <= lo < hi <= 2 ** 64 - 1
+        for trial in range(3):
+            keys = rng.integers(0, 2 ** 64, size=C, dtype=np.uint64)
+            kth = int(np.partition(keys, k - 1)[k - 1])
+            below = int((keys < np.uint64(lo)).sum())
+            inside = int(((keys >= np.uint64(lo)) & (keys < np.uint64(hi))).sum())
+            assert below < k <= below + inside            # what the kernel checks before it trusts the bracket
+            assert lo <= kth < hi
+            assert inside <= 32768
+    assert mst.mst_rand_bracket(0, 100, 6.0, 32768) is None
+    assert mst.mst_rand_bracket(101, 100, 6.0, 32768) is None
+    assert mst.mst_rand_bracket(50, 100, 0.0, 32768) is None           # switched off
+    assert mst.mst_rand_bracket(4_000_000, 8_000_000, 6.0, 32768) is None   # the list would not fit
+    assert mst.mst_rand_bracket(50, 100, 6.0, 32768) == (0, 2 ** 64 - 1)     # k + m beyond the candidates: everything
+    narrow, wide = mst.mst_rand_bracket(10_000, 1_000_000, 1.0, 32768), mst.mst_rand_bracket(10_000, 1_000_000, 6.0, 32768)
+    assert wide[0] < narrow[0] < narrow[1] < wide[1]
