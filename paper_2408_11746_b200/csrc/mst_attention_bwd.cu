@@ -7,7 +7,7 @@
 //   dV_j = sum_i P_ij dOut_i      dK_j = sum_i dS_ij q_i / sqrt(d)      dQ_i = sum_j dS_ij k_j / sqrt(d)
 //
 // Three launches, no atomics (every output element has one owner and a fixed summation order):
-//   1. delta: one warp per (token, head).
+//   1. delta: eight lanes per (token, head) row, 16-byte loads.
 //   2. dQ, query-centric: a block owns 64 queries of one (sequence, head) and walks the key tiles of their window
 //      (stride / 64 + 1 tiles of 64 keys; the tile that starts `stride` positions back also holds the first strided
 //      key of every query).  Per tile: S = Q K^T and dP = dOut V^T on the tensor cores (warp-level mma.sync
@@ -64,20 +64,38 @@ __device__ __forceinline__ void load_floats_async(float* dst, const float* src, 
 __device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
-__global__ void attn_delta_kernel(BwdParams P) {
-  const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;   // (token, head)
-  const int lane = threadIdx.x & 31;
-  const int64_t rows = (int64_t)P.batch * P.seq;
-  if (w >= rows * P.heads) return;
-  const int64_t t = w / P.heads;
-  const int h = (int)(w - t * P.heads);
-  const __nv_bfloat162 o = *reinterpret_cast<const __nv_bfloat162*>(P.Out + t * P.ldo + h * D + 2 * lane);
-  const __nv_bfloat162 g = *reinterpret_cast<const __nv_bfloat162*>(P.dOut + t * P.lddo + h * D + 2 * lane);
-  float s = __bfloat162float(o.x) * __bfloat162float(g.x) + __bfloat162float(o.y) * __bfloat162float(g.y);
-  for (int off = 16; off; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-  const int64_t b = t / P.seq;
-  const int i = (int)(t - b * P.seq);
-  if (lane == 0) P.delta[(b * P.heads + h) * P.seq + i] = s;
+// delta[b, h, i] = dOut_i . Out_i per head: eight lanes per (token, head) row of 64 elements, 16 bytes per lane and
+// tensor, four rows per warp and trip
+__global__ void __launch_bounds__(256) attn_delta_kernel(BwdParams P) {
+  const int lane = threadIdx.x & 31, grp = lane >> 3, piece = lane & 7;
+  const int64_t rows = (int64_t)P.batch * P.seq * P.heads;
+  const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t w0 = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * 4; w0 < rows; w0 += warps * 4) {
+    const int64_t w = w0 + grp;          // (token, head)
+    float s = 0.f;
+    int64_t t = 0;
+    int h = 0;
+    if (w < rows) {
+      t = w / P.heads;
+      h = (int)(w - t * P.heads);
+      const uint4 o = *reinterpret_cast<const uint4*>(P.Out + t * P.ldo + h * D + piece * 8);
+      const uint4 g = *reinterpret_cast<const uint4*>(P.dOut + t * P.lddo + h * D + piece * 8);
+      const uint32_t ow[4] = {o.x, o.y, o.z, o.w}, gw[4] = {g.x, g.y, g.z, g.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        s = fmaf(__uint_as_float(ow[j] << 16), __uint_as_float(gw[j] << 16), s);
+        s = fmaf(__uint_as_float(ow[j] & 0xFFFF0000u), __uint_as_float(gw[j] & 0xFFFF0000u), s);
+      }
+    }
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
+    s += __shfl_xor_sync(0xffffffffu, s, 4);
+    if (piece == 0 && w < rows) {
+      const int64_t b = t / P.seq;
+      const int i = (int)(t - b * P.seq);
+      P.delta[(b * P.heads + h) * P.seq + i] = s;
+    }
+  }
 }
 
 // Warp-level tensor-core pieces (mma.sync m16n8k16, bf16 in, fp32 accumulate) with the published fragment layouts:
@@ -491,8 +509,9 @@ extern "C" mst_status_t mst_strided_attention_bwd(const void* Q, const void* K, 
   P.dQ = (__nv_bfloat16*)dQ; P.dK = (__nv_bfloat16*)dK; P.dV = (__nv_bfloat16*)dV;
   P.ldg = ldg;
   P.batch = batch; P.seq = seq_len; P.heads = heads; P.stride = stride;
-  const int64_t warps = (int64_t)batch * seq_len * heads;
-  attn_delta_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, s>>>(P); MST_COUNT_LAUNCH();
+  const int64_t delta_rows = (int64_t)batch * seq_len * heads;
+  const int64_t delta_blocks = (delta_rows / 4 + 7) / 8 + 1;   // eight warps per block, four rows per warp and trip
+  attn_delta_kernel<<<(unsigned)(delta_blocks < 148 * 16 ? delta_blocks : 148 * 16), 256, 0, s>>>(P); MST_COUNT_LAUNCH();
   static_assert(2 * TS * LDF * 4 <= 4 * TS * LDB * 2, "the staged gradients must fit the tile buffers");
   const size_t smem_q = (size_t)(6 * TS * LDB) * 2 + 128;
   const size_t smem_kv = (size_t)(6 * TS * LDB) * 2 + 128;
