@@ -2167,6 +2167,7 @@ mst_status_t launch_cooperative(const void* fn, void** args, int grid_blocks, si
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = mst_pdl_enabled() ? 2 : 1;
+  if (getenv("MST_DEBUG")) fprintf(stderr, "libmst: cooperative launch grid %d block %d dynamic shared memory %zu\n", grid_blocks, FUSED_THREADS, smem);
   MST_CUDA_TRY(cudaLaunchKernelExC(&cfg, fn, args));
   MST_COUNT_LAUNCH();
   return MST_OK;
@@ -2207,7 +2208,10 @@ mst_status_t launch_single_update(const UpdatePlan& pl, cudaStream_t s, bool* fu
             const int64_t per_k = (L->nwords + g - 1) / g;
             const size_t need = (size_t)per_k * (20 + 128);
             if (need + 10 * 1024 > (size_t)optin) continue;
-            if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need) != cudaSuccess) continue;
+            // never below the default limit: the attribute stays with the function, and a later launch that needs less
+            // than 48 KiB does not set it again
+            const size_t attr_bytes = need > 48 * 1024 ? need : 48 * 1024;
+            if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)attr_bytes) != cudaSuccess) continue;
             int occ = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, fn, FUSED_THREADS, need) != cudaSuccess || occ < 1) continue;
             if ((int64_t)occ * sms < g) continue;   // all blocks must be resident at once

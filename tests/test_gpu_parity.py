@@ -235,6 +235,24 @@ def test_update_is_bit_exact_over_consecutive_steps(O, I, dtype, density, kind, 
     L.close()
 
 
+def test_update_of_a_larger_layer_after_a_small_one_with_another_form():
+    # the cooperative kernel's shared-memory limit is a property of the function, not of a launch: a small layer updated
+    # with the key cache in shared memory must not leave a limit behind that a later, larger layer (updated with
+    # regrowth of just-pruned links, hence one selection after the other and no key cache) exceeds
+    small = _problem(33, 95, 4, "bf16", 0.3, 61)
+    Ls = make_layer(small)
+    Ws = np.where(small.mask == 1, small.W, np.float32(0)).astype(np.float32)
+    _update_both(Ls, small, Ws, small.mask.copy(), np.ones((33, 95), np.float32), 0.3, -1, 0.25, 3, 0)
+    big = _problem(794, 865, 4, "bf16", 0.0, 62)
+    Lb = make_layer(big)
+    rng = np.random.default_rng(4)
+    G = rng.standard_normal((794, 865)).astype(np.float32)
+    Wb = np.zeros((794, 865), np.float32)
+    _update_both(Lb, big, Wb, big.mask.copy(), G, 0.3, 170320, 0.25, 3, 0, allow=True)     # growth from an empty mask
+    Ls.close()
+    Lb.close()
+
+
 def test_update_changes_density_both_ways_and_reaches_dense_and_empty():
     O, I = 80, 96
     p = _problem(O, I, 4, "bf16", 0.3, 55)
