@@ -93,3 +93,16 @@ def test_attention_bwd_is_deterministic_and_checks_arguments():
     with pytest.raises(mst.MstError) as e:      # sequence length not a multiple of 64
         mst.mst_strided_attention_bwd(x, x, x, 192, x, 192, x, 192, lse, 1, 200, 1, 64, 128, x, x, x, 192)
     assert e.value.status == 2
+
+
+def test_attention_bwd_random_shapes():
+    # sequence lengths and strides drawn at random (multiples of 64), one call after the other in one process
+    rng = np.random.default_rng(21)
+    for case in range(14):
+        n = 64 * int(rng.integers(1, 13))
+        stride = 64 * int(rng.integers(1, n // 64 + 1))
+        B, H = int(rng.integers(1, 3)), int(rng.integers(1, 4))
+        pad = int(rng.choice([0, 8]))
+        got, ref, _ = _run(B, n, H, stride, 1300 + case, pad, float(rng.choice([0.5, 1.0, 1.5])))
+        for a, b, name in zip(got, ref, ("dQ", "dK", "dV")):
+            assert rel_err(a, b) <= 2e-2, (case, name, B, n, H, stride, pad)
