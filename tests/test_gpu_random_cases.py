@@ -90,3 +90,74 @@ def test_random_products_on_every_kernel_family(seed):
             assert rel_err(host(dW)[: p.nnz], Gr[rows, cols]) <= TOL[dtype], what
         assert mst.mst_device_error_flags() == 0, what
         L.close()
+
+
+def test_random_sequences_of_calls_on_one_layer():
+    # products on changing kernel families, updates, in-place value changes and value tracking in random order on
+    # the same layer: cached operands (dense image, compressed 2:4 operand and its places, CSC view, longest row) must
+    # follow every change
+    from cuda.bindings import runtime as cudart
+    rng = np.random.default_rng(8)
+    paths = [mst.MST_PATH_AUTO, mst.MST_PATH_CUDA_CORE, mst.MST_PATH_TENSOR_CORE, mst.MST_PATH_SPARSE_TC]
+    for case in range(24):
+        O, I, T = 8 * int(rng.integers(4, 60)), 8 * int(rng.integers(4, 70)), int(rng.integers(8, 400))
+        dtype = "bf16" if rng.random() < 0.75 else "f32"
+        density = float(rng.choice([0.03, 0.1, 0.25, 0.5]))
+        zipf = rng.random() < 0.25
+        p = (mst_inputs.zipf_layer if zipf else mst_inputs.uniform_layer)("t", case % 5, O, I, T, dtype, density, 11000 + case)
+        L = make_layer(p)
+        W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+        if dtype == "bf16":
+            W = mst_inputs.bf16_bits_to_f32(mst_inputs.f32_to_bf16_bits(W))
+        M = p.mask.copy()
+        X, dY = to_dev(p, "X"), to_dev(p, "dY")
+        track, log = False, []
+        for op_i in range(12):
+            op = str(rng.choice(["prod", "prod", "update", "path", "scale", "track"]))
+            log.append(op)
+            if op == "path":
+                L.set_path(int(rng.choice(paths)))
+            elif op == "track":
+                track = not track
+                L.track_values(track)
+            elif op == "scale":          # an optimizer step in place: every stored value doubled (exact)
+                ptr, nnz = mst.mst_values(L.handle)
+                if nnz:
+                    _, _, v = oracle.to_csr(W, M)
+                    v2 = (2.0 * v).astype(np.float32)
+                    src = (torch.from_numpy(mst_inputs.f32_to_bf16_bits(v2).view(np.int16)) if dtype == "bf16" else torch.from_numpy(v2)).to(dev())
+                    torch.cuda.synchronize()
+                    (err,) = cudart.cudaMemcpy(ptr, src.data_ptr(), (2 if dtype == "bf16" else 4) * nnz,
+                                               cudart.cudaMemcpyKind.cudaMemcpyDeviceToDevice)
+                    assert int(err) == 0
+                    W = (2.0 * W).astype(np.float32)
+                    if track:
+                        L.values_changed()
+            elif op == "update":
+                zeta, R = float(rng.choice([0.1, 0.3, 0.5])), float(rng.choice([0.0, 0.25, 1.0]))
+                tgt = -1 if rng.random() < 0.6 else int(rng.integers(1, O * I // 2))
+                G = rng.standard_normal((O, I)).astype(np.float32)
+                c = oracle.mg_counts(zeta, int(M.sum()), tgt, O * I, R)
+                mst.mst_topology_update(L.handle, zeta, tgt, R, 5, op_i, False, torch.from_numpy(G).to(dev()),
+                                        want_stats=bool(rng.random() < 0.5))
+                W, M, *_ = oracle.mg_update(W, M, G, c[0], c[3], c[2], 5, op_i, p.layer_id, False, 0.0)
+            else:
+                nnz = int(M.sum())
+                Y = torch.full((T, O), float("nan"), dtype=tdtype(p), device=dev())
+                dX = torch.full((T, I), float("nan"), dtype=tdtype(p), device=dev())
+                dW = torch.full((max(nnz, 1),), float("nan"), dtype=torch.float32, device=dev())
+                L.fwd(X, Y, T)
+                L.bwd_x(dY, dX, T)
+                L.sddmm(dY, X, T, dW)
+                torch.cuda.synchronize()
+                what = (case, O, I, T, dtype, density, log)
+                assert rel_err(host(Y), oracle.fwd(p.X, W, M)) <= TOL[dtype], what
+                assert rel_err(host(dX), oracle.bwd_x(p.dY, W, M)) <= TOL[dtype], what
+                if nnz:
+                    rows, cols = np.nonzero(M)
+                    assert rel_err(host(dW)[:nnz], oracle.dense_grad(p.dY, p.X)[rows, cols]) <= TOL[dtype], what
+        rp, ci, vb = export_csr(L, dtype)
+        rp_r, ci_r, v_r = oracle.to_csr(W, M)
+        assert np.array_equal(rp, rp_r) and np.array_equal(ci, ci_r) and np.array_equal(vb, value_bits(v_r, dtype)), (case, log)
+        assert mst.mst_device_error_flags() == 0, (case, log)
+        L.close()
