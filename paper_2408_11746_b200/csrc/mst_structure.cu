@@ -344,6 +344,10 @@ mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s) {
 // and reuses it until the mask or the values change.
 mst_status_t mst_densify(const mst_layer* L, cudaStream_t s, const uint16_t** image) {
   const int c = L->cur;
+  if (L->nnz == L->N) {  // every entry kept: the CSR values in row-major order are the dense matrix
+    *image = (const uint16_t*)L->vals[c];
+    return MST_OK;
+  }
   uint16_t* dst = nullptr;
   if (L->track_values) {
     MST_TRY(mst_alloc_dense(const_cast<mst_layer*>(L)));

@@ -57,6 +57,7 @@ struct Params {
   void* pre;
   int64_t ldpre;
   int tma_out;  // rows leave through shared memory and TMA stores (tensor map tmC) instead of per-thread stores
+  int sampled_stage_min;  // sampled output: a 32 x 32 chunk with at least this many kept entries leaves row by row
 };
 
 // PTX wrappers live in mst_tc_ptx.cuh; waits in this file report to g_tc_error
@@ -219,6 +220,67 @@ __device__ __forceinline__ void epilogue_tile(const Params& P, uint32_t tmem_bas
           }
         }
       }
+    }
+  }
+}
+
+// The sampled accumulator (weight gradient under the mask).  A chunk is 32 rows x one mask word.  Chunks with few
+// entries are written by the row-owning lanes, entry by entry.  Denser chunks leave through the warp's staging box:
+// the lanes turn from rows to columns, so that each store instruction writes the kept entries of ONE row, which are
+// neighbours in CSR order; a row-per-lane store touches 32 lines per instruction and costs the memory pipeline as many
+// passes, which at high density slows the concurrent main loop.
+__device__ __forceinline__ void epilogue_tile_sampled(const Params& P, uint32_t stage, uint32_t tmem_base, int acc, int q,
+                                                      int c0, int lane, int64_t m0, int n0, int split) {
+  const int64_t m = (int64_t)m0 + q * 32 + lane;
+  const bool row_ok = m < P.M;
+  const uint32_t my_row = stage + (uint32_t)lane * 128u;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  const uint32_t lt = (1u << lane) - 1u;
+  float* out = P.splits > 1 ? P.partial + (int64_t)split * P.nnz : reinterpret_cast<float*>(P.out);
+#pragma unroll 1
+  for (int c = c0; c < BN / 32; c += EPI_WARPS / 4) {
+    const int n = n0 + c * 32;
+    if (n >= P.N) break;  // uniform
+    uint32_t word = 0;
+    int32_t at = 0;
+    if (row_ok) {
+      const int64_t wi = m * P.wpr + (n >> 5);
+      word = P.bits[wi];
+      at = P.wscan[wi];
+    }
+    uint32_t r[32];
+    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+    const int kept = __reduce_add_sync(0xFFFFFFFFu, __popc(word));
+    if (kept < P.sampled_stage_min) {
+      float* dst = out + at;
+      int rank = 0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        if ((word >> j) & 1u) {
+          dst[rank] = __uint_as_float(r[j]);
+          ++rank;
+        }
+      }
+      continue;
+    }
+    __syncwarp();  // the previous chunk has been read out of the box
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+      const uint32_t piece = (uint32_t)v ^ sw;
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(my_row + piece * 16u), "r"(r[4 * v]), "r"(r[4 * v + 1]),
+                   "r"(r[4 * v + 2]), "r"(r[4 * v + 3])
+                   : "memory");
+    }
+    __syncwarp();
+#pragma unroll 4
+    for (int rr = 0; rr < 32; ++rr) {
+      const uint32_t w = __shfl_sync(0xFFFFFFFFu, word, rr);
+      const int32_t base = __shfl_sync(0xFFFFFFFFu, at, rr);
+      if (w == 0) continue;  // uniform
+      const uint32_t piece = (uint32_t)(lane >> 2) ^ (uint32_t)(rr & 7);
+      uint32_t v;
+      asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(stage + (uint32_t)rr * 128u + piece * 16u + (uint32_t)(lane & 3) * 4u) : "memory");
+      if ((w >> lane) & 1u) out[base + __popc(w & lt)] = __uint_as_float(v);
     }
   }
 }
@@ -427,6 +489,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (use_tma)
         epilogue_tile_tma(P, &tmC, out_base + (uint32_t)(warp - 2) * OUT_BOX_BYTES, tmem_base, acc, q, (warp - 2) >> 2, lane, m0,
                           n0, split);
+      else if (P.epilogue == MST_TC_OUT_SAMPLED)
+        epilogue_tile_sampled(P, out_base + (uint32_t)(warp - 2) * OUT_BOX_BYTES, tmem_base, acc, q, (warp - 2) >> 2, lane, m0,
+                              n0, split);
       else
         epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
       tc_fence_before();
@@ -631,6 +696,9 @@ tc_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (use_tma)
         epilogue_tile_tma(P, &tmC, out_base + (uint32_t)(warp - 2) * OUT_BOX_BYTES, tmem_base, acc, q, (warp - 2) >> 2, lane, m0,
                           n0, split);
+      else if (P.epilogue == MST_TC_OUT_SAMPLED)
+        epilogue_tile_sampled(P, out_base + (uint32_t)(warp - 2) * OUT_BOX_BYTES, tmem_base, acc, q, (warp - 2) >> 2, lane, m0,
+                              n0, split);
       else
         epilogue_tile(P, tmem_base, acc, q, (warp - 2) >> 2, lane, m0, n0, split);
       tc_fence_before();
@@ -837,6 +905,8 @@ mst_status_t mst_tc_gemm(const mst_tc_gemm_args& a, cudaStream_t s) {
   P.pre = a.pre;
   P.ldpre = a.ldpre;
   if (P.act == MST_ACT_GELU_GRAD && !P.pre) return MST_ERR_INVALID_ARG;
+  P.sampled_stage_min = 384;  // measured: row-by-row stores pay from a density of about 0.4
+  if (const char* e = getenv("MST_TC_SAMPLED_STAGE")) P.sampled_stage_min = atoi(e);  // measurement override
   if (a.epilogue != MST_TC_OUT_BF16) {
     // few output tiles: cut the contraction range so that all SMs work; partial sums go to the shared scratch buffer
     const int64_t works1 = pair ? (int64_t)((P.m_tiles + 1) / 2) * P.n_tiles : (int64_t)P.m_tiles * P.n_tiles;

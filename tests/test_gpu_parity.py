@@ -91,7 +91,10 @@ def _run_products(p, L, ldx=None, ldy=None):
     (3, 5, 7, "f32", 0.6, "uniform", 0),
     (70, 1100, 260, "bf16", 0.15, "uniform", 0),
     (520, 328, 900, "bf16", 0.1, "uniform", 0),      # three N tiles / two K-tail blocks on the tensor-core path
-    (1024, 768, 1024, "bf16", 0.05, "zipf", 0)])
+    (1024, 768, 1024, "bf16", 0.05, "zipf", 0),
+    (520, 328, 900, "bf16", 0.7, "uniform", 0),      # dense chunks of the sampled weight gradient: row-by-row stores
+    (300, 1000, 2100, "bf16", 0.45, "uniform", 8),   # chunks on both sides of the row-by-row threshold
+    (264, 520, 640, "bf16", 1.0, "uniform", 0)])     # all-ones mask over several tiles: the values are the dense image
 def test_products_match_oracle(O, I, T, dtype, density, kind, pad):
     p = _problem(O, I, T, dtype, density, 1000 + O + I + T, kind)
     L = make_layer(p)
