@@ -48,6 +48,36 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the tcgen05 contraction launches of ONE step of the
+# default workload, by call kind, summed over the block's four layers: one ncu capture of
+#     python bench.py --steps 1 --warmup 3 --no-sweeps --no-cpu-baseline
+# (launch list and command in profiles/tc_gemm_pair_dram_traffic_gpt2medium_block_T16384.md).  The figures belong to the
+# kernel sources with the digest below; with any other sources the bench line reports no traffic.
+NCU_TRAFFIC = {
+    "sources": ("mst_tc_gemm.cu", "mst_tc_gemm.cuh", "mst_tc_ptx.cuh"),
+    "sha256_16": "58ce9e9d8b745fb1",
+    "launches_per_kind": 4,
+    "read": {"spmm_fwd": 262971392, "spmm_bwd_x": 331241216, "sddmm_dw": 552359680, "dense_grad": 550548992},
+    "write": {"spmm_fwd": 144084992, "spmm_bwd_x": 106702848, "sddmm_dw": 2329344, "dense_grad": 21459968},
+}
+
+
+def captured_traffic(kind: str, workload: str):
+    """Average DRAM bytes of one launch of this call kind from the committed capture, or None when the kernel sources or
+    the workload are not the captured ones."""
+    import hashlib
+    h = hashlib.sha256()
+    try:
+        for f in NCU_TRAFFIC["sources"]:
+            with open(os.path.join(ROOT, "paper_2408_11746_b200", "csrc", f), "rb") as fh:
+                h.update(fh.read())
+    except OSError:
+        return None
+    if h.hexdigest()[:16] != NCU_TRAFFIC["sha256_16"] or workload != WORKLOAD or kind not in NCU_TRAFFIC["read"]:
+        return None
+    return (NCU_TRAFFIC["read"][kind] + NCU_TRAFFIC["write"][kind]) / NCU_TRAFFIC["launches_per_kind"]
+
+
 # ------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -784,8 +814,16 @@ def main() -> None:
     else:
         roof["kernel"] = ("tc_sp24_pair_kernel" if paths == ["sparse_tc"] else "tc_gemm_pair_kernel") + " as " + dom
     roof["family_ms_per_step"] = fam_ms
-    roof["traffic_note"] = ("dram bytes of one launch are in profiles/ (ncu capture of the same kernel on a smaller case); "
-                            "not repeated here because the capture is not regenerated with every kernel change")
+    traffic = captured_traffic(dom, WORKLOAD) if dom_family == "contraction" and paths == ["dense_tiles"] else None
+    roof["traffic"] = traffic
+    if traffic is not None:
+        roof["algorithmic_bytes"] = sum(algorithmic(dom, s)[1] for s in slots) / len(slots)
+        roof["traffic_note"] = ("bytes per launch, mean over the block's four layers like `achieved`; one ncu capture of this "
+                                "workload with the kernel sources as they are now (digest checked).  Output lines still dirty "
+                                "in L2 when a launch ends are written back under a later launch, so products with large outputs "
+                                "show less than their algorithmic bytes")
+    else:
+        roof["traffic_note"] = "no capture of this kernel, workload and source digest is committed"
     if dom_family == "contraction":
         # what the tensor pipe itself sustains: executed dense flops of this call kind over its time
         dense_fl = sum(2.0 * T * s.O * s.I for ss, _, _ in timers[dom] for s in ss)
