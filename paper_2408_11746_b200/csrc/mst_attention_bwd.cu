@@ -23,18 +23,12 @@
 // they enter a tensor-core product (as the forward kernel does with P).
 #include <cuda_bf16.h>
 
+#include "mst_attention_mma.cuh"
 #include "mst_internal.cuh"
 #include "mst_tc_gemm.cuh"
 
 namespace {
-
-
-constexpr int D = 64;        // head dimension
-constexpr int TS = 64;       // tile side (queries and keys)
-constexpr int BW_THREADS = 128;
-constexpr int LDB = 72;      // row pitch of the bf16 tiles in shared memory (64 + 8: rows 144 bytes apart, no bank aliasing)
-constexpr int LDF = 68;      // row pitch of the fp32 tiles
-constexpr float SCALE = 0.125f;   // 1 / sqrt(64)
+using namespace mst_attn;
 
 struct BwdParams {
   const __nv_bfloat16 *Q, *K, *V, *Out, *dOut;
@@ -45,24 +39,6 @@ struct BwdParams {
   int64_t ldg;
   int batch, seq, heads, stride;
 };
-
-// rows [r0, r0 + 64) of one head's 64 columns -> dst[64][LDB] (row-major, bf16), issued asynchronously (cp.async, 16 bytes per
-// request); complete after async_wait_all + a barrier
-__device__ __forceinline__ void load_tile_async(__nv_bfloat16* dst, const __nv_bfloat16* src, int64_t ld, int64_t r0) {
-  for (int e = threadIdx.x; e < TS * D / 8; e += BW_THREADS) {
-    const int r = e >> 3, c = (e & 7) * 8;
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + r * LDB + c);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + (r0 + r) * ld + c) : "memory");
-  }
-}
-__device__ __forceinline__ void load_floats_async(float* dst, const float* src, int n) {
-  for (int e = threadIdx.x; e < n; e += BW_THREADS) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + e);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(src + e) : "memory");
-  }
-}
-__device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 // delta[b, h, i] = dOut_i . Out_i per head: eight lanes per (token, head) row of 64 elements, 16 bytes per lane and
 // tensor, four rows per warp and trip
@@ -95,68 +71,6 @@ __global__ void __launch_bounds__(256) attn_delta_kernel(BwdParams P) {
       const int i = (int)(t - b * P.seq);
       P.delta[(b * P.heads + h) * P.seq + i] = s;
     }
-  }
-}
-
-// Warp-level tensor-core pieces (mma.sync m16n8k16, bf16 in, fp32 accumulate) with the published fragment layouts:
-// with g = lane / 4 and t = lane % 4, an accumulator tile (16 x 8) holds rows g, g + 8 and columns 2t, 2t + 1 in its
-// four registers, and an A operand (16 x 16, row-major) holds the same rows and columns 2t, 2t + 1, 2t + 8, 2t + 9 —
-// so two neighbouring accumulator tiles, rounded to bf16, ARE the A operand of the next product and the scores never
-// leave the registers.
-__device__ __forceinline__ void ldsm_x4(uint32_t (&r)[4], const __nv_bfloat16* p) {
-  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t (&r)[4], const __nv_bfloat16* p) {
-  const uint32_t a = (uint32_t)__cvta_generic_to_shared(p);
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(a));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-constexpr float SCALE_LOG2E = SCALE * 1.4426950408889634f;   // exp(s / sqrt(d) - lse) = 2^(s * SCALE_LOG2E - lse * log2(e))
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<const uint32_t*>(&v);
-}
-// A operand: rows r0 .. r0 + 16, columns 16 kb .. 16 kb + 16 of a bf16 tile with row pitch LDB
-__device__ __forceinline__ void load_a(uint32_t (&a)[4], const __nv_bfloat16* tile, int r0, int kb, int lane) {
-  ldsm_x4(a, tile + (r0 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDB + kb * 16 + (lane >> 4) * 8);
-}
-// c[16 x 8] += A strip (four k-steps over the 64 head dimensions, in registers) * rows n0 .. n0 + 8 of `tile`, transposed
-__device__ __forceinline__ void mma_rows(float (&c)[4], const uint32_t (&a)[4][4], const __nv_bfloat16* tile, int n0, int lane) {
-#pragma unroll
-  for (int k2 = 0; k2 < 2; ++k2) {
-    uint32_t b[4];
-    ldsm_x4(b, tile + (n0 + (lane & 7)) * LDB + k2 * 32 + (lane >> 3) * 8);
-    mma_bf16(c, a[2 * k2], b[0], b[1]);
-    mma_bf16(c, a[2 * k2 + 1], b[2], b[3]);
-  }
-}
-// acc[16 x 64] += A (16 x 16, in registers) * rows k0 .. k0 + 16 of `tile` (64 columns)
-__device__ __forceinline__ void mma_cols(float (&acc)[8][4], const uint32_t (&a)[4], const __nv_bfloat16* tile, int k0, int lane) {
-#pragma unroll
-  for (int n2 = 0; n2 < 4; ++n2) {
-    uint32_t b[4];
-    ldsm_x4_t(b, tile + (k0 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDB + n2 * 16 + (lane >> 4) * 8);
-    mma_bf16(acc[2 * n2], a, b[0], b[1]);
-    mma_bf16(acc[2 * n2 + 1], a, b[2], b[3]);
-  }
-}
-// accumulators (16 x 64) -> fp32 tile in shared memory, rows r0 .. r0 + 16
-__device__ __forceinline__ void store_acc(float* out, const float (&acc)[8][4], int r0, int lane) {
-  const int g = lane >> 2, t = lane & 3;
-#pragma unroll
-  for (int nb = 0; nb < 8; ++nb) {
-    *reinterpret_cast<float2*>(out + (r0 + g) * LDF + nb * 8 + 2 * t) = make_float2(acc[nb][0], acc[nb][1]);
-    *reinterpret_cast<float2*>(out + (r0 + g + 8) * LDF + nb * 8 + 2 * t) = make_float2(acc[nb][2], acc[nb][3]);
   }
 }
 
@@ -231,9 +145,9 @@ __global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P)
       for (int nb = 0; nb < 2; ++nb) {
         sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
         dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
-        mma_rows(sc[nb], qa, Ks, c0 + nb * 8, lane);
-        mma_rows(dp[nb], ga, Vs, c0 + nb * 8, lane);
       }
+      mma_rows_wide<2>(sc, qa, Ks, c0, lane);
+      mma_rows_wide<2>(dp, ga, Vs, c0, lane);
 #pragma unroll
       for (int nb = 0; nb < 2; ++nb) {
 #pragma unroll
@@ -264,9 +178,9 @@ __global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P)
       for (int nb = 0; nb < 4; ++nb) {
         sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
         dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
-        mma_rows(sc[nb], qa, Ks, half * 32 + nb * 8, lane);
-        mma_rows(dp[nb], ga, Vs, half * 32 + nb * 8, lane);
       }
+      mma_rows_wide<4>(sc, qa, Ks, half * 32, lane);
+      mma_rows_wide<4>(dp, ga, Vs, half * 32, lane);
       if (full) {
 #pragma unroll
         for (int nb = 0; nb < 4; ++nb) {
@@ -283,7 +197,7 @@ __global__ void __launch_bounds__(BW_THREADS, 4) attn_bwd_dq_kernel(BwdParams P)
           for (int i = 0; i < 4; ++i) {
             const int back = back0 + (i >> 1) * 8 - (half * 32 + nb * 8 + (i & 1));
             float ds = 0.f;
-            if (back >= back_lo && back <= back_hi) {
+            if ((unsigned)(back - back_lo) <= (unsigned)(back_hi - back_lo)) {
               const float p = ex2_approx(fmaf(sc[nb][i], SCALE_LOG2E, (i >> 1) ? nl1 : nl0));
               ds = p * (dp[nb][i] - ((i >> 1) ? del1 : del0));
             }
@@ -382,9 +296,9 @@ __global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dkv_kernel(BwdParams P
       for (int nb = 0; nb < 2; ++nb) {
         st[nb][0] = st[nb][1] = st[nb][2] = st[nb][3] = 0.f;
         dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
-        mma_rows(st[nb], ka, Qs, c0 + nb * 8, lane);
-        mma_rows(dp[nb], va, Gs, c0 + nb * 8, lane);
       }
+      mma_rows_wide<2>(st, ka, Qs, c0, lane);
+      mma_rows_wide<2>(dp, va, Gs, c0, lane);
 #pragma unroll
       for (int nb = 0; nb < 2; ++nb) {
         const int c = c0 + nb * 8 + 2 * t;
@@ -422,9 +336,9 @@ __global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dkv_kernel(BwdParams P
       for (int nb = 0; nb < 4; ++nb) {
         st[nb][0] = st[nb][1] = st[nb][2] = st[nb][3] = 0.f;
         dp[nb][0] = dp[nb][1] = dp[nb][2] = dp[nb][3] = 0.f;
-        mma_rows(st[nb], ka, Qs, half * 32 + nb * 8, lane);
-        mma_rows(dp[nb], va, Gs, half * 32 + nb * 8, lane);
       }
+      mma_rows_wide<4>(st, ka, Qs, half * 32, lane);
+      mma_rows_wide<4>(dp, va, Gs, half * 32, lane);
 #pragma unroll
       for (int nb = 0; nb < 4; ++nb) {
         const int c = half * 32 + nb * 8 + 2 * t;
@@ -444,7 +358,7 @@ __global__ void __launch_bounds__(BW_THREADS, 3) attn_bwd_dkv_kernel(BwdParams P
           for (int i = 0; i < 4; ++i) {
             const int back = back0 + (half * 32 + nb * 8 + (i & 1)) - (i >> 1) * 8;
             float p = 0.f, ds = 0.f;
-            if (back >= back_lo && back <= back_hi) {
+            if ((unsigned)(back - back_lo) <= (unsigned)(back_hi - back_lo)) {
               p = ex2_approx(fmaf(st[nb][i], SCALE_LOG2E, (i & 1) ? ls.y : ls.x));
               ds = p * (dp[nb][i] - ((i & 1) ? dl.y : dl.x));
             }

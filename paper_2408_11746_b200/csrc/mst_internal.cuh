@@ -168,6 +168,10 @@ mst_status_t mst_build_csc(mst_layer* L, cudaStream_t s);
 mst_status_t mst_ensure_csc(const mst_layer* L, cudaStream_t s);  // builds the CSC view if it is stale
 mst_status_t mst_combine_update_bits(mst_layer* L, int new_set, cudaStream_t s);
 mst_status_t mst_densify(const mst_layer* L, cudaStream_t s, const uint16_t** image);
+// strided attention forward on warp-level products (mst_attention_fwd_mma.cu); the caller has checked pointers and
+// leading dimensions
+mst_status_t mst_attention_fwd_mma(const void* Q, const void* K, const void* V, int64_t ld, int32_t batch, int32_t seq_len,
+                                   int32_t heads, int32_t stride, void* Out, int64_t ldo, float* lse, cudaStream_t s);
 bool mst_use_tensor_path(const mst_layer* L);
 bool mst_use_sparse_tc_path(const mst_layer* L);
 

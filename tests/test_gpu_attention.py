@@ -38,8 +38,25 @@ def _run(p, stride, want_lse=True, pad=0):
     (3, 256, 2, 256, 8),       # stride = n: plain causal attention inside one window; padded leading dimensions
     (2, 128, 1, 128, 0),       # a single query block
     (1, 1024, 1, 128, 0),      # seven strided positions
-    (1, 2048, 2, 256, 0)])     # the longest supported sequence for l = 256: six positions outside the tile
-def test_forward_matches_oracle(batch, seq, heads, stride, pad):
+    (1, 2048, 2, 256, 0)])     # the longest sequence the tensor-memory kernel takes for l = 256: six positions outside the tile
+@pytest.mark.parametrize("kernel", ["warp", "tcgen05"])
+def test_forward_matches_oracle(batch, seq, heads, stride, pad, kernel, monkeypatch):
+    monkeypatch.setenv("MST_ATTN_FWD", kernel)
+    _check_forward(batch, seq, heads, stride, pad)
+
+
+@pytest.mark.parametrize("batch,seq,heads,stride,pad", [
+    (1, 512, 2, 64, 0),        # stride of one tile: seven strided positions per half block
+    (2, 384, 1, 192, 8),       # stride an odd multiple of 64: the two halves of a block reach back differently
+    (1, 640, 2, 320, 0),
+    (1, 1024, 1, 512, 0),      # window longer than a block's span
+    (2, 256, 2, 1024, 0),      # stride beyond the sequence: plain causal attention
+    (1, 4096, 1, 128, 0)])     # 31 strided positions
+def test_forward_strides_of_the_warp_level_kernel(batch, seq, heads, stride, pad):
+    _check_forward(batch, seq, heads, stride, pad)
+
+
+def _check_forward(batch, seq, heads, stride, pad):
     p = mst_inputs.attention_problem(batch, seq, heads, 64, seed=900 + seq + stride)
     out, lse = _run(p, stride, pad=pad)
     Q, K, V = p.split()
@@ -51,7 +68,9 @@ def test_forward_matches_oracle(batch, seq, heads, stride, pad):
     np.testing.assert_array_equal(out[:, :, 0], V[:, :, 0])
 
 
-def test_larger_scores_and_run_to_run_identity():
+@pytest.mark.parametrize("kernel", ["warp", "tcgen05"])
+def test_larger_scores_and_run_to_run_identity(kernel, monkeypatch):
+    monkeypatch.setenv("MST_ATTN_FWD", kernel)
     p = mst_inputs.attention_problem(2, 512, 2, 64, seed=77, std=2.0)      # scaled scores of variance 16: peaked rows
     a, _ = _run(p, 256, want_lse=False)
     b, _ = _run(p, 256, want_lse=False)
@@ -61,8 +80,10 @@ def test_larger_scores_and_run_to_run_identity():
     assert rel_err(a, ref) <= TOL["bf16"]
 
 
+@pytest.mark.parametrize("kernel", ["warp", "tcgen05"])
 @pytest.mark.parametrize("stride", [256, 128])
-def test_gpt2_small_full_size_sampled(stride):
+def test_gpt2_small_full_size_sampled(stride, kernel, monkeypatch):
+    monkeypatch.setenv("MST_ATTN_FWD", kernel)
     # 16 sequences of 1024 tokens, 12 heads: the attention input of the benchmark's 16384-token batch
     rng = np.random.default_rng(12 + stride)
     p = mst_inputs.attention_problem(16, 1024, 12, 64)
@@ -79,7 +100,7 @@ def test_argument_errors():
     p = mst_inputs.attention_problem(1, 128, 1, 64)
     x = torch.zeros((128, 192), dtype=torch.bfloat16, device=dev())
     o = torch.zeros((128, 64), dtype=torch.bfloat16, device=dev())
-    for kwargs in (dict(seq_len=100), dict(head_dim=32), dict(stride=64), dict(stride=384), dict(ld=60)):
+    for kwargs in (dict(seq_len=100), dict(head_dim=32), dict(stride=96), dict(stride=0), dict(ld=60)):
         a = dict(ld=192, batch=1, seq_len=128, heads=1, head_dim=64, stride=128)
         a.update(kwargs)
         with pytest.raises(mst.MstError) as e:
