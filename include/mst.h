@@ -177,9 +177,10 @@ mst_status_t mst_spmm_bwd_x_gelu(const mst_layer_t* layer, const void* dY, int64
  * head h in columns h*head_dim .. (so the three column slices of a fused qkv activation can be passed as they are);
  * token b*seq_len + i is position i of sequence b.  Out: device bf16 [batch*seq_len x ldo], same column layout.
  * lse (device float [batch, heads, seq_len], may be NULL) receives log sum_j exp(q_i . k_j / sqrt(d)) for a backward
- * pass.  Supported: head_dim = 64, seq_len a multiple of 128, stride l = 128 or 256, seq_len <= 8 l, ld and ldo
+ * pass.  Supported: head_dim = 64, seq_len a multiple of 128, stride l a positive multiple of 64, ld and ldo
  * multiples of 8, 16-byte aligned pointers; anything else MST_ERR_SHAPE.  Scores and sums are fp32, the softmax
- * weights are rounded to bf16 before they multiply the values. */
+ * weights are rounded to bf16 before they multiply the values.  Two kernels serve the call (a tcgen05 one for
+ * l = 256 with seq_len <= 8 l, a warp-level one for everything else); which one runs does not change the contract. */
 mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, const void* V, int64_t ld, int32_t batch,
                                        int32_t seq_len, int32_t heads, int32_t head_dim, int32_t stride, void* Out,
                                        int64_t ldo, float* lse, mst_stream_t stream);

@@ -549,7 +549,7 @@ extern "C" mst_status_t mst_strided_attention_fwd(const void* Q, const void* K, 
   // Two kernels, same results up to rounding order.  The tcgen05 one (whole window scored at once in tensor memory)
   // takes strides 128 and 256 up to 8 strides of sequence; the warp-level one (running softmax over 64-key tiles) takes
   // every stride that is a multiple of 64 and any length.  Measured at 16 x 1024 tokens, 12 heads: stride 256 - 68 us
-  // against 89 us, stride 128 - 99 us against 89 us; so the tcgen05 kernel runs where it can at strides from 256 and
+  // against 72 us, stride 128 - 99 us against 64 us; so the tcgen05 kernel runs where it can at strides from 256 and
   // the warp-level one elsewhere.  MST_ATTN_FWD=tcgen05 / warp forces one of them.
   const bool tm_can = stride % KB == 0 && stride + KB <= O_COL && seq_len / stride - 2 <= MAX_FAR;
   bool tensor_memory_kernel = tm_can && stride >= 256;

@@ -1,17 +1,20 @@
 // Strided sparse self-attention, forward (Sec. 3.3), on warp-level tensor-core products:
 //   Out[i] = sum_{j in S_i} P_ij v_j,   P = softmax over S_i of q_i . k_j / sqrt(d),
 //   S_i = { j <= i : i - j < l  or  (i - j) mod l == 0 }.
-// A block owns 128 queries of one (sequence, head); each of its four warps owns 32 of them as two 16-row strips, so
-// every key / value fragment fetched from shared memory (ldmatrix) feeds two products and the fetches stay at half of
-// the shared-memory bandwidth the products could consume.  The block walks 64-key tiles: first the tiles of the
-// window (keys q0 - l .. q0 + 127; the tile that starts l positions back also holds the first strided key of every
-// query), then one tile per strided position further back (i - 2l, i - 3l, ...) and 64-query half of the block, of
-// which only the diagonal is attended: a warp forms the two 16 x 8 score tiles in line with a strip's rows and one
-// 16-key step of the second product.  A warp skips the window tiles none of its rows can see.  The softmax is the
-// running one (maximum and sum carried per row, the output rescaled when the maximum moves), in base 2 with the
-// scale folded into one multiply-add; scores never leave the registers: two neighbouring accumulator tiles, rounded
-// to bf16, are the A operand of P V.  K / V tiles are double-buffered with cp.async; the query tile passes through
-// the second buffer once.  No atomics; the order of every sum is fixed.
+// A block owns 64 queries of one (sequence, head) and each of its four warps a 16-row strip of them (the kernel is
+// also built for 128-query blocks and for two strips per warp, which share every key / value fragment between two
+// products; measured within 2 % of each other or slower, see MST_ATTN_FWD_SHAPE below).  The block walks 64-key tiles
+// of the window (keys q0 - l .. q0 + 63; the tile that starts l positions back also holds the first strided key of
+// every query); riding along with window tile `it` comes the tile of the strided position i - (it + 2) l, of which only
+// the diagonal is attended: a warp forms the two 16 x 8 score tiles in line with its rows and one 16-key step of the
+// second product.  Window tiles are scored 32 keys at a time, and a warp skips the keys none of its rows can see.
+// The softmax is the running one in base 2 with the scale folded into one multiply-add; its reference follows the
+// running maximum lazily (see softmax_step), so the output rows are rescaled rarely.  Scores never leave the
+// registers: two neighbouring accumulator tiles, rounded to bf16, are the A operand of P V.  K / V tiles are
+// double-buffered with cp.async, every thread copying the same piece of every tile (addresses formed once); the
+// query tile passes through the second buffer once.  No atomics; the order of every sum is fixed.
+// The kernel is bound by instruction issue, not by a pipe: per score it spends about 16 thread instructions of which
+// the two products are one (executed-opcode counts in the profile summary).
 #include <cuda_bf16.h>
 
 #include <cstdlib>
@@ -22,10 +25,6 @@
 namespace {
 using namespace mst_attn;
 
-constexpr int FQ = 128;   // queries per block
-#ifndef MST_ATTN_FWD_BLOCKS
-#define MST_ATTN_FWD_BLOCKS 2   // resident blocks per SM (110 KB of tiles each)
-#endif
 
 struct FwdParams {
   const __nv_bfloat16 *Q, *K, *V;
@@ -86,13 +85,15 @@ __device__ __forceinline__ void softmax_step(float (&x)[NB][4], float (&acc)[8][
   sum[1] += s1;
 }
 
-// NS = 16-row strips per warp: the block's 128 queries are shared by 8 / NS warps
-template <int NS>
-__global__ void __launch_bounds__(256 / NS, MST_ATTN_FWD_BLOCKS) attn_fwd_mma_kernel(FwdParams P) {
+// NS = 16-row strips per warp, HALVES = 64-query halves per block: a block's 64 HALVES queries are shared by
+// 4 HALVES / NS warps
+template <int NS, int HALVES>
+__global__ void __launch_bounds__(128 * HALVES / NS, HALVES == 1 ? 3 : 2) attn_fwd_mma_kernel(FwdParams P) {
   constexpr int WR = 16 * NS;        // rows per warp
   constexpr int HW = 4 / NS;         // warps per 64-query half
+  constexpr int FQ = 64 * HALVES;    // queries per block
   extern __shared__ __align__(128) unsigned char smem[];
-  __nv_bfloat16* KV = reinterpret_cast<__nv_bfloat16*>(smem);   // twelve tiles of [64][LDB], see `slot`
+  __nv_bfloat16* KV = reinterpret_cast<__nv_bfloat16*>(smem);   // 4 + 4 HALVES tiles of [64][LDB], see `slot`
 
   const int qt = (int)gridDim.x - 1 - (int)blockIdx.x;   // the blocks with the most tiles start first
   const int h = blockIdx.y, b = blockIdx.z;
@@ -105,12 +106,14 @@ __global__ void __launch_bounds__(256 / NS, MST_ATTN_FWD_BLOCKS) attn_fwd_mma_ke
   // Trip `it` of the block's loop brings window tile `it` (keys k_first + 64 it ...) and, riding along, the strided
   // position m = it + 2 of both 64-query halves (keys q0 + 64 half - m l ...), as long as each exists
   const int k_first = q0 - l > 0 ? q0 - l : 0;
-  const int n_near = (q0 + TS - k_first) / TS + 1;
-  const int far0 = q0 / l > 1 ? q0 / l - 1 : 0, far1 = (q0 + TS) / l > 1 ? (q0 + TS) / l - 1 : 0;   // far0 <= far1
-  const int n_trips = n_near > far1 ? n_near : far1;
-  auto slot = [&](int i) { return KV + i * TS * LDB; };   // 0..3: window K, V of buffers 0 and 1; 4..11: far K, V per buffer and half
+  const int n_near = (q0 + (HALVES - 1) * TS - k_first) / TS + 1;
+  const int far0 = q0 / l > 1 ? q0 / l - 1 : 0;
+  const int far1 = HALVES == 2 && (q0 + TS) / l > 1 ? (q0 + TS) / l - 1 : 0;   // two halves: far0 <= far1
+  const int far_max = far0 > far1 ? far0 : far1;
+  const int n_trips = n_near > far_max ? n_near : far_max;
+  auto slot = [&](int i) { return KV + i * TS * LDB; };   // 0..3: window K, V of buffers 0 and 1; from 4: far K, V per buffer and half
   // this thread's piece of every tile copy: row threadIdx.x / 8 (+ multiples of THREADS / 8), 16-byte column threadIdx.x % 8
-  constexpr int THREADS = 256 / NS;
+  constexpr int THREADS = 128 * HALVES / NS;
   const uint32_t s_thr = (uint32_t)__cvta_generic_to_shared(KV + (threadIdx.x >> 3) * LDB + (threadIdx.x & 7) * 8);
   const int64_t g_thr = (row0 + (threadIdx.x >> 3)) * P.ld + h * D + (threadIdx.x & 7) * 8;
   const __nv_bfloat16 *Kt = P.K + g_thr, *Vt = P.V + g_thr;
@@ -123,17 +126,17 @@ __global__ void __launch_bounds__(256 / NS, MST_ATTN_FWD_BLOCKS) attn_fwd_mma_ke
       copy(2 * bf + 1, Vt, k_first + it * TS);
     }
     if (it < far0) {
-      copy(4 + 4 * bf, Kt, q0 - (it + 2) * l);
-      copy(5 + 4 * bf, Vt, q0 - (it + 2) * l);
+      copy(4 + 2 * HALVES * bf, Kt, q0 - (it + 2) * l);
+      copy(5 + 2 * HALVES * bf, Vt, q0 - (it + 2) * l);
     }
-    if (it < far1) {
+    if (HALVES == 2 && it < far1) {
       copy(6 + 4 * bf, Kt, q0 + TS - (it + 2) * l);
       copy(7 + 4 * bf, Vt, q0 + TS - (it + 2) * l);
     }
     async_commit();
   };
   copy(2, P.Q + g_thr, q0);             // queries through the second window buffer
-  copy(3, P.Q + g_thr, q0 + TS);
+  if (HALVES == 2) copy(3, P.Q + g_thr, q0 + TS);
   fetch(0, 0);
   async_wait_all();
   __syncthreads();
@@ -161,7 +164,7 @@ __global__ void __launch_bounds__(256 / NS, MST_ATTN_FWD_BLOCKS) attn_fwd_mma_ke
     if (it + 1 < n_trips) fetch(it + 1, buf ^ 1);
     if (it < (warp / HW ? far1 : far0)) {
       // the strided position: query r of this half sees key r of the half's tile only
-      const __nv_bfloat16* Ks = slot(4 + 4 * buf + 2 * (warp / HW));
+      const __nv_bfloat16* Ks = slot(4 + 2 * HALVES * buf + 2 * (warp / HW));
       const __nv_bfloat16* Vs = Ks + TS * LDB;
       const int c0 = (warp % HW) * WR;   // strip s: the 16 keys c0 + 16 s ... in line with its rows
       float sc[NS][2][4];
@@ -301,7 +304,7 @@ __global__ void __launch_bounds__(256 / NS, MST_ATTN_FWD_BLOCKS) attn_fwd_mma_ke
 // positive multiple of 64, 16-byte aligned pointers, leading dimensions multiples of 8.
 mst_status_t mst_attention_fwd_mma(const void* Q, const void* K, const void* V, int64_t ld, int32_t batch, int32_t seq_len,
                                    int32_t heads, int32_t stride, void* Out, int64_t ldo, float* lse, cudaStream_t s) {
-  if (seq_len % FQ != 0 || stride <= 0 || stride % TS != 0 || heads > 65535 || batch > 65535) return MST_ERR_SHAPE;
+  if (seq_len % 128 != 0 || stride <= 0 || stride % TS != 0 || heads > 65535 || batch > 65535) return MST_ERR_SHAPE;
   FwdParams P;
   P.Q = (const __nv_bfloat16*)Q; P.K = (const __nv_bfloat16*)K; P.V = (const __nv_bfloat16*)V;
   P.ld = ld;
@@ -309,17 +312,23 @@ mst_status_t mst_attention_fwd_mma(const void* Q, const void* K, const void* V, 
   P.ldo = ldo;
   P.lse = lse;
   P.batch = batch; P.seq = seq_len; P.heads = heads; P.stride = stride;
-  const size_t smem = (size_t)(12 * TS * LDB) * 2;
-  dim3 grid((unsigned)(seq_len / FQ), (unsigned)heads, (unsigned)batch);
-  int strips = 1;   // 16 rows per warp, eight warps per block
-  if (const char* e = getenv("MST_ATTN_FWD_STRIPS")) strips = atoi(e) == 2 ? 2 : 1;   // measurement override
-  if (strips == 2) {
-    MST_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_mma_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_fwd_mma_kernel<2><<<grid, 128, smem, s>>>(P); MST_COUNT_LAUNCH();
-  } else {
-    MST_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_mma_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attn_fwd_mma_kernel<1><<<grid, 256, smem, s>>>(P); MST_COUNT_LAUNCH();
+  int halves = 1, strips = 1;   // 64 queries per block, 16 rows per warp: four warps
+  if (const char* e = getenv("MST_ATTN_FWD_SHAPE")) {   // measurement override: "<halves><strips>", e.g. 21
+    halves = e[0] == '2' ? 2 : 1;
+    strips = e[0] && e[1] == '2' ? 2 : 1;
   }
+  const size_t smem = (size_t)((4 + 4 * halves) * TS * LDB) * 2;
+  dim3 grid((unsigned)(seq_len / (64 * halves)), (unsigned)heads, (unsigned)batch);
+#define MST_ATTN_LAUNCH(NS_, H_)                                                                                              \
+  do {                                                                                                                        \
+    MST_CUDA_TRY(cudaFuncSetAttribute(attn_fwd_mma_kernel<NS_, H_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));  \
+    attn_fwd_mma_kernel<NS_, H_><<<grid, 128 * H_ / NS_, smem, s>>>(P); MST_COUNT_LAUNCH();                                    \
+  } while (0)
+  if (halves == 2 && strips == 2) MST_ATTN_LAUNCH(2, 2);
+  else if (halves == 2) MST_ATTN_LAUNCH(1, 2);
+  else if (strips == 2) MST_ATTN_LAUNCH(2, 1);
+  else MST_ATTN_LAUNCH(1, 1);
+#undef MST_ATTN_LAUNCH
   MST_CUDA_TRY(cudaGetLastError());
   return MST_OK;
 }

@@ -72,18 +72,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ void load_a(uint32_t (&a)[4], const __nv_bfloat16* tile, int r0, int kb, int lane) {
   ldsm_x4(a, tile + (r0 + (lane & 7) + ((lane >> 3) & 1) * 8) * LDB + kb * 16 + (lane >> 4) * 8);
 }
-// c[16 x 8] += A strip (four k-steps over the 64 head dimensions, in registers) * rows n0 .. n0 + 8 of `tile`, transposed
-__device__ __forceinline__ void mma_rows(float (&c)[4], const uint32_t (&a)[4][4], const __nv_bfloat16* tile, int n0, int lane) {
-#pragma unroll
-  for (int k2 = 0; k2 < 2; ++k2) {
-    uint32_t b[4];
-    ldsm_x4(b, tile + (n0 + (lane & 7)) * LDB + k2 * 32 + (lane >> 3) * 8);
-    mma_bf16(c, a[2 * k2], b[0], b[1]);
-    mma_bf16(c, a[2 * k2 + 1], b[2], b[3]);
-  }
-}
-// The same product for NB neighbouring blocks of eight rows (n0 .. n0 + 8 NB) at once, k-step by k-step, so that
-// consecutive products go to different accumulators and none waits for the one issued just before it
+// c[nb][16 x 8] += A strip (four k-steps over the 64 head dimensions, in registers) * rows n0 + 8 nb .. + 8 of `tile`,
+// transposed, for NB neighbouring blocks of eight rows at once, k-step by k-step, so that consecutive products go to
+// different accumulators and none waits for the one issued just before it
 template <int NB>
 __device__ __forceinline__ void mma_rows_wide(float (&c)[NB][4], const uint32_t (&a)[4][4], const __nv_bfloat16* tile, int n0, int lane) {
 #pragma unroll

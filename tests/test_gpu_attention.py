@@ -56,8 +56,17 @@ def test_forward_strides_of_the_warp_level_kernel(batch, seq, heads, stride, pad
     _check_forward(batch, seq, heads, stride, pad)
 
 
-def _check_forward(batch, seq, heads, stride, pad):
-    p = mst_inputs.attention_problem(batch, seq, heads, 64, seed=900 + seq + stride)
+def test_forward_random_shapes_and_strides():
+    rng = np.random.default_rng(20241)
+    for case in range(10):
+        batch, heads = int(rng.integers(1, 3)), int(rng.integers(1, 3))
+        seq = 128 * int(rng.integers(1, 7))
+        stride = 64 * int(rng.integers(1, 9))
+        _check_forward(batch, seq, heads, stride, 8 * int(rng.integers(0, 2)), seed=5000 + case)
+
+
+def _check_forward(batch, seq, heads, stride, pad, seed=None):
+    p = mst_inputs.attention_problem(batch, seq, heads, 64, seed=900 + seq + stride if seed is None else seed)
     out, lse = _run(p, stride, pad=pad)
     Q, K, V = p.split()
     ref, lse_ref = att.strided_attention(Q, K, V, stride)
