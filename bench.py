@@ -231,10 +231,15 @@ def run_attention(args) -> None:
                                                             H, d, stride, gb, gb + 2 * C, gb + 4 * C, 3 * C))
         kept = sum(min(i, stride - 1) + 1 + i // stride for i in range(n))        # |S_i| summed over positions
         useful = 4.0 * d * kept * B * H                                            # scores + weighted sum, kept pairs
-        executed = 4.0 * d * n * (stride + 128) * B * H                            # the two tile products as issued
+        # the two tile products as issued: the tcgen05 kernel scores stride + 128 keys per query, the warp-level one
+        # stride + 32 (32-key steps around a 16-row strip's window); which one runs follows the entry point's rule
+        forced = os.environ.get("MST_ATTN_FWD", "")
+        kernel = forced if forced in ("tcgen05", "warp") else ("tcgen05" if stride >= 256 else "warp")
+        executed = 4.0 * d * n * (stride + (128 if kernel == "tcgen05" else 32)) * B * H
         bytes_alg = 4.0 * B * n * C * 2 + 4.0 * B * H * n
         print(json.dumps({
             "report": "strided_attention_fwd", "stride": stride, "batch": B, "seq_len": n, "heads": H, "head_dim": d,
+            "forward_kernel": kernel,
             "us": t * 1e6, "useful_tflops": useful / t / 1e12, "executed_tflops": executed / t / 1e12,
             "kept_fraction": kept / float(n * n),
             "roofline": {"bound": "hbm", "achieved": bytes_alg / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
