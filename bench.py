@@ -916,7 +916,7 @@ def main() -> None:
     }
     if rank == 0 and world == 1 and not args.no_sweeps:
         out["density_sweep"] = sweep_report("large", mst_inputs.CONFIG5_DENSITIES, args.sweep_reps, peaks, dev)
-        out["density_sweep_medium"] = sweep_report("medium", (0.25, 0.1, 0.05, 0.02), args.sweep_reps, peaks, dev)
+        out["density_sweep_medium"] = sweep_report("medium", mst_inputs.CONFIG5_DENSITIES, args.sweep_reps, peaks, dev)
         out["other_workloads"] = other_legs(args.sweep_reps, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline()
