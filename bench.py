@@ -375,9 +375,15 @@ def sweep_report(width_name: str, densities, reps: int, peaks, dev, path: str = 
                 L.set_path({"cuda_core": mst.MST_PATH_CUDA_CORE, "dense_tiles": mst.MST_PATH_TENSOR_CORE,
                             "sparse_tc": mst.MST_PATH_SPARSE_TC}[path])
             dW = torch.empty(max(nnz, 1), device=dev, dtype=torch.float32)
+            once = path in ("auto", "dense_tiles")
+            if once:
+                L.track_values(True)    # as in a training step: the values change once per repetition, so the dense
+                                        # image of W.M is rebuilt once for the forward and the input gradient together
 
             def all3():
                 X, dY = nxt()
+                if once:
+                    L.values_changed()
                 L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW)
             t, tmin = median_ms(all3, reps)
             path = mst.path_name(L.path_in_use())
@@ -405,7 +411,8 @@ def sweep_report(width_name: str, densities, reps: int, peaks, dev, path: str = 
                     "speedup_vs_dense_cublas": round(pt["dense_cublas_ms"] / pt["ms"], 3), "layers": pt["layers"]})
     return {"shapes": "gpt2-%s block (d_model %d), T=%d, bf16, uniform masks" % (width_name, width, T), "reps": reps,
             "requested_path": path,
-            "timing": "median of %d calls, CUDA events; inputs rotate over buffer sets larger than L2" % reps,
+            "timing": "median of %d repetitions of the three products, CUDA events; inputs rotate over buffer sets larger "
+                      "than L2; mst_values_changed once per repetition (one optimizer step)" % reps,
             "roofline_peaks": "measured HBM copy bandwidth and burst bf16 GEMM (%s)" % peaks["source"], "points": out}
 
 
