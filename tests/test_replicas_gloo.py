@@ -52,3 +52,18 @@ def test_single_process_needs_no_group():
     import bench
     assert bench.max_over_ranks(3.5, None, None) == 3.5
     assert bench.aggregate_value(1e12, 2, 1, 1000.0) == pytest.approx(2.0)
+
+
+def test_captured_traffic_is_tied_to_kernel_sources_and_workload(tmp_path, monkeypatch):
+    """The bench line prints DRAM traffic only for the kernel sources, workload and call kind the capture was taken on."""
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.captured_traffic("spmm_fwd", "another workload") is None
+    assert bench.captured_traffic("topology_update", bench.WORKLOAD) is None
+    t = bench.captured_traffic("sddmm_dw", bench.WORKLOAD)
+    if t is not None:                      # sources unchanged since the capture
+        per = bench.NCU_TRAFFIC["launches_per_kind"]
+        assert t == (bench.NCU_TRAFFIC["read"]["sddmm_dw"] + bench.NCU_TRAFFIC["write"]["sddmm_dw"]) / per
+    # any other digest of the sources: no figure
+    monkeypatch.setitem(bench.NCU_TRAFFIC, "sha256_16", "0" * 16)
+    assert bench.captured_traffic("sddmm_dw", bench.WORKLOAD) is None
