@@ -618,6 +618,52 @@ def test_value_tracking_reuses_and_refreshes_derived_operands():
         L.close()
 
 
+@pytest.mark.parametrize("track", [False, True])
+def test_products_through_the_fully_dense_state_and_back(track):
+    """A layer restored to every entry kept passes its values as the dense operand: products must follow in-place value
+    changes there with and without value tracking, and the image must come back when the layer is sparsified again."""
+    from cuda.bindings import runtime as cudart
+    O, I, T = 264, 328, 520
+    p = _problem(O, I, T, "bf16", 0.3, 8642)
+    L = make_layer(p)                         # capacity = O*I
+    L.set_path(mst.MST_PATH_TENSOR_CORE)
+    L.track_values(track)
+    X, dY = to_dev(p, "X"), to_dev(p, "dY")
+    Y = torch.empty((T, O), dtype=torch.bfloat16, device=dev())
+    dX = torch.empty((T, I), dtype=torch.bfloat16, device=dev())
+
+    def check(W, M):
+        dW = torch.empty((max(int(M.sum()), 1),), dtype=torch.float32, device=dev())
+        L.fwd(X, Y, T); L.bwd_x(dY, dX, T); L.sddmm(dY, X, T, dW)
+        torch.cuda.synchronize()
+        rows, cols = np.nonzero(M)
+        assert rel_err(host(Y), oracle.fwd(p.X, W, M)) <= TOL["bf16"]
+        assert rel_err(host(dX), oracle.bwd_x(p.dY, W, M)) <= TOL["bf16"]
+        assert rel_err(host(dW)[: len(rows)], oracle.dense_grad(p.dY, p.X)[rows, cols]) <= TOL["bf16"]
+
+    W = np.where(p.mask == 1, p.W, np.float32(0)).astype(np.float32)
+    M = p.mask.copy()
+    check(W, M)
+    rng = np.random.default_rng(3)
+    G = rng.standard_normal((O, I)).astype(np.float32)
+    W, M = _update_both(L, p, W, M, G, 0.1, O * I, 0.25, 9, 0)           # restored: every entry kept, grown ones zero
+    assert int(M.sum()) == O * I
+    check(W, M)
+    # an optimizer step in the dense state: new values written in place
+    W = mst_inputs.bf16_bits_to_f32(mst_inputs.f32_to_bf16_bits((0.02 * rng.standard_normal((O, I))).astype(np.float32)))
+    ptr, nnz = mst.mst_values(L.handle)
+    assert nnz == O * I
+    bits = torch.from_numpy(mst_inputs.f32_to_bf16_bits(W).view(np.int16)).to(dev())      # CSR order of a full matrix = row-major
+    (err,) = cudart.cudaMemcpy(ptr, bits.data_ptr(), 2 * nnz, cudart.cudaMemcpyKind.cudaMemcpyDeviceToDevice)
+    assert int(err) == 0
+    L.values_changed()
+    check(W, M)
+    W, M = _update_both(L, p, W, M, G, 0.2, int(0.4 * O * I), 0.25, 9, 1)  # sparsified again
+    check(W, M)
+    assert mst.mst_device_error_flags() == 0
+    L.close()
+
+
 def test_path_in_use_reports_the_resolved_path():
     p = _problem(64, 64, 8, "bf16", 0.1, 1)
     L = make_layer(p)
